@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the forward-convolution hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-general]
+
+One "step" is one pass of the single-channel hot path over the large single-channel
+configuration (1 x 1 x 4096 x 4096 image, 32 filters of 5 x 5): filter staging, tile staging,
+register-window FMA loop and vector stores, all inside conv2d_fwd_single_channel.  The general-case
+configurations are timed as well (tensor-core and fp32 variants) and reported under "general" in the
+same JSON line.  Prints exactly one JSON line on stdout (rank 0).
+
+Multi-GPU: the path has no exchange step; with --gpus N every rank runs an independent replica of the
+workload on its own GPU (weak scaling, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import numpy as np  # noqa: E402
+
+from workloads import CONFIGS, make_inputs  # noqa: E402
+
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+TF32_FLOP_PER_CLK_PER_SM = 4096     # dense TF32 = half the bf16 rate per clock
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_TF32_TFLOPS = 1125.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def load_peaks():
+    path = ROOT / "MEASURED_PEAKS.json"
+    if path.exists():
+        p = json.loads(path.read_text())
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS, bf16_tflops_sustained=1400.0,
+                sm_max_mhz=1965.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock, power and throttle reasons through NVML in a thread while the timed region runs."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, gpu_index: int, period_s: float = 0.002):
+        self.gpu_index, self.period_s = gpu_index, period_s
+        self.samples, self.reasons, self.power = [], set(), []
+        self.sm_max = None
+        self._stop = False
+        self._thread = None
+        self._active = False
+
+    def _run(self, nv, handle):
+        while not self._stop:
+            if self._active:
+                try:
+                    self.samples.append(nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM))
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(handle)
+                    for bit, name in self.REASONS.items():
+                        if mask & bit:
+                            self.reasons.add(name)
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(handle) / 1000.0)
+                except Exception:
+                    pass
+            time.sleep(self.period_s)
+
+    def start(self):
+        """Starts the thread (idle); mark the timed region with begin()/end()."""
+        try:
+            import threading
+            import pynvml as nv
+            nv.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            index = self.gpu_index
+            if visible:
+                ids = [v.strip() for v in visible.split(",") if v.strip()]
+                if self.gpu_index < len(ids) and ids[self.gpu_index].isdigit():
+                    index = int(ids[self.gpu_index])
+            handle = nv.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM)
+            self._thread = threading.Thread(target=self._run, args=(nv, handle), daemon=True)
+            self._thread.start()
+        except Exception:
+            self._thread = None
+
+    def begin(self):
+        self._active = True
+
+    def end(self):
+        self._active = False
+
+    def stop(self) -> dict:
+        self._stop = True
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": sorted(self.reasons), "samples": len(self.samples),
+               "power_w_max": max(self.power) if self.power else None}
+        if self.samples:
+            out["sm_mhz"] = statistics.median(self.samples)
+        return out
+
+
+def cpu_model():
+    try:
+        for line in Path("/proc/cpuinfo").read_text().splitlines():
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def time_oracle_sample(cfg, target_seconds: float):
+    """Times the oracle, as it stands, on a bounded sample of output maps of `cfg`."""
+    import oracle
+    x, w = make_inputs(cfg)
+    flops_per_map = 2 * cfg.N * cfg.C * cfg.R * cfg.S * cfg.P * cfg.Q
+    t0 = time.perf_counter()
+    oracle.conv2d_oracle_range(x, w, k_range=(0, 1))
+    t1 = time.perf_counter() - t0
+    maps = int(max(1, min(cfg.K - 1, round(target_seconds / max(t1, 1e-6)))))
+    t0 = time.perf_counter()
+    oracle.conv2d_oracle_range(x, w, k_range=(1, 1 + maps))
+    t = time.perf_counter() - t0
+    return dict(value=flops_per_map * maps / t / 1e9, unit="GFLOP/s", cores=oracle.oracle_threads(),
+                kind="oracle", sample=f"{cfg.name}: all outputs of {maps} of {cfg.K} maps, {t:.1f} s, {cpu_model()}")
+
+
+def run_reference(args, rank: int):
+    """The reference arm: the CPU oracle on the host cores, bounded sample per step."""
+    if rank != 0:
+        return
+    import oracle
+    cfg = CONFIGS[args.workload]
+    x, w = make_inputs(cfg)
+    maps = 2
+    flops = 2 * cfg.N * cfg.C * cfg.R * cfg.S * cfg.P * cfg.Q * maps
+    for _ in range(min(args.warmup, 1)):
+        oracle.conv2d_oracle_range(x, w, k_range=(0, maps))
+    steps = min(args.steps, 5)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.conv2d_oracle_range(x, w, k_range=(0, maps))
+    t = (time.perf_counter() - t0) / steps
+    val = flops / t / 1e9
+    sample = f"{cfg.name}: all outputs of {maps} of {cfg.K} maps per step, {cpu_model()}"
+    print(json.dumps({
+        "impl": "reference", "metric": "conv_fwd_gflops", "value": val, "unit": "GFLOP/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": t * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, **cfg.as_dict()},
+        "cpu_baseline": {"value": val, "unit": "GFLOP/s", "cores": oracle.oracle_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def event_ms(fn, torch, iters=1):
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(iters):
+        fn()
+    stop.record()
+    stop.synchronize()
+    return start.elapsed_time(stop) / iters
+
+
+def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
+    """Times every general-case configuration, tensor-core and fp32 variants, cold and warm L2."""
+    out = []
+    dev = torch.device("cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    for name in ["cfg3", "cfg4", "cfg5_r1", "cfg5_r3", "cfg5_r5", "cfg5_r7"]:
+        cfg = CONFIGS[name]
+        x, w = make_inputs(cfg)
+        xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
+        yd = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), device=dev, dtype=torch.float32)
+        for algo_name, algo in (("tf32", lib.ALGO_TF32), ("ffma", lib.ALGO_FFMA)):
+            try:
+                ws_bytes = lib.conv2d_fwd_workspace_size(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, algo)
+            except lib.Conv2dError:
+                out.append({"workload": name, "algo": algo_name, "unavailable": "no instance"})
+                continue
+            ws = torch.zeros(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+
+            def call(flags=0):
+                lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
+                                       cfg.K, cfg.R, cfg.S, algo, ws.data_ptr(), ws_bytes, flags, stream)
+            for _ in range(3):
+                call()
+            lib.conv2d_get_status(ws.data_ptr(), stream)
+            cold = []
+            for _ in range(10):
+                flush.zero_()
+                cold.append(event_ms(call, torch))
+            warm = event_ms(call, torch, iters=20)
+            packed = event_ms(lambda: call(lib.FLAG_WEIGHTS_PACKED), torch, iters=20) if algo == lib.ALGO_TF32 else None
+            lib.conv2d_get_status(ws.data_ptr(), stream)
+            t_cold, t_warm = statistics.median(cold), warm
+            if algo == lib.ALGO_TF32:
+                pipe_peak = peaks["bf16_tflops"] / 2.0     # TF32 dense rate is half of bf16 per clock
+                bound = "tensor"
+            else:
+                pipe_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+                bound = "alu"
+            t_pipe = cfg.flops / (pipe_peak * 1e12) * 1e3
+            t_hbm = cfg.compulsory_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+            entry = {
+                "workload": name, "algo": algo_name, "ms_cold_l2": t_cold, "ms_warm_l2": t_warm,
+                "gflops_cold": cfg.flops / t_cold / 1e6, "gflops_warm": cfg.flops / t_warm / 1e6,
+                "roofline": {"bound": bound if t_pipe >= t_hbm else "hbm",
+                             "pipe_peak_tflops": pipe_peak, "pipe_frac_warm": t_pipe / t_warm,
+                             "pipe_frac_cold": t_pipe / t_cold, "hbm_frac_cold": t_hbm / t_cold,
+                             "frac": max(t_pipe, t_hbm) / t_cold, "peaks": peaks["source"]},
+            }
+            if packed is not None:
+                entry["ms_warm_l2_weights_prepacked"] = packed
+            out.append(entry)
+        del xd, wd, yd
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
+    ap.add_argument("--no-general", action="store_true", help="skip the general-case configurations")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import paper_1705_10591_b200 as lib
+    from paper_1705_10591_b200 import build as lib_build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    lib_build.build()
+    lib.load_library()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+
+    cfg = CONFIGS[args.workload]
+    single = cfg.C == 1
+    x, w = make_inputs(cfg)
+    x_host = torch.from_numpy(x).pin_memory()
+    w_host = torch.from_numpy(w).pin_memory()
+    xd, wd = x_host.to(dev), w_host.to(dev)
+    yd = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), device=dev, dtype=torch.float32)
+    algo = lib.ALGO_FFMA if single else lib.ALGO_AUTO
+    ws_bytes = 0 if single else lib.conv2d_fwd_workspace_size(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, algo)
+    ws = torch.zeros(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
+
+    def step():
+        if single:
+            lib.conv2d_fwd_single_channel(xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.H, cfg.W,
+                                          cfg.K, cfg.R, cfg.S, 0, 0, 0, stream)
+        else:
+            lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
+                                   cfg.K, cfg.R, cfg.S, algo, ws.data_ptr(), ws_bytes, 0, stream)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    working_set = cfg.compulsory_bytes
+    flush_between = working_set < 2 * 126 * 1024 * 1024
+    for _ in range(args.warmup):
+        step()
+    lib.conv2d_get_status(ws.data_ptr() if ws_bytes else 0, stream)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    barrier()
+    sampler.begin()
+    launches0 = lib.conv2d_launch_count()
+    per_step = []
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if flush_between:
+        for _ in range(args.steps):
+            flush.zero_()
+            per_step.append(event_ms(step, torch))
+        total_ms = sum(per_step)
+    else:
+        start.record()
+        for _ in range(args.steps):
+            step()
+        stop.record()
+        stop.synchronize()
+        total_ms = start.elapsed_time(stop)
+    barrier()
+    sampler.end()
+    launches = lib.conv2d_launch_count() - launches0
+    clocks = sampler.stop()
+    lib.conv2d_get_status(ws.data_ptr() if ws_bytes else 0, stream)
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * cfg.flops / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    y_host = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), dtype=torch.float32).pin_memory()
+
+    def e2e_step():
+        lib.conv2d_fwd_host(x_host.data_ptr(), w_host.data_ptr(), y_host.data_ptr(),
+                            xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
+                            cfg.K, cfg.R, cfg.S, algo, ws.data_ptr() if ws_bytes else 0, ws_bytes, stream)
+    e2e_step()
+    e2e_steps = max(2, min(args.steps, 5))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()          # synchronises the stream itself
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * cfg.flops / e2e_s / 1e9, "unit": "GFLOP/s",
+           "h2d_bytes_per_step": int(x.nbytes + w.nbytes), "d2h_bytes_per_step": int(y_host.numel() * 4),
+           "ms_per_step": e2e_s * 1e3}
+
+    # ---- roofline of the dominant kernel (per launch = one step)
+    t_kernel_s = ms_per_step * 1e-3
+    fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # TFLOP/s at max clock
+    t_hbm = cfg.compulsory_bytes / (peaks["hbm_gbs"] * 1e9)
+    if single:
+        t_pipe, pipe_name, pipe_peak = cfg.flops / (fp32_peak * 1e12), "alu", fp32_peak
+    else:
+        pipe_peak = peaks["bf16_tflops"] / 2.0
+        t_pipe, pipe_name = cfg.flops / (pipe_peak * 1e12), "tensor"
+    if t_pipe >= t_hbm:
+        roof = {"bound": pipe_name, "achieved": cfg.flops / t_kernel_s / 1e12, "peak": pipe_peak, "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": cfg.compulsory_bytes / t_kernel_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof.update({
+        "traffic": None, "peaks": peaks["source"],
+        "algorithmic_bytes_per_launch": cfg.compulsory_bytes, "flops_per_launch": cfg.flops,
+        "hbm_gbs_achieved": cfg.compulsory_bytes / t_kernel_s / 1e9,
+        "hbm_frac_of_measured": cfg.compulsory_bytes / t_kernel_s / 1e9 / peaks["hbm_gbs"],
+        "hbm_frac_of_nominal_8tbs": cfg.compulsory_bytes / t_kernel_s / 1e9 / 8000.0,
+        "alu_tflops_achieved": cfg.flops / t_kernel_s / 1e12,
+        "alu_frac_at_max_clock": cfg.flops / t_kernel_s / 1e12 / fp32_peak,
+    })
+    traffic_file = ROOT / "profiles" / "traffic.json"
+    if traffic_file.exists():
+        roof["traffic"] = json.loads(traffic_file.read_text()).get(args.workload)
+    if clocks.get("sm_mhz"):
+        at_clock = SM_COUNT * FP32_LANES_PER_SM * 2 * clocks["sm_mhz"] * 1e6 / 1e12
+        roof["alu_frac_at_sampled_clock"] = cfg.flops / t_kernel_s / 1e12 / at_clock
+
+    result = {
+        "metric": "conv_fwd_gflops", "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, **cfg.as_dict(), "parallelism": f"replicas x{world}",
+                   "l2": "flushed between timed steps" if flush_between else
+                         "inputs+outputs per step (2.2 GB) exceed the 126 MB L2"},
+        "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "power_w_max")},
+        "e2e": e2e, "gpu_launches": int(launches), "roofline": roof,
+    }
+
+    if rank == 0 and world == 1:
+        if not args.no_general:
+            result["general"] = bench_general(torch, lib, peaks, flush, clocks.get("sm_mhz"))
+        if not args.no_cpu_baseline:
+            result["cpu_baseline"] = time_oracle_sample(cfg, 12.0)
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

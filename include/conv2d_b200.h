@@ -1,0 +1,149 @@
+/*
+ * conv2d_b200 -- forward 2-D convolution for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The operation is the one optimised by Chen, Chen, Chen and Hu, "Optimizing
+ * Memory Efficiency for Convolution Kernels on Kepler GPUs" (DAC 2017): a
+ * C-channel image convolved with a bank of filters, one output map per filter
+ * (Fig. 3a), in the paper's two cases -- one input channel (Section 3,
+ * Algorithm 1) and many input channels (Section 4, Algorithm 2).
+ *
+ *     y[n,k,p,q] = sum_{c,r,s} x[n,c,p+r,q+s] * w[k,c,r,s]
+ *     P = H-R+1, Q = W-S+1        (stride 1, no padding, filter not flipped)
+ *
+ * Symbols: N images, C input channels, H x W image, K filters, R x S taps,
+ * P x Q output map.  (The paper has no batch, calls the filter count F and the
+ * square filter size K, and uses H, W for its thread-block tile.)  Outputs are
+ * anchored at the top-left pixel of their window: a tile needs extra input
+ * only beyond its right and bottom edges (Section 3.1).
+ *
+ * Conventions shared by every entry point
+ *   - x, w, y and workspace are DEVICE pointers unless an argument is named
+ *     *_host.  Tensors are dense, contiguous, row-major fp32: x[N][C][H][W],
+ *     w[K][C][R][S], y[N][K][P][Q].  Base addresses must be 16-byte aligned.
+ *   - All memory is owned by the caller.  y must not overlap x, w or the
+ *     workspace.  y is overwritten (no accumulation into prior contents).
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*;
+ *     NULL is the default stream) and return without synchronising, except
+ *     conv2d_get_status and conv2d_fwd_host, which wait for the stream.
+ *   - The library allocates no device memory.  There is no CPU fallback: on
+ *     a machine without a usable sm_100 device every launch entry returns
+ *     CONV2D_ERR_ARCH or CONV2D_ERR_CUDA.
+ *   - Errors are reported by return code only; nothing is thrown.  Argument
+ *     errors are detected before anything is enqueued.
+ */
+#ifndef CONV2D_B200_H
+#define CONV2D_B200_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CONV2D_OK = 0,
+    CONV2D_ERR_NULL = 1,           /* a required pointer is NULL */
+    CONV2D_ERR_SHAPE = 2,          /* non-positive extent, R > H, S > W, or a size beyond 32-bit element indexing */
+    CONV2D_ERR_ALIGN = 3,          /* x, w, y or workspace not 16-byte aligned */
+    CONV2D_ERR_WORKSPACE = 4,      /* workspace smaller than conv2d_fwd_workspace_size reports */
+    CONV2D_ERR_UNSUPPORTED = 5,    /* no kernel instance for this algorithm/shape combination */
+    CONV2D_ERR_ARCH = 6,           /* current device is not compute capability 10.x */
+    CONV2D_ERR_CUDA = 7,           /* a CUDA runtime call failed (cudaGetLastError is left set) */
+    CONV2D_ERR_DEVICE_TIMEOUT = 8  /* a bounded on-device wait expired; outputs of that launch are invalid */
+} conv2d_status_t;
+
+typedef enum {
+    CONV2D_ALGO_AUTO = 0,  /* tensor cores (TF32) where an instance exists, else fp32 FMA */
+    CONV2D_ALGO_FFMA = 1,  /* fp32 fused multiply-add on the CUDA cores; error <= 1e-5 * sum|x*w| */
+    CONV2D_ALGO_TF32 = 2   /* operands rounded to TF32, fp32 accumulation on tcgen05; error <= 2e-3 * sum|x*w| */
+} conv2d_algo_t;
+
+/* `flags` bits */
+enum {
+    /* The workspace already holds the filters of this exact call (same w contents,
+       K, C, R, S and algorithm) in the kernel's internal order, left there by an
+       earlier call: skip the re-ordering launch. */
+    CONV2D_FLAG_WEIGHTS_PACKED = 1u
+};
+
+/*
+ * Workspace query (host only, touches no device).
+ * Writes to *bytes the workspace size conv2d_fwd_general needs for this shape
+ * and algorithm: 0 for CONV2D_ALGO_FFMA; for TF32 (and AUTO) a 256-byte status
+ * block followed by the filters re-ordered for the tensor-core kernel (the
+ * counterpart of the transposed, padded filter block that Section 4.2 / Fig. 6
+ * builds in shared memory, done once per call instead of once per thread block).
+ * Returns CONV2D_ERR_UNSUPPORTED if `algo` is TF32 and no instance fits.
+ */
+conv2d_status_t conv2d_fwd_workspace_size(int N, int C, int H, int W, int K, int R, int S,
+                                          conv2d_algo_t algo, size_t* bytes);
+
+/*
+ * Special case, one input channel (Section 3, Algorithm 1).
+ *   x [N][1][H][W], w [K][1][R][S], y [N][K][P][Q]; fp32 FMA arithmetic.
+ * The filters are first copied (device to device, on the stream) into a
+ * constant-memory bank of 16384 floats that the whole device shares
+ * (Section 3.2: the filters of this case are small and live in constant
+ * memory); K*R*S must not exceed 16384 (CONV2D_ERR_UNSUPPORTED otherwise).
+ * Because that bank is one per device, single-channel calls issued on
+ * DIFFERENT streams must not overlap in time; calls on one stream are ordered.
+ * workspace may be NULL (none is used); flags must be 0.
+ */
+conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float* y,
+                                          int N, int H, int W, int K, int R, int S,
+                                          void* workspace, size_t workspace_bytes,
+                                          unsigned flags, void* cuda_stream);
+
+/*
+ * General case, C input channels (Section 4, Algorithm 2).
+ *   x [N][C][H][W], w [K][C][R][S], y [N][K][P][Q].
+ * algo = FFMA: register-tiled fp32 kernel (each thread accumulates a block of
+ *   filters x horizontally adjacent outputs, as in Section 4.1-4.2); no workspace.
+ * algo = TF32: implicit-GEMM on the tcgen05 tensor cores with the accumulator
+ *   in tensor memory; needs the workspace reported by conv2d_fwd_workspace_size
+ *   (16-byte aligned).  Its first 256 bytes are a status block that each call
+ *   clears on the stream before launching.
+ * algo = AUTO: TF32 when an instance exists and the workspace suffices, else FFMA.
+ * C == 1 is accepted and gives the same result as the single-channel entry.
+ */
+conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
+                                   int N, int C, int H, int W, int K, int R, int S,
+                                   conv2d_algo_t algo,
+                                   void* workspace, size_t workspace_bytes,
+                                   unsigned flags, void* cuda_stream);
+
+/*
+ * Host-buffer convenience path (no counterpart in the paper): x_host and
+ * w_host are copied to the caller's device buffers x, w on the stream, the
+ * convolution runs (single-channel kernel when C == 1, else conv2d_fwd_general
+ * with `algo`), y is copied back into y_host and the stream is synchronised.
+ * Host buffers should be page-locked for the copies to run at full speed.
+ * Returns the first error met, or the device status after synchronising.
+ */
+conv2d_status_t conv2d_fwd_host(const float* x_host, const float* w_host, float* y_host,
+                                float* x, float* w, float* y,
+                                int N, int C, int H, int W, int K, int R, int S,
+                                conv2d_algo_t algo,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Waits for `cuda_stream`, then reads the status block at the start of
+ * `workspace` (NULL workspace: only waits).  Returns CONV2D_OK,
+ * CONV2D_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded wait, or
+ * CONV2D_ERR_CUDA if the stream reported an error.
+ */
+conv2d_status_t conv2d_get_status(const void* workspace, void* cuda_stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char* conv2d_status_string(conv2d_status_t status);
+
+/*
+ * Number of kernels this library has launched in the calling process since it
+ * was loaded (all entry points, all streams); for accounting in benchmarks.
+ */
+unsigned long long conv2d_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONV2D_B200_H */

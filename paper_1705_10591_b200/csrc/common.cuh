@@ -1,0 +1,37 @@
+// Internal declarations shared by the translation units of libconv2d_b200.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "conv2d_b200.h"
+
+namespace conv2d_b200 {
+
+// Problem extents, library symbols (N images, C channels, H x W image, K filters, R x S taps).
+struct Shape {
+    int N, C, H, W, K, R, S, P, Q;
+};
+
+// Capacity of the per-device constant-memory filter bank of the single-channel kernel, in floats.
+constexpr int kConstFilterFloats = 16384;
+
+// Bytes reserved at the start of the workspace for the device status word.
+constexpr size_t kStatusBytes = 256;
+
+// Every kernel launch goes through this so that conv2d_launch_count() is exact.
+void count_launch(int launches = 1);
+
+// Launchers.  Each returns CONV2D_OK, CONV2D_ERR_UNSUPPORTED (no instance) or CONV2D_ERR_CUDA.
+conv2d_status_t launch_single_channel(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);
+conv2d_status_t launch_general_ffma(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);
+conv2d_status_t launch_direct_fallback(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);
+
+// Tensor-core path.
+bool tf32_supported(const Shape& sh);
+size_t tf32_workspace_bytes(const Shape& sh);   // includes the status block
+conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
+                                    void* workspace, bool weights_packed, cudaStream_t stream);
+
+}  // namespace conv2d_b200

@@ -1,0 +1,168 @@
+// C-ABI boundary: argument validation, dispatch and the host-buffer convenience path.
+#include <atomic>
+
+#include "common.cuh"
+
+namespace conv2d_b200 {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int launches) { g_launches.fetch_add((unsigned long long)launches, std::memory_order_relaxed); }
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates extents and fills the derived output size.
+conv2d_status_t make_shape(int N, int C, int H, int W, int K, int R, int S, Shape* sh)
+{
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || R <= 0 || S <= 0) return CONV2D_ERR_SHAPE;
+    if (R > H || S > W) return CONV2D_ERR_SHAPE;
+    const long long P = H - R + 1, Q = W - S + 1;
+    const long long lim = 0x7fffffffLL;   // kernels index single tensors with 32-bit element counts per image plane set
+    if ((long long)N * C * H * W > 4 * lim || (long long)N * K * P * Q > 4 * lim) return CONV2D_ERR_SHAPE;
+    if ((long long)C * H * W > lim || (long long)K * P * Q > lim || (long long)K * C * R * S > lim) return CONV2D_ERR_SHAPE;
+    *sh = Shape{N, C, H, W, K, R, S, (int)P, (int)Q};
+    return CONV2D_OK;
+}
+
+conv2d_status_t check_device()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return CONV2D_ERR_CUDA;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return CONV2D_ERR_CUDA;
+    return major == 10 ? CONV2D_OK : CONV2D_ERR_ARCH;
+}
+
+}  // namespace
+}  // namespace conv2d_b200
+
+using namespace conv2d_b200;
+
+extern "C" {
+
+conv2d_status_t conv2d_fwd_workspace_size(int N, int C, int H, int W, int K, int R, int S,
+                                          conv2d_algo_t algo, size_t* bytes)
+{
+    if (!bytes) return CONV2D_ERR_NULL;
+    *bytes = 0;
+    Shape sh;
+    conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
+    if (st != CONV2D_OK) return st;
+    switch (algo) {
+        case CONV2D_ALGO_FFMA: return CONV2D_OK;
+        case CONV2D_ALGO_TF32:
+            if (!tf32_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
+            *bytes = tf32_workspace_bytes(sh);
+            return CONV2D_OK;
+        case CONV2D_ALGO_AUTO:
+            if (tf32_supported(sh)) *bytes = tf32_workspace_bytes(sh);
+            return CONV2D_OK;
+        default: return CONV2D_ERR_UNSUPPORTED;
+    }
+}
+
+conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float* y,
+                                          int N, int H, int W, int K, int R, int S,
+                                          void* workspace, size_t workspace_bytes,
+                                          unsigned flags, void* cuda_stream)
+{
+    (void)workspace; (void)workspace_bytes;
+    if (!x || !w || !y) return CONV2D_ERR_NULL;
+    Shape sh;
+    conv2d_status_t st = make_shape(N, 1, H, W, K, R, S, &sh);
+    if (st != CONV2D_OK) return st;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return CONV2D_ERR_ALIGN;
+    if (flags != 0) return CONV2D_ERR_UNSUPPORTED;
+    if (N > 65535) return CONV2D_ERR_UNSUPPORTED;
+    st = check_device();
+    if (st != CONV2D_OK) return st;
+    return launch_single_channel(x, w, y, sh, static_cast<cudaStream_t>(cuda_stream));
+}
+
+conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
+                                   int N, int C, int H, int W, int K, int R, int S,
+                                   conv2d_algo_t algo,
+                                   void* workspace, size_t workspace_bytes,
+                                   unsigned flags, void* cuda_stream)
+{
+    if (!x || !w || !y) return CONV2D_ERR_NULL;
+    Shape sh;
+    conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
+    if (st != CONV2D_OK) return st;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (flags & ~(unsigned)CONV2D_FLAG_WEIGHTS_PACKED) return CONV2D_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    bool use_tf32 = false;
+    if (algo == CONV2D_ALGO_TF32) {
+        if (!tf32_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
+        if (!workspace) return CONV2D_ERR_NULL;
+        if (workspace_bytes < tf32_workspace_bytes(sh)) return CONV2D_ERR_WORKSPACE;
+        use_tf32 = true;
+    } else if (algo == CONV2D_ALGO_AUTO) {
+        use_tf32 = tf32_supported(sh) && workspace && workspace_bytes >= tf32_workspace_bytes(sh);
+    } else if (algo != CONV2D_ALGO_FFMA) {
+        return CONV2D_ERR_UNSUPPORTED;
+    }
+    st = check_device();
+    if (st != CONV2D_OK) return st;
+    if (use_tf32)
+        return launch_general_tf32(x, w, y, sh, workspace, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0, stream);
+    return launch_general_ffma(x, w, y, sh, stream);
+}
+
+conv2d_status_t conv2d_fwd_host(const float* x_host, const float* w_host, float* y_host,
+                                float* x, float* w, float* y,
+                                int N, int C, int H, int W, int K, int R, int S,
+                                conv2d_algo_t algo,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!x_host || !w_host || !y_host || !x || !w || !y) return CONV2D_ERR_NULL;
+    Shape sh;
+    conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
+    if (st != CONV2D_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t xb = (size_t)N * C * H * W * sizeof(float);
+    const size_t wb = (size_t)K * C * R * S * sizeof(float);
+    const size_t yb = (size_t)N * K * sh.P * sh.Q * sizeof(float);
+    if (cudaMemcpyAsync(x, x_host, xb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CONV2D_ERR_CUDA;
+    if (cudaMemcpyAsync(w, w_host, wb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CONV2D_ERR_CUDA;
+    if (C == 1 && algo != CONV2D_ALGO_TF32)
+        st = conv2d_fwd_single_channel(x, w, y, N, H, W, K, R, S, nullptr, 0, 0, cuda_stream);
+    else
+        st = conv2d_fwd_general(x, w, y, N, C, H, W, K, R, S, algo, workspace, workspace_bytes, 0, cuda_stream);
+    if (st != CONV2D_OK) return st;
+    if (cudaMemcpyAsync(y_host, y, yb, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return CONV2D_ERR_CUDA;
+    return conv2d_get_status(workspace, cuda_stream);
+}
+
+conv2d_status_t conv2d_get_status(const void* workspace, void* cuda_stream)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return CONV2D_ERR_CUDA;
+    if (!workspace) return CONV2D_OK;
+    unsigned word = 0;
+    if (cudaMemcpy(&word, workspace, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) return CONV2D_ERR_CUDA;
+    return word == 0 ? CONV2D_OK : CONV2D_ERR_DEVICE_TIMEOUT;
+}
+
+const char* conv2d_status_string(conv2d_status_t status)
+{
+    switch (status) {
+        case CONV2D_OK: return "ok";
+        case CONV2D_ERR_NULL: return "a required pointer is NULL";
+        case CONV2D_ERR_SHAPE: return "invalid shape (non-positive extent, filter larger than image, or too large)";
+        case CONV2D_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case CONV2D_ERR_WORKSPACE: return "workspace too small";
+        case CONV2D_ERR_UNSUPPORTED: return "no kernel instance for this algorithm/shape/flags";
+        case CONV2D_ERR_ARCH: return "device is not compute capability 10.x (B200)";
+        case CONV2D_ERR_CUDA: return "CUDA runtime error";
+        case CONV2D_ERR_DEVICE_TIMEOUT: return "a bounded on-device wait expired";
+        default: return "unknown status";
+    }
+}
+
+unsigned long long conv2d_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,199 @@
+// General case on the fp32 CUDA cores (Section 4, Algorithm 2), plus a shape-agnostic direct kernel.
+//
+// Kept from the paper's design:
+//   * grid = (blocks of filters) x (image blocks); a thread block covers the same image block
+//     over all C channels for kTileK adjacent filters (Section 4.1);
+//   * channels are staged kCB at a time in shared memory: the image block with its right/bottom
+//     halo as it lies in memory, the filters transposed so that adjacent filters are adjacent
+//     words (Section 4.2, Fig. 6);
+//   * a thread accumulates kThrK filters x kThrQ horizontally adjacent outputs in registers,
+//     keeps one input row segment of kThrQ+S-1 pixels in registers and reuses it for the S
+//     horizontal taps (Section 4.2); filter values are read as 128-bit units, image pixels are
+//     broadcast to the threads that differ only in their filter group.
+// Changed for B200: register tile 8 x 8 with 128-bit shared-memory reads on both operands;
+// the output is written with 128-bit stores per filter row segment where alignment allows.
+#include "common.cuh"
+
+namespace conv2d_b200 {
+namespace {
+
+constexpr int kTileK = 64;    // filters per thread block (the paper's F_TB)
+constexpr int kTileW = 32;    // output columns per thread block
+constexpr int kTileH = 8;     // output rows per thread block
+constexpr int kThrK = 8;      // filters per thread (F_T)
+constexpr int kThrQ = 8;      // adjacent outputs per thread (W_T)
+constexpr int kThreads = (kTileK / kThrK) * (kTileW * kTileH / kThrQ);   // 8 x 32 = 256
+
+template <int R, int S, int CB>
+struct Smem {
+    static constexpr int kRows = kTileH + R - 1;
+    static constexpr int kPitch = (kTileW + S - 1 + 3 + 3) / 4 * 4;   // room for whole 128-bit reads past the halo
+    float img[CB][kRows][kPitch];
+    float flt[CB][R * S][kTileK + 4];   // +4: transposed filter stores spread over banks, 128-bit reads stay aligned
+};
+
+template <int R, int S, int CB>
+__global__ void __launch_bounds__(kThreads)
+general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
+                    int C, int H, int W, int K, int P, int Q, int tiles_q, int vec_st)
+{
+    using SM = Smem<R, S, CB>;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SM& sm = *reinterpret_cast<SM*>(smem_raw);
+
+    const int tid = threadIdx.x;
+    const int tx = tid % (kTileK / kThrK);            // filter group: adjacent threads, adjacent filter units
+    const int ty = tid / (kTileK / kThrK);            // output segment
+    const int seg_row = ty / (kTileW / kThrQ);
+    const int seg_col = (ty % (kTileW / kThrQ)) * kThrQ;
+
+    const int k0 = blockIdx.y * kTileK;
+    const int tq = blockIdx.x % tiles_q, tp = blockIdx.x / tiles_q;
+    const int p0 = tp * kTileH, q0 = tq * kTileW;
+    const int n = blockIdx.z;
+    const float* xin = x + (size_t)n * C * H * W;
+
+    float acc[kThrK][kThrQ];
+#pragma unroll
+    for (int i = 0; i < kThrK; ++i)
+#pragma unroll
+        for (int j = 0; j < kThrQ; ++j) acc[i][j] = 0.f;
+
+    constexpr int NV = (kThrQ + S - 1 + 3) / 4;       // 128-bit reads per input row segment
+
+    for (int c0 = 0; c0 < C; c0 += CB) {
+        // ---- stage CB channels: image block with halo, filters transposed to [tap][filter] ----
+        for (int idx = tid; idx < CB * SM::kRows * SM::kPitch; idx += kThreads) {
+            const int col = idx % SM::kPitch;
+            const int row = (idx / SM::kPitch) % SM::kRows;
+            const int cc = idx / (SM::kPitch * SM::kRows);
+            const int c = c0 + cc, h = p0 + row, ww = q0 + col;
+            float v = 0.f;
+            if (c < C && h < H && ww < W) v = __ldg(xin + ((size_t)c * H + h) * W + ww);
+            sm.img[cc][row][col] = v;
+        }
+        for (int idx = tid; idx < CB * R * S * kTileK; idx += kThreads) {
+            // consecutive threads walk the taps of one filter (contiguous in memory), then the channels
+            const int t = idx % (R * S);
+            const int cc = (idx / (R * S)) % CB;
+            const int kk = idx / (R * S * CB);
+            const int c = c0 + cc, k = k0 + kk;
+            float v = 0.f;
+            if (c < C && k < K) v = __ldg(w + ((size_t)k * C + c) * (R * S) + t);
+            sm.flt[cc][t][kk] = v;
+        }
+        __syncthreads();
+
+#pragma unroll 1
+        for (int cc = 0; cc < CB; ++cc) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float img[4 * NV];
+                const float4* src = reinterpret_cast<const float4*>(&sm.img[cc][seg_row + r][seg_col]);
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const float4 t = src[v];
+                    img[4 * v + 0] = t.x; img[4 * v + 1] = t.y; img[4 * v + 2] = t.z; img[4 * v + 3] = t.w;
+                }
+#pragma unroll
+                for (int s = 0; s < S; ++s) {
+                    float flt[kThrK];
+                    const float4* fs = reinterpret_cast<const float4*>(&sm.flt[cc][r * S + s][tx * kThrK]);
+#pragma unroll
+                    for (int v = 0; v < kThrK / 4; ++v) {
+                        const float4 t = fs[v];
+                        flt[4 * v + 0] = t.x; flt[4 * v + 1] = t.y; flt[4 * v + 2] = t.z; flt[4 * v + 3] = t.w;
+                    }
+#pragma unroll
+                    for (int i = 0; i < kThrK; ++i)
+#pragma unroll
+                        for (int j = 0; j < kThrQ; ++j) acc[i][j] = fmaf(flt[i], img[s + j], acc[i][j]);
+                }
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- write the register tile ----
+    const int p = p0 + seg_row, q = q0 + seg_col;
+    if (p >= P || q >= Q) return;
+#pragma unroll
+    for (int i = 0; i < kThrK; ++i) {
+        const int k = k0 + tx * kThrK + i;
+        if (k >= K) break;
+        float* o = y + (((size_t)n * K + k) * P + p) * Q + q;
+        if (vec_st && q + kThrQ <= Q) {
+#pragma unroll
+            for (int v = 0; v < kThrQ / 4; ++v)
+                *reinterpret_cast<float4*>(o + 4 * v) =
+                    make_float4(acc[i][4 * v], acc[i][4 * v + 1], acc[i][4 * v + 2], acc[i][4 * v + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kThrQ; ++j)
+                if (q + j < Q) o[j] = acc[i][j];
+        }
+    }
+}
+
+template <int R, int S, int CB>
+conv2d_status_t launch_instance(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
+{
+    auto kern = general_ffma_kernel<R, S, CB>;
+    const size_t smem = sizeof(Smem<R, S, CB>);
+    if (smem > 48 * 1024) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return CONV2D_ERR_CUDA;
+    }
+    const int tiles_q = (sh.Q + kTileW - 1) / kTileW, tiles_p = (sh.P + kTileH - 1) / kTileH;
+    dim3 grid(tiles_q * tiles_p, (sh.K + kTileK - 1) / kTileK, sh.N);
+    const int vec_st = (sh.Q % 4 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
+    kern<<<grid, kThreads, smem, stream>>>(x, w, y, sh.C, sh.H, sh.W, sh.K, sh.P, sh.Q, tiles_q, vec_st);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
+// One thread per output, loops over c, r, s in that order: correct for every shape, tuned for none.
+__global__ void direct_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
+                              int C, int H, int W, int K, int R, int S, int P, int Q, long long total)
+{
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += stride) {
+        const int q = (int)(o % Q);
+        const int p = (int)((o / Q) % P);
+        const int k = (int)((o / ((long long)Q * P)) % K);
+        const int n = (int)(o / ((long long)Q * P * K));
+        const float* xb = x + ((size_t)n * C * H + p) * W + q;
+        const float* wb = w + (size_t)k * C * R * S;
+        float acc = 0.f;
+        for (int c = 0; c < C; ++c)
+            for (int r = 0; r < R; ++r)
+                for (int s = 0; s < S; ++s)
+                    acc = fmaf(__ldg(xb + ((size_t)c * H + r) * W + s), __ldg(wb + ((size_t)c * R + r) * S + s), acc);
+        y[o] = acc;
+    }
+}
+
+}  // namespace
+
+conv2d_status_t launch_direct_fallback(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
+{
+    const long long total = (long long)sh.N * sh.K * sh.P * sh.Q;
+    const int threads = 256;
+    long long blocks = (total + threads - 1) / threads;
+    if (blocks > 148LL * 64) blocks = 148LL * 64;
+    direct_kernel<<<(unsigned)blocks, threads, 0, stream>>>(x, w, y, sh.C, sh.H, sh.W, sh.K, sh.R, sh.S, sh.P, sh.Q, total);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
+conv2d_status_t launch_general_ffma(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
+{
+    if (sh.N > 65535 || (sh.K + kTileK - 1) / kTileK > 65535) return launch_direct_fallback(x, w, y, sh, stream);
+    if (sh.R == 1 && sh.S == 1) return launch_instance<1, 1, 16>(x, w, y, sh, stream);
+    if (sh.R == 3 && sh.S == 3) return launch_instance<3, 3, 8>(x, w, y, sh, stream);
+    if (sh.R == 5 && sh.S == 5) return launch_instance<5, 5, 4>(x, w, y, sh, stream);
+    if (sh.R == 7 && sh.S == 7) return launch_instance<7, 7, 2>(x, w, y, sh, stream);
+    return launch_direct_fallback(x, w, y, sh, stream);
+}
+
+}  // namespace conv2d_b200

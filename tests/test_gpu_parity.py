@@ -1,0 +1,190 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs.
+
+Bars: integer-valued inputs must match bit for bit; real-valued inputs within
+|y - y_ref| <= 1e-5 * sum|x*w| (fp32 FMA paths) or 2e-3 * sum|x*w| (TF32 tensor-core path), elementwise.
+"""
+import numpy as np
+import pytest
+
+from helpers import FFMA_TOL, TF32_TOL, assert_parity, run_library
+from workloads import CONFIGS, make_inputs, small_integers, uniform
+
+pytestmark = pytest.mark.gpu
+
+ALGO_AUTO, ALGO_FFMA, ALGO_TF32 = 0, 1, 2
+
+
+# ---------------------------------------------------------------- special case (one input channel)
+
+SINGLE_SHAPES = [
+    # N, H, W, K, R, S
+    (1, 64, 64, 8, 3, 3),        # cfg1 shape
+    (1, 9, 10, 3, 3, 3),         # W % 4 != 0, tiny
+    (2, 37, 53, 5, 5, 5),        # odd everything, Q % 4 != 0
+    (1, 19, 1031, 2, 3, 3),      # three column tiles with a ragged last one
+    (3, 40, 520, 4, 7, 7),       # Q = 514: second column tile nearly empty
+    (1, 33, 36, 1, 1, 1),        # 1x1: no data sharing at all
+    (1, 5, 5, 7, 5, 5),          # filter as large as the image: one output per map
+    (2, 21, 24, 3, 3, 5),        # rectangular taps -> shape-agnostic kernel
+    (1, 70, 16, 6, 5, 5),        # more rows than one tile, Q = 12 (vector stores)
+]
+
+
+@pytest.mark.parametrize("dims", SINGLE_SHAPES)
+def test_single_channel_exact_on_integers(oracle, dims):
+    N, H, W, K, R, S = dims
+    x, w = small_integers((N, 1, H, W), 301), small_integers((K, 1, R, S), 302)
+    y_ref, _ = oracle.conv2d_oracle(x, w)
+    y = run_library(x, w, entry="single")
+    np.testing.assert_array_equal(y.astype(np.float64), y_ref)
+
+
+@pytest.mark.parametrize("dims", SINGLE_SHAPES)
+def test_single_channel_within_tolerance(oracle, dims):
+    N, H, W, K, R, S = dims
+    x, w = uniform((N, 1, H, W), 303), uniform((K, 1, R, S), 304)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="single"), y_ref, yabs, FFMA_TOL, f"single {dims}")
+
+
+@pytest.mark.parametrize("knobs", [dict(CONV2D_B200_SC_WSRC="0"), dict(CONV2D_B200_SC_ROWS="1"),
+                                   dict(CONV2D_B200_SC_TILE_H="5", CONV2D_B200_SC_WSRC="0", CONV2D_B200_SC_ROWS="1")])
+def test_single_channel_variants_agree(oracle, monkeypatch, knobs):
+    for k, v in knobs.items():
+        monkeypatch.setenv(k, v)
+    for dims in [(1, 64, 64, 8, 3, 3), (2, 37, 53, 5, 5, 5), (1, 19, 1031, 2, 3, 3)]:
+        N, H, W, K, R, S = dims
+        x, w = small_integers((N, 1, H, W), 305), small_integers((K, 1, R, S), 306)
+        y_ref, _ = oracle.conv2d_oracle(x, w)
+        np.testing.assert_array_equal(run_library(x, w, entry="single").astype(np.float64), y_ref)
+
+
+def test_cfg1_single_channel(oracle):
+    x, w = make_inputs(CONFIGS["cfg1"])
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="single"), y_ref, yabs, FFMA_TOL, "cfg1")
+
+
+def test_general_entry_with_one_channel_matches_single_channel_entry(oracle):
+    x, w = make_inputs(CONFIGS["cfg1"])
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    y_g = run_library(x, w, entry="general", algo=ALGO_FFMA)
+    assert_parity(y_g, y_ref, yabs, FFMA_TOL, "cfg1 via general")
+    xi, wi = small_integers(x.shape, 307), small_integers(w.shape, 308)
+    np.testing.assert_array_equal(run_library(xi, wi, entry="general", algo=ALGO_FFMA),
+                                  run_library(xi, wi, entry="single"))
+
+
+def test_cfg2_full_size_sampled_rows(oracle):
+    """Full 4096 x 4096, 32 filters of 5 x 5, in the launch configuration the benchmark times."""
+    cfg = CONFIGS["cfg2"]
+    x, w = make_inputs(cfg)
+    y = run_library(x, w, entry="single")
+    worst = 0.0
+    # first/last rows, rows around tile seams, and a seeded scatter; all maps
+    rows = sorted({0, 1, 15, 16, 17, 31, 32, 2047, 2048, 4090, 4091} | set(int(v) for v in
+                  (uniform((24,), 309, 0, 1) * cfg.P).astype(np.int64)))
+    for p in rows:
+        y_ref, yabs = oracle.conv2d_oracle_range(x, w, p_range=(p, p + 1))
+        worst = max(worst, assert_parity(y[:, :, p:p + 1], y_ref, yabs, FFMA_TOL, f"cfg2 row {p}"))
+    # properties that hold at any size: the last column tile is ragged (Q = 4092), nothing is NaN
+    assert y.shape == (1, 32, 4092, 4092)
+    assert np.isfinite(y).all()
+    print(f"cfg2 max ratio {worst:.3e}")
+
+
+# ---------------------------------------------------------------- general case
+
+GENERAL_SHAPES = [
+    # N, C, H, W, K, R, S
+    (1, 3, 12, 13, 5, 3, 3),
+    (2, 17, 20, 21, 70, 3, 3),     # K and C not multiples of the tiles
+    (1, 8, 41, 37, 64, 5, 5),
+    (2, 6, 15, 44, 9, 7, 7),
+    (3, 32, 9, 9, 16, 1, 1),
+    (1, 4, 11, 10, 3, 2, 4),       # rectangular taps -> shape-agnostic kernel
+    (2, 5, 3, 3, 4, 3, 3),         # one output per map
+    (1, 64, 14, 14, 96, 3, 3),
+]
+
+
+@pytest.mark.parametrize("dims", GENERAL_SHAPES)
+@pytest.mark.parametrize("algo", [ALGO_FFMA, ALGO_AUTO])
+def test_general_exact_on_integers(oracle, dims, algo):
+    N, C, H, W, K, R, S = dims
+    x, w = small_integers((N, C, H, W), 401), small_integers((K, C, R, S), 402)
+    y_ref, _ = oracle.conv2d_oracle(x, w)
+    y = run_library(x, w, entry="general", algo=algo)
+    np.testing.assert_array_equal(y.astype(np.float64), y_ref)
+
+
+@pytest.mark.parametrize("dims", GENERAL_SHAPES)
+def test_general_ffma_within_tolerance(oracle, dims):
+    N, C, H, W, K, R, S = dims
+    x, w = uniform((N, C, H, W), 403), uniform((K, C, R, S), 404)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_FFMA), y_ref, yabs, FFMA_TOL, f"ffma {dims}")
+
+
+def _tf32_available(cfg_dims):
+    import paper_1705_10591_b200 as lib
+    try:
+        return lib.conv2d_fwd_workspace_size(*cfg_dims, ALGO_TF32) > 0
+    except lib.Conv2dError:
+        return False
+
+
+@pytest.mark.parametrize("dims", GENERAL_SHAPES)
+def test_general_tf32_within_tolerance(oracle, dims):
+    if not _tf32_available(dims):
+        pytest.skip("no tensor-core instance for this shape")
+    from oracle.conv2d_oracle import MODE_TF32_RNA
+    N, C, H, W, K, R, S = dims
+    x, w = uniform((N, C, H, W), 405), uniform((K, C, R, S), 406)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    y = run_library(x, w, entry="general", algo=ALGO_TF32)
+    assert_parity(y, y_ref, yabs, TF32_TOL, f"tf32 {dims}")
+    # Diagnostic, far tighter than the bar: against the oracle fed TF32-rounded operands only the
+    # fp32 accumulation order differs.
+    y_rna, yabs_rna = oracle.conv2d_oracle(x, w, mode=MODE_TF32_RNA)
+    assert_parity(y, y_rna, yabs_rna, 2e-5, f"tf32 vs rounded-operand oracle {dims}")
+
+
+FULL = ["cfg3", "cfg4", "cfg5_r1", "cfg5_r3", "cfg5_r5", "cfg5_r7"]
+
+
+def _sampled_planes(cfg, count, seed):
+    n = (uniform((count,), seed, 0, 1) * cfg.N).astype(np.int64)
+    k = (uniform((count,), seed + 1, 0, 1) * cfg.K).astype(np.int64)
+    picks = {(0, 0), (cfg.N - 1, cfg.K - 1)} | set(zip(n.tolist(), k.tolist()))
+    return sorted(picks)
+
+
+@pytest.mark.parametrize("name", FULL)
+@pytest.mark.parametrize("algo", [ALGO_FFMA, ALGO_TF32])
+def test_full_size_configs(oracle, name, algo):
+    """Benchmark shapes at full size; every output of a seeded sample of (image, map) planes is checked."""
+    cfg = CONFIGS[name]
+    dims = (cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S)
+    if algo == ALGO_TF32 and not _tf32_available(dims):
+        pytest.skip("no tensor-core instance for this shape")
+    x, w = make_inputs(cfg)
+    y = run_library(x, w, entry="general", algo=algo)
+    tol = FFMA_TOL if algo == ALGO_FFMA else TF32_TOL
+    worst = 0.0
+    for n, k in _sampled_planes(cfg, 48, 500 + cfg.seed):
+        y_ref, yabs = oracle.conv2d_oracle_range(x, w, n_range=(n, n + 1), k_range=(k, k + 1))
+        worst = max(worst, assert_parity(y[n:n + 1, k:k + 1], y_ref, yabs, tol, f"{name} plane {(n, k)}"))
+    assert np.isfinite(y).all()
+    print(f"{name} algo={algo} max ratio {worst:.3e}")
+
+
+def test_relu_zero_windows_give_exact_zero(oracle):
+    """Where every product is zero the result must be exactly zero in every path."""
+    x = np.zeros((1, 16, 12, 12), np.float32)
+    x[:, :, 8:, 8:] = uniform((1, 16, 4, 4), 411)
+    w = uniform((32, 16, 3, 3), 412)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    for algo in (ALGO_FFMA, ALGO_AUTO):
+        y = run_library(x, w, entry="general", algo=algo)
+        assert np.all(y[yabs == 0] == 0)
