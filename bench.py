@@ -231,6 +231,32 @@ def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
     return out
 
 
+def run_e2e(torch, lib, cfg, algo, x_host, w_host, xd, wd, yd, ws, ws_bytes, stream, args, world, dev, barrier):
+    """Same metric through conv2d_fwd_host: pinned host buffers, H2D and D2H copies inside the timed region."""
+    y_host = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), dtype=torch.float32).pin_memory()
+
+    def e2e_step():
+        lib.conv2d_fwd_host(x_host.data_ptr(), w_host.data_ptr(), y_host.data_ptr(),
+                            xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
+                            cfg.K, cfg.R, cfg.S, algo, ws.data_ptr() if ws_bytes else 0, ws_bytes, stream)
+    e2e_step()
+    e2e_steps = max(2, min(args.steps, 5))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()          # synchronises the stream itself
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    return {"value": world * cfg.flops / e2e_s / 1e9, "unit": "GFLOP/s",
+            "h2d_bytes_per_step": int(x_host.numel() * 4 + w_host.numel() * 4),
+            "d2h_bytes_per_step": int(y_host.numel() * 4), "ms_per_step": e2e_s * 1e3, "steps": e2e_steps}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -240,6 +266,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
     ap.add_argument("--no-general", action="store_true", help="skip the general-case configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -333,28 +360,9 @@ def main():
     value = world * cfg.flops / (ms_per_step * 1e-3) / 1e9
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
-    y_host = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), dtype=torch.float32).pin_memory()
-
-    def e2e_step():
-        lib.conv2d_fwd_host(x_host.data_ptr(), w_host.data_ptr(), y_host.data_ptr(),
-                            xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
-                            cfg.K, cfg.R, cfg.S, algo, ws.data_ptr() if ws_bytes else 0, ws_bytes, stream)
-    e2e_step()
-    e2e_steps = max(2, min(args.steps, 5))
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()          # synchronises the stream itself
-    barrier()
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * cfg.flops / e2e_s / 1e9, "unit": "GFLOP/s",
-           "h2d_bytes_per_step": int(x.nbytes + w.nbytes), "d2h_bytes_per_step": int(y_host.numel() * 4),
-           "ms_per_step": e2e_s * 1e3}
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(torch, lib, cfg, algo, x_host, w_host, xd, wd, yd, ws, ws_bytes, stream, args, world, dev, barrier)
 
     # ---- roofline of the dominant kernel (per launch = one step)
     t_kernel_s = ms_per_step * 1e-3

@@ -113,6 +113,41 @@ conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
                                    unsigned flags, void* cuda_stream);
 
 /*
+ * General case on the tensor cores for callers that cannot hand over scratch memory.
+ * (The paper has no counterpart; this is a packaging variant of conv2d_fwd_general with
+ * algo = CONV2D_ALGO_TF32, same kernels, same results.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- inside a
+ * latency-critical loop that must not touch the allocator, in a process whose memory pool was
+ * sized up front and is fully handed out, or in a plug-in that is only given its input and
+ * output buffers.  Such callers cannot call cudaMalloc (or a framework allocator) to obtain the
+ * workspace that conv2d_fwd_general asks for.
+ *
+ * Here the status block and the re-ordered filters live in a fixed array of
+ * 256 + 8 MiB bytes inside the library's device image: every GPU on which the library is
+ * loaded gives up that much memory until the process exits.  The call allocates and frees
+ * nothing, on the device or through any library.  Shapes whose re-ordered filters
+ * need more (conv2d_fwd_workspace_size(..., CONV2D_ALGO_TF32) > 256 + 8 MiB) are rejected with
+ * CONV2D_ERR_WORKSPACE before anything is enqueued; shapes without a tensor-core instance with
+ * CONV2D_ERR_UNSUPPORTED.
+ *
+ * The first call on each device looks up the array's device address (a one-time set-up under a
+ * lock, with that device current); make that first call outside any stream capture.
+ * The array is shared by all calls on a device and keeps the previous call's contents: each
+ * call clears the status block and rewrites every filter word it will read, so stale contents
+ * are never used, but two calls whose kernels can overlap on the GPU (calls on different
+ * streams without an ordering between them) race on it.  Issue these calls on one stream per
+ * device, or order them with events.
+ *
+ * x, w, y: device pointers as for conv2d_fwd_general.  wait = 0: enqueue and return;
+ * wait != 0: also wait for the stream and return CONV2D_ERR_DEVICE_TIMEOUT if a bounded
+ * on-device wait expired.
+ */
+conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float* y,
+                                           int N, int C, int H, int W, int K, int R, int S,
+                                           int wait, void* cuda_stream);
+
+/*
  * Host-buffer convenience path (no counterpart in the paper): x_host and
  * w_host are copied to the caller's device buffers x, w on the stream, the
  * convolution runs (single-channel kernel when C == 1, else conv2d_fwd_general

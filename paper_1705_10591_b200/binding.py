@@ -46,6 +46,8 @@ def load_library() -> ctypes.CDLL:
     lib.conv2d_fwd_single_channel.restype = i
     lib.conv2d_fwd_general.argtypes = [vp, vp, vp] + [i] * 7 + [i, vp, sz, u, vp]
     lib.conv2d_fwd_general.restype = i
+    lib.conv2d_fwd_general_noalloc.argtypes = [vp, vp, vp] + [i] * 7 + [i, vp]
+    lib.conv2d_fwd_general_noalloc.restype = i
     lib.conv2d_fwd_host.argtypes = [vp] * 6 + [i] * 7 + [i, vp, sz, vp]
     lib.conv2d_fwd_host.restype = i
     lib.conv2d_get_status.argtypes = [vp, vp]
@@ -90,6 +92,13 @@ def conv2d_fwd_general(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, algo=ALGO_AUTO,
     _check(load_library().conv2d_fwd_general(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, algo,
                                              workspace_ptr or None, workspace_bytes, flags, stream or None),
            "conv2d_fwd_general")
+
+
+def conv2d_fwd_general_noalloc(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, wait=0, stream=0) -> None:
+    """Tensor-core convolution whose scratch is the library's own fixed device array (see the header)."""
+    _check(load_library().conv2d_fwd_general_noalloc(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S,
+                                                     int(wait), stream or None),
+           "conv2d_fwd_general_noalloc")
 
 
 def conv2d_fwd_host(x_host_ptr, w_host_ptr, y_host_ptr, x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S,

@@ -34,4 +34,9 @@ size_t tf32_workspace_bytes(const Shape& sh);   // includes the status block
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
                                     void* workspace, bool weights_packed, cudaStream_t stream);
 
+// Variant of the tensor-core path whose scratch is a fixed array inside the library image.
+constexpr size_t kNoAllocScratchBytes = kStatusBytes + (size_t)8 * 1024 * 1024;
+conv2d_status_t launch_general_tf32_noalloc(const float* x, const float* w, float* y, const Shape& sh,
+                                            bool wait, cudaStream_t stream);
+
 }  // namespace conv2d_b200

@@ -112,6 +112,22 @@ conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
     return launch_general_ffma(x, w, y, sh, stream);
 }
 
+conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float* y,
+                                           int N, int C, int H, int W, int K, int R, int S,
+                                           int wait, void* cuda_stream)
+{
+    if (!x || !w || !y) return CONV2D_ERR_NULL;
+    Shape sh;
+    conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
+    if (st != CONV2D_OK) return st;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return CONV2D_ERR_ALIGN;
+    if (!tf32_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
+    if (tf32_workspace_bytes(sh) > kNoAllocScratchBytes) return CONV2D_ERR_WORKSPACE;
+    st = check_device();
+    if (st != CONV2D_OK) return st;
+    return launch_general_tf32_noalloc(x, w, y, sh, wait != 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
 conv2d_status_t conv2d_fwd_host(const float* x_host, const float* w_host, float* y_host,
                                 float* x, float* w, float* y,
                                 int N, int C, int H, int W, int K, int R, int S,

@@ -29,6 +29,8 @@
 //     the coalesced write-back that Section 4.2 leaves out).
 //   * Every wait is bounded; on expiry the block raises a flag, skips its stores, frees its tensor
 //     memory and the status word in the workspace becomes non-zero.
+#include <mutex>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -357,6 +359,42 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
     general_tf32_kernel<<<grid, kThreads, p.smem_bytes, stream>>>(a);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------- variant without caller-provided scratch
+// Scratch of conv2d_fwd_general_noalloc: status block + re-ordered filters.  It lives in the module's
+// device image, so every GPU that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+conv2d_status_t launch_general_tf32_noalloc(const float* x, const float* w, float* y, const Shape& sh,
+                                            bool wait, cudaStream_t stream)
+{
+    if (!tf32_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
+    if (tf32_workspace_bytes(sh) > kNoAllocScratchBytes) return CONV2D_ERR_WORKSPACE;
+
+    // In host code the array's name is only a handle; the device address has to be asked for, once per
+    // device, with that device current.
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void* scratch_of_device[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CONV2D_ERR_CUDA;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!scratch_of_device[dev]) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return CONV2D_ERR_CUDA;
+            scratch_of_device[dev] = p;
+        }
+        scratch = scratch_of_device[dev];
+    }
+    conv2d_status_t st = launch_general_tf32(x, w, y, sh, scratch, /*weights_packed=*/false, stream);
+    if (st != CONV2D_OK || !wait) return st;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return CONV2D_ERR_CUDA;
+    unsigned word = 0;
+    if (cudaMemcpy(&word, scratch, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) return CONV2D_ERR_CUDA;
+    return word == 0 ? CONV2D_OK : CONV2D_ERR_DEVICE_TIMEOUT;
 }
 
 }  // namespace conv2d_b200

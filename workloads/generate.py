@@ -111,6 +111,8 @@ CONFIGS = {
     "cfg2": ConvShape("cfg2", 1, 1, 4096, 4096, 32, 5, 5, "uniform_pm1", 0.2, 2),
     "cfg3": ConvShape("cfg3", 32, 64, 56, 56, 64, 3, 3, "relu_normal", (2.0 / (64 * 9)) ** 0.5, 3),
     "cfg4": ConvShape("cfg4", 32, 256, 14, 14, 256, 3, 3, "relu_normal", (2.0 / (256 * 9)) ** 0.5, 4),
+    # profiling-size stand-in for cfg2 (same kernel instance, output 536 MB: still far beyond L2)
+    "cfg2_half": ConvShape("cfg2_half", 1, 1, 2048, 2048, 32, 5, 5, "uniform_pm1", 0.2, 2),
     "cfg5_r1": _cfg5(1),
     "cfg5_r3": _cfg5(3),
     "cfg5_r5": _cfg5(5),
