@@ -20,6 +20,10 @@ constexpr int kConstFilterFloats = 16384;
 // Bytes reserved at the start of the workspace for the device status word.
 constexpr size_t kStatusBytes = 256;
 
+// Reads and clears the device word that kernels without a workspace raise when a bounded wait expires.
+// Returns cudaSuccess and sets *raised, or the CUDA error.  The stream must already be idle.
+cudaError_t consume_device_timeout(bool* raised);
+
 // Every kernel launch goes through this so that conv2d_launch_count() is exact.
 void count_launch(int launches = 1);
 

@@ -157,6 +157,9 @@ conv2d_status_t conv2d_get_status(const void* workspace, void* cuda_stream)
 {
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaStreamSynchronize(stream) != cudaSuccess) return CONV2D_ERR_CUDA;
+    bool raised = false;
+    if (consume_device_timeout(&raised) != cudaSuccess) return CONV2D_ERR_CUDA;
+    if (raised) return CONV2D_ERR_DEVICE_TIMEOUT;
     if (!workspace) return CONV2D_OK;
     unsigned word = 0;
     if (cudaMemcpy(&word, workspace, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) return CONV2D_ERR_CUDA;

@@ -15,8 +15,12 @@
 // fetched feeds 8 FMAs; output stores are 128-bit streaming stores (the output is 97 % of the
 // traffic and is never read back).
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace conv2d_b200 {
+
+// Raised by a kernel whose bounded wait expired; read and cleared by conv2d_get_status.
+__device__ unsigned g_device_timeout;
 
 __constant__ float c_filters[kConstFilterFloats];
 
@@ -29,6 +33,24 @@ constexpr int kPitch = kTileW + 8;            // staged columns per row (halo S-
 constexpr int kPitch4 = kPitch / 4;
 
 __device__ __forceinline__ void store4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+
+// Stores the n = 4 adjacent outputs of one thread at columns q0..q0+3 of a row of Q outputs with the
+// widest unit the row alignment allows: `unit` = 4 when Q % 4 == 0 (every row 16-byte aligned),
+// 2 when Q % 2 == 0, else 1.  q0 is a multiple of 4.
+__device__ __forceinline__ void store_outputs(float* o, float a0, float a1, float a2, float a3, int q0, int Q, int unit)
+{
+    if (unit == 4 && q0 + 3 < Q) {
+        store4(o, make_float4(a0, a1, a2, a3));
+    } else if (unit >= 2) {
+        if (q0 + 1 < Q) __stcs(reinterpret_cast<float2*>(o), make_float2(a0, a1));
+        if (q0 + 3 < Q) __stcs(reinterpret_cast<float2*>(o + 2), make_float2(a2, a3));
+    } else {
+        if (q0 + 0 < Q) __stcs(o + 0, a0);
+        if (q0 + 1 < Q) __stcs(o + 1, a1);
+        if (q0 + 2 < Q) __stcs(o + 2, a2);
+        if (q0 + 3 < Q) __stcs(o + 3, a3);
+    }
+}
 
 // WSRC: 0 = filter taps read from the constant bank, 1 = from a shared-memory copy (128-bit broadcast loads).
 template <int R, int S, int TR, int WSRC>
@@ -155,6 +177,165 @@ single_channel_kernel(const float* __restrict__ x, const float* __restrict__ w, 
     }
 }
 
+// Packed-FMA variant.  B200 issues fp32 FMAs at full rate only as two-wide packed instructions
+// (fma.rn.f32x2): a scalar-FMA loop tops out near 82 % of the fp32 peak, a packed one near 99 %,
+// and the packed form leaves issue slots for the loads, stores and address arithmetic.  The two
+// lanes of a packed FMA are two adjacent FILTERS applied to the same pixel: the pixel window is
+// held as (x, x) pairs (built once per row step, reused by all filters) and the taps of filters
+// 2i and 2i+1 are interleaved in shared memory so that one 128-bit broadcast load brings two taps
+// for both filters.  Everything else is as in the kernel above.
+template <int R, int S, int TR>
+__global__ void __launch_bounds__(kThreads)
+single_channel_packed_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
+                             int H, int W, int K, int P, int Q, int tile_h, int vec_ld, int vec_st)
+{
+    constexpr int NV = (S + kVec - 1 + 3) / 4;          // float4 loads per window row
+    constexpr int WC = 4 * NV;
+    constexpr int WR = R - 1 + TR;
+    constexpr int RS = R * S;
+    constexpr int RS2 = (RS + 1) / 2;                   // 128-bit units per filter pair (two taps each)
+
+    extern __shared__ float4 smem4[];
+    float4* tile4 = smem4;
+    const int tid = threadIdx.x;
+    const int col0 = blockIdx.x * kTileW;
+    const int row0 = blockIdx.y * tile_h;
+    const int n = blockIdx.z;
+    const int th = min(tile_h, P - row0);
+    const int rows_in = th + R - 1;
+    const float* xin = x + (size_t)n * H * W;
+
+    for (int idx = tid; idx < rows_in * kPitch4; idx += kThreads) {
+        const int row = idx / kPitch4, c4 = idx - row * kPitch4;
+        const int col = col0 + 4 * c4;
+        const float* src = xin + (size_t)(row0 + row) * W + col;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (vec_ld && col + 3 < W) {
+            v = __ldg(reinterpret_cast<const float4*>(src));
+        } else {
+            if (col + 0 < W) v.x = __ldg(src + 0);
+            if (col + 1 < W) v.y = __ldg(src + 1);
+            if (col + 2 < W) v.z = __ldg(src + 2);
+            if (col + 3 < W) v.w = __ldg(src + 3);
+        }
+        tile4[idx] = v;
+    }
+    // taps of filter pair i: [i][unit u] = (w[2i][2u], w[2i+1][2u], w[2i][2u+1], w[2i+1][2u+1]); zero past K or RS
+    float4* wsm4 = smem4 + (size_t)(tile_h + R - 1) * kPitch4;
+    const int pairs = (K + 1) / 2;
+    for (int idx = tid; idx < pairs * RS2; idx += kThreads) {
+        const int i = idx / RS2, u = idx - i * RS2;
+        const int f0 = 2 * i, f1 = 2 * i + 1, t0 = 2 * u, t1 = 2 * u + 1;
+        float4 v;
+        v.x = __ldg(w + (size_t)f0 * RS + t0);
+        v.y = (f1 < K) ? __ldg(w + (size_t)f1 * RS + t0) : 0.f;
+        v.z = (t1 < RS) ? __ldg(w + (size_t)f0 * RS + t1) : 0.f;
+        v.w = (t1 < RS && f1 < K) ? __ldg(w + (size_t)f1 * RS + t1) : 0.f;
+        wsm4[idx] = v;
+    }
+    __syncthreads();
+
+    const int q0 = col0 + kVec * tid;
+    if (q0 >= Q) return;
+
+    float2 win[WR][WC];                                   // (x, x) pairs
+#pragma unroll
+    for (int r = 0; r < R - 1; ++r)
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const float4 t = tile4[r * kPitch4 + tid + v];
+            win[r][4 * v + 0] = make_float2(t.x, t.x); win[r][4 * v + 1] = make_float2(t.y, t.y);
+            win[r][4 * v + 2] = make_float2(t.z, t.z); win[r][4 * v + 3] = make_float2(t.w, t.w);
+        }
+
+    const size_t plane = (size_t)P * Q;
+    const bool vec_ok = vec_st && (q0 + 3 < Q);
+    for (int p = 0; p < th; p += TR) {
+#pragma unroll
+        for (int tr = 0; tr < TR; ++tr) {
+            const int row = p + R - 1 + tr;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (row < rows_in) t = tile4[row * kPitch4 + tid + v];
+                win[R - 1 + tr][4 * v + 0] = make_float2(t.x, t.x); win[R - 1 + tr][4 * v + 1] = make_float2(t.y, t.y);
+                win[R - 1 + tr][4 * v + 2] = make_float2(t.z, t.z); win[R - 1 + tr][4 * v + 3] = make_float2(t.w, t.w);
+            }
+        }
+        bool row_ok[TR];
+#pragma unroll
+        for (int tr = 0; tr < TR; ++tr) row_ok[tr] = (p + tr < th);
+
+        float* yout = y + ((size_t)n * K * P + (size_t)(row0 + p)) * Q + q0;
+        const float4* wf = wsm4;
+#pragma unroll 1
+        for (int i = 0; i < pairs; ++i, yout += 2 * plane, wf += RS2) {
+            float2 acc[TR][kVec];
+#pragma unroll
+            for (int tr = 0; tr < TR; ++tr)
+#pragma unroll
+                for (int j = 0; j < kVec; ++j) acc[tr][j] = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < RS2; ++u) {
+                const float4 w2 = wf[u];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int t = 2 * u + h;
+                    if (t < RS) {
+                        const int r = t / S, s2 = t % S;
+                        const float2 wv = h == 0 ? make_float2(w2.x, w2.y) : make_float2(w2.z, w2.w);
+#pragma unroll
+                        for (int tr = 0; tr < TR; ++tr)
+#pragma unroll
+                            for (int j = 0; j < kVec; ++j)
+                                acc[tr][j] = __ffma2_rn(win[tr + r][s2 + j], wv, acc[tr][j]);
+                    }
+                }
+            }
+            const bool second = (2 * i + 1 < K);
+#pragma unroll
+            for (int tr = 0; tr < TR; ++tr) {
+                if (row_ok[tr]) {
+                    float* o = yout + (size_t)tr * Q;
+                    if (vec_ok) {
+                        store4(o, make_float4(acc[tr][0].x, acc[tr][1].x, acc[tr][2].x, acc[tr][3].x));
+                        if (second) store4(o + plane, make_float4(acc[tr][0].y, acc[tr][1].y, acc[tr][2].y, acc[tr][3].y));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < kVec; ++j)
+                            if (q0 + j < Q) {
+                                __stcs(o + j, acc[tr][j].x);
+                                if (second) __stcs(o + plane + j, acc[tr][j].y);
+                            }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R - 1; ++r)
+#pragma unroll
+            for (int c = 0; c < WC; ++c) win[r][c] = win[r + TR][c];
+    }
+}
+
+template <int R, int S, int TR>
+conv2d_status_t launch_packed(const float* x, const float* w, float* y, const Shape& sh, int tile_h, cudaStream_t stream)
+{
+    constexpr int RS2 = (R * S + 1) / 2;
+    const size_t smem = (size_t)(tile_h + R - 1) * kPitch * sizeof(float) + (size_t)((sh.K + 1) / 2) * RS2 * sizeof(float4);
+    auto kern = single_channel_packed_kernel<R, S, TR>;
+    if (smem > 48 * 1024) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return CONV2D_ERR_CUDA;
+    }
+    dim3 grid((sh.Q + kTileW - 1) / kTileW, (sh.P + tile_h - 1) / tile_h, sh.N);
+    const int vec_ld = (sh.W % 4 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0);
+    const int vec_st = (sh.Q % 4 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
+    kern<<<grid, kThreads, smem, stream>>>(x, w, y, sh.H, sh.W, sh.K, sh.P, sh.Q, tile_h, vec_ld, vec_st);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
 template <int R, int S, int TR, int WSRC>
 conv2d_status_t launch_instance(const float* x, const float* w, float* y, const Shape& sh, int tile_h, cudaStream_t stream)
 {
@@ -174,6 +355,198 @@ conv2d_status_t launch_instance(const float* x, const float* w, float* y, const 
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
 }
 
+// Wide persistent variant for large images.
+//
+// Measured on B200: the output (97 % of the bytes) reaches HBM at 6.1-6.8 TB/s only when the pieces
+// written close together in time form long contiguous runs (a thread block writing 8-16 KB of one
+// output row at a time, its warps in step); 128-thread blocks writing 512-byte pieces into K planes
+// reach 4.5-5.2 TB/s however cheap the arithmetic.  So here one 512-thread block owns kRowsW = 2048
+// adjacent output columns and walks over row bands of `band_h` output rows; blocks are persistent and
+// take bands round-robin, so the blocks running at any moment cover adjacent rows.  The input band
+// (with halo) is brought in by 1-D bulk (TMA) copies, one per image row, into a double buffer guarded
+// by mbarriers: the copy of the next band runs under the FMA loop of the current one (the prefetch of
+// Algorithm 1, done by the copy engine instead of registers).  Arithmetic as in the packed kernel.
+constexpr int kRowsThreads = 512;
+constexpr int kRowsW = kRowsThreads * kVec;            // 2048 output columns per block
+constexpr int kRowsPitch = kRowsW + 8;                 // staged floats per row
+constexpr int kRowsPitch4 = kRowsPitch / 4;
+
+template <int R, int S, int TR>
+__global__ void __launch_bounds__(kRowsThreads, 1)
+single_channel_rows_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
+                           int N, int H, int W, int K, int P, int Q, int band_h, int col_tiles, int items, int unit)
+{
+    constexpr int NV = (S + kVec - 1 + 3) / 4;
+    constexpr int WC = 4 * NV;
+    constexpr int WR = R - 1 + TR;
+    constexpr int RS = R * S;
+    constexpr int RS2 = (RS + 1) / 2;
+
+    extern __shared__ float4 smem4[];
+    const int stage_f4 = (band_h + R - 1) * kRowsPitch4;
+    float4* tiles4 = smem4;                                          // [2][band_h+R-1][kRowsPitch4]
+    float4* wsm4 = smem4 + 2 * (size_t)stage_f4;
+    const int pairs = (K + 1) / 2;
+    uint64_t* full = reinterpret_cast<uint64_t*>(wsm4 + (size_t)pairs * RS2);   // [2]
+    volatile uint32_t* abort_flag = reinterpret_cast<uint32_t*>(full + 2);
+
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        ptx::mbar_init(&full[0], 1);
+        ptx::mbar_init(&full[1], 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    for (int idx = tid; idx < pairs * RS2; idx += kRowsThreads) {
+        const int i = idx / RS2, u = idx - i * RS2;
+        const int f0 = 2 * i, f1 = 2 * i + 1, t0 = 2 * u, t1 = 2 * u + 1;
+        float4 v;
+        v.x = __ldg(w + (size_t)f0 * RS + t0);
+        v.y = (f1 < K) ? __ldg(w + (size_t)f1 * RS + t0) : 0.f;
+        v.z = (t1 < RS) ? __ldg(w + (size_t)f0 * RS + t1) : 0.f;
+        v.w = (t1 < RS && f1 < K) ? __ldg(w + (size_t)f1 * RS + t1) : 0.f;
+        wsm4[idx] = v;
+    }
+    __syncthreads();
+
+    const int bands = (P + band_h - 1) / band_h;
+    // item -> (image, band, column tile); the column tile varies fastest
+    auto issue = [&](int item, int stage) {               // thread 0 only
+        const int ct = item % col_tiles;
+        const int band = (item / col_tiles) % bands;
+        const int n = item / (col_tiles * bands);
+        const int row0 = band * band_h, col0 = ct * kRowsW;
+        const int rows_in = min(band_h, P - row0) + R - 1;
+        const int cols = min(kRowsPitch, W - col0);                   // multiple of 4 (W % 4 == 0)
+        const uint32_t row_bytes = (uint32_t)cols * 4u;
+        ptx::mbar_arrive_expect_tx(&full[stage], row_bytes * (uint32_t)rows_in);
+        const float* src = x + ((size_t)n * H + row0) * W + col0;
+        float4* dst = tiles4 + (size_t)stage * stage_f4;
+        for (int r = 0; r < rows_in; ++r)
+            ptx::bulk_g2s(dst + (size_t)r * kRowsPitch4, src + (size_t)r * W, row_bytes, &full[stage]);
+    };
+
+    int it = blockIdx.x;
+    if (tid == 0 && it < items) issue(it, 0);
+    const size_t plane = (size_t)P * Q;
+    bool alive = true;
+    for (int local = 0; it < items; it += gridDim.x, ++local) {
+        const int stage = local & 1;
+        __syncthreads();                                              // everyone is done reading the other buffer
+        if (tid == 0 && it + (int)gridDim.x < items) issue(it + gridDim.x, stage ^ 1);
+        if (alive && !ptx::mbar_wait_bounded(&full[stage], (uint32_t)(local >> 1) & 1u, abort_flag)) alive = false;
+        if (!alive) continue;                                         // keep meeting the barriers, do no work
+
+        const int ct = it % col_tiles;
+        const int band = (it / col_tiles) % bands;
+        const int n = it / (col_tiles * bands);
+        const int row0 = band * band_h, col0 = ct * kRowsW;
+        const int th = min(band_h, P - row0);
+        const int rows_in = th + R - 1;
+        const int q0 = col0 + kVec * tid;
+        if (q0 >= Q) continue;
+        const float4* tile4 = tiles4 + (size_t)stage * stage_f4;
+
+        float2 win[WR][WC];
+#pragma unroll
+        for (int r = 0; r < R - 1; ++r)
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const float4 t = tile4[r * kRowsPitch4 + tid + v];
+                win[r][4 * v + 0] = make_float2(t.x, t.x); win[r][4 * v + 1] = make_float2(t.y, t.y);
+                win[r][4 * v + 2] = make_float2(t.z, t.z); win[r][4 * v + 3] = make_float2(t.w, t.w);
+            }
+        for (int p = 0; p < th; p += TR) {
+#pragma unroll
+            for (int tr = 0; tr < TR; ++tr) {
+                const int row = p + R - 1 + tr;
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (row < rows_in) t = tile4[row * kRowsPitch4 + tid + v];
+                    win[R - 1 + tr][4 * v + 0] = make_float2(t.x, t.x); win[R - 1 + tr][4 * v + 1] = make_float2(t.y, t.y);
+                    win[R - 1 + tr][4 * v + 2] = make_float2(t.z, t.z); win[R - 1 + tr][4 * v + 3] = make_float2(t.w, t.w);
+                }
+            }
+            bool row_ok[TR];
+#pragma unroll
+            for (int tr = 0; tr < TR; ++tr) row_ok[tr] = (p + tr < th);
+
+            float* yout = y + ((size_t)n * K * P + (size_t)(row0 + p)) * Q + q0;
+            const float4* wf = wsm4;
+#pragma unroll 1
+            for (int i = 0; i < pairs; ++i, yout += 2 * plane, wf += RS2) {
+                float2 acc[TR][kVec];
+#pragma unroll
+                for (int tr = 0; tr < TR; ++tr)
+#pragma unroll
+                    for (int j = 0; j < kVec; ++j) acc[tr][j] = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < RS2; ++u) {
+                    const float4 w2 = wf[u];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int t = 2 * u + h;
+                        if (t < RS) {
+                            const int r = t / S, s2 = t % S;
+                            const float2 wv = h == 0 ? make_float2(w2.x, w2.y) : make_float2(w2.z, w2.w);
+#pragma unroll
+                            for (int tr = 0; tr < TR; ++tr)
+#pragma unroll
+                                for (int j = 0; j < kVec; ++j)
+                                    acc[tr][j] = __ffma2_rn(win[tr + r][s2 + j], wv, acc[tr][j]);
+                        }
+                    }
+                }
+                const bool second = (2 * i + 1 < K);
+#pragma unroll
+                for (int tr = 0; tr < TR; ++tr) {
+                    if (row_ok[tr]) {
+                        float* o = yout + (size_t)tr * Q;
+                        store_outputs(o, acc[tr][0].x, acc[tr][1].x, acc[tr][2].x, acc[tr][3].x, q0, Q, unit);
+                        if (second)
+                            store_outputs(o + plane, acc[tr][0].y, acc[tr][1].y, acc[tr][2].y, acc[tr][3].y, q0, Q, unit);
+                    }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < R - 1; ++r)
+#pragma unroll
+                for (int c = 0; c < WC; ++c) win[r][c] = win[r + TR][c];
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && *abort_flag) {
+        // a copy may still be in flight into this block's shared memory: give it a bounded time to land
+        uint32_t dummy = 0;
+        ptx::mbar_wait_bounded(&full[0], 0u, &dummy, 1u << 12);
+        ptx::mbar_wait_bounded(&full[1], 0u, &dummy, 1u << 12);
+        atomicExch(&g_device_timeout, 1u);
+    }
+}
+
+template <int R, int S, int TR>
+conv2d_status_t launch_rows(const float* x, const float* w, float* y, const Shape& sh, int band_h, cudaStream_t stream)
+{
+    constexpr int RS2 = (R * S + 1) / 2;
+    const size_t smem = 2 * (size_t)(band_h + R - 1) * kRowsPitch * sizeof(float)
+                      + (size_t)((sh.K + 1) / 2) * RS2 * sizeof(float4) + 64;
+    if (smem > 227 * 1024) return CONV2D_ERR_UNSUPPORTED;
+    auto kern = single_channel_rows_kernel<R, S, TR>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return CONV2D_ERR_CUDA;
+    const int col_tiles = (sh.Q + kRowsW - 1) / kRowsW;
+    const long long items = (long long)sh.N * ((sh.P + band_h - 1) / band_h) * col_tiles;
+    if (items > 0x7fffffffLL) return CONV2D_ERR_UNSUPPORTED;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int grid = (int)(items < sms ? items : sms);
+    const int unit = (reinterpret_cast<uintptr_t>(y) % 16 != 0) ? 1 : (sh.Q % 4 == 0 ? 4 : (sh.Q % 2 == 0 ? 2 : 1));
+    kern<<<grid, kRowsThreads, smem, stream>>>(x, w, y, sh.N, sh.H, sh.W, sh.K, sh.P, sh.Q, band_h, col_tiles, (int)items, unit);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
 int env_int(const char* name, int dflt)
 {
     const char* v = getenv(name);
@@ -183,12 +556,28 @@ int env_int(const char* name, int dflt)
 template <int R, int S>
 conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
 {
-    // Tuning knobs (benchmark ablations only): tile height, rows per step, tap source.
-    int tile_h = env_int("CONV2D_B200_SC_TILE_H", 16);
+    // Tuning knobs (benchmark ablations only): tile height, rows per step, packed/scalar FMA, tap source.
+    int tile_h = env_int("CONV2D_B200_SC_TILE_H", 8);
     if (tile_h < 1) tile_h = 1;
     if (tile_h > 64) tile_h = 64;
     if (tile_h > sh.P) tile_h = sh.P;
-    const int tr = env_int("CONV2D_B200_SC_ROWS", 2);
+    const int tr = env_int("CONV2D_B200_SC_ROWS", R >= 7 ? 1 : 2);
+    constexpr int RS2 = (R * S + 1) / 2;
+    // Large images: the wide persistent kernel (needs 16-byte aligned input rows for the bulk copies).
+    const bool rows_ok = sh.W % 4 == 0 && sh.Q >= 1024 && reinterpret_cast<uintptr_t>(x) % 16 == 0;
+    if (rows_ok && env_int("CONV2D_B200_SC_WIDE", 1) != 0) {
+        int band_h = env_int("CONV2D_B200_SC_BAND_H", 8);
+        if (band_h < 1) band_h = 1;
+        if (band_h > 16) band_h = 16;
+        const conv2d_status_t st = (tr == 1 || R >= 7) ? launch_rows<R, S, 1>(x, w, y, sh, band_h, stream)
+                                                       : launch_rows<R, S, 2>(x, w, y, sh, band_h, stream);
+        if (st != CONV2D_ERR_UNSUPPORTED) return st;
+    }
+    if (env_int("CONV2D_B200_SC_PACKED", 1) != 0 &&
+        (size_t)((sh.K + 1) / 2) * RS2 * sizeof(float4) <= 96 * 1024) {
+        return (tr == 1 || R >= 7) ? launch_packed<R, S, 1>(x, w, y, sh, tile_h, stream)
+                                   : launch_packed<R, S, 2>(x, w, y, sh, tile_h, stream);
+    }
     constexpr int RSP = (R * S + 3) / 4 * 4;
     int wsrc = env_int("CONV2D_B200_SC_WSRC", 1);
     if ((size_t)sh.K * RSP * sizeof(float) > 64 * 1024) wsrc = 0;       // too many taps for the shared copy
@@ -205,6 +594,19 @@ conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shap
 }
 
 }  // namespace
+
+cudaError_t consume_device_timeout(bool* raised)
+{
+    unsigned flag = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(&flag, g_device_timeout, sizeof flag);
+    if (e != cudaSuccess) return e;
+    *raised = flag != 0;
+    if (flag != 0) {
+        const unsigned zero = 0;
+        e = cudaMemcpyToSymbol(g_device_timeout, &zero, sizeof zero);
+    }
+    return e;
+}
 
 conv2d_status_t launch_single_channel(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
 {

@@ -27,6 +27,10 @@ SINGLE_SHAPES = [
     (1, 5, 5, 7, 5, 5),          # filter as large as the image: one output per map
     (2, 21, 24, 3, 3, 5),        # rectangular taps -> shape-agnostic kernel
     (1, 70, 16, 6, 5, 5),        # more rows than one tile, Q = 12 (vector stores)
+    (1, 23, 2100, 3, 5, 5),      # wide persistent kernel: two column tiles (2048 + 48), 128-bit stores
+    (2, 11, 1032, 5, 3, 3),      # wide kernel, Q = 1030: 64-bit stores, odd filter count
+    (1, 9, 1028, 2, 7, 7),       # wide kernel, 7 x 7, band taller than the image's output rows
+    (1, 14, 1040, 4, 1, 1),      # wide kernel, 1 x 1
 ]
 
 
@@ -47,12 +51,15 @@ def test_single_channel_within_tolerance(oracle, dims):
     assert_parity(run_library(x, w, entry="single"), y_ref, yabs, FFMA_TOL, f"single {dims}")
 
 
-@pytest.mark.parametrize("knobs", [dict(CONV2D_B200_SC_WSRC="0"), dict(CONV2D_B200_SC_ROWS="1"),
-                                   dict(CONV2D_B200_SC_TILE_H="5", CONV2D_B200_SC_WSRC="0", CONV2D_B200_SC_ROWS="1")])
+@pytest.mark.parametrize("knobs", [
+    dict(CONV2D_B200_SC_ROWS="1"), dict(CONV2D_B200_SC_TILE_H="5"),                       # packed-FMA kernel
+    dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_WSRC="0"),                              # scalar-FMA kernel
+    dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_WSRC="1", CONV2D_B200_SC_ROWS="1"),
+    dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_TILE_H="5", CONV2D_B200_SC_WSRC="0", CONV2D_B200_SC_ROWS="1")])
 def test_single_channel_variants_agree(oracle, monkeypatch, knobs):
     for k, v in knobs.items():
         monkeypatch.setenv(k, v)
-    for dims in [(1, 64, 64, 8, 3, 3), (2, 37, 53, 5, 5, 5), (1, 19, 1031, 2, 3, 3)]:
+    for dims in [(1, 64, 64, 8, 3, 3), (2, 37, 53, 5, 5, 5), (1, 19, 1031, 2, 3, 3), (1, 30, 40, 3, 7, 7)]:
         N, H, W, K, R, S = dims
         x, w = small_integers((N, 1, H, W), 305), small_integers((K, 1, R, S), 306)
         y_ref, _ = oracle.conv2d_oracle(x, w)
