@@ -231,6 +231,22 @@ def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
     return out
 
 
+def reduce_max(value: float, device=None) -> float:
+    """Max of a per-rank scalar over all ranks (identity when torch.distributed is not initialised)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(flops_per_replica: int, world: int, seconds_per_step: float) -> float:
+    """Whole-job GFLOP/s of `world` independent replicas that each finish a step in `seconds_per_step`."""
+    return world * flops_per_replica / seconds_per_step / 1e9
+
+
 def run_e2e(torch, lib, cfg, algo, x_host, w_host, xd, wd, yd, ws, ws_bytes, stream, args, world, dev, barrier):
     """Same metric through conv2d_fwd_host: pinned host buffers, H2D and D2H copies inside the timed region."""
     y_host = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), dtype=torch.float32).pin_memory()
@@ -247,12 +263,8 @@ def run_e2e(torch, lib, cfg, algo, x_host, w_host, xd, wd, yd, ws, ws_bytes, str
         e2e_step()          # synchronises the stream itself
     barrier()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    return {"value": world * cfg.flops / e2e_s / 1e9, "unit": "GFLOP/s",
+    e2e_s = reduce_max(e2e_s, dev)
+    return {"value": job_throughput(cfg.flops, world, e2e_s), "unit": "GFLOP/s",
             "h2d_bytes_per_step": int(x_host.numel() * 4 + w_host.numel() * 4),
             "d2h_bytes_per_step": int(y_host.numel() * 4), "ms_per_step": e2e_s * 1e3, "steps": e2e_steps}
 
@@ -351,13 +363,9 @@ def main():
     clocks = sampler.stop()
     lib.conv2d_get_status(ws.data_ptr() if ws_bytes else 0, stream)
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = reduce_max(total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * cfg.flops / (ms_per_step * 1e-3) / 1e9
+    value = job_throughput(cfg.flops, world, ms_per_step * 1e-3)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
