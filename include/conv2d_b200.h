@@ -101,8 +101,9 @@ conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float*
  *   filters x horizontally adjacent outputs, as in Section 4.1-4.2); no workspace.
  * algo = TF32: implicit-GEMM on the tcgen05 tensor cores with the accumulator
  *   in tensor memory; needs the workspace reported by conv2d_fwd_workspace_size
- *   (16-byte aligned).  Its first 256 bytes are a status block that each call
- *   clears on the stream before launching.
+ *   (16-byte aligned).  Its first 256 bytes are a status block: the filter
+ *   re-ordering step of each call clears it, a call with CONV2D_FLAG_WEIGHTS_PACKED
+ *   leaves it as it is (so a time-out stays visible until the next full call).
  * algo = AUTO: TF32 when an instance exists and the workspace suffices, else FFMA.
  * C == 1 is accepted and gives the same result as the single-channel entry.
  */
