@@ -4,15 +4,15 @@
 // Mapping of the paper's design onto B200
 //   * GEMM view: rows = output pixels, columns = filters, contraction over (channel, tap).
 //     The accumulator block rAcc[F_T][W_T] of Algorithm 2 becomes a 128-pixel x n_tile-filter
-//     fp32 tile in tensor memory; a thread block owns `mt` such tiles for adjacent pixels.
+//     fp32 tile in tensor memory; a work item is `mt` such tiles for adjacent pixels.
 //   * Pixels are numbered in one flat sequence j = (n*H + h)*W + w over the whole batch.  For tap
 //     (r,s) the input needed by output j is the pixel j + r*W + s of the same channel, a pure
-//     shift.  A thread block therefore stages, per block of kCB channels, ONE run of
-//     mt*128 + (R-1)*W + (S-1) pixels ("block plus halo to the right and below", Section 3.1/4.1)
-//     and every tap reads it through a descriptor whose start address is shifted by r*W + s rows:
-//     the row reuse of Section 4.2 (one staged input row serves all horizontal taps) extended to
-//     the vertical taps, with no im2col buffer.  Outputs whose window wraps over the right or
-//     bottom image edge are computed but not stored.
+//     shift.  Per block of kCB channels ONE run of mt*128 + (R-1)*W + (S-1) pixels is staged
+//     ("block plus halo to the right and below", Section 3.1/4.1) and every tap reads it through
+//     a descriptor whose start address is shifted by r*W + s rows: the row reuse of Section 4.2
+//     (one staged input row serves all horizontal taps) extended to the vertical taps, with no
+//     im2col buffer.  Outputs whose window wraps over the right or bottom image edge are
+//     computed but not stored.
 //   * Shared-memory operand layout: K-major, no swizzle: [channel/4][row][4 channels], i.e. each
 //     row (pixel or filter) of a 4-channel chunk is one 16-byte unit and rows are 16 bytes apart.
 //     This is the transposed staging of Fig. 6 (adjacent units belong to adjacent rows) in the
@@ -23,12 +23,17 @@
 //     NCHW has the pixels, not the channels, contiguous, and a tiled copy cannot transpose nor
 //     start at a 4-byte offset; eight producer warps gather them (coalesced along pixels),
 //     round to TF32 and write 16-byte units.
-//   * Warp roles: warp 0 streams filter chunks, warp 1 (one thread) issues tcgen05.mma and owns
-//     the tensor-memory allocation, warps 2-9 stage activations and afterwards drain the
-//     accumulators (lane = pixel, so the 32 lanes of a warp store 32 adjacent outputs of one map:
-//     the coalesced write-back that Section 4.2 leaves out).
-//   * Every wait is bounded; on expiry the block raises a flag, skips its stores, frees its tensor
+//   * Persistent blocks, one per SM, walk over the work items round-robin.  Warp roles: warp 0
+//     streams filter stages, warp 1 (one thread) issues tcgen05.mma and owns the tensor-memory
+//     allocation, eight warps stage activations, four warps drain finished accumulators (lane =
+//     pixel, so a warp stores 32 adjacent outputs of one map: the coalesced write-back that
+//     Section 4.2 leaves out).  All rings run across item boundaries, so the loads of the next
+//     item proceed under the MMAs of the current one (the prefetch of Algorithm 2), and where two
+//     accumulator sets fit into the 512 tensor-memory columns the write-back of item i overlaps
+//     the MMAs of item i+1.
+//   * Every wait is bounded; on expiry the block raises a flag, stops storing, frees its tensor
 //     memory and the status word in the workspace becomes non-zero.
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -52,35 +57,60 @@ constexpr int kCB = 16;                     // channels per staged block (two UM
 constexpr int kChunks = kCB / 4;            // 16-byte channel chunks per block
 constexpr int kProducerWarps = 8;
 constexpr int kProducers = kProducerWarps * 32;
-constexpr int kThreads = 64 + kProducers;   // warp 0: filter copies, warp 1: MMA issue, then the workers
+constexpr int kEpilogueWarps = 4;
+// Warp roles by warp index.  An SM has four warp schedulers and warp w is served by scheduler w % 4.  The
+// single thread that issues the MMAs (warp 1) must never wait for an issue slot behind arithmetic-heavy
+// warps -- measured: sharing its scheduler with two producer warps stretched each MMA issue from ~64 to
+// 120-180 cycles -- so scheduler 1 hosts only that warp, one epilogue warp and two warps that exit at once.
+//   warp 0           filter copies (one thread)
+//   warp 1           MMA issue (one thread), owner of the tensor-memory allocation
+//   warps 4-7        epilogue, tensor-memory lane quarter = warp % 4
+//   warps 2,3,8,10,11,12,14,15   activation producers (schedulers 0, 2, 3)
+//   warps 9, 13      no work
+constexpr int kThreads = 512;
+__device__ __forceinline__ int producer_index(int warp)     // 0..7 for producer warps, -1 otherwise
+{
+    switch (warp) {
+        case 2: return 0; case 3: return 1; case 8: return 2; case 10: return 3;
+        case 11: return 4; case 12: return 5; case 14: return 6; case 15: return 7;
+        default: return -1;
+    }
+}
 constexpr int kMaxBStages = 16;
 constexpr int kMaxAStages = 4;
-constexpr int kUnitsPerThread = 3;           // (pixel, channel block) units a producer thread keeps in flight per pass
+constexpr int kUnitsPerThread = 3;          // (pixel, channel block) units a producer thread keeps in flight per pass
 constexpr size_t kSmemLimit = 227 * 1024;
-constexpr size_t kSmemLimitHalf = 113 * 1024;    // two blocks per SM
 
 struct Plan {
-    int n_tile;       // filters per thread block (UMMA N), multiple of 16
-    int n_blocks;     // thread-block columns over the filters
-    int mt;           // accumulator tiles per thread block
+    int n_tile;       // filters per work item (UMMA N), multiple of 16
+    int n_blocks;     // work-item columns over the filters
+    int mt;           // accumulator tiles per work item
+    int nbuf;         // accumulator sets in tensor memory (2: write-back overlaps the next item)
     int npix;         // staged pixel rows per channel chunk
     int cblks;        // channel blocks
     int taps;
     int a_stages;
     int b_stages;
     int tps;          // taps per filter stage
-    int blocks_per_sm;
     int cbg;          // channel blocks per activation stage
+    int resident;     // 1: the whole filter block stays in shared memory for the life of the thread block
     int tmem_cols;    // power of two >= 32
-    int supertiles;   // thread-block rows over the flat pixel sequence
+    int supertiles;   // work-item rows over the flat pixel sequence
+    int grid;
     size_t smem_bytes;
     bool ok;
 };
 
-// b_stages counts filter stages of `tps` taps each
-size_t smem_need(int a_stages, int npix, int n_tile, int b_stages, int tps = 1, int cbg = 1)
+// b_stages counts filter stages of `tps` taps each; an activation stage holds `cbg` channel blocks.
+size_t smem_need(int a_stages, int npix, int n_tile, int b_stages, int tps, int cbg)
 {
     return (size_t)a_stages * cbg * kCB * npix * 4 + (size_t)b_stages * tps * kCB * n_tile * 4 + 512;
+}
+
+int env_int(const char* name, int dflt)
+{
+    const char* v = getenv(name);
+    return (v && *v) ? atoi(v) : dflt;
 }
 
 Plan make_plan(const Shape& sh)
@@ -92,75 +122,100 @@ Plan make_plan(const Shape& sh)
     const int kp16 = (sh.K + 15) / 16 * 16;
     p.n_blocks = (kp16 + 255) / 256;
     p.n_tile = ((sh.K + p.n_blocks - 1) / p.n_blocks + 15) / 16 * 16;
-    if (p.n_blocks > 65535) return p;
     p.cblks = (sh.C + kCB - 1) / kCB;
     p.taps = sh.R * sh.S;
-    p.b_stages = 2;
-    p.tps = 1;
     const long long halo = (long long)(sh.R - 1) * sh.W + (sh.S - 1);
     const long long tiles = (total_pix + kTileM - 1) / kTileM;
-    // Tiles per block.  Heavy tiles (many taps x channel blocks): as many as tensor memory holds, so a
-    // streamed filter stage is reused by up to 4 tiles, picked to minimise (waves x tiles per block).
-    // Light tiles (1x1-like): the block is dominated by memory latency and write-back, so small blocks,
-    // two resident per SM, overlap one block's loads and stores with the other's MMAs.
-    const bool light = (long long)p.taps * p.cblks <= 16;
-    int best_mt = 0;
-    long long best_cost = 0;
-    for (int mt = 4; mt >= 1; mt >>= 1) {
-        if (mt * p.n_tile > 512) continue;
-        if (light && mt > 1 && (tiles + mt - 1) / mt * p.n_blocks < 4 * 148) continue;
-        const long long npix = ((long long)mt * kTileM + halo + 7) / 8 * 8;
-        if (npix > 16000) continue;
-        if (smem_need(2, (int)npix, p.n_tile, 2) > kSmemLimit) continue;
-        const long long ctas = (tiles + mt - 1) / mt * p.n_blocks;
-        const long long waves = (ctas + 147) / 148;
-        const long long cost = waves * mt;
-        if (best_mt == 0 || cost < best_cost) { best_mt = mt; best_cost = cost; }
+    const int chunk = kCB * p.n_tile * 4;
+    const int sms = 148;
+
+    const int forced_mt = env_int("CONV2D_B200_TF32_MT", 0);      // benchmark ablations only
+    const size_t wbytes = (size_t)p.cblks * p.taps * chunk;        // re-ordered filters of one filter block
+    auto npix_of = [&](int mt) { return (int)(((long long)mt * kTileM + halo + 7) / 8 * 8); };
+
+    // Small filter banks stay resident in shared memory: nothing is streamed, so one tile per item is
+    // best (finest balance over the SMs, two accumulator sets), and the rest of shared memory becomes a
+    // deep activation ring whose stages carry several channel blocks (these items are bound by memory
+    // latency: one producer pass should have 32-48 loads per thread in flight).
+    p.resident = 0;
+    if (env_int("CONV2D_B200_TF32_RESIDENT", 1) != 0 && p.n_blocks == 1 && wbytes <= 152 * 1024) {
+        const int mt = forced_mt ? forced_mt : 1;
+        const int npix = npix_of(mt);
+        if (mt * p.n_tile <= 512 && npix <= 16000 && wbytes + (size_t)2 * kCB * npix * 4 + 512 <= kSmemLimit) {
+            p.resident = 1;
+            p.mt = mt;
+            p.npix = npix;
+            p.cbg = 1;
+            p.a_stages = 2;
+            p.b_stages = 1;
+            p.tps = p.taps;
+            auto need = [&](int a_stages, int cbg) { return wbytes + (size_t)a_stages * cbg * kCB * npix * 4 + 512; };
+            while (p.cbg * 2 <= p.cblks && npix * p.cbg * 2 <= kProducers * kUnitsPerThread &&
+                   need(p.a_stages, p.cbg * 2) <= kSmemLimit) p.cbg *= 2;
+            while (p.a_stages < kMaxAStages && need(p.a_stages + 1, p.cbg) <= kSmemLimit) ++p.a_stages;
+            p.smem_bytes = need(p.a_stages, p.cbg);
+        }
     }
-    if (best_mt == 0) return p;
-    p.mt = best_mt;
-    p.npix = (int)(((long long)p.mt * kTileM + halo + 7) / 8 * 8);
+
+    if (!p.resident) {
+        // Streamed filters.  Measured: all SMs together draw filter stages from L2 at no more than
+        // ~5-6 TB/s, i.e. a 8 KB stage costs ~120 cycles on top of the MMAs that consume it unless it is
+        // reused by several tiles.  More tiles per item (mt) amortise that; fewer tiles leave room for a
+        // second accumulator set (hidden write-back) and balance better.  Cost in units of one tile's MMA
+        // time: rounds x mt x (1 + stage cost / MMA time) + exposed write-back.
+        const double mma_cycles = p.n_tile > 128 ? p.n_tile / 2 : 64;
+        const double tile_cycles = (double)p.taps * p.cblks * 2 * mma_cycles;
+        int best_mt = 0;
+        double best_cost = 0;
+        for (int mt = 4; mt >= 1; mt >>= 1) {
+            if (forced_mt && mt != forced_mt) continue;
+            if (mt * p.n_tile > 512) continue;
+            const int npix = npix_of(mt);
+            if (npix > 16000) continue;
+            if (smem_need(2, npix, p.n_tile, 2, 1, 1) > kSmemLimit) continue;
+            const long long items = (tiles + mt - 1) / mt * p.n_blocks;
+            const long long rounds = (items + sms - 1) / sms;
+            const int nbuf = (2 * mt * p.n_tile <= 512) ? 2 : 1;
+            const double stream = 1.0 + (chunk / 66.0) / (mt * 2 * mma_cycles);
+            const double writeback = (nbuf == 1 ? 1.0 : 0.15) * mt * (3000.0 * p.n_tile / 128.0) / tile_cycles;
+            const double cost = rounds * (mt * stream + 0.5 * writeback);
+            if (best_mt == 0 || cost < best_cost) { best_mt = mt; best_cost = cost; }
+        }
+        if (best_mt == 0) return p;
+        p.mt = best_mt;
+        p.npix = npix_of(p.mt);
+        // Filter stages: several taps per stage (up to 32 KB) so that the single MMA-issuing thread pays
+        // its per-stage bookkeeping (barrier wait, commit) once per 16-32 MMAs; the ring should hold
+        // 64-128 KB in flight to cover the L2 latency.
+        p.a_stages = 2;
+        p.cbg = 1;
+        p.tps = 32 * 1024 / chunk;
+        if (p.tps < 1) p.tps = 1;
+        if (p.tps > p.taps) p.tps = p.taps;
+        p.b_stages = 2;
+        while (p.tps > 1 && smem_need(p.a_stages, p.npix, p.n_tile, 3, p.tps, 1) > kSmemLimit) --p.tps;
+        while (p.b_stages < 4 && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps, 1) <= kSmemLimit) ++p.b_stages;
+        while (p.a_stages < kMaxAStages && p.taps <= 3 &&
+               smem_need(p.a_stages + 1, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg) <= kSmemLimit - 32 * 1024) ++p.a_stages;
+        while (p.b_stages < kMaxBStages && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps, p.cbg) <= kSmemLimit &&
+               (size_t)p.b_stages * p.tps * chunk < 128 * 1024) ++p.b_stages;
+        p.smem_bytes = smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg);
+    }
+
+    p.nbuf = (2 * p.mt * p.n_tile <= 512) ? 2 : 1;
     p.supertiles = (int)((tiles + p.mt - 1) / p.mt);
-    int cols = p.mt * p.n_tile;
+    const long long items = (long long)p.supertiles * p.n_blocks;
+    if (items > 0x7fffffffLL) return p;
+    p.grid = (int)(items < sms ? items : sms);
+    int cols = p.nbuf * p.mt * p.n_tile;
     p.tmem_cols = 32;
     while (p.tmem_cols < cols) p.tmem_cols <<= 1;
-
-    // Two blocks per SM when tensor memory (512 columns) and shared memory allow it.
-    const int chunk = kCB * p.n_tile * 4;
-    size_t limit = kSmemLimit;
-    p.blocks_per_sm = 1;
-    if (p.tmem_cols <= 256 && smem_need(2, p.npix, p.n_tile, 2, 1) <= kSmemLimitHalf &&
-        (size_t)2 * chunk * (p.taps < 4 ? p.taps : 4) + (size_t)2 * kCB * p.npix * 4 + 512 <= kSmemLimitHalf) {
-        p.blocks_per_sm = 2;
-        limit = kSmemLimitHalf;
-    }
-    p.a_stages = 2;
-    // Filter stages: several taps per stage (up to 32 KB) so that the single MMA-issuing thread pays its
-    // per-stage bookkeeping (barrier wait, commit) once per 16-32 MMAs; the ring should hold 64-128 KB in
-    // flight to cover the L2 latency.
-    p.tps = 32 * 1024 / chunk;
-    if (p.tps < 1) p.tps = 1;
-    if (p.tps > p.taps) p.tps = p.taps;
-    p.b_stages = 2;
-    while (p.tps > 1 && smem_need(p.a_stages, p.npix, p.n_tile, 3, p.tps) > limit) --p.tps;
-    while (p.b_stages < 4 && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps) <= limit) ++p.b_stages;
-    // Light tiles: an activation stage carries several channel blocks, so that one producer pass has
-    // 32-48 loads per thread in flight (the block is bound by memory latency, not by the MMAs).
-    p.cbg = 1;
-    if (light) {
-        while (p.cbg * 2 <= p.cblks && p.npix * p.cbg * 2 <= kProducers * kUnitsPerThread &&
-               smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg * 2) <= limit) p.cbg *= 2;
-    }
-    while (p.b_stages < kMaxBStages && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps, p.cbg) <= limit &&
-           (size_t)p.b_stages * p.tps * chunk < 128 * 1024) ++p.b_stages;
-    p.smem_bytes = smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg);
     p.ok = true;
     return p;
 }
 
-size_t packed_floats(const Shape& sh, const Plan& p)
+size_t packed_floats(const Plan& p)
 {
-    (void)sh;
     return (size_t)p.n_blocks * p.cblks * p.taps * kCB * p.n_tile;
 }
 
@@ -195,8 +250,10 @@ struct KernelArgs {
     int N, C, H, W, K, R, S, P, Q;
     int HW;
     int total_pix;
-    int n_tile, mt, npix, cblks, taps, a_stages, b_stages, tps;
+    int n_tile, n_blocks, mt, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
     int cbg, groups;        // channel blocks per activation stage, number of such groups
+    int resident;           // filters loaded once per thread block instead of streamed
+    int items;              // work items = supertiles x n_blocks
     unsigned tmem_cols;
 };
 
@@ -246,34 +303,33 @@ __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* 
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 general_tf32_kernel(const KernelArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     const uint32_t a_block_bytes = (uint32_t)kCB * a.npix * 4;          // one channel block of a stage
     const uint32_t a_stage_bytes = a_block_bytes * (uint32_t)a.cbg;
-    const uint32_t b_chunk_bytes = (uint32_t)kCB * a.n_tile * 4;     // one (channel block, tap)
+    const uint32_t b_chunk_bytes = (uint32_t)kCB * a.n_tile * 4;        // one (channel block, tap)
     const uint32_t b_stage_bytes = b_chunk_bytes * (uint32_t)a.tps;
     unsigned char* a_smem = smem;
     unsigned char* b_smem = smem + (size_t)a.a_stages * a_stage_bytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(b_smem + (size_t)a.b_stages * b_stage_bytes);
-    uint64_t* a_full = bars;                 // [kMaxAStages]
-    uint64_t* a_empty = bars + kMaxAStages;  // [kMaxAStages]
-    uint64_t* b_full = bars + 2 * kMaxAStages;             // [kMaxBStages]
-    uint64_t* b_empty = b_full + kMaxBStages;
-    uint64_t* acc_full = b_empty + kMaxBStages;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+    const size_t b_region_bytes = a.resident ? (size_t)a.cblks * a.taps * b_chunk_bytes : (size_t)a.b_stages * b_stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(b_smem + b_region_bytes);
+    uint64_t* a_full = bars;                               // [kMaxAStages]
+    uint64_t* a_empty = a_full + kMaxAStages;              // [kMaxAStages]
+    uint64_t* b_full = a_empty + kMaxAStages;              // [kMaxBStages]
+    uint64_t* b_empty = b_full + kMaxBStages;              // [kMaxBStages]
+    uint64_t* acc_full = b_empty + kMaxBStages;            // [2]
+    uint64_t* acc_empty = acc_full + 2;                    // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const long long t_entry = clock_now();
-    const int nb = blockIdx.y;
-    const int j0 = blockIdx.x * a.mt * kTileM;              // first flat pixel of this block
 
     if (tid == 0) {
         for (int i = 0; i < a.a_stages; ++i) { mbar_init(&a_full[i], kProducers); mbar_init(&a_empty[i], 1); }
         for (int i = 0; i < a.b_stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
-        mbar_init(acc_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpilogueWarps); }
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -284,37 +340,52 @@ general_tf32_kernel(const KernelArgs a)
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
-    const int steps = a.cblks * a.taps;                     // filter chunks this block consumes
-    const int grp_first = (int)(blockIdx.x % (unsigned)a.groups);  // channel-block group this block starts with
+    // Work item -> (supertile, filter block); blocks rotate the order of the channel-block groups by the
+    // item number, so that at any moment they stream different parts of the filter bank.
+    const int acc_cols = a.mt * a.n_tile;                   // tensor-memory columns of one accumulator set
 
     if (warp == 0) {
         // ---------------- filters: global -> shared by bulk copy, up to `tps` taps of one channel block per stage
         if (lane == 0) {
-            const unsigned char* src = reinterpret_cast<const unsigned char*>(a.wp) + (size_t)nb * steps * b_chunk_bytes;
             int s = 0, issued = 0;
             uint32_t ph = 0;
             bool alive = true;
-            // Blocks start at different channel-block groups (grp_first), so that at any moment they stream
-            // different parts of the filter bank.  Order: groups rotated, channel blocks inside a group
-            // ascending, taps ascending -- the order in which the MMA thread consumes them.
-            for (int grp = 0; grp < a.groups && alive; ++grp) {
-                int gr = grp + grp_first;
-                if (gr >= a.groups) gr -= a.groups;
-                for (int g = 0; g < a.cbg && alive; ++g) {
-                    const int cbr = gr * a.cbg + g;
-                    if (cbr >= a.cblks) break;
-                    for (int t0 = 0; t0 < a.taps; t0 += a.tps) {
-                        const int nt = min(a.tps, a.taps - t0);
-                        if (!mbar_wait_bounded(&b_empty[s], ph ^ 1u, abort_flag)) { alive = false; break; }
-                        const uint32_t bytes = b_chunk_bytes * (uint32_t)nt;
-                        mbar_arrive_expect_tx(&b_full[s], bytes);
-                        bulk_g2s(b_smem + (size_t)s * b_stage_bytes, src + ((size_t)cbr * a.taps + t0) * b_chunk_bytes, bytes, &b_full[s]);
-                        ++issued;
-                        if (++s == a.b_stages) { s = 0; ph ^= 1u; }
+            if (a.resident) {
+                // the whole filter bank (a single filter block in this mode), once, one bulk copy per channel
+                // block, all on one barrier
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(a.wp);
+                const uint32_t piece = b_chunk_bytes * (uint32_t)a.taps;
+                mbar_arrive_expect_tx(&b_full[0], piece * (uint32_t)a.cblks);
+                for (int cb = 0; cb < a.cblks; ++cb)
+                    bulk_g2s(b_smem + (size_t)cb * piece, src + (size_t)cb * piece, piece, &b_full[0]);
+                alive = false;          // nothing to stream
+                if (*abort_flag) { uint32_t dummy = 0; mbar_wait_bounded(&b_full[0], 0u, &dummy, 1u << 16); }
+            }
+            for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
+                const int nb = item % a.n_blocks;
+                const int grp_first = item % a.groups;
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(a.wp)
+                                         + (size_t)nb * a.cblks * a.taps * b_chunk_bytes;
+                for (int grp = 0; grp < a.groups && alive; ++grp) {
+                    int gr = grp + grp_first;
+                    if (gr >= a.groups) gr -= a.groups;
+                    for (int g = 0; g < a.cbg && alive; ++g) {
+                        const int cbr = gr * a.cbg + g;
+                        if (cbr >= a.cblks) break;
+                        for (int t0 = 0; t0 < a.taps; t0 += a.tps) {
+                            const int nt = min(a.tps, a.taps - t0);
+                            if (!mbar_wait_bounded(&b_empty[s], ph ^ 1u, abort_flag)) { alive = false; break; }
+                            const uint32_t bytes = b_chunk_bytes * (uint32_t)nt;
+                            mbar_arrive_expect_tx(&b_full[s], bytes);
+                            bulk_g2s(b_smem + (size_t)s * b_stage_bytes, src + ((size_t)cbr * a.taps + t0) * b_chunk_bytes,
+                                     bytes, &b_full[s]);
+                            ++issued;
+                            if (++s == a.b_stages) { s = 0; ph ^= 1u; }
+                        }
                     }
                 }
             }
-            if (*abort_flag) {
+            if (*abort_flag && !a.resident) {
                 // let copies already in flight land before the block's shared memory is released
                 const int pending = issued < a.b_stages ? issued : a.b_stages;
                 for (int i = 0; i < pending; ++i) {
@@ -337,89 +408,126 @@ general_tf32_kernel(const KernelArgs a)
             const uint32_t a_kstep = 2u * (uint32_t)a.npix;                     // 8 channels further, in 16-byte units
             const uint32_t b_kstep = 2u * (uint32_t)a.n_tile;
             bool alive = true;
-            long long t_first_mma = 0, wait_a = 0, wait_b = 0;   // diagnostics: operand-wait cycles of this thread
-            int as = 0, bs = 0;
-            uint32_t a_phase = 0, b_phase = 0, accumulate = 0;
-            for (int grp = 0; grp < a.groups && alive; ++grp) {
-                long long tw = clock_now();
-                if (!mbar_wait_bounded(&a_full[as], a_phase, abort_flag)) { alive = false; break; }
+            int as = 0, bs = 0, buf = 0;
+            uint32_t a_phase = 0, b_phase = 0, acc_phase0 = 0, acc_phase1 = 0;
+            // diagnostics of block 0 (status words 2..5): cycles this thread waited for activations and for a
+            // free accumulator set, its total cycles, its item count
+            long long wait_a = 0, wait_acc = 0;
+            const long long t_begin = clock_now();
+            int n_items = 0;
+            if (a.resident) {
+                if (!mbar_wait_bounded(&b_full[0], 0u, abort_flag)) alive = false;
                 tc_fence_after_sync();
-                wait_a += clock_now() - tw;
-                if (grp == 0) t_first_mma = clock_now();
-                int gr = grp + grp_first;
-                if (gr >= a.groups) gr -= a.groups;
-                uint32_t a_lo_block = a_lo_fixed | (smem_u32(a_smem + (size_t)as * a_stage_bytes) >> 4);
-                for (int g = 0; g < a.cbg && alive; ++g, a_lo_block += a_block_bytes >> 4) {
-                    if (gr * a.cbg + g >= a.cblks) break;
-                    uint32_t row_shift = 0;                                      // r * W, in pixels (= 16-byte units)
-                    int sx = 0;
-                    for (int t0 = 0; t0 < a.taps; t0 += a.tps) {
-                        const int nt = min(a.tps, a.taps - t0);
-                        tw = clock_now();
-                        if (!mbar_wait_bounded(&b_full[bs], b_phase, abort_flag)) { alive = false; break; }
-                        tc_fence_after_sync();
-                        wait_b += clock_now() - tw;
-                        uint32_t b_lo = b_lo_fixed | (smem_u32(b_smem + (size_t)bs * b_stage_bytes) >> 4);
-                        for (int t = 0; t < nt; ++t, b_lo += b_chunk_bytes >> 4) {
-                            uint32_t a_lo = a_lo_block + row_shift + (uint32_t)sx;
-                            uint32_t d = tmem;
-                            for (int m = 0; m < a.mt; ++m, a_lo += kTileM, d += (uint32_t)a.n_tile) {
-                                mma_tf32(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, accumulate != 0);
-                                mma_tf32(d, ((uint64_t)desc_hi << 32) | (a_lo + a_kstep), ((uint64_t)desc_hi << 32) | (b_lo + b_kstep), idesc, true);
-                            }
-                            accumulate = 1;
-                            if (++sx == a.S) { sx = 0; row_shift += (uint32_t)a.W; }
-                        }
-                        mma_commit(&b_empty[bs]);   // frees the filter stage when these MMAs have read it
-                        if (++bs == a.b_stages) { bs = 0; b_phase ^= 1u; }
-                    }
-                }
-                if (alive) mma_commit(&a_empty[as]);
-                if (++as == a.a_stages) { as = 0; a_phase ^= 1u; }
             }
-            if (alive) mma_commit(acc_full);
-            if (blockIdx.x == 0 && blockIdx.y == 0) {
-                // diagnostic time stamps of block (0,0), cycles since kernel entry: status words 2, 3
-                a.status[2] = (unsigned)(t_first_mma - t_entry);
-                a.status[3] = (unsigned)(clock_now() - t_entry);
-                a.status[7] = (unsigned)wait_a;
-                a.status[8] = (unsigned)wait_b;
+            for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
+                const int grp_first = item % a.groups;
+                // the accumulator set must have been drained by the epilogue of its previous item
+                const uint32_t acc_phase = buf ? acc_phase1 : acc_phase0;
+                long long tw = clock_now();
+                if (!mbar_wait_bounded(&acc_empty[buf], acc_phase ^ 1u, abort_flag)) { alive = false; break; }
+                tc_fence_after_sync();
+                wait_acc += clock_now() - tw;
+                const uint32_t d0 = tmem + (uint32_t)(buf * acc_cols);
+                uint32_t accumulate = 0;
+                for (int grp = 0; grp < a.groups && alive; ++grp) {
+                    tw = clock_now();
+                    if (!mbar_wait_bounded(&a_full[as], a_phase, abort_flag)) { alive = false; break; }
+                    tc_fence_after_sync();
+                    wait_a += clock_now() - tw;
+                    int gr = grp + grp_first;
+                    if (gr >= a.groups) gr -= a.groups;
+                    uint32_t a_lo_block = a_lo_fixed | (smem_u32(a_smem + (size_t)as * a_stage_bytes) >> 4);
+                    for (int g = 0; g < a.cbg && alive; ++g, a_lo_block += a_block_bytes >> 4) {
+                        if (gr * a.cbg + g >= a.cblks) break;
+                        uint32_t row_shift = 0;                                  // r * W, in pixels (= 16-byte units)
+                        int sx = 0;
+                        for (int t0 = 0; t0 < a.taps; t0 += a.tps) {
+                            const int nt = min(a.tps, a.taps - t0);
+                            uint32_t b_lo;
+                            if (a.resident) {
+                                b_lo = b_lo_fixed | (smem_u32(b_smem + (size_t)(gr * a.cbg + g) * a.taps * b_chunk_bytes) >> 4);
+                            } else {
+                                if (!mbar_wait_bounded(&b_full[bs], b_phase, abort_flag)) { alive = false; break; }
+                                tc_fence_after_sync();
+                                b_lo = b_lo_fixed | (smem_u32(b_smem + (size_t)bs * b_stage_bytes) >> 4);
+                            }
+                            for (int t = 0; t < nt; ++t, b_lo += b_chunk_bytes >> 4) {
+                                uint32_t a_lo = a_lo_block + row_shift + (uint32_t)sx;
+                                uint32_t d = d0;
+                                for (int m = 0; m < a.mt; ++m, a_lo += kTileM, d += (uint32_t)a.n_tile) {
+                                    mma_tf32(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, accumulate != 0);
+                                    mma_tf32(d, ((uint64_t)desc_hi << 32) | (a_lo + a_kstep),
+                                             ((uint64_t)desc_hi << 32) | (b_lo + b_kstep), idesc, true);
+                                }
+                                accumulate = 1;
+                                if (++sx == a.S) { sx = 0; row_shift += (uint32_t)a.W; }
+                            }
+                            if (!a.resident) {
+                                mma_commit(&b_empty[bs]);   // frees the filter stage when these MMAs have read it
+                                if (++bs == a.b_stages) { bs = 0; b_phase ^= 1u; }
+                            }
+                        }
+                    }
+                    if (alive) mma_commit(&a_empty[as]);
+                    if (++as == a.a_stages) { as = 0; a_phase ^= 1u; }
+                }
+                if (alive) mma_commit(&acc_full[buf]);
+                if (buf) acc_phase1 ^= 1u; else acc_phase0 ^= 1u;
+                if (++buf == a.nbuf) buf = 0;
+                ++n_items;
+            }
+            if (blockIdx.x == 0) {
+                a.status[2] = (unsigned)wait_a;
+                a.status[3] = (unsigned)wait_acc;
+                a.status[4] = (unsigned)(clock_now() - t_begin);
+                a.status[5] = (unsigned)n_items;
             }
         }
-    } else {
-        // ---------------- workers: stage activations, then drain the accumulators
-        const int wtid = tid - 64;
+    } else if (producer_index(warp) >= 0) {
+        // ---------------- producers: stage activations, running ahead across item boundaries
+        const int wtid = producer_index(warp) * 32 + lane;
         bool alive = true;
         int as = 0;
         uint32_t a_phase = 0;
-        // One stage = cbg consecutive channel blocks.  All loads of a pass (kUnitsPerThread units of 16
-        // channels per thread) are issued before its first store, so a pass costs one memory round trip.
         const int units = a.npix * a.cbg;
-        for (int grp = 0; grp < a.groups && alive; ++grp) {
-            if (!mbar_wait_bounded(&a_empty[as], a_phase ^ 1u, abort_flag)) { alive = false; break; }
-            float4* dst = reinterpret_cast<float4*>(a_smem + (size_t)as * a_stage_bytes);
-            int gr = grp + grp_first;
-            if (gr >= a.groups) gr -= a.groups;
-            for (int first = 0; first < units; first += kProducers * kUnitsPerThread) {
-                float v[kUnitsPerThread][kCB];
-                load_units(v, a, j0, gr * a.cbg, first, wtid);
-                store_units(v, dst, a, first, wtid);
+        for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
+            const int j0 = (item / a.n_blocks) * a.mt * kTileM;          // first flat pixel of the item
+            const int grp_first = item % a.groups;
+            // One stage = cbg consecutive channel blocks.  All loads of a pass (kUnitsPerThread units of
+            // 16 channels per thread) are issued before its first store: a pass costs one memory round trip.
+            for (int grp = 0; grp < a.groups && alive; ++grp) {
+                if (!mbar_wait_bounded(&a_empty[as], a_phase ^ 1u, abort_flag)) { alive = false; break; }
+                float4* dst = reinterpret_cast<float4*>(a_smem + (size_t)as * a_stage_bytes);
+                int gr = grp + grp_first;
+                if (gr >= a.groups) gr -= a.groups;
+                for (int first = 0; first < units; first += kProducers * kUnitsPerThread) {
+                    float v[kUnitsPerThread][kCB];
+                    load_units(v, a, j0, gr * a.cbg, first, wtid);
+                    store_units(v, dst, a, first, wtid);
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(&a_full[as]);
+                if (++as == a.a_stages) { as = 0; a_phase ^= 1u; }
             }
-            fence_proxy_async_smem();
-            mbar_arrive(&a_full[as]);
-            if (++as == a.a_stages) { as = 0; a_phase ^= 1u; }
         }
-
-        // tcgen05.ld is warp-collective: take the decision for the whole warp
-        if (__all_sync(0xffffffffu, alive && mbar_wait_bounded(acc_full, 0u, abort_flag))) {
+    } else if (warp >= 4 && warp < 4 + kEpilogueWarps) {
+        // ---------------- epilogue: drain finished accumulator sets (lane = pixel)
+        const int quarter = warp & 3;                       // tensor-memory lanes this warp may read
+        const size_t plane = (size_t)a.P * a.Q;
+        const int chunks_per_tile = a.n_tile / 16;
+        const int total_chunks = a.mt * chunks_per_tile;
+        int buf = 0;
+        uint32_t acc_phase0 = 0, acc_phase1 = 0;
+        bool alive = true;
+        for (int item = blockIdx.x; item < a.items; item += gridDim.x) {
+            const int j0 = (item / a.n_blocks) * a.mt * kTileM;
+            const int nb = item % a.n_blocks;
+            // tcgen05.ld is warp-collective: take the decision for the whole warp
+            const uint32_t acc_phase = buf ? acc_phase1 : acc_phase0;
+            alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag));
+            if (!alive) break;
             tc_fence_after_sync();
-            if (tid == 64 && blockIdx.x == 0 && blockIdx.y == 0) a.status[4] = (unsigned)(clock_now() - t_entry);
-            const int quarter = warp & 3;                    // tensor-memory lanes this warp may read
-            const int half = (warp - 2) >> 2;                // the two warps of a quarter split the columns
-            const size_t plane = (size_t)a.P * a.Q;
-            const int chunks_per_tile = a.n_tile / 16;
-            const int total_chunks = a.mt * chunks_per_tile;
-            const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+            const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * acc_cols);
             int cur_m = -1;
             bool ok = false;
             float* yb = a.y;
@@ -452,26 +560,29 @@ general_tf32_kernel(const KernelArgs a)
             };
             // Two register buffers: the load of the next chunk is in flight while the current one is stored.
             uint32_t va[16], vb[16];
-            int c = half;
-            if (c < total_chunks) load_chunk(va, c);
+            int c = 0;
+            load_chunk(va, c);
             while (c < total_chunks) {
                 tmem_ld_wait();
-                if (c + 2 < total_chunks) load_chunk(vb, c + 2);
+                if (c + 1 < total_chunks) load_chunk(vb, c + 1);
                 store_chunk(va, c);
-                c += 2;
-                if (c >= total_chunks) break;
+                if (++c >= total_chunks) break;
                 tmem_ld_wait();
-                if (c + 2 < total_chunks) load_chunk(va, c + 2);
+                if (c + 1 < total_chunks) load_chunk(va, c + 1);
                 store_chunk(vb, c);
-                c += 2;
+                ++c;
             }
-            if (tid == 64 && blockIdx.x == 0 && blockIdx.y == 0) a.status[6] = (unsigned)(clock_now() - t_entry);
+            // all of this warp's reads of the accumulator set are complete: hand it back to the MMA thread
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            if (buf) acc_phase1 ^= 1u; else acc_phase0 ^= 1u;
+            if (++buf == a.nbuf) buf = 0;
         }
     }
 
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) a.status[5] = (unsigned)(clock_now() - t_entry);
     if (warp == 1) tmem_dealloc(tmem, a.tmem_cols);
     if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
 }
@@ -487,7 +598,7 @@ size_t tf32_workspace_bytes(const Shape& sh)
 {
     const Plan p = make_plan(sh);
     if (!p.ok) return kStatusBytes;
-    return kStatusBytes + packed_floats(sh, p) * sizeof(float);
+    return kStatusBytes + packed_floats(p) * sizeof(float);
 }
 
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
@@ -499,7 +610,7 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
     float* wp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
 
     if (!weights_packed) {
-        const long long total = (long long)packed_floats(sh, p);
+        const long long total = (long long)packed_floats(p);
         long long blocks = (total + 255) / 256;
         if (blocks > 148 * 16) blocks = 148 * 16;
         repack_filters_kernel<<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, sh.C, p.taps, p.n_tile, p.cblks, total);
@@ -518,12 +629,13 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
     a.N = sh.N; a.C = sh.C; a.H = sh.H; a.W = sh.W; a.K = sh.K; a.R = sh.R; a.S = sh.S; a.P = sh.P; a.Q = sh.Q;
     a.HW = sh.H * sh.W;
     a.total_pix = sh.N * sh.H * sh.W;
-    a.n_tile = p.n_tile; a.mt = p.mt; a.npix = p.npix; a.cblks = p.cblks; a.taps = p.taps;
+    a.n_tile = p.n_tile; a.n_blocks = p.n_blocks; a.mt = p.mt; a.nbuf = p.nbuf; a.npix = p.npix;
+    a.cblks = p.cblks; a.taps = p.taps;
     a.a_stages = p.a_stages; a.b_stages = p.b_stages; a.tps = p.tps;
-    a.cbg = p.cbg; a.groups = (p.cblks + p.cbg - 1) / p.cbg;
+    a.cbg = p.cbg; a.groups = (p.cblks + p.cbg - 1) / p.cbg; a.resident = p.resident;
+    a.items = p.supertiles * p.n_blocks;
     a.tmem_cols = (unsigned)p.tmem_cols;
-    dim3 grid((unsigned)p.supertiles, (unsigned)p.n_blocks, 1);
-    general_tf32_kernel<<<grid, kThreads, p.smem_bytes, stream>>>(a);
+    general_tf32_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
 }
