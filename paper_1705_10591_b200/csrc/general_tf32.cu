@@ -80,6 +80,8 @@ constexpr int kMaxBStages = 16;
 constexpr int kMaxAStages = 4;
 constexpr int kUnitsPerThread = 3;          // (pixel, channel block) units a producer thread keeps in flight per pass
 constexpr size_t kSmemLimit = 227 * 1024;
+constexpr int kXposePitch = 36;             // floats per row of the epilogue's transposition tile (16-byte aligned, conflict-free)
+constexpr size_t kXposeBytes = (size_t)kEpilogueWarps * 32 * kXposePitch * 4;
 
 struct Plan {
     int n_tile;       // filters per work item (UMMA N), multiple of 16
@@ -94,6 +96,7 @@ struct Plan {
     int tps;          // taps per filter stage
     int cbg;          // channel blocks per activation stage
     int resident;     // 1: the whole filter block stays in shared memory for the life of the thread block
+    int swap;         // 1: filters are the MMA's M operand, 256 pixels its N operand (K <= 128)
     int tmem_cols;    // power of two >= 32
     int supertiles;   // work-item rows over the flat pixel sequence
     int grid;
@@ -122,8 +125,15 @@ Plan make_plan(const Shape& sh)
     const int kp16 = (sh.K + 15) / 16 * 16;
     p.n_blocks = (kp16 + 255) / 256;
     p.n_tile = ((sh.K + p.n_blocks - 1) / p.n_blocks + 15) / 16 * 16;
+    // Operand roles.  One tcgen05.mma costs its issuing thread ~60 cycles whatever its size (measured), so
+    // an instruction must carry >= 128 cycles of tensor-pipe work to keep the pipe busy: N = 256.  With up
+    // to 128 filters that is only possible with the pixels as the N operand: M = 128 filters (padded),
+    // N = 256 pixels, accumulator lanes = filters.  With more filters the pixels stay the M operand.
+    p.swap = (kp16 <= 128 && env_int("CONV2D_B200_TF32_SWAP", 1) != 0) ? 1 : 0;
+    if (p.swap) { p.n_blocks = 1; p.n_tile = 128; }
     p.cblks = (sh.C + kCB - 1) / kCB;
     p.taps = sh.R * sh.S;
+    const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
     const long long halo = (long long)(sh.R - 1) * sh.W + (sh.S - 1);
     const long long tiles = (total_pix + kTileM - 1) / kTileM;
     const int chunk = kCB * p.n_tile * 4;
@@ -139,9 +149,9 @@ Plan make_plan(const Shape& sh)
     // latency: one producer pass should have 32-48 loads per thread in flight).
     p.resident = 0;
     if (env_int("CONV2D_B200_TF32_RESIDENT", 1) != 0 && p.n_blocks == 1 && wbytes <= 152 * 1024) {
-        const int mt = forced_mt ? forced_mt : 1;
+        const int mt = forced_mt ? forced_mt : (p.swap ? 2 : 1);
         const int npix = npix_of(mt);
-        if (mt * p.n_tile <= 512 && npix <= 16000 && wbytes + (size_t)2 * kCB * npix * 4 + 512 <= kSmemLimit) {
+        if (mt * p.n_tile <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * npix * 4 + 512 <= kSmemLimit) {
             p.resident = 1;
             p.mt = mt;
             p.npix = npix;
@@ -149,7 +159,7 @@ Plan make_plan(const Shape& sh)
             p.a_stages = 2;
             p.b_stages = 1;
             p.tps = p.taps;
-            auto need = [&](int a_stages, int cbg) { return wbytes + (size_t)a_stages * cbg * kCB * npix * 4 + 512; };
+            auto need = [&](int a_stages, int cbg) { return wbytes + extra + (size_t)a_stages * cbg * kCB * npix * 4 + 512; };
             while (p.cbg * 2 <= p.cblks && npix * p.cbg * 2 <= kProducers * kUnitsPerThread &&
                    need(p.a_stages, p.cbg * 2) <= kSmemLimit) p.cbg *= 2;
             while (p.a_stages < kMaxAStages && need(p.a_stages + 1, p.cbg) <= kSmemLimit) ++p.a_stages;
@@ -163,16 +173,18 @@ Plan make_plan(const Shape& sh)
         // reused by several tiles.  More tiles per item (mt) amortise that; fewer tiles leave room for a
         // second accumulator set (hidden write-back) and balance better.  Cost in units of one tile's MMA
         // time: rounds x mt x (1 + stage cost / MMA time) + exposed write-back.
-        const double mma_cycles = p.n_tile > 128 ? p.n_tile / 2 : 64;
+        const double mma_cycles = p.swap ? 64 : (p.n_tile > 128 ? p.n_tile / 2 : 90);   // per 128-pixel tile and K step
         const double tile_cycles = (double)p.taps * p.cblks * 2 * mma_cycles;
         int best_mt = 0;
         double best_cost = 0;
+        const size_t kLimit = kSmemLimit - extra;
         for (int mt = 4; mt >= 1; mt >>= 1) {
             if (forced_mt && mt != forced_mt) continue;
+            if (p.swap && mt < 2) continue;
             if (mt * p.n_tile > 512) continue;
             const int npix = npix_of(mt);
             if (npix > 16000) continue;
-            if (smem_need(2, npix, p.n_tile, 2, 1, 1) > kSmemLimit) continue;
+            if (smem_need(2, npix, p.n_tile, 2, 1, 1) > kLimit) continue;
             const long long items = (tiles + mt - 1) / mt * p.n_blocks;
             const long long rounds = (items + sms - 1) / sms;
             const int nbuf = (2 * mt * p.n_tile <= 512) ? 2 : 1;
@@ -193,13 +205,13 @@ Plan make_plan(const Shape& sh)
         if (p.tps < 1) p.tps = 1;
         if (p.tps > p.taps) p.tps = p.taps;
         p.b_stages = 2;
-        while (p.tps > 1 && smem_need(p.a_stages, p.npix, p.n_tile, 3, p.tps, 1) > kSmemLimit) --p.tps;
-        while (p.b_stages < 4 && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps, 1) <= kSmemLimit) ++p.b_stages;
+        while (p.tps > 1 && smem_need(p.a_stages, p.npix, p.n_tile, 3, p.tps, 1) > kLimit) --p.tps;
+        while (p.b_stages < 4 && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps, 1) <= kLimit) ++p.b_stages;
         while (p.a_stages < kMaxAStages && p.taps <= 3 &&
-               smem_need(p.a_stages + 1, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg) <= kSmemLimit - 32 * 1024) ++p.a_stages;
-        while (p.b_stages < kMaxBStages && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps, p.cbg) <= kSmemLimit &&
+               smem_need(p.a_stages + 1, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg) <= kLimit - 32 * 1024) ++p.a_stages;
+        while (p.b_stages < kMaxBStages && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps, p.cbg) <= kLimit &&
                (size_t)p.b_stages * p.tps * chunk < 128 * 1024) ++p.b_stages;
-        p.smem_bytes = smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg);
+        p.smem_bytes = smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg) + extra;
     }
 
     p.nbuf = (2 * p.mt * p.n_tile <= 512) ? 2 : 1;
@@ -253,6 +265,7 @@ struct KernelArgs {
     int n_tile, n_blocks, mt, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
     int cbg, groups;        // channel blocks per activation stage, number of such groups
     int resident;           // filters loaded once per thread block instead of streamed
+    int swap;               // operand roles swapped: accumulator lanes = filters, columns = pixels
     int items;              // work items = supertiles x n_blocks
     unsigned tmem_cols;
 };
@@ -314,7 +327,8 @@ general_tf32_kernel(const KernelArgs a)
     unsigned char* a_smem = smem;
     unsigned char* b_smem = smem + (size_t)a.a_stages * a_stage_bytes;
     const size_t b_region_bytes = a.resident ? (size_t)a.cblks * a.taps * b_chunk_bytes : (size_t)a.b_stages * b_stage_bytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(b_smem + b_region_bytes);
+    float* xpose = reinterpret_cast<float*>(b_smem + b_region_bytes);            // only present (and used) when a.swap
+    uint64_t* bars = reinterpret_cast<uint64_t*>(b_smem + b_region_bytes + (a.swap ? kXposeBytes : 0));
     uint64_t* a_full = bars;                               // [kMaxAStages]
     uint64_t* a_empty = a_full + kMaxAStages;              // [kMaxAStages]
     uint64_t* b_full = a_empty + kMaxAStages;              // [kMaxBStages]
@@ -401,7 +415,7 @@ general_tf32_kernel(const KernelArgs a)
             // Per MMA this thread only adds small constants to the low word of a descriptor: everything
             // that does not change is folded into a_lo_fixed / b_lo_fixed / desc_hi beforehand, because a
             // single thread issuing ~40 dependent integer instructions per MMA was slower than the MMA.
-            const uint32_t idesc = idesc_tf32(kTileM, (uint32_t)a.n_tile);
+            const uint32_t idesc = a.swap ? idesc_tf32(128u, 256u) : idesc_tf32(kTileM, (uint32_t)a.n_tile);
             const uint32_t desc_hi = (128u >> 4) | (1u << 14);                  // SBO = 128 B, descriptor version 1
             const uint32_t a_lo_fixed = ((uint32_t)a.npix & 0x3FFFu) << 16;     // LBO = npix * 16 B
             const uint32_t b_lo_fixed = ((uint32_t)a.n_tile & 0x3FFFu) << 16;   // LBO = n_tile * 16 B
@@ -454,10 +468,19 @@ general_tf32_kernel(const KernelArgs a)
                             for (int t = 0; t < nt; ++t, b_lo += b_chunk_bytes >> 4) {
                                 uint32_t a_lo = a_lo_block + row_shift + (uint32_t)sx;
                                 uint32_t d = d0;
-                                for (int m = 0; m < a.mt; ++m, a_lo += kTileM, d += (uint32_t)a.n_tile) {
-                                    mma_tf32(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, accumulate != 0);
-                                    mma_tf32(d, ((uint64_t)desc_hi << 32) | (a_lo + a_kstep),
-                                             ((uint64_t)desc_hi << 32) | (b_lo + b_kstep), idesc, true);
+                                if (a.swap) {
+                                    // M operand = the 128 filters of this stage, N operand = 256 staged pixels
+                                    for (int m = 0; m < a.mt; m += 2, a_lo += 2 * kTileM, d += 2 * kTileM) {
+                                        mma_tf32(d, ((uint64_t)desc_hi << 32) | b_lo, ((uint64_t)desc_hi << 32) | a_lo, idesc, accumulate != 0);
+                                        mma_tf32(d, ((uint64_t)desc_hi << 32) | (b_lo + b_kstep),
+                                                 ((uint64_t)desc_hi << 32) | (a_lo + a_kstep), idesc, true);
+                                    }
+                                } else {
+                                    for (int m = 0; m < a.mt; ++m, a_lo += kTileM, d += (uint32_t)a.n_tile) {
+                                        mma_tf32(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, accumulate != 0);
+                                        mma_tf32(d, ((uint64_t)desc_hi << 32) | (a_lo + a_kstep),
+                                                 ((uint64_t)desc_hi << 32) | (b_lo + b_kstep), idesc, true);
+                                    }
                                 }
                                 accumulate = 1;
                                 if (++sx == a.S) { sx = 0; row_shift += (uint32_t)a.W; }
@@ -528,6 +551,63 @@ general_tf32_kernel(const KernelArgs a)
             if (!alive) break;
             tc_fence_after_sync();
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * acc_cols);
+            if (a.swap) {
+                // Lanes are filters, columns pixels: this thread holds adjacent pixels of ONE map.  A
+                // warp-private shared-memory tile turns a 32-filter x 32-pixel block around so that each
+                // store instruction again writes 32 adjacent pixels of one map.
+                float* tile = xpose + (size_t)(warp - 4) * 32 * kXposePitch;
+                const int blocks = a.mt * kTileM / 32;
+                auto load_block = [&](uint32_t (&v0)[16], uint32_t (&v1)[16], int b) {
+                    tmem_ld16(lane_base + (uint32_t)(b * 32), v0);
+                    tmem_ld16(lane_base + (uint32_t)(b * 32 + 16), v1);
+                };
+                auto store_block = [&](const uint32_t (&v0)[16], const uint32_t (&v1)[16], int b) {
+                    __syncwarp();                                   // the previous block has been read out
+                    float4* row = reinterpret_cast<float4*>(tile + lane * kXposePitch);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        row[i] = make_float4(__uint_as_float(v0[4 * i]), __uint_as_float(v0[4 * i + 1]),
+                                             __uint_as_float(v0[4 * i + 2]), __uint_as_float(v0[4 * i + 3]));
+                        row[4 + i] = make_float4(__uint_as_float(v1[4 * i]), __uint_as_float(v1[4 * i + 1]),
+                                                 __uint_as_float(v1[4 * i + 2]), __uint_as_float(v1[4 * i + 3]));
+                    }
+                    __syncwarp();
+                    const int j = j0 + b * 32 + lane;               // this lane's pixel of the block
+                    bool ok = j < a.total_pix;
+                    float* o = a.y;
+                    if (ok) {
+                        const int n = j / a.HW, off = j - n * a.HW;
+                        const int p = off / a.W, q = off - p * a.W;
+                        ok = (p < a.P) && (q < a.Q);
+                        o = a.y + (((size_t)n * a.K + quarter * 32) * a.P + p) * a.Q + q;
+                    }
+                    if (ok) {
+                        const int kmax = a.K - quarter * 32;        // maps of this quarter that exist
+#pragma unroll 8
+                        for (int r = 0; r < 32; ++r, o += plane)
+                            if (r < kmax) *o = tile[r * kXposePitch + lane];
+                    }
+                };
+                uint32_t va0[16], va1[16], vb0[16], vb1[16];
+                int b = 0;
+                load_block(va0, va1, b);
+                while (b < blocks) {
+                    tmem_ld_wait();
+                    if (b + 1 < blocks) load_block(vb0, vb1, b + 1);
+                    store_block(va0, va1, b);
+                    if (++b >= blocks) break;
+                    tmem_ld_wait();
+                    if (b + 1 < blocks) load_block(va0, va1, b + 1);
+                    store_block(vb0, vb1, b);
+                    ++b;
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                if (buf) acc_phase1 ^= 1u; else acc_phase0 ^= 1u;
+                if (++buf == a.nbuf) buf = 0;
+                continue;
+            }
             int cur_m = -1;
             bool ok = false;
             float* yb = a.y;
@@ -632,7 +712,7 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
     a.n_tile = p.n_tile; a.n_blocks = p.n_blocks; a.mt = p.mt; a.nbuf = p.nbuf; a.npix = p.npix;
     a.cblks = p.cblks; a.taps = p.taps;
     a.a_stages = p.a_stages; a.b_stages = p.b_stages; a.tps = p.tps;
-    a.cbg = p.cbg; a.groups = (p.cblks + p.cbg - 1) / p.cbg; a.resident = p.resident;
+    a.cbg = p.cbg; a.groups = (p.cblks + p.cbg - 1) / p.cbg; a.resident = p.resident; a.swap = p.swap;
     a.items = p.supertiles * p.n_blocks;
     a.tmem_cols = (unsigned)p.tmem_cols;
     general_tf32_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
