@@ -129,7 +129,7 @@ Plan make_plan(const Shape& sh)
     // an instruction must carry >= 128 cycles of tensor-pipe work to keep the pipe busy: N = 256.  With up
     // to 128 filters that is only possible with the pixels as the N operand: M = 128 filters (padded),
     // N = 256 pixels, accumulator lanes = filters.  With more filters the pixels stay the M operand.
-    p.swap = (kp16 <= 128 && env_int("CONV2D_B200_TF32_SWAP", 1) != 0) ? 1 : 0;
+    p.swap = (kp16 > 64 && kp16 <= 128 && env_int("CONV2D_B200_TF32_SWAP", 1) != 0) ? 1 : 0;   // <= 64 filters: padding to 128 would double the work
     if (p.swap) { p.n_blocks = 1; p.n_tile = 128; }
     p.cblks = (sh.C + kCB - 1) / kCB;
     p.taps = sh.R * sh.S;
@@ -143,12 +143,14 @@ Plan make_plan(const Shape& sh)
     const size_t wbytes = (size_t)p.cblks * p.taps * chunk;        // re-ordered filters of one filter block
     auto npix_of = [&](int mt) { return (int)(((long long)mt * kTileM + halo + 7) / 8 * 8); };
 
-    // Small filter banks stay resident in shared memory: nothing is streamed, so one tile per item is
-    // best (finest balance over the SMs, two accumulator sets), and the rest of shared memory becomes a
-    // deep activation ring whose stages carry several channel blocks (these items are bound by memory
-    // latency: one producer pass should have 32-48 loads per thread in flight).
+    // Light problems (1x1-like: few taps x channel blocks) with a small filter bank keep it resident in
+    // shared memory: nothing is streamed, items are small (finest balance over the SMs, two accumulator
+    // sets), and the rest of shared memory becomes a deep activation ring whose stages carry several
+    // channel blocks (these items are bound by memory latency: one producer pass should have 32-48 loads
+    // per thread in flight).  Measured: for 3x3 with 64 filters streaming with two tiles per item is faster.
     p.resident = 0;
-    if (env_int("CONV2D_B200_TF32_RESIDENT", 1) != 0 && p.n_blocks == 1 && wbytes <= 152 * 1024) {
+    if (env_int("CONV2D_B200_TF32_RESIDENT", 1) != 0 && p.n_blocks == 1 && wbytes <= 152 * 1024 &&
+        (long long)p.taps * p.cblks <= 16) {
         const int mt = forced_mt ? forced_mt : (p.swap ? 2 : 1);
         const int npix = npix_of(mt);
         if (mt * p.n_tile <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * npix * 4 + 512 <= kSmemLimit) {
@@ -266,6 +268,7 @@ struct KernelArgs {
     int cbg, groups;        // channel blocks per activation stage, number of such groups
     int resident;           // filters loaded once per thread block instead of streamed
     int swap;               // operand roles swapped: accumulator lanes = filters, columns = pixels
+    int vec;                // swap mode: adjacent pixels a lane stores as one unit (1, 2 or 4)
     int items;              // work items = supertiles x n_blocks
     unsigned tmem_cols;
 };
@@ -552,6 +555,7 @@ general_tf32_kernel(const KernelArgs a)
             tc_fence_after_sync();
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * acc_cols);
             if (a.swap) {
+                const long long t_epi = clock_now();
                 // Lanes are filters, columns pixels: this thread holds adjacent pixels of ONE map.  A
                 // warp-private shared-memory tile turns a 32-filter x 32-pixel block around so that each
                 // store instruction again writes 32 adjacent pixels of one map.
@@ -572,20 +576,37 @@ general_tf32_kernel(const KernelArgs a)
                                                  __uint_as_float(v1[4 * i + 2]), __uint_as_float(v1[4 * i + 3]));
                     }
                     __syncwarp();
-                    const int j = j0 + b * 32 + lane;               // this lane's pixel of the block
+                    // Each lane stores `vec` adjacent pixels of one map, so one instruction covers `vec` maps:
+                    // per-warp store throughput is bounded by instructions in flight, not bytes (measured
+                    // ~2.7 B/clk per warp with 4-byte lanes), hence the widest unit the alignment allows.
+                    const int vec = a.vec;                          // 1, 2 or 4 (W, Q, P*Q multiples of vec)
+                    const int lanes_per_row = 32 / vec;
+                    const int row_sub = lane / lanes_per_row, pg = lane - row_sub * lanes_per_row;
+                    const int j = j0 + b * 32 + pg * vec;           // this lane's first pixel of the block
                     bool ok = j < a.total_pix;
                     float* o = a.y;
                     if (ok) {
                         const int n = j / a.HW, off = j - n * a.HW;
                         const int p = off / a.W, q = off - p * a.W;
                         ok = (p < a.P) && (q < a.Q);
-                        o = a.y + (((size_t)n * a.K + quarter * 32) * a.P + p) * a.Q + q;
+                        o = a.y + (((size_t)n * a.K + quarter * 32 + row_sub) * a.P + p) * a.Q + q;
                     }
                     if (ok) {
                         const int kmax = a.K - quarter * 32;        // maps of this quarter that exist
+                        const float* src = tile + row_sub * kXposePitch + pg * vec;
+                        if (vec == 4) {
+#pragma unroll
+                            for (int r = 0; r < 32; r += 4, o += 4 * plane, src += 4 * kXposePitch)
+                                if (r + row_sub < kmax) *reinterpret_cast<float4*>(o) = *reinterpret_cast<const float4*>(src);
+                        } else if (vec == 2) {
 #pragma unroll 8
-                        for (int r = 0; r < 32; ++r, o += plane)
-                            if (r < kmax) *o = tile[r * kXposePitch + lane];
+                            for (int r = 0; r < 32; r += 2, o += 2 * plane, src += 2 * kXposePitch)
+                                if (r + row_sub < kmax) *reinterpret_cast<float2*>(o) = *reinterpret_cast<const float2*>(src);
+                        } else {
+#pragma unroll 8
+                            for (int r = 0; r < 32; ++r, o += plane, src += kXposePitch)
+                                if (r < kmax) *o = *src;
+                        }
                     }
                 };
                 uint32_t va0[16], va1[16], vb0[16], vb1[16];
@@ -604,6 +625,7 @@ general_tf32_kernel(const KernelArgs a)
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                if (blockIdx.x == 0 && warp == 4 && lane == 0) a.status[6] = (unsigned)(clock_now() - t_epi);
                 if (buf) acc_phase1 ^= 1u; else acc_phase0 ^= 1u;
                 if (++buf == a.nbuf) buf = 0;
                 continue;
@@ -713,6 +735,10 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
     a.cblks = p.cblks; a.taps = p.taps;
     a.a_stages = p.a_stages; a.b_stages = p.b_stages; a.tps = p.tps;
     a.cbg = p.cbg; a.groups = (p.cblks + p.cbg - 1) / p.cbg; a.resident = p.resident; a.swap = p.swap;
+    a.vec = 1;
+    for (int v = 4; v >= 2; v >>= 1)
+        if (sh.W % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
+            reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
     a.items = p.supertiles * p.n_blocks;
     a.tmem_cols = (unsigned)p.tmem_cols;
     general_tf32_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
