@@ -111,7 +111,12 @@ GENERAL_SHAPES = [
     (3, 32, 9, 9, 16, 1, 1),
     (1, 4, 11, 10, 3, 2, 4),       # rectangular taps -> shape-agnostic kernel
     (2, 5, 3, 3, 4, 3, 3),         # one output per map
-    (1, 64, 14, 14, 96, 3, 3),
+    (1, 64, 14, 14, 96, 3, 3),     # 96 filters: operand-swap path with zero-padded filters
+    (2, 20, 10, 12, 300, 3, 3),    # 300 filters: two filter blocks, partial last channel block
+    (1, 40, 16, 16, 130, 1, 7),    # 1 x 7 taps, 130 filters (pixels stay the M operand)
+    (5, 33, 7, 9, 128, 3, 3),      # batch*H*W = 315 pixels: ragged last tile, images change inside a tile
+    (1, 16, 6, 70, 72, 5, 3),      # wide rows: horizontal wrap inside a tile
+    (2, 48, 12, 12, 128, 1, 1),    # 1 x 1 with resident filters
 ]
 
 
@@ -184,6 +189,34 @@ def test_full_size_configs(oracle, name, algo):
         worst = max(worst, assert_parity(y[n:n + 1, k:k + 1], y_ref, yabs, tol, f"{name} plane {(n, k)}"))
     assert np.isfinite(y).all()
     print(f"{name} algo={algo} max ratio {worst:.3e}")
+
+
+def test_auto_falls_back_to_fp32_when_no_tensor_core_instance_fits(oracle):
+    """A very wide image needs a staged halo beyond shared memory: AUTO must still give the right answer."""
+    import paper_1705_10591_b200 as lib
+    dims = (1, 4, 6, 6000, 8, 5, 5)
+    assert not _tf32_available(dims)
+    with pytest.raises(lib.Conv2dError) as e:
+        lib.conv2d_fwd_workspace_size(*dims, ALGO_TF32)
+    assert e.value.status == 5
+    N, C, H, W, K, R, S = dims
+    x, w = small_integers((N, C, H, W), 421), small_integers((K, C, R, S), 422)
+    y_ref, _ = oracle.conv2d_oracle(x, w)
+    np.testing.assert_array_equal(run_library(x, w, entry="general", algo=ALGO_AUTO).astype(np.float64), y_ref)
+
+
+def test_prepacked_filters_flag_reuses_the_workspace(oracle):
+    import torch
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K, R, S = 2, 32, 12, 12, 128, 3, 3
+    x1, x2 = uniform((N, C, H, W), 431), uniform((N, C, H, W), 432)
+    w = uniform((K, C, R, S), 433)
+    ws = torch.zeros(lib.conv2d_fwd_workspace_size(N, C, H, W, K, R, S, ALGO_TF32), dtype=torch.uint8, device="cuda:0")
+    y1 = run_library(x1, w, entry="general", algo=ALGO_TF32, workspace=ws)
+    y2 = run_library(x2, w, entry="general", algo=ALGO_TF32, workspace=ws, flags=1)   # filters already re-ordered
+    for x, y in ((x1, y1), (x2, y2)):
+        y_ref, yabs = oracle.conv2d_oracle(x, w)
+        assert_parity(y, y_ref, yabs, TF32_TOL, "prepacked")
 
 
 def test_relu_zero_windows_give_exact_zero(oracle):
