@@ -97,6 +97,7 @@ struct Plan {
     int cbg;          // channel blocks per activation stage
     int resident;     // 1: the whole filter block stays in shared memory for the life of the thread block
     int swap;         // 1: filters are the MMA's M operand, 256 pixels its N operand (K <= 128)
+    int ksplit;       // 2: the channel blocks of a tile are shared by two work items that add into y
     int tmem_cols;    // power of two >= 32
     int supertiles;   // work-item rows over the flat pixel sequence
     int grid;
@@ -126,11 +127,12 @@ Plan make_plan(const Shape& sh)
     p.n_blocks = (kp16 + 255) / 256;
     p.n_tile = ((sh.K + p.n_blocks - 1) / p.n_blocks + 15) / 16 * 16;
     // Operand roles.  One tcgen05.mma costs its issuing thread ~60 cycles whatever its size (measured), so
-    // an instruction must carry >= 128 cycles of tensor-pipe work to keep the pipe busy: N = 256.  With up
-    // to 128 filters that is only possible with the pixels as the N operand: M = 128 filters (padded),
-    // N = 256 pixels, accumulator lanes = filters.  With more filters the pixels stay the M operand.
-    p.swap = (kp16 > 64 && kp16 <= 128 && env_int("CONV2D_B200_TF32_SWAP", 1) != 0) ? 1 : 0;   // <= 64 filters: padding to 128 would double the work
-    if (p.swap) { p.n_blocks = 1; p.n_tile = 128; }
+    // an instruction must carry >= 128 cycles of tensor-pipe work to keep the pipe busy: N = 256.  For any
+    // filter count that is possible with the pixels as the N operand: M = a block of 128 filters (zero
+    // padded), N = 256 pixels, accumulator lanes = filters.  It also halves the filter bytes an item streams
+    // per pixel compared with 128 pixels x 256 filters.
+    p.swap = (kp16 > 64 && env_int("CONV2D_B200_TF32_SWAP", 1) != 0) ? 1 : 0;   // <= 64 filters: padding to 128 would double the work
+    if (p.swap) { p.n_blocks = (kp16 + 127) / 128; p.n_tile = 128; }
     p.cblks = (sh.C + kCB - 1) / kCB;
     p.taps = sh.R * sh.S;
     const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
@@ -218,7 +220,12 @@ Plan make_plan(const Shape& sh)
 
     p.nbuf = (2 * p.mt * p.n_tile <= 512) ? 2 : 1;
     p.supertiles = (int)((tiles + p.mt - 1) / p.mt);
-    const long long items = (long long)p.supertiles * p.n_blocks;
+    // Too few tiles for the machine (e.g. 14 x 14 images): two work items per tile, each contracting half of
+    // the channel-block groups and adding into a zeroed output.
+    const int n_groups = (p.cblks + p.cbg - 1) / p.cbg;
+    p.ksplit = ((long long)p.supertiles * p.n_blocks * 2 <= sms && n_groups >= 2 &&
+                env_int("CONV2D_B200_TF32_KSPLIT", 1) != 0) ? 2 : 1;
+    const long long items = (long long)p.supertiles * p.n_blocks * p.ksplit;
     if (items > 0x7fffffffLL) return p;
     p.grid = (int)(items < sms ? items : sms);
     int cols = p.nbuf * p.mt * p.n_tile;
@@ -269,6 +276,9 @@ struct KernelArgs {
     int resident;           // filters loaded once per thread block instead of streamed
     int swap;               // operand roles swapped: accumulator lanes = filters, columns = pixels
     int vec;                // swap mode: adjacent pixels a lane stores as one unit (1, 2 or 4)
+    int ksplit;             // items per output tile (split of the contraction): 1 or 2
+    unsigned max_polls;     // bound of every barrier wait
+    int test_drop_stage;    // test hook: the filter copy with this ordinal is armed but never issued (-1: none)
     int items;              // work items = supertiles x n_blocks
     unsigned tmem_cols;
 };
@@ -317,6 +327,25 @@ __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* 
                                              to_tf32_rna(v[u][4 * ch + 2]), to_tf32_rna(v[u][4 * ch + 3]));
         }
     }
+}
+
+// Work item -> (supertile, filter block, part of the contraction).  With ksplit = 2 two items share an
+// output tile, each contracts half of the channel-block groups and both add their partial sums into y
+// (zeroed beforehand); 0 + a + b does not depend on the order, so the result stays deterministic.
+struct ItemInfo {
+    int supertile, nb, g_begin, n_groups, rot;
+};
+__device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
+{
+    ItemInfo it;
+    const int part = item % a.ksplit;
+    const int rest = item / a.ksplit;
+    it.nb = rest % a.n_blocks;
+    it.supertile = rest / a.n_blocks;
+    it.g_begin = part * a.groups / a.ksplit;
+    it.n_groups = (part + 1) * a.groups / a.ksplit - it.g_begin;
+    it.rot = rest % it.n_groups;        // blocks stream the filter bank in rotated order (see kernel)
+    return it;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -379,23 +408,25 @@ general_tf32_kernel(const KernelArgs a)
                 if (*abort_flag) { uint32_t dummy = 0; mbar_wait_bounded(&b_full[0], 0u, &dummy, 1u << 16); }
             }
             for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
-                const int nb = item % a.n_blocks;
-                const int grp_first = item % a.groups;
+                const ItemInfo ii = decode_item(a, item);
+                const int nb = ii.nb;
                 const unsigned char* src = reinterpret_cast<const unsigned char*>(a.wp)
                                          + (size_t)nb * a.cblks * a.taps * b_chunk_bytes;
-                for (int grp = 0; grp < a.groups && alive; ++grp) {
-                    int gr = grp + grp_first;
-                    if (gr >= a.groups) gr -= a.groups;
+                for (int grp = 0; grp < ii.n_groups && alive; ++grp) {
+                    int gr = grp + ii.rot;
+                    if (gr >= ii.n_groups) gr -= ii.n_groups;
+                    gr += ii.g_begin;
                     for (int g = 0; g < a.cbg && alive; ++g) {
                         const int cbr = gr * a.cbg + g;
                         if (cbr >= a.cblks) break;
                         for (int t0 = 0; t0 < a.taps; t0 += a.tps) {
                             const int nt = min(a.tps, a.taps - t0);
-                            if (!mbar_wait_bounded(&b_empty[s], ph ^ 1u, abort_flag)) { alive = false; break; }
+                            if (!mbar_wait_bounded(&b_empty[s], ph ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                             const uint32_t bytes = b_chunk_bytes * (uint32_t)nt;
                             mbar_arrive_expect_tx(&b_full[s], bytes);
-                            bulk_g2s(b_smem + (size_t)s * b_stage_bytes, src + ((size_t)cbr * a.taps + t0) * b_chunk_bytes,
-                                     bytes, &b_full[s]);
+                            if (issued != a.test_drop_stage)     // (test hook: a dropped copy makes the consumer's wait expire)
+                                bulk_g2s(b_smem + (size_t)s * b_stage_bytes, src + ((size_t)cbr * a.taps + t0) * b_chunk_bytes,
+                                         bytes, &b_full[s]);
                             ++issued;
                             if (++s == a.b_stages) { s = 0; ph ^= 1u; }
                         }
@@ -433,26 +464,27 @@ general_tf32_kernel(const KernelArgs a)
             const long long t_begin = clock_now();
             int n_items = 0;
             if (a.resident) {
-                if (!mbar_wait_bounded(&b_full[0], 0u, abort_flag)) alive = false;
+                if (!mbar_wait_bounded(&b_full[0], 0u, abort_flag, a.max_polls)) alive = false;
                 tc_fence_after_sync();
             }
             for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
-                const int grp_first = item % a.groups;
+                const ItemInfo ii = decode_item(a, item);
                 // the accumulator set must have been drained by the epilogue of its previous item
                 const uint32_t acc_phase = buf ? acc_phase1 : acc_phase0;
                 long long tw = clock_now();
-                if (!mbar_wait_bounded(&acc_empty[buf], acc_phase ^ 1u, abort_flag)) { alive = false; break; }
+                if (!mbar_wait_bounded(&acc_empty[buf], acc_phase ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                 tc_fence_after_sync();
                 wait_acc += clock_now() - tw;
                 const uint32_t d0 = tmem + (uint32_t)(buf * acc_cols);
                 uint32_t accumulate = 0;
-                for (int grp = 0; grp < a.groups && alive; ++grp) {
+                for (int grp = 0; grp < ii.n_groups && alive; ++grp) {
                     tw = clock_now();
-                    if (!mbar_wait_bounded(&a_full[as], a_phase, abort_flag)) { alive = false; break; }
+                    if (!mbar_wait_bounded(&a_full[as], a_phase, abort_flag, a.max_polls)) { alive = false; break; }
                     tc_fence_after_sync();
                     wait_a += clock_now() - tw;
-                    int gr = grp + grp_first;
-                    if (gr >= a.groups) gr -= a.groups;
+                    int gr = grp + ii.rot;
+                    if (gr >= ii.n_groups) gr -= ii.n_groups;
+                    gr += ii.g_begin;
                     uint32_t a_lo_block = a_lo_fixed | (smem_u32(a_smem + (size_t)as * a_stage_bytes) >> 4);
                     for (int g = 0; g < a.cbg && alive; ++g, a_lo_block += a_block_bytes >> 4) {
                         if (gr * a.cbg + g >= a.cblks) break;
@@ -464,7 +496,7 @@ general_tf32_kernel(const KernelArgs a)
                             if (a.resident) {
                                 b_lo = b_lo_fixed | (smem_u32(b_smem + (size_t)(gr * a.cbg + g) * a.taps * b_chunk_bytes) >> 4);
                             } else {
-                                if (!mbar_wait_bounded(&b_full[bs], b_phase, abort_flag)) { alive = false; break; }
+                                if (!mbar_wait_bounded(&b_full[bs], b_phase, abort_flag, a.max_polls)) { alive = false; break; }
                                 tc_fence_after_sync();
                                 b_lo = b_lo_fixed | (smem_u32(b_smem + (size_t)bs * b_stage_bytes) >> 4);
                             }
@@ -517,15 +549,16 @@ general_tf32_kernel(const KernelArgs a)
         uint32_t a_phase = 0;
         const int units = a.npix * a.cbg;
         for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
-            const int j0 = (item / a.n_blocks) * a.mt * kTileM;          // first flat pixel of the item
-            const int grp_first = item % a.groups;
+            const ItemInfo ii = decode_item(a, item);
+            const int j0 = ii.supertile * a.mt * kTileM;                 // first flat pixel of the item
             // One stage = cbg consecutive channel blocks.  All loads of a pass (kUnitsPerThread units of
             // 16 channels per thread) are issued before its first store: a pass costs one memory round trip.
-            for (int grp = 0; grp < a.groups && alive; ++grp) {
-                if (!mbar_wait_bounded(&a_empty[as], a_phase ^ 1u, abort_flag)) { alive = false; break; }
+            for (int grp = 0; grp < ii.n_groups && alive; ++grp) {
+                if (!mbar_wait_bounded(&a_empty[as], a_phase ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                 float4* dst = reinterpret_cast<float4*>(a_smem + (size_t)as * a_stage_bytes);
-                int gr = grp + grp_first;
-                if (gr >= a.groups) gr -= a.groups;
+                int gr = grp + ii.rot;
+                if (gr >= ii.n_groups) gr -= ii.n_groups;
+                gr += ii.g_begin;
                 for (int first = 0; first < units; first += kProducers * kUnitsPerThread) {
                     float v[kUnitsPerThread][kCB];
                     load_units(v, a, j0, gr * a.cbg, first, wtid);
@@ -546,11 +579,13 @@ general_tf32_kernel(const KernelArgs a)
         uint32_t acc_phase0 = 0, acc_phase1 = 0;
         bool alive = true;
         for (int item = blockIdx.x; item < a.items; item += gridDim.x) {
-            const int j0 = (item / a.n_blocks) * a.mt * kTileM;
-            const int nb = item % a.n_blocks;
+            const ItemInfo ii = decode_item(a, item);
+            const int j0 = ii.supertile * a.mt * kTileM;
+            const int nb = ii.nb;
+            const bool add = a.ksplit > 1;                   // partial sums: add into the zeroed output
             // tcgen05.ld is warp-collective: take the decision for the whole warp
             const uint32_t acc_phase = buf ? acc_phase1 : acc_phase0;
-            alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag));
+            alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag, a.max_polls));
             if (!alive) break;
             tc_fence_after_sync();
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * acc_cols);
@@ -589,23 +624,31 @@ general_tf32_kernel(const KernelArgs a)
                         const int n = j / a.HW, off = j - n * a.HW;
                         const int p = off / a.W, q = off - p * a.W;
                         ok = (p < a.P) && (q < a.Q);
-                        o = a.y + (((size_t)n * a.K + quarter * 32 + row_sub) * a.P + p) * a.Q + q;
+                        o = a.y + (((size_t)n * a.K + nb * 128 + quarter * 32 + row_sub) * a.P + p) * a.Q + q;
                     }
                     if (ok) {
-                        const int kmax = a.K - quarter * 32;        // maps of this quarter that exist
+                        const int kmax = a.K - nb * 128 - quarter * 32;   // maps of this quarter that exist
                         const float* src = tile + row_sub * kXposePitch + pg * vec;
                         if (vec == 4) {
 #pragma unroll
                             for (int r = 0; r < 32; r += 4, o += 4 * plane, src += 4 * kXposePitch)
-                                if (r + row_sub < kmax) *reinterpret_cast<float4*>(o) = *reinterpret_cast<const float4*>(src);
+                                if (r + row_sub < kmax) {
+                                    const float4 t = *reinterpret_cast<const float4*>(src);
+                                    if (add) { atomicAdd(o, t.x); atomicAdd(o + 1, t.y); atomicAdd(o + 2, t.z); atomicAdd(o + 3, t.w); }
+                                    else *reinterpret_cast<float4*>(o) = t;
+                                }
                         } else if (vec == 2) {
 #pragma unroll 8
                             for (int r = 0; r < 32; r += 2, o += 2 * plane, src += 2 * kXposePitch)
-                                if (r + row_sub < kmax) *reinterpret_cast<float2*>(o) = *reinterpret_cast<const float2*>(src);
+                                if (r + row_sub < kmax) {
+                                    const float2 t = *reinterpret_cast<const float2*>(src);
+                                    if (add) { atomicAdd(o, t.x); atomicAdd(o + 1, t.y); }
+                                    else *reinterpret_cast<float2*>(o) = t;
+                                }
                         } else {
 #pragma unroll 8
                             for (int r = 0; r < 32; ++r, o += plane, src += kXposePitch)
-                                if (r < kmax) *o = *src;
+                                if (r < kmax) { if (add) atomicAdd(o, *src); else *o = *src; }
                         }
                     }
                 };
@@ -657,7 +700,7 @@ general_tf32_kernel(const KernelArgs a)
                     float* o = yb + (size_t)k0 * plane;
 #pragma unroll
                     for (int i = 0; i < 16; ++i, o += plane)
-                        if (k0 + i < a.K) *o = __uint_as_float(v[i]);
+                        if (k0 + i < a.K) { if (add) atomicAdd(o, __uint_as_float(v[i])); else *o = __uint_as_float(v[i]); }
                 }
             };
             // Two register buffers: the load of the next chunk is in flight while the current one is stored.
@@ -739,8 +782,16 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
     for (int v = 4; v >= 2; v >>= 1)
         if (sh.W % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
-    a.items = p.supertiles * p.n_blocks;
+    a.items = p.supertiles * p.n_blocks * p.ksplit;
+    a.ksplit = p.ksplit;
+    // Failure-detection test hooks (host-side injection only): a short wait bound and one filter copy that is
+    // never issued, so that a bounded wait expires and the time-out path can be checked without hanging anything.
+    a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
+    a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
     a.tmem_cols = (unsigned)p.tmem_cols;
+    if (p.ksplit > 1 &&
+        cudaMemsetAsync(y, 0, (size_t)sh.N * sh.K * sh.P * sh.Q * sizeof(float), stream) != cudaSuccess)
+        return CONV2D_ERR_CUDA;
     general_tf32_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
