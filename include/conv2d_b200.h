@@ -81,12 +81,15 @@ conv2d_status_t conv2d_fwd_workspace_size(int N, int C, int H, int W, int K, int
 /*
  * Special case, one input channel (Section 3, Algorithm 1).
  *   x [N][1][H][W], w [K][1][R][S], y [N][K][P][Q]; fp32 FMA arithmetic.
- * The filters are first copied (device to device, on the stream) into a
- * constant-memory bank of 16384 floats that the whole device shares
- * (Section 3.2: the filters of this case are small and live in constant
- * memory); K*R*S must not exceed 16384 (CONV2D_ERR_UNSUPPORTED otherwise).
- * Because that bank is one per device, single-channel calls issued on
- * DIFFERENT streams must not overlap in time; calls on one stream are ordered.
+ * The filters are small in this case (Section 3.2) and are kept on chip for the
+ * whole call: every thread block copies them into shared memory and reads them
+ * with broadcast loads.  Tuned instances exist for R = S in {1, 3, 5, 7}; images
+ * with W % 4 == 0 and at least 1024 output columns take the wide kernel that
+ * stages input rows with bulk (TMA) copies; every other shape is computed by a
+ * slower shape-agnostic kernel, never rejected.  N must not exceed 65535.
+ * (A benchmark-only variant selected by an environment switch keeps the filters
+ * in a per-device constant-memory bank instead; calls using it on different
+ * streams must not overlap.)
  * workspace may be NULL (none is used); flags must be 0.
  */
 conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float* y,

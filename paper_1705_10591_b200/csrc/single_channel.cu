@@ -177,6 +177,92 @@ single_channel_kernel(const float* __restrict__ x, const float* __restrict__ w, 
     }
 }
 
+// Per-thread unit ablation (the matched / unmatched experiment of Section 5.1): the same row-walking
+// scheme with a per-thread unit of UNIT adjacent outputs (1 = float, 2 = float2, 4 = float4) read, computed
+// and written as one piece.  On Kepler the unit had to match the 8-byte bank; on B200 banks are 4 bytes
+// wide, so any difference comes from instruction count and store width.  Benchmark use only
+// (CONV2D_B200_SC_UNIT); scalar FMA, one output row per step, taps in shared memory.
+template <int R, int S, int UNIT>
+__global__ void __launch_bounds__(kThreads)
+single_channel_unit_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
+                           int H, int W, int K, int P, int Q, int tile_h, int vec_st)
+{
+    constexpr int TW = kThreads * UNIT;                 // output columns per block
+    constexpr int PITCH = TW + 8;                       // staged floats per row
+    constexpr int WC = S + UNIT - 1;                    // window columns
+    constexpr int RS = R * S;
+    extern __shared__ float4 smem4[];
+    float* tile = reinterpret_cast<float*>(smem4);
+    const int tid = threadIdx.x;
+    const int col0 = blockIdx.x * TW, row0 = blockIdx.y * tile_h, n = blockIdx.z;
+    const int th = min(tile_h, P - row0);
+    const int rows_in = th + R - 1;
+    const float* xin = x + (size_t)n * H * W;
+    for (int idx = tid; idx < rows_in * PITCH; idx += kThreads) {
+        const int row = idx / PITCH, c = idx - row * PITCH;
+        const int col = col0 + c;
+        tile[idx] = (col < W) ? __ldg(xin + (size_t)(row0 + row) * W + col) : 0.f;
+    }
+    float* wsm = tile + (size_t)(tile_h + R - 1) * PITCH;
+    for (int idx = tid; idx < K * RS; idx += kThreads) wsm[idx] = __ldg(w + idx);
+    __syncthreads();
+    const int q0 = col0 + UNIT * tid;
+    if (q0 >= Q) return;
+    float win[R][WC];
+#pragma unroll
+    for (int r = 0; r < R - 1; ++r)
+#pragma unroll
+        for (int c = 0; c < WC; ++c) win[r][c] = tile[r * PITCH + UNIT * tid + c];
+    const size_t plane = (size_t)P * Q;
+    for (int p = 0; p < th; ++p) {
+#pragma unroll
+        for (int c = 0; c < WC; ++c) win[R - 1][c] = tile[(p + R - 1) * PITCH + UNIT * tid + c];
+        float* yout = y + ((size_t)n * K * P + (size_t)(row0 + p)) * Q + q0;
+#pragma unroll 1
+        for (int f = 0; f < K; ++f, yout += plane) {
+            float acc[UNIT];
+#pragma unroll
+            for (int j = 0; j < UNIT; ++j) acc[j] = 0.f;
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int s2 = 0; s2 < S; ++s2) {
+                    const float wv = wsm[f * RS + r * S + s2];
+#pragma unroll
+                    for (int j = 0; j < UNIT; ++j) acc[j] = fmaf(win[r][s2 + j], wv, acc[j]);
+                }
+            if (vec_st && q0 + UNIT <= Q) {
+                if (UNIT == 4) store4(yout, make_float4(acc[0], acc[1 % UNIT], acc[2 % UNIT], acc[3 % UNIT]));
+                else if (UNIT == 2) __stcs(reinterpret_cast<float2*>(yout), make_float2(acc[0], acc[1 % UNIT]));
+                else __stcs(yout, acc[0]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < UNIT; ++j)
+                    if (q0 + j < Q) __stcs(yout + j, acc[j]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R - 1; ++r)
+#pragma unroll
+            for (int c = 0; c < WC; ++c) win[r][c] = win[r + 1][c];
+    }
+}
+
+template <int R, int S, int UNIT>
+conv2d_status_t launch_unit(const float* x, const float* w, float* y, const Shape& sh, int tile_h, cudaStream_t stream)
+{
+    constexpr int TW = kThreads * UNIT;
+    const size_t smem = ((size_t)(tile_h + R - 1) * (TW + 8) + (size_t)sh.K * R * S) * sizeof(float);
+    if (smem > 200 * 1024) return CONV2D_ERR_UNSUPPORTED;
+    auto kern = single_channel_unit_kernel<R, S, UNIT>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return CONV2D_ERR_CUDA;
+    dim3 grid((sh.Q + TW - 1) / TW, (sh.P + tile_h - 1) / tile_h, sh.N);
+    const int vec_st = (sh.Q % UNIT == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
+    kern<<<grid, kThreads, smem, stream>>>(x, w, y, sh.H, sh.W, sh.K, sh.P, sh.Q, tile_h, vec_st);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
 // Packed-FMA variant.  B200 issues fp32 FMAs at full rate only as two-wide packed instructions
 // (fma.rn.f32x2): a scalar-FMA loop tops out near 82 % of the fp32 peak, a packed one near 99 %,
 // and the packed form leaves issue slots for the loads, stores and address arithmetic.  The two
@@ -557,12 +643,26 @@ template <int R, int S>
 conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
 {
     // Tuning knobs (benchmark ablations only): tile height, rows per step, packed/scalar FMA, tap source.
-    int tile_h = env_int("CONV2D_B200_SC_TILE_H", 8);
+    int tile_h = env_int("CONV2D_B200_SC_TILE_H", 0);
+    if (tile_h <= 0) {
+        // 8 rows per block unless that leaves the machine short of blocks (small images): then fewer rows,
+        // down to 2, aiming at four blocks per SM
+        tile_h = 8;
+        const long long col_tiles = (sh.Q + kTileW - 1) / kTileW;
+        while (tile_h > 2 && col_tiles * ((sh.P + tile_h - 1) / tile_h) * sh.N < 4 * 148) tile_h >>= 1;
+    }
     if (tile_h < 1) tile_h = 1;
     if (tile_h > 64) tile_h = 64;
     if (tile_h > sh.P) tile_h = sh.P;
     const int tr = env_int("CONV2D_B200_SC_ROWS", R >= 7 ? 1 : 2);
     constexpr int RS2 = (R * S + 1) / 2;
+    const int unit = env_int("CONV2D_B200_SC_UNIT", 0);      // per-thread unit ablation (benchmark only)
+    if (unit == 1 || unit == 2 || unit == 4) {
+        const conv2d_status_t st = unit == 1 ? launch_unit<R, S, 1>(x, w, y, sh, tile_h, stream)
+                                 : unit == 2 ? launch_unit<R, S, 2>(x, w, y, sh, tile_h, stream)
+                                             : launch_unit<R, S, 4>(x, w, y, sh, tile_h, stream);
+        if (st != CONV2D_ERR_UNSUPPORTED) return st;
+    }
     // Large images: the wide persistent kernel (needs 16-byte aligned input rows for the bulk copies).
     const bool rows_ok = sh.W % 4 == 0 && sh.Q >= 1024 && reinterpret_cast<uintptr_t>(x) % 16 == 0;
     if (rows_ok && env_int("CONV2D_B200_SC_WIDE", 1) != 0) {
@@ -582,7 +682,7 @@ conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shap
     int wsrc = env_int("CONV2D_B200_SC_WSRC", 1);
     if ((size_t)sh.K * RSP * sizeof(float) > 64 * 1024) wsrc = 0;       // too many taps for the shared copy
     if (wsrc == 0) {
-        if ((size_t)sh.K * R * S > (size_t)kConstFilterFloats) return CONV2D_ERR_UNSUPPORTED;
+        if ((size_t)sh.K * R * S > (size_t)kConstFilterFloats) return launch_direct_fallback(x, w, y, sh, stream);
         if (cudaMemcpyToSymbolAsync(c_filters, w, (size_t)sh.K * R * S * sizeof(float), 0,
                                     cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
             return CONV2D_ERR_CUDA;

@@ -53,13 +53,16 @@ def test_single_channel_within_tolerance(oracle, dims):
 
 @pytest.mark.parametrize("knobs", [
     dict(CONV2D_B200_SC_ROWS="1"), dict(CONV2D_B200_SC_TILE_H="5"),                       # packed-FMA kernel
+    dict(CONV2D_B200_SC_UNIT="1"), dict(CONV2D_B200_SC_UNIT="2"), dict(CONV2D_B200_SC_UNIT="4"),   # unit ablation
+    dict(CONV2D_B200_SC_WIDE="0"),                                                        # tile kernel on wide images
     dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_WSRC="0"),                              # scalar-FMA kernel
     dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_WSRC="1", CONV2D_B200_SC_ROWS="1"),
     dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_TILE_H="5", CONV2D_B200_SC_WSRC="0", CONV2D_B200_SC_ROWS="1")])
 def test_single_channel_variants_agree(oracle, monkeypatch, knobs):
     for k, v in knobs.items():
         monkeypatch.setenv(k, v)
-    for dims in [(1, 64, 64, 8, 3, 3), (2, 37, 53, 5, 5, 5), (1, 19, 1031, 2, 3, 3), (1, 30, 40, 3, 7, 7)]:
+    for dims in [(1, 64, 64, 8, 3, 3), (2, 37, 53, 5, 5, 5), (1, 19, 1031, 2, 3, 3), (1, 30, 40, 3, 7, 7),
+                 (1, 12, 1100, 3, 5, 5)]:
         N, H, W, K, R, S = dims
         x, w = small_integers((N, 1, H, W), 305), small_integers((K, 1, R, S), 306)
         y_ref, _ = oracle.conv2d_oracle(x, w)
