@@ -31,6 +31,9 @@ SINGLE_SHAPES = [
     (2, 11, 1032, 5, 3, 3),      # wide kernel, Q = 1030: 64-bit stores, odd filter count
     (1, 9, 1028, 2, 7, 7),       # wide kernel, 7 x 7, band taller than the image's output rows
     (1, 14, 1040, 4, 1, 1),      # wide kernel, 1 x 1
+    (1, 12, 1032, 3, 3, 3),      # shifted wide kernel: Q = 1030 (8-byte aligned rows), odd filter count
+    (2, 20, 2100, 5, 3, 3),      # shifted wide kernel: Q = 2098, two column tiles, three bands
+    (1, 14, 1040, 4, 7, 7),      # wide kernel, 7 x 7, Q = 1034: 64-bit stores
 ]
 
 
@@ -55,6 +58,7 @@ def test_single_channel_within_tolerance(oracle, dims):
     dict(CONV2D_B200_SC_ROWS="1"), dict(CONV2D_B200_SC_TILE_H="5"),                       # packed-FMA kernel
     dict(CONV2D_B200_SC_UNIT="1"), dict(CONV2D_B200_SC_UNIT="2"), dict(CONV2D_B200_SC_UNIT="4"),   # unit ablation
     dict(CONV2D_B200_SC_WIDE="0"),                                                        # tile kernel on wide images
+    dict(CONV2D_B200_SC_SHIFT="0"),                                                       # wide kernel with 64-bit stores
     dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_WSRC="0"),                              # scalar-FMA kernel
     dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_WSRC="1", CONV2D_B200_SC_ROWS="1"),
     dict(CONV2D_B200_SC_PACKED="0", CONV2D_B200_SC_TILE_H="5", CONV2D_B200_SC_WSRC="0", CONV2D_B200_SC_ROWS="1")])
@@ -62,7 +66,7 @@ def test_single_channel_variants_agree(oracle, monkeypatch, knobs):
     for k, v in knobs.items():
         monkeypatch.setenv(k, v)
     for dims in [(1, 64, 64, 8, 3, 3), (2, 37, 53, 5, 5, 5), (1, 19, 1031, 2, 3, 3), (1, 30, 40, 3, 7, 7),
-                 (1, 12, 1100, 3, 5, 5)]:
+                 (1, 12, 1100, 3, 5, 5), (1, 12, 1032, 3, 3, 3)]:
         N, H, W, K, R, S = dims
         x, w = small_integers((N, 1, H, W), 305), small_integers((K, 1, R, S), 306)
         y_ref, _ = oracle.conv2d_oracle(x, w)
