@@ -131,8 +131,15 @@ Plan make_plan(const Shape& sh)
     // filter count that is possible with the pixels as the N operand: M = a block of 128 filters (zero
     // padded), N = 256 pixels, accumulator lanes = filters.  It also halves the filter bytes an item streams
     // per pixel compared with 128 pixels x 256 filters.
-    p.swap = (kp16 > 64 && env_int("CONV2D_B200_TF32_SWAP", 1) != 0) ? 1 : 0;   // <= 64 filters: padding to 128 would double the work
-    if (p.swap) { p.n_blocks = (kp16 + 127) / 128; p.n_tile = 128; }
+    // Up to 64 filters use M = 64 (one tcgen05.mma then covers 64 filters x 256 pixels; its accumulator
+    // occupies lanes 0-15 of each 32-lane quarter -- established with a probe).
+    p.swap = env_int("CONV2D_B200_TF32_SWAP", 1) != 0 ? 1 : 0;
+    if (p.swap && kp16 <= 64 && env_int("CONV2D_B200_TF32_M64", 1) == 0) p.swap = 0;
+    if (p.swap) {
+        p.n_tile = kp16 <= 64 ? 64 : 128;                  // filters per block = rows of the M operand
+        p.n_blocks = (kp16 + p.n_tile - 1) / p.n_tile;
+    }
+    const int set_cols = p.swap ? kTileM : p.n_tile;      // tensor-memory columns of one 128-pixel tile
     p.cblks = (sh.C + kCB - 1) / kCB;
     p.taps = sh.R * sh.S;
     const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
@@ -149,13 +156,15 @@ Plan make_plan(const Shape& sh)
     // shared memory: nothing is streamed, items are small (finest balance over the SMs, two accumulator
     // sets), and the rest of shared memory becomes a deep activation ring whose stages carry several
     // channel blocks (these items are bound by memory latency: one producer pass should have 32-48 loads
-    // per thread in flight).  Measured: for 3x3 with 64 filters streaming with two tiles per item is faster.
+    // per thread in flight).  Any other bank that fits next to a two-stage activation ring is kept resident too
+    // (64 filters of 64 x 3 x 3: 39 us resident vs 43 us streamed).
     p.resident = 0;
-    if (env_int("CONV2D_B200_TF32_RESIDENT", 1) != 0 && p.n_blocks == 1 && wbytes <= 152 * 1024 &&
-        (long long)p.taps * p.cblks <= 16) {
+    const int resident_mode = env_int("CONV2D_B200_TF32_RESIDENT", 2);      // 0 never, 1 light problems only, 2 whenever it fits
+    if (resident_mode != 0 && p.n_blocks == 1 && wbytes <= 152 * 1024 &&
+        ((long long)p.taps * p.cblks <= 16 || resident_mode == 2)) {
         const int mt = forced_mt ? forced_mt : (p.swap ? 2 : 1);
         const int npix = npix_of(mt);
-        if (mt * p.n_tile <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * npix * 4 + 512 <= kSmemLimit) {
+        if (mt * set_cols <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * npix * 4 + 512 <= kSmemLimit) {
             p.resident = 1;
             p.mt = mt;
             p.npix = npix;
@@ -185,13 +194,13 @@ Plan make_plan(const Shape& sh)
         for (int mt = 4; mt >= 1; mt >>= 1) {
             if (forced_mt && mt != forced_mt) continue;
             if (p.swap && mt < 2) continue;
-            if (mt * p.n_tile > 512) continue;
+            if (mt * set_cols > 512) continue;
             const int npix = npix_of(mt);
             if (npix > 16000) continue;
             if (smem_need(2, npix, p.n_tile, 2, 1, 1) > kLimit) continue;
             const long long items = (tiles + mt - 1) / mt * p.n_blocks;
             const long long rounds = (items + sms - 1) / sms;
-            const int nbuf = (2 * mt * p.n_tile <= 512) ? 2 : 1;
+            const int nbuf = (2 * mt * set_cols <= 512) ? 2 : 1;
             const double stream = 1.0 + (chunk / 66.0) / (mt * 2 * mma_cycles);
             const double writeback = (nbuf == 1 ? 1.0 : 0.15) * mt * (3000.0 * p.n_tile / 128.0) / tile_cycles;
             const double cost = rounds * (mt * stream + 0.5 * writeback);
@@ -218,7 +227,7 @@ Plan make_plan(const Shape& sh)
         p.smem_bytes = smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg) + extra;
     }
 
-    p.nbuf = (2 * p.mt * p.n_tile <= 512) ? 2 : 1;
+    p.nbuf = (2 * p.mt * set_cols <= 512) ? 2 : 1;
     p.supertiles = (int)((tiles + p.mt - 1) / p.mt);
     // Too few tiles for the machine (e.g. 14 x 14 images): two work items per tile, each contracting half of
     // the channel-block groups and adding into a zeroed output.
@@ -228,7 +237,7 @@ Plan make_plan(const Shape& sh)
     const long long items = (long long)p.supertiles * p.n_blocks * p.ksplit;
     if (items > 0x7fffffffLL) return p;
     p.grid = (int)(items < sms ? items : sms);
-    int cols = p.nbuf * p.mt * p.n_tile;
+    int cols = p.nbuf * p.mt * set_cols;
     p.tmem_cols = 32;
     while (p.tmem_cols < cols) p.tmem_cols <<= 1;
     p.ok = true;
@@ -388,7 +397,7 @@ general_tf32_kernel(const KernelArgs a)
 
     // Work item -> (supertile, filter block); blocks rotate the order of the channel-block groups by the
     // item number, so that at any moment they stream different parts of the filter bank.
-    const int acc_cols = a.mt * a.n_tile;                   // tensor-memory columns of one accumulator set
+    const int acc_cols = a.mt * (a.swap ? kTileM : a.n_tile);   // tensor-memory columns of one accumulator set
 
     if (warp == 0) {
         // ---------------- filters: global -> shared by bulk copy, up to `tps` taps of one channel block per stage
@@ -449,7 +458,7 @@ general_tf32_kernel(const KernelArgs a)
             // Per MMA this thread only adds small constants to the low word of a descriptor: everything
             // that does not change is folded into a_lo_fixed / b_lo_fixed / desc_hi beforehand, because a
             // single thread issuing ~40 dependent integer instructions per MMA was slower than the MMA.
-            const uint32_t idesc = a.swap ? idesc_tf32(128u, 256u) : idesc_tf32(kTileM, (uint32_t)a.n_tile);
+            const uint32_t idesc = a.swap ? idesc_tf32((uint32_t)a.n_tile, 256u) : idesc_tf32(kTileM, (uint32_t)a.n_tile);
             const uint32_t desc_hi = (128u >> 4) | (1u << 14);                  // SBO = 128 B, descriptor version 1
             const uint32_t a_lo_fixed = ((uint32_t)a.npix & 0x3FFFu) << 16;     // LBO = npix * 16 B
             const uint32_t b_lo_fixed = ((uint32_t)a.n_tile & 0x3FFFu) << 16;   // LBO = n_tile * 16 B
@@ -595,6 +604,7 @@ general_tf32_kernel(const KernelArgs a)
                 // warp-private shared-memory tile turns a 32-filter x 32-pixel block around so that each
                 // store instruction again writes 32 adjacent pixels of one map.
                 float* tile = xpose + (size_t)(warp - 4) * 32 * kXposePitch;
+                const int rpq = a.n_tile / 4;      // filter rows per lane quarter: 32 (M = 128) or 16 (M = 64, lanes 0-15)
                 const int blocks = a.mt * kTileM / 32;
                 auto load_block = [&](uint32_t (&v0)[16], uint32_t (&v1)[16], int b) {
                     tmem_ld16(lane_base + (uint32_t)(b * 32), v0);
@@ -624,10 +634,10 @@ general_tf32_kernel(const KernelArgs a)
                         const int n = j / a.HW, off = j - n * a.HW;
                         const int p = off / a.W, q = off - p * a.W;
                         ok = (p < a.P) && (q < a.Q);
-                        o = a.y + (((size_t)n * a.K + nb * 128 + quarter * 32 + row_sub) * a.P + p) * a.Q + q;
+                        o = a.y + (((size_t)n * a.K + nb * a.n_tile + quarter * rpq + row_sub) * a.P + p) * a.Q + q;
                     }
                     if (ok) {
-                        const int kmax = a.K - nb * 128 - quarter * 32;   // maps of this quarter that exist
+                        const int kmax = min(rpq, a.K - nb * a.n_tile - quarter * rpq);   // maps of this quarter that exist
                         const float* src = tile + row_sub * kXposePitch + pg * vec;
                         if (vec == 4) {
 #pragma unroll
