@@ -10,7 +10,8 @@
 //     keeps one input row segment of kThrQ+S-1 pixels in registers and reuses it for the S
 //     horizontal taps (Section 4.2); filter values are read as 128-bit units, image pixels are
 //     broadcast to the threads that differ only in their filter group.
-// Changed for B200: register tile 8 x 8 with 128-bit shared-memory reads on both operands;
+// Changed for B200: register tile 8 x 8 with 128-bit shared-memory reads on both operands and packed
+// two-filter FMAs;
 // the output is written with 128-bit stores per filter row segment where alignment allows.
 #include "common.cuh"
 
@@ -33,7 +34,7 @@ struct Smem {
 };
 
 template <int R, int S, int CB>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
                     int C, int H, int W, int K, int P, int Q, int tiles_q, int vec_st)
 {
@@ -53,11 +54,13 @@ general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
     const int n = blockIdx.z;
     const float* xin = x + (size_t)n * C * H * W;
 
-    float acc[kThrK][kThrQ];
+    // Accumulators as (filter 2i, filter 2i+1) pairs: B200 reaches its fp32 FMA peak only with the two-wide
+    // packed instruction (fma.rn.f32x2); the pixel is duplicated, the two filter taps are adjacent in shFlt.
+    float2 acc[kThrK / 2][kThrQ];
 #pragma unroll
-    for (int i = 0; i < kThrK; ++i)
+    for (int i = 0; i < kThrK / 2; ++i)
 #pragma unroll
-        for (int j = 0; j < kThrQ; ++j) acc[i][j] = 0.f;
+        for (int j = 0; j < kThrQ; ++j) acc[i][j] = make_float2(0.f, 0.f);
 
     constexpr int NV = (kThrQ + S - 1 + 3) / 4;       // 128-bit reads per input row segment
 
@@ -88,26 +91,27 @@ general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
         for (int cc = 0; cc < CB; ++cc) {
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                float img[4 * NV];
+                float2 img[4 * NV];                              // (x, x)
                 const float4* src = reinterpret_cast<const float4*>(&sm.img[cc][seg_row + r][seg_col]);
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     const float4 t = src[v];
-                    img[4 * v + 0] = t.x; img[4 * v + 1] = t.y; img[4 * v + 2] = t.z; img[4 * v + 3] = t.w;
+                    img[4 * v + 0] = make_float2(t.x, t.x); img[4 * v + 1] = make_float2(t.y, t.y);
+                    img[4 * v + 2] = make_float2(t.z, t.z); img[4 * v + 3] = make_float2(t.w, t.w);
                 }
 #pragma unroll
                 for (int s = 0; s < S; ++s) {
-                    float flt[kThrK];
+                    float2 flt[kThrK / 2];                       // taps of filters (2i, 2i+1)
                     const float4* fs = reinterpret_cast<const float4*>(&sm.flt[cc][r * S + s][tx * kThrK]);
 #pragma unroll
                     for (int v = 0; v < kThrK / 4; ++v) {
                         const float4 t = fs[v];
-                        flt[4 * v + 0] = t.x; flt[4 * v + 1] = t.y; flt[4 * v + 2] = t.z; flt[4 * v + 3] = t.w;
+                        flt[2 * v + 0] = make_float2(t.x, t.y); flt[2 * v + 1] = make_float2(t.z, t.w);
                     }
 #pragma unroll
-                    for (int i = 0; i < kThrK; ++i)
+                    for (int i = 0; i < kThrK / 2; ++i)
 #pragma unroll
-                        for (int j = 0; j < kThrQ; ++j) acc[i][j] = fmaf(flt[i], img[s + j], acc[i][j]);
+                        for (int j = 0; j < kThrQ; ++j) acc[i][j] = __ffma2_rn(img[s + j], flt[i], acc[i][j]);
                 }
             }
         }
@@ -122,15 +126,17 @@ general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
         const int k = k0 + tx * kThrK + i;
         if (k >= K) break;
         float* o = y + (((size_t)n * K + k) * P + p) * Q + q;
+        float row[kThrQ];
+#pragma unroll
+        for (int j = 0; j < kThrQ; ++j) row[j] = (i & 1) ? acc[i / 2][j].y : acc[i / 2][j].x;
         if (vec_st && q + kThrQ <= Q) {
 #pragma unroll
             for (int v = 0; v < kThrQ / 4; ++v)
-                *reinterpret_cast<float4*>(o + 4 * v) =
-                    make_float4(acc[i][4 * v], acc[i][4 * v + 1], acc[i][4 * v + 2], acc[i][4 * v + 3]);
+                *reinterpret_cast<float4*>(o + 4 * v) = make_float4(row[4 * v], row[4 * v + 1], row[4 * v + 2], row[4 * v + 3]);
         } else {
 #pragma unroll
             for (int j = 0; j < kThrQ; ++j)
-                if (q + j < Q) o[j] = acc[i][j];
+                if (q + j < Q) o[j] = row[j];
         }
     }
 }
