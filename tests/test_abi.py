@@ -89,3 +89,25 @@ def test_product_package_does_not_touch_the_oracle():
     for path in (ROOT / "paper_1705_10591_b200").rglob("*"):
         if path.suffix in {".py", ".cu", ".cuh", ".h", ".cpp"}:
             assert "oracle" not in path.read_text().lower(), f"{path} mentions the oracle"
+
+
+def test_workspace_query_over_many_shapes_is_consistent(lib):
+    """The tensor-core planner runs on the host: sweep it over odd shapes (no device needed)."""
+    import itertools
+    seen = 0
+    for N, C, HW, K, R in itertools.product((1, 3, 32), (1, 3, 16, 17, 300), (7, 14, 57), (1, 8, 64, 65, 129, 257, 600), (1, 3, 7)):
+        if R > HW:
+            continue
+        try:
+            tf32 = lib.conv2d_fwd_workspace_size(N, C, HW, HW, K, R, R, lib.ALGO_TF32)
+        except lib.Conv2dError as e:
+            assert e.status == 5                      # no instance: must be reported, not guessed
+            assert lib.conv2d_fwd_workspace_size(N, C, HW, HW, K, R, R, lib.ALGO_AUTO) == 0
+            continue
+        seen += 1
+        # status block + re-ordered filters: at least one float per real filter tap, padded to whole blocks
+        assert tf32 >= 256 + 4 * K * C * R * R
+        assert tf32 % 16 == 0
+        assert lib.conv2d_fwd_workspace_size(N, C, HW, HW, K, R, R, lib.ALGO_AUTO) == tf32
+        assert lib.conv2d_fwd_workspace_size(N, C, HW, HW, K, R, R, lib.ALGO_FFMA) == 0
+    assert seen > 100
