@@ -58,6 +58,10 @@ conv2d_status_t conv2d_fwd_workspace_size(int N, int C, int H, int W, int K, int
         case CONV2D_ALGO_AUTO:
             if (tf32_supported(sh)) *bytes = tf32_workspace_bytes(sh);
             return CONV2D_OK;
+        case CONV2D_ALGO_BF16:
+            if (!bf16_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
+            *bytes = bf16_workspace_bytes(sh);
+            return CONV2D_OK;
         default: return CONV2D_ERR_UNSUPPORTED;
     }
 }
@@ -110,6 +114,25 @@ conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
     if (use_tf32)
         return launch_general_tf32(x, w, y, sh, workspace, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0, stream);
     return launch_general_ffma(x, w, y, sh, stream);
+}
+
+conv2d_status_t conv2d_fwd_general_bf16(const void* x_bf16, const void* w_bf16, float* y,
+                                        int N, int C, int H, int W, int K, int R, int S,
+                                        void* workspace, size_t workspace_bytes,
+                                        unsigned flags, void* cuda_stream)
+{
+    if (!x_bf16 || !w_bf16 || !y || !workspace) return CONV2D_ERR_NULL;
+    Shape sh;
+    conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
+    if (st != CONV2D_OK) return st;
+    if (!aligned16(x_bf16) || !aligned16(w_bf16) || !aligned16(y) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (flags & ~(unsigned)CONV2D_FLAG_WEIGHTS_PACKED) return CONV2D_ERR_UNSUPPORTED;
+    if (!bf16_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
+    if (workspace_bytes < bf16_workspace_bytes(sh)) return CONV2D_ERR_WORKSPACE;
+    st = check_device();
+    if (st != CONV2D_OK) return st;
+    return launch_general_bf16(x_bf16, w_bf16, y, sh, workspace, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0,
+                               static_cast<cudaStream_t>(cuda_stream));
 }
 
 conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float* y,

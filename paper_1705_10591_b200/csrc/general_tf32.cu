@@ -117,7 +117,9 @@ int env_int(const char* name, int dflt)
     return (v && *v) ? atoi(v) : dflt;
 }
 
-Plan make_plan(const Shape& sh)
+// bf16: the operands are bf16 (16-byte unit = 8 channels, 32 channels per staged block, K = 16 per MMA); the
+// byte layout of every stage is the same as for TF32 (16 channels of 4 bytes).
+Plan make_plan(const Shape& sh, bool bf16 = false)
 {
     Plan p{};
     p.ok = false;
@@ -140,7 +142,8 @@ Plan make_plan(const Shape& sh)
         p.n_blocks = (kp16 + p.n_tile - 1) / p.n_tile;
     }
     const int set_cols = p.swap ? kTileM : p.n_tile;      // tensor-memory columns of one 128-pixel tile
-    p.cblks = (sh.C + kCB - 1) / kCB;
+    const int cbc = bf16 ? 2 * kCB : kCB;                 // channels per staged block
+    p.cblks = (sh.C + cbc - 1) / cbc;
     p.taps = sh.R * sh.S;
     const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
     const long long halo = (long long)(sh.R - 1) * sh.W + (sh.S - 1);
@@ -272,6 +275,28 @@ __global__ void repack_filters_kernel(const float* __restrict__ w, float* __rest
     }
 }
 
+// bf16 variant: wp[nb][cb][t][chunk][f][e] = w[nb*n_tile + f][cb*32 + 8*chunk + e][t] (16-bit elements).
+__global__ void repack_filters_bf16_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ wp,
+                                           unsigned* __restrict__ status, int K, int C, int taps, int n_tile, int cblks,
+                                           long long total)
+{
+    if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        long long r = i;
+        const int e = (int)(r % 8); r /= 8;
+        const int f = (int)(r % n_tile); r /= n_tile;
+        const int chunk = (int)(r % kChunks); r /= kChunks;
+        const int t = (int)(r % taps); r /= taps;
+        const int cb = (int)(r % cblks); r /= cblks;
+        const int nb = (int)r;
+        const int k = nb * n_tile + f, c = cb * 2 * kCB + 8 * chunk + e;
+        unsigned short v = 0;
+        if (k < K && c < C) v = __ldg(w + ((size_t)k * C + c) * taps + t);
+        wp[i] = v;
+    }
+}
+
 struct KernelArgs {
     const float* x;
     const float* wp;
@@ -296,7 +321,7 @@ struct KernelArgs {
 // [channel block][chunk][pixel] in 16-byte units.  A work unit is (channel block g, pixel jj), numbered
 // i = g * npix + jj; thread t of the 256 producers owns units first + t, first + t + 256, ...  Consecutive
 // lanes read consecutive pixels of one channel (coalesced) and write consecutive 16-byte units.
-template <int CNT>
+template <bool BF16, int CNT>
 __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArgs& a, int j0, int cb0, int first, int wtid)
 {
     const int units = a.npix * a.cbg;
@@ -308,19 +333,35 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
         if (i < units) {
             const int g = i / a.npix, jj = i - g * a.npix;
             const int j = j0 + jj;
-            const int c0 = (cb0 + g) * kCB;
-            if (j < a.total_pix && c0 < a.C) {
-                const int n = j / a.HW, off = j - n * a.HW;
-                const float* src = a.x + ((size_t)n * a.C + c0) * a.HW + off;
+            if (BF16) {
+                // 32 bf16 channels of this pixel, packed two per 32-bit word (lower channel in the low half)
+                const int c0 = (cb0 + g) * 2 * kCB;
+                if (j < a.total_pix && c0 < a.C) {
+                    const int n = j / a.HW, off = j - n * a.HW;
+                    const unsigned short* src = reinterpret_cast<const unsigned short*>(a.x) + ((size_t)n * a.C + c0) * a.HW + off;
 #pragma unroll
-                for (int e = 0; e < kCB; ++e)
-                    if (c0 + e < a.C) v[u][e] = __ldg(src + (size_t)e * a.HW);
+                    for (int e = 0; e < kCB; ++e) {
+                        unsigned lo = 0, hi = 0;
+                        if (c0 + 2 * e < a.C) lo = __ldg(src + (size_t)(2 * e) * a.HW);
+                        if (c0 + 2 * e + 1 < a.C) hi = __ldg(src + (size_t)(2 * e + 1) * a.HW);
+                        v[u][e] = __uint_as_float(lo | (hi << 16));
+                    }
+                }
+            } else {
+                const int c0 = (cb0 + g) * kCB;
+                if (j < a.total_pix && c0 < a.C) {
+                    const int n = j / a.HW, off = j - n * a.HW;
+                    const float* src = a.x + ((size_t)n * a.C + c0) * a.HW + off;
+#pragma unroll
+                    for (int e = 0; e < kCB; ++e)
+                        if (c0 + e < a.C) v[u][e] = __ldg(src + (size_t)e * a.HW);
+                }
             }
         }
     }
 }
 
-template <int CNT>
+template <bool BF16, int CNT>
 __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* dst, const KernelArgs& a, int first, int wtid)
 {
     const int units = a.npix * a.cbg;
@@ -332,8 +373,9 @@ __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* 
             float4* d = dst + (size_t)g * kChunks * a.npix + jj;
 #pragma unroll
             for (int ch = 0; ch < kChunks; ++ch)
-                d[ch * a.npix] = make_float4(to_tf32_rna(v[u][4 * ch]), to_tf32_rna(v[u][4 * ch + 1]),
-                                             to_tf32_rna(v[u][4 * ch + 2]), to_tf32_rna(v[u][4 * ch + 3]));
+                d[ch * a.npix] = BF16 ? make_float4(v[u][4 * ch], v[u][4 * ch + 1], v[u][4 * ch + 2], v[u][4 * ch + 3])
+                                      : make_float4(to_tf32_rna(v[u][4 * ch]), to_tf32_rna(v[u][4 * ch + 1]),
+                                                    to_tf32_rna(v[u][4 * ch + 2]), to_tf32_rna(v[u][4 * ch + 3]));
         }
     }
 }
@@ -357,8 +399,9 @@ __device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
     return it;
 }
 
+template <bool BF16>
 __global__ void __launch_bounds__(kThreads, 1)
-general_tf32_kernel(const KernelArgs a)
+general_tc_kernel(const KernelArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     const uint32_t a_block_bytes = (uint32_t)kCB * a.npix * 4;          // one channel block of a stage
@@ -458,7 +501,12 @@ general_tf32_kernel(const KernelArgs a)
             // Per MMA this thread only adds small constants to the low word of a descriptor: everything
             // that does not change is folded into a_lo_fixed / b_lo_fixed / desc_hi beforehand, because a
             // single thread issuing ~40 dependent integer instructions per MMA was slower than the MMA.
-            const uint32_t idesc = a.swap ? idesc_tf32((uint32_t)a.n_tile, 256u) : idesc_tf32(kTileM, (uint32_t)a.n_tile);
+            const uint32_t m_rows = a.swap ? (uint32_t)a.n_tile : (uint32_t)kTileM;
+            const uint32_t n_cols = a.swap ? 256u : (uint32_t)a.n_tile;
+            const uint32_t idesc = BF16 ? idesc_bf16(m_rows, n_cols) : idesc_tf32(m_rows, n_cols);
+            auto mma = [](uint32_t d, uint64_t ad, uint64_t bd, uint32_t id, bool acc) {
+                if (BF16) mma_bf16(d, ad, bd, id, acc); else mma_tf32(d, ad, bd, id, acc);
+            };
             const uint32_t desc_hi = (128u >> 4) | (1u << 14);                  // SBO = 128 B, descriptor version 1
             const uint32_t a_lo_fixed = ((uint32_t)a.npix & 0x3FFFu) << 16;     // LBO = npix * 16 B
             const uint32_t b_lo_fixed = ((uint32_t)a.n_tile & 0x3FFFu) << 16;   // LBO = n_tile * 16 B
@@ -515,14 +563,14 @@ general_tf32_kernel(const KernelArgs a)
                                 if (a.swap) {
                                     // M operand = the 128 filters of this stage, N operand = 256 staged pixels
                                     for (int m = 0; m < a.mt; m += 2, a_lo += 2 * kTileM, d += 2 * kTileM) {
-                                        mma_tf32(d, ((uint64_t)desc_hi << 32) | b_lo, ((uint64_t)desc_hi << 32) | a_lo, idesc, accumulate != 0);
-                                        mma_tf32(d, ((uint64_t)desc_hi << 32) | (b_lo + b_kstep),
+                                        mma(d, ((uint64_t)desc_hi << 32) | b_lo, ((uint64_t)desc_hi << 32) | a_lo, idesc, accumulate != 0);
+                                        mma(d, ((uint64_t)desc_hi << 32) | (b_lo + b_kstep),
                                                  ((uint64_t)desc_hi << 32) | (a_lo + a_kstep), idesc, true);
                                     }
                                 } else {
                                     for (int m = 0; m < a.mt; ++m, a_lo += kTileM, d += (uint32_t)a.n_tile) {
-                                        mma_tf32(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, accumulate != 0);
-                                        mma_tf32(d, ((uint64_t)desc_hi << 32) | (a_lo + a_kstep),
+                                        mma(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, accumulate != 0);
+                                        mma(d, ((uint64_t)desc_hi << 32) | (a_lo + a_kstep),
                                                  ((uint64_t)desc_hi << 32) | (b_lo + b_kstep), idesc, true);
                                     }
                                 }
@@ -570,8 +618,8 @@ general_tf32_kernel(const KernelArgs a)
                 gr += ii.g_begin;
                 for (int first = 0; first < units; first += kProducers * kUnitsPerThread) {
                     float v[kUnitsPerThread][kCB];
-                    load_units(v, a, j0, gr * a.cbg, first, wtid);
-                    store_units(v, dst, a, first, wtid);
+                    load_units<BF16>(v, a, j0, gr * a.cbg, first, wtid);
+                    store_units<BF16>(v, dst, a, first, wtid);
                 }
                 fence_proxy_async_smem();
                 mbar_arrive(&a_full[as]);
@@ -756,10 +804,25 @@ size_t tf32_workspace_bytes(const Shape& sh)
     return kStatusBytes + packed_floats(p) * sizeof(float);
 }
 
-conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
-                                    void* workspace, bool weights_packed, cudaStream_t stream)
+bool bf16_supported(const Shape& sh)
 {
-    const Plan p = make_plan(sh);
+    return make_plan(sh, true).ok;
+}
+
+size_t bf16_workspace_bytes(const Shape& sh)
+{
+    const Plan p = make_plan(sh, true);
+    if (!p.ok) return kStatusBytes;
+    return kStatusBytes + packed_floats(p) * sizeof(float);
+}
+
+namespace {
+conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* y, const Shape& sh, bool bf16,
+                                   void* workspace, bool weights_packed, cudaStream_t stream)
+{
+    const float* x = static_cast<const float*>(x_any);   // bf16: re-read as 16-bit elements inside the kernel
+    const float* w = static_cast<const float*>(w_any);
+    const Plan p = make_plan(sh, bf16);
     if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
     unsigned* status = static_cast<unsigned*>(workspace);
     float* wp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
@@ -768,14 +831,20 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
         const long long total = (long long)packed_floats(p);
         long long blocks = (total + 255) / 256;
         if (blocks > 148 * 16) blocks = 148 * 16;
-        repack_filters_kernel<<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, sh.C, p.taps, p.n_tile, p.cblks, total);
+        if (bf16)
+            repack_filters_bf16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+                static_cast<const unsigned short*>(w_any), reinterpret_cast<unsigned short*>(wp), status, sh.K, sh.C,
+                p.taps, p.n_tile, p.cblks, 2 * total);
+        else
+            repack_filters_kernel<<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, sh.C, p.taps, p.n_tile, p.cblks, total);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
     }
 
     static bool attr_set = false;   // per process; the attribute is per function and device-wide
     if (!attr_set) {
-        if (cudaFuncSetAttribute(general_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
+        if (cudaFuncSetAttribute(general_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(general_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
             return CONV2D_ERR_CUDA;
         attr_set = true;
     }
@@ -802,9 +871,25 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
     if (p.ksplit > 1 &&
         cudaMemsetAsync(y, 0, (size_t)sh.N * sh.K * sh.P * sh.Q * sizeof(float), stream) != cudaSuccess)
         return CONV2D_ERR_CUDA;
-    general_tf32_kernel<<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
+    if (bf16)
+        general_tc_kernel<true><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
+    else
+        general_tc_kernel<false><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+}  // namespace
+
+conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
+                                    void* workspace, bool weights_packed, cudaStream_t stream)
+{
+    return launch_tensor_core(x, w, y, sh, false, workspace, weights_packed, stream);
+}
+
+conv2d_status_t launch_general_bf16(const void* x, const void* w, float* y, const Shape& sh,
+                                    void* workspace, bool weights_packed, cudaStream_t stream)
+{
+    return launch_tensor_core(x, w, y, sh, true, workspace, weights_packed, stream);
 }
 
 // ---------------------------------------------------------------- variant without caller-provided scratch

@@ -9,6 +9,17 @@ FFMA_TOL = 1e-5   # |y - y_ref| <= 1e-5 * sum|x*w|   (fp32 FMA paths)
 TF32_TOL = 2e-3   # |y - y_ref| <= 2e-3 * sum|x*w|   (TF32 tensor-core path)
 
 
+BF16_TOL = 1e-5   # bf16 operands, exact products, fp32 accumulation: same bar as the fp32 FMA paths
+
+
+def bf16_values(a: np.ndarray):
+    """Rounds fp32 to the nearest bf16 (ties to even).  Returns (the values as fp32, their 16-bit patterns)."""
+    bits = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    bits = (bits + 0x7FFF + ((bits >> 16) & 1)) >> 16
+    pat = bits.astype(np.uint16)
+    return (pat.astype(np.uint32) << 16).view(np.float32).reshape(a.shape), pat.reshape(a.shape)
+
+
 def run_library(x: np.ndarray, w: np.ndarray, entry: str = "general", algo: int = 1, flags: int = 0,
                 workspace=None, repeat: int = 1):
     """Runs one convolution through the C ABI on cuda:0 and returns y as a numpy array [N,K,P,Q].
@@ -23,8 +34,13 @@ def run_library(x: np.ndarray, w: np.ndarray, entry: str = "general", algo: int 
     K, _, R, S = w.shape
     P, Q = H - R + 1, W - S + 1
     dev = torch.device("cuda:0")
-    xd = torch.from_numpy(np.ascontiguousarray(x)).to(dev)
-    wd = torch.from_numpy(np.ascontiguousarray(w)).to(dev)
+    if entry == "bf16":     # x, w hold bf16 values; the device gets their 16-bit patterns
+        xd = torch.from_numpy(bf16_values(x)[1].view(np.int16)).to(dev)
+        wd = torch.from_numpy(bf16_values(w)[1].view(np.int16)).to(dev)
+        algo = 3
+    else:
+        xd = torch.from_numpy(np.ascontiguousarray(x)).to(dev)
+        wd = torch.from_numpy(np.ascontiguousarray(w)).to(dev)
     numel = N * K * P * Q
     payload = np.array([0x7FC0BEEF], dtype=np.uint32).view(np.float32)[0]
     buf = torch.full((numel + 2 * GUARD,), float("nan"), device=dev, dtype=torch.float32)
@@ -32,7 +48,7 @@ def run_library(x: np.ndarray, w: np.ndarray, entry: str = "general", algo: int 
     y_ptr = buf.data_ptr() + 4 * GUARD
     stream = torch.cuda.current_stream().cuda_stream
     ws_ptr, ws_bytes = 0, 0
-    if entry == "general":
+    if entry in ("general", "bf16"):
         ws_bytes = lib.conv2d_fwd_workspace_size(N, C, H, W, K, R, S, algo)
         if workspace is None and ws_bytes:
             workspace = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
@@ -41,6 +57,9 @@ def run_library(x: np.ndarray, w: np.ndarray, entry: str = "general", algo: int 
         if entry == "single":
             assert C == 1
             lib.conv2d_fwd_single_channel(xd.data_ptr(), wd.data_ptr(), y_ptr, N, H, W, K, R, S, 0, 0, flags, stream)
+        elif entry == "bf16":
+            lib.conv2d_fwd_general_bf16(xd.data_ptr(), wd.data_ptr(), y_ptr, N, C, H, W, K, R, S,
+                                        ws_ptr, ws_bytes, flags, stream)
         else:
             lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), y_ptr, N, C, H, W, K, R, S, algo,
                                    ws_ptr, ws_bytes, flags, stream)

@@ -32,3 +32,14 @@ def test_config_shapes_and_weight_scale():
     assert CONFIGS["cfg5_r7"].Q == 26
     x5, w5 = make_inputs(CONFIGS["cfg5_r3"], batch=1)
     assert 0.0 <= x5.min() and x5.max() < 1.0 and w5.shape == (128, 128, 3, 3)
+
+
+def test_bf16_rounding_helper_matches_torch():
+    import torch
+    from helpers import bf16_values
+    from workloads import uniform
+    a = uniform((4097,), 431, -3.0, 3.0)
+    vals, pat = bf16_values(a)
+    t = torch.from_numpy(a).to(torch.bfloat16)
+    np.testing.assert_array_equal(vals, t.float().numpy())
+    np.testing.assert_array_equal(pat.view(np.int16), t.view(torch.int16).numpy())
