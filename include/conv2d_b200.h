@@ -56,8 +56,13 @@ typedef enum {
     CONV2D_ALGO_AUTO = 0,  /* tensor cores (TF32) where an instance exists, else fp32 FMA */
     CONV2D_ALGO_FFMA = 1,  /* fp32 fused multiply-add on the CUDA cores; error <= 1e-5 * sum|x*w| */
     CONV2D_ALGO_TF32 = 2,  /* operands rounded to TF32, fp32 accumulation on tcgen05; error <= 2e-3 * sum|x*w| */
-    CONV2D_ALGO_BF16 = 3   /* workspace query only: the size conv2d_fwd_general_bf16 needs */
+    CONV2D_ALGO_16BIT = 3  /* workspace query only: the size conv2d_fwd_general_16bit needs */
 } conv2d_algo_t;
+
+typedef enum {
+    CONV2D_OPERAND_BF16 = 0,  /* bfloat16: the upper 16 bits of an IEEE fp32 */
+    CONV2D_OPERAND_FP16 = 1   /* IEEE binary16 */
+} conv2d_operand_t;
 
 /* `flags` bits */
 enum {
@@ -121,19 +126,22 @@ conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
  * General case with 16-bit operands (Section 4, Algorithm 2, with the shorter data types
  * that Section 6 names as the next step).  Section 2.1's rule -- make the unit a thread
  * moves as wide as the memory's access width -- is applied to the tensor-core operand
- * layout: one 16-byte unit holds 8 bf16 channels where the TF32 path holds 4 fp32.
- *   x_bf16 [N][C][H][W], w_bf16 [K][C][R][S]: bfloat16 (the upper 16 bits of an IEEE fp32),
+ * layout: one 16-byte unit holds 8 channels where the TF32 path holds 4 fp32.
+ *   x16 [N][C][H][W], w16 [K][C][R][S]: both of the element type `operand` names,
  *   y [N][K][P][Q]: fp32.  Products are exact, accumulation is fp32 on tcgen05 (kind::f16):
- *   for inputs that are bf16 values the error against exact arithmetic is <= 1e-5 * sum|x*w|.
+ *   the error against exact arithmetic on the given 16-bit values is <= 1e-5 * sum|x*w|.
  * Same kernel, tiling and status block as CONV2D_ALGO_TF32; the workspace size comes from
- * conv2d_fwd_workspace_size(..., CONV2D_ALGO_BF16, ...), and CONV2D_FLAG_WEIGHTS_PACKED has the
- * same meaning.  All four pointers are device pointers and must be 16-byte aligned.
- * Returns CONV2D_ERR_UNSUPPORTED when no tensor-core instance fits the shape.
+ * conv2d_fwd_workspace_size(..., CONV2D_ALGO_16BIT, ...), and CONV2D_FLAG_WEIGHTS_PACKED has the
+ * same meaning (same operand type included).  All four pointers are device pointers and must
+ * be 16-byte aligned; workspace is required.
+ * Returns CONV2D_ERR_UNSUPPORTED when no tensor-core instance fits the shape or `operand`
+ * is not one of the two values.
  */
-conv2d_status_t conv2d_fwd_general_bf16(const void* x_bf16, const void* w_bf16, float* y,
-                                        int N, int C, int H, int W, int K, int R, int S,
-                                        void* workspace, size_t workspace_bytes,
-                                        unsigned flags, void* cuda_stream);
+conv2d_status_t conv2d_fwd_general_16bit(const void* x16, const void* w16, float* y,
+                                         int N, int C, int H, int W, int K, int R, int S,
+                                         conv2d_operand_t operand,
+                                         void* workspace, size_t workspace_bytes,
+                                         unsigned flags, void* cuda_stream);
 
 /*
  * General case on the tensor cores for callers that cannot hand over scratch memory.

@@ -10,7 +10,8 @@ from __future__ import annotations
 import ctypes
 from pathlib import Path
 
-ALGO_AUTO, ALGO_FFMA, ALGO_TF32, ALGO_BF16 = 0, 1, 2, 3
+ALGO_AUTO, ALGO_FFMA, ALGO_TF32, ALGO_16BIT = 0, 1, 2, 3
+OPERAND_BF16, OPERAND_FP16 = 0, 1
 FLAG_WEIGHTS_PACKED = 1
 
 _LIB_PATH = Path(__file__).resolve().parent / "libconv2d_b200.so"
@@ -46,8 +47,8 @@ def load_library() -> ctypes.CDLL:
     lib.conv2d_fwd_single_channel.restype = i
     lib.conv2d_fwd_general.argtypes = [vp, vp, vp] + [i] * 7 + [i, vp, sz, u, vp]
     lib.conv2d_fwd_general.restype = i
-    lib.conv2d_fwd_general_bf16.argtypes = [vp, vp, vp] + [i] * 7 + [vp, sz, u, vp]
-    lib.conv2d_fwd_general_bf16.restype = i
+    lib.conv2d_fwd_general_16bit.argtypes = [vp, vp, vp] + [i] * 7 + [i, vp, sz, u, vp]
+    lib.conv2d_fwd_general_16bit.restype = i
     lib.conv2d_fwd_general_noalloc.argtypes = [vp, vp, vp] + [i] * 7 + [i, vp]
     lib.conv2d_fwd_general_noalloc.restype = i
     lib.conv2d_fwd_host.argtypes = [vp] * 6 + [i] * 7 + [i, vp, sz, vp]
@@ -96,12 +97,12 @@ def conv2d_fwd_general(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, algo=ALGO_AUTO,
            "conv2d_fwd_general")
 
 
-def conv2d_fwd_general_bf16(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S,
-                            workspace_ptr=0, workspace_bytes=0, flags=0, stream=0) -> None:
-    """x, w: device bf16 tensors; y: device fp32 tensor."""
-    _check(load_library().conv2d_fwd_general_bf16(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S,
-                                                  workspace_ptr or None, workspace_bytes, flags, stream or None),
-           "conv2d_fwd_general_bf16")
+def conv2d_fwd_general_16bit(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, operand=OPERAND_BF16,
+                             workspace_ptr=0, workspace_bytes=0, flags=0, stream=0) -> None:
+    """x, w: device tensors of bf16 or fp16 elements (as `operand` says); y: device fp32 tensor."""
+    _check(load_library().conv2d_fwd_general_16bit(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, operand,
+                                                   workspace_ptr or None, workspace_bytes, flags, stream or None),
+           "conv2d_fwd_general_16bit")
 
 
 def conv2d_fwd_general_noalloc(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, wait=0, stream=0) -> None:

@@ -38,11 +38,11 @@ size_t tf32_workspace_bytes(const Shape& sh);   // includes the status block
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
                                     void* workspace, bool weights_packed, cudaStream_t stream);
 
-// Same kernel with bf16 operands (x, w hold 16-bit elements in the same NCHW / KCRS order), fp32 output.
-bool bf16_supported(const Shape& sh);
-size_t bf16_workspace_bytes(const Shape& sh);
-conv2d_status_t launch_general_bf16(const void* x, const void* w, float* y, const Shape& sh,
-                                    void* workspace, bool weights_packed, cudaStream_t stream);
+// Same kernel with 16-bit operands (x, w hold bf16 or fp16 elements in the same NCHW / KCRS order), fp32 output.
+bool b16_supported(const Shape& sh);
+size_t b16_workspace_bytes(const Shape& sh);
+conv2d_status_t launch_general_b16(const void* x, const void* w, float* y, const Shape& sh, bool fp16,
+                                   void* workspace, bool weights_packed, cudaStream_t stream);
 
 // Variant of the tensor-core path whose scratch is a fixed array inside the library image.
 constexpr size_t kNoAllocScratchBytes = kStatusBytes + (size_t)8 * 1024 * 1024;

@@ -58,9 +58,9 @@ conv2d_status_t conv2d_fwd_workspace_size(int N, int C, int H, int W, int K, int
         case CONV2D_ALGO_AUTO:
             if (tf32_supported(sh)) *bytes = tf32_workspace_bytes(sh);
             return CONV2D_OK;
-        case CONV2D_ALGO_BF16:
-            if (!bf16_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
-            *bytes = bf16_workspace_bytes(sh);
+        case CONV2D_ALGO_16BIT:
+            if (!b16_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
+            *bytes = b16_workspace_bytes(sh);
             return CONV2D_OK;
         default: return CONV2D_ERR_UNSUPPORTED;
     }
@@ -116,23 +116,24 @@ conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
     return launch_general_ffma(x, w, y, sh, stream);
 }
 
-conv2d_status_t conv2d_fwd_general_bf16(const void* x_bf16, const void* w_bf16, float* y,
-                                        int N, int C, int H, int W, int K, int R, int S,
-                                        void* workspace, size_t workspace_bytes,
-                                        unsigned flags, void* cuda_stream)
+conv2d_status_t conv2d_fwd_general_16bit(const void* x16, const void* w16, float* y,
+                                         int N, int C, int H, int W, int K, int R, int S,
+                                         conv2d_operand_t operand, void* workspace, size_t workspace_bytes,
+                                         unsigned flags, void* cuda_stream)
 {
-    if (!x_bf16 || !w_bf16 || !y || !workspace) return CONV2D_ERR_NULL;
+    if (!x16 || !w16 || !y || !workspace) return CONV2D_ERR_NULL;
     Shape sh;
     conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
     if (st != CONV2D_OK) return st;
-    if (!aligned16(x_bf16) || !aligned16(w_bf16) || !aligned16(y) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (!aligned16(x16) || !aligned16(w16) || !aligned16(y) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
     if (flags & ~(unsigned)CONV2D_FLAG_WEIGHTS_PACKED) return CONV2D_ERR_UNSUPPORTED;
-    if (!bf16_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
-    if (workspace_bytes < bf16_workspace_bytes(sh)) return CONV2D_ERR_WORKSPACE;
+    if (operand != CONV2D_OPERAND_BF16 && operand != CONV2D_OPERAND_FP16) return CONV2D_ERR_UNSUPPORTED;
+    if (!b16_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
+    if (workspace_bytes < b16_workspace_bytes(sh)) return CONV2D_ERR_WORKSPACE;
     st = check_device();
     if (st != CONV2D_OK) return st;
-    return launch_general_bf16(x_bf16, w_bf16, y, sh, workspace, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0,
-                               static_cast<cudaStream_t>(cuda_stream));
+    return launch_general_b16(x16, w16, y, sh, operand == CONV2D_OPERAND_FP16, workspace,
+                              (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
 conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float* y,

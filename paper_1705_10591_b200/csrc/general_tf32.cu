@@ -117,9 +117,9 @@ int env_int(const char* name, int dflt)
     return (v && *v) ? atoi(v) : dflt;
 }
 
-// bf16: the operands are bf16 (16-byte unit = 8 channels, 32 channels per staged block, K = 16 per MMA); the
+// b16: the operands are 16-bit floats, bf16 or fp16 (16-byte unit = 8 channels, 32 channels per staged block, K = 16 per MMA); the
 // byte layout of every stage is the same as for TF32 (16 channels of 4 bytes).
-Plan make_plan(const Shape& sh, bool bf16 = false)
+Plan make_plan(const Shape& sh, bool b16 = false)
 {
     Plan p{};
     p.ok = false;
@@ -142,7 +142,7 @@ Plan make_plan(const Shape& sh, bool bf16 = false)
         p.n_blocks = (kp16 + p.n_tile - 1) / p.n_tile;
     }
     const int set_cols = p.swap ? kTileM : p.n_tile;      // tensor-memory columns of one 128-pixel tile
-    const int cbc = bf16 ? 2 * kCB : kCB;                 // channels per staged block
+    const int cbc = b16 ? 2 * kCB : kCB;                 // channels per staged block
     p.cblks = (sh.C + cbc - 1) / cbc;
     p.taps = sh.R * sh.S;
     const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
@@ -275,8 +275,8 @@ __global__ void repack_filters_kernel(const float* __restrict__ w, float* __rest
     }
 }
 
-// bf16 variant: wp[nb][cb][t][chunk][f][e] = w[nb*n_tile + f][cb*32 + 8*chunk + e][t] (16-bit elements).
-__global__ void repack_filters_bf16_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ wp,
+// 16-bit variant: wp[nb][cb][t][chunk][f][e] = w[nb*n_tile + f][cb*32 + 8*chunk + e][t] (16-bit elements).
+__global__ void repack_filters_b16_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ wp,
                                            unsigned* __restrict__ status, int K, int C, int taps, int n_tile, int cblks,
                                            long long total)
 {
@@ -306,6 +306,8 @@ struct KernelArgs {
     int HW;
     int total_pix;
     int n_tile, n_blocks, mt, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
+    int fp16;         // 16-bit operands only: 1 = IEEE half, 0 = bf16
+    int pair;         // 16-bit operands only: producers load two adjacent pixels per 32-bit word (needs H*W even)
     int cbg, groups;        // channel blocks per activation stage, number of such groups
     int resident;           // filters loaded once per thread block instead of streamed
     int swap;               // operand roles swapped: accumulator lanes = filters, columns = pixels
@@ -321,7 +323,7 @@ struct KernelArgs {
 // [channel block][chunk][pixel] in 16-byte units.  A work unit is (channel block g, pixel jj), numbered
 // i = g * npix + jj; thread t of the 256 producers owns units first + t, first + t + 256, ...  Consecutive
 // lanes read consecutive pixels of one channel (coalesced) and write consecutive 16-byte units.
-template <bool BF16, int CNT>
+template <bool B16, int CNT>
 __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArgs& a, int j0, int cb0, int first, int wtid)
 {
     const int units = a.npix * a.cbg;
@@ -333,8 +335,22 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
         if (i < units) {
             const int g = i / a.npix, jj = i - g * a.npix;
             const int j = j0 + jj;
-            if (BF16) {
-                // 32 bf16 channels of this pixel, packed two per 32-bit word (lower channel in the low half)
+            if (B16 && a.pair) {
+                // Unit = 2 adjacent pixels x 16 channels: every load is one aligned 32-bit word holding the
+                // two pixels of one channel (H*W even keeps pairs aligned and inside one image).
+                const int half_n = a.npix >> 1;
+                const int h = jj / half_n, pp = jj - h * half_n;
+                const int jp = j0 + 2 * pp;
+                const int c0 = (cb0 + g) * 2 * kCB + kCB * h;
+                if (jp < a.total_pix && c0 < a.C) {
+                    const int n = jp / a.HW, off = jp - n * a.HW;
+                    const unsigned short* src = reinterpret_cast<const unsigned short*>(a.x) + ((size_t)n * a.C + c0) * a.HW + off;
+#pragma unroll
+                    for (int e = 0; e < kCB; ++e)
+                        if (c0 + e < a.C) v[u][e] = __uint_as_float(__ldg(reinterpret_cast<const unsigned*>(src + (size_t)e * a.HW)));
+                }
+            } else if (B16) {
+                // 32 16-bit channels of this pixel, packed two per 32-bit word (lower channel in the low half)
                 const int c0 = (cb0 + g) * 2 * kCB;
                 if (j < a.total_pix && c0 < a.C) {
                     const int n = j / a.HW, off = j - n * a.HW;
@@ -361,7 +377,7 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
     }
 }
 
-template <bool BF16, int CNT>
+template <bool B16, int CNT>
 __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* dst, const KernelArgs& a, int first, int wtid)
 {
     const int units = a.npix * a.cbg;
@@ -370,10 +386,28 @@ __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* 
         const int i = first + u * kProducers + wtid;
         if (i < units) {
             const int g = i / a.npix, jj = i - g * a.npix;
+            if (B16 && a.pair) {
+                const int half_n = a.npix >> 1;
+                const int h = jj / half_n, pp = jj - h * half_n;
+                float4* d = dst + ((size_t)g * kChunks + 2 * h) * a.npix + 2 * pp;
+#pragma unroll
+                for (int m = 0; m < 2; ++m) {       // 8 channels per 16-byte unit; word k = channels 2k, 2k+1
+                    unsigned lo[4], hi[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const unsigned w0 = __float_as_uint(v[u][8 * m + 2 * k]), w1 = __float_as_uint(v[u][8 * m + 2 * k + 1]);
+                        lo[k] = __byte_perm(w0, w1, 0x5410);     // first pixel: low halves
+                        hi[k] = __byte_perm(w0, w1, 0x7632);     // second pixel: high halves
+                    }
+                    d[m * a.npix] = make_float4(__uint_as_float(lo[0]), __uint_as_float(lo[1]), __uint_as_float(lo[2]), __uint_as_float(lo[3]));
+                    d[m * a.npix + 1] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(hi[2]), __uint_as_float(hi[3]));
+                }
+                continue;
+            }
             float4* d = dst + (size_t)g * kChunks * a.npix + jj;
 #pragma unroll
             for (int ch = 0; ch < kChunks; ++ch)
-                d[ch * a.npix] = BF16 ? make_float4(v[u][4 * ch], v[u][4 * ch + 1], v[u][4 * ch + 2], v[u][4 * ch + 3])
+                d[ch * a.npix] = B16 ? make_float4(v[u][4 * ch], v[u][4 * ch + 1], v[u][4 * ch + 2], v[u][4 * ch + 3])
                                       : make_float4(to_tf32_rna(v[u][4 * ch]), to_tf32_rna(v[u][4 * ch + 1]),
                                                     to_tf32_rna(v[u][4 * ch + 2]), to_tf32_rna(v[u][4 * ch + 3]));
         }
@@ -399,7 +433,7 @@ __device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
     return it;
 }
 
-template <bool BF16>
+template <bool B16>
 __global__ void __launch_bounds__(kThreads, 1)
 general_tc_kernel(const KernelArgs a)
 {
@@ -503,9 +537,9 @@ general_tc_kernel(const KernelArgs a)
             // single thread issuing ~40 dependent integer instructions per MMA was slower than the MMA.
             const uint32_t m_rows = a.swap ? (uint32_t)a.n_tile : (uint32_t)kTileM;
             const uint32_t n_cols = a.swap ? 256u : (uint32_t)a.n_tile;
-            const uint32_t idesc = BF16 ? idesc_bf16(m_rows, n_cols) : idesc_tf32(m_rows, n_cols);
+            const uint32_t idesc = B16 ? idesc_b16(m_rows, n_cols, a.fp16 != 0) : idesc_tf32(m_rows, n_cols);
             auto mma = [](uint32_t d, uint64_t ad, uint64_t bd, uint32_t id, bool acc) {
-                if (BF16) mma_bf16(d, ad, bd, id, acc); else mma_tf32(d, ad, bd, id, acc);
+                if (B16) mma_b16(d, ad, bd, id, acc); else mma_tf32(d, ad, bd, id, acc);
             };
             const uint32_t desc_hi = (128u >> 4) | (1u << 14);                  // SBO = 128 B, descriptor version 1
             const uint32_t a_lo_fixed = ((uint32_t)a.npix & 0x3FFFu) << 16;     // LBO = npix * 16 B
@@ -618,8 +652,8 @@ general_tc_kernel(const KernelArgs a)
                 gr += ii.g_begin;
                 for (int first = 0; first < units; first += kProducers * kUnitsPerThread) {
                     float v[kUnitsPerThread][kCB];
-                    load_units<BF16>(v, a, j0, gr * a.cbg, first, wtid);
-                    store_units<BF16>(v, dst, a, first, wtid);
+                    load_units<B16>(v, a, j0, gr * a.cbg, first, wtid);
+                    store_units<B16>(v, dst, a, first, wtid);
                 }
                 fence_proxy_async_smem();
                 mbar_arrive(&a_full[as]);
@@ -804,12 +838,12 @@ size_t tf32_workspace_bytes(const Shape& sh)
     return kStatusBytes + packed_floats(p) * sizeof(float);
 }
 
-bool bf16_supported(const Shape& sh)
+bool b16_supported(const Shape& sh)
 {
     return make_plan(sh, true).ok;
 }
 
-size_t bf16_workspace_bytes(const Shape& sh)
+size_t b16_workspace_bytes(const Shape& sh)
 {
     const Plan p = make_plan(sh, true);
     if (!p.ok) return kStatusBytes;
@@ -817,12 +851,12 @@ size_t bf16_workspace_bytes(const Shape& sh)
 }
 
 namespace {
-conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* y, const Shape& sh, bool bf16,
+conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* y, const Shape& sh, bool b16, bool fp16,
                                    void* workspace, bool weights_packed, cudaStream_t stream)
 {
-    const float* x = static_cast<const float*>(x_any);   // bf16: re-read as 16-bit elements inside the kernel
+    const float* x = static_cast<const float*>(x_any);   // 16-bit operands: re-read as such inside the kernel
     const float* w = static_cast<const float*>(w_any);
-    const Plan p = make_plan(sh, bf16);
+    const Plan p = make_plan(sh, b16);
     if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
     unsigned* status = static_cast<unsigned*>(workspace);
     float* wp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
@@ -831,8 +865,8 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         const long long total = (long long)packed_floats(p);
         long long blocks = (total + 255) / 256;
         if (blocks > 148 * 16) blocks = 148 * 16;
-        if (bf16)
-            repack_filters_bf16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+        if (b16)
+            repack_filters_b16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
                 static_cast<const unsigned short*>(w_any), reinterpret_cast<unsigned short*>(wp), status, sh.K, sh.C,
                 p.taps, p.n_tile, p.cblks, 2 * total);
         else
@@ -861,6 +895,8 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     for (int v = 4; v >= 2; v >>= 1)
         if (sh.W % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
+    a.fp16 = fp16 ? 1 : 0;
+    a.pair = (b16 && (sh.H * sh.W) % 2 == 0 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
     a.items = p.supertiles * p.n_blocks * p.ksplit;
     a.ksplit = p.ksplit;
     // Failure-detection test hooks (host-side injection only): a short wait bound and one filter copy that is
@@ -871,7 +907,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     if (p.ksplit > 1 &&
         cudaMemsetAsync(y, 0, (size_t)sh.N * sh.K * sh.P * sh.Q * sizeof(float), stream) != cudaSuccess)
         return CONV2D_ERR_CUDA;
-    if (bf16)
+    if (b16)
         general_tc_kernel<true><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
     else
         general_tc_kernel<false><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
@@ -883,13 +919,13 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
                                     void* workspace, bool weights_packed, cudaStream_t stream)
 {
-    return launch_tensor_core(x, w, y, sh, false, workspace, weights_packed, stream);
+    return launch_tensor_core(x, w, y, sh, false, false, workspace, weights_packed, stream);
 }
 
-conv2d_status_t launch_general_bf16(const void* x, const void* w, float* y, const Shape& sh,
-                                    void* workspace, bool weights_packed, cudaStream_t stream)
+conv2d_status_t launch_general_b16(const void* x, const void* w, float* y, const Shape& sh, bool fp16,
+                                   void* workspace, bool weights_packed, cudaStream_t stream)
 {
-    return launch_tensor_core(x, w, y, sh, true, workspace, weights_packed, stream);
+    return launch_tensor_core(x, w, y, sh, true, fp16, workspace, weights_packed, stream);
 }
 
 // ---------------------------------------------------------------- variant without caller-provided scratch

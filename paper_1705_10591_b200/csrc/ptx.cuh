@@ -92,8 +92,8 @@ __device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint6
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
 }
-// Same with bf16 operands (kind::f16, K = 16 per instruction).
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate)
+// Same with 16-bit operands, bf16 or fp16 as the instruction descriptor says (kind::f16, K = 16 per instruction).
+__device__ __forceinline__ void mma_b16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -140,12 +140,12 @@ __host__ __device__ constexpr uint32_t idesc_tf32(uint32_t m, uint32_t n)
          | ((m >> 4) << 24);
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
-__host__ __device__ constexpr uint32_t idesc_bf16(uint32_t m, uint32_t n)
+// Instruction descriptor: 16-bit x 16-bit -> fp32 (operand format 0 = fp16, 1 = bf16), both operands K-major.
+__host__ __device__ constexpr uint32_t idesc_b16(uint32_t m, uint32_t n, bool fp16)
 {
-    return (1u << 4)            // accumulator format fp32
-         | (1u << 7)            // A format bf16
-         | (1u << 10)           // B format bf16
+    return (1u << 4)                    // accumulator format fp32
+         | ((fp16 ? 0u : 1u) << 7)      // A format
+         | ((fp16 ? 0u : 1u) << 10)     // B format
          | ((n >> 3) << 17)
          | ((m >> 4) << 24);
 }

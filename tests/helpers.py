@@ -9,7 +9,7 @@ FFMA_TOL = 1e-5   # |y - y_ref| <= 1e-5 * sum|x*w|   (fp32 FMA paths)
 TF32_TOL = 2e-3   # |y - y_ref| <= 2e-3 * sum|x*w|   (TF32 tensor-core path)
 
 
-BF16_TOL = 1e-5   # bf16 operands, exact products, fp32 accumulation: same bar as the fp32 FMA paths
+B16_TOL = 1e-5    # 16-bit operands, exact products, fp32 accumulation: same bar as the fp32 FMA paths
 
 
 def bf16_values(a: np.ndarray):
@@ -18,6 +18,12 @@ def bf16_values(a: np.ndarray):
     bits = (bits + 0x7FFF + ((bits >> 16) & 1)) >> 16
     pat = bits.astype(np.uint16)
     return (pat.astype(np.uint32) << 16).view(np.float32).reshape(a.shape), pat.reshape(a.shape)
+
+
+def fp16_values(a: np.ndarray):
+    """Rounds fp32 to the nearest IEEE half (numpy's conversion, ties to even).  Returns (values as fp32, patterns)."""
+    h = np.ascontiguousarray(a, dtype=np.float32).astype(np.float16)
+    return h.astype(np.float32), h.view(np.uint16)
 
 
 def run_library(x: np.ndarray, w: np.ndarray, entry: str = "general", algo: int = 1, flags: int = 0,
@@ -34,9 +40,10 @@ def run_library(x: np.ndarray, w: np.ndarray, entry: str = "general", algo: int 
     K, _, R, S = w.shape
     P, Q = H - R + 1, W - S + 1
     dev = torch.device("cuda:0")
-    if entry == "bf16":     # x, w hold bf16 values; the device gets their 16-bit patterns
-        xd = torch.from_numpy(bf16_values(x)[1].view(np.int16)).to(dev)
-        wd = torch.from_numpy(bf16_values(w)[1].view(np.int16)).to(dev)
+    if entry in ("bf16", "fp16"):     # x, w hold 16-bit values; the device gets their 16-bit patterns
+        conv = bf16_values if entry == "bf16" else fp16_values
+        xd = torch.from_numpy(conv(x)[1].view(np.int16)).to(dev)
+        wd = torch.from_numpy(conv(w)[1].view(np.int16)).to(dev)
         algo = 3
     else:
         xd = torch.from_numpy(np.ascontiguousarray(x)).to(dev)
@@ -48,7 +55,7 @@ def run_library(x: np.ndarray, w: np.ndarray, entry: str = "general", algo: int 
     y_ptr = buf.data_ptr() + 4 * GUARD
     stream = torch.cuda.current_stream().cuda_stream
     ws_ptr, ws_bytes = 0, 0
-    if entry in ("general", "bf16"):
+    if entry in ("general", "bf16", "fp16"):
         ws_bytes = lib.conv2d_fwd_workspace_size(N, C, H, W, K, R, S, algo)
         if workspace is None and ws_bytes:
             workspace = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
@@ -57,9 +64,10 @@ def run_library(x: np.ndarray, w: np.ndarray, entry: str = "general", algo: int 
         if entry == "single":
             assert C == 1
             lib.conv2d_fwd_single_channel(xd.data_ptr(), wd.data_ptr(), y_ptr, N, H, W, K, R, S, 0, 0, flags, stream)
-        elif entry == "bf16":
-            lib.conv2d_fwd_general_bf16(xd.data_ptr(), wd.data_ptr(), y_ptr, N, C, H, W, K, R, S,
-                                        ws_ptr, ws_bytes, flags, stream)
+        elif entry in ("bf16", "fp16"):
+            lib.conv2d_fwd_general_16bit(xd.data_ptr(), wd.data_ptr(), y_ptr, N, C, H, W, K, R, S,
+                                         lib.OPERAND_BF16 if entry == "bf16" else lib.OPERAND_FP16,
+                                         ws_ptr, ws_bytes, flags, stream)
         else:
             lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), y_ptr, N, C, H, W, K, R, S, algo,
                                    ws_ptr, ws_bytes, flags, stream)
