@@ -186,7 +186,8 @@ def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
         x, w = make_inputs(cfg)
         xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
         yd = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), device=dev, dtype=torch.float32)
-        for algo_name, algo in (("tf32", lib.ALGO_TF32), ("ffma", lib.ALGO_FFMA)):
+        xd16 = wd16 = None
+        for algo_name, algo in (("tf32", lib.ALGO_TF32), ("bf16", lib.ALGO_16BIT), ("ffma", lib.ALGO_FFMA)):
             try:
                 ws_bytes = lib.conv2d_fwd_workspace_size(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, algo)
             except lib.Conv2dError:
@@ -194,9 +195,18 @@ def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
                 continue
             ws = torch.zeros(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
 
+            tensor_core = algo in (lib.ALGO_TF32, lib.ALGO_16BIT)
+            if algo == lib.ALGO_16BIT and xd16 is None:     # same synthetic values, rounded once to bf16
+                xd16, wd16 = xd.to(torch.bfloat16).contiguous(), wd.to(torch.bfloat16).contiguous()
+
             def call(flags=0):
-                lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
-                                       cfg.K, cfg.R, cfg.S, algo, ws.data_ptr(), ws_bytes, flags, stream)
+                if algo == lib.ALGO_16BIT:
+                    lib.conv2d_fwd_general_16bit(xd16.data_ptr(), wd16.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H,
+                                                 cfg.W, cfg.K, cfg.R, cfg.S, lib.OPERAND_BF16, ws.data_ptr(), ws_bytes,
+                                                 flags, stream)
+                else:
+                    lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
+                                           cfg.K, cfg.R, cfg.S, algo, ws.data_ptr(), ws_bytes, flags, stream)
             for _ in range(3):
                 call()
             lib.conv2d_get_status(ws.data_ptr(), stream)
@@ -205,17 +215,22 @@ def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
                 flush.zero_()
                 cold.append(event_ms(call, torch))
             warm = event_ms(call, torch, iters=20)
-            packed = event_ms(lambda: call(lib.FLAG_WEIGHTS_PACKED), torch, iters=20) if algo == lib.ALGO_TF32 else None
+            packed = event_ms(lambda: call(lib.FLAG_WEIGHTS_PACKED), torch, iters=20) if tensor_core else None
             lib.conv2d_get_status(ws.data_ptr(), stream)
             t_cold, t_warm = statistics.median(cold), warm
+            nbytes = cfg.compulsory_bytes
             if algo == lib.ALGO_TF32:
                 pipe_peak = peaks["bf16_tflops"] / 2.0     # TF32 dense rate is half of bf16 per clock
                 bound = "tensor"
+            elif algo == lib.ALGO_16BIT:
+                pipe_peak = peaks["bf16_tflops"]
+                bound = "tensor"
+                nbytes = 2 * (x.size + w.size) + 4 * yd.numel()     # 2-byte operands, fp32 output
             else:
                 pipe_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
                 bound = "alu"
             t_pipe = cfg.flops / (pipe_peak * 1e12) * 1e3
-            t_hbm = cfg.compulsory_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+            t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9) * 1e3
             entry = {
                 "workload": name, "algo": algo_name, "ms_cold_l2": t_cold, "ms_warm_l2": t_warm,
                 "gflops_cold": cfg.flops / t_cold / 1e6, "gflops_warm": cfg.flops / t_warm / 1e6,
@@ -227,7 +242,7 @@ def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
             if packed is not None:
                 entry["ms_warm_l2_weights_prepacked"] = packed
             out.append(entry)
-        del xd, wd, yd
+        del xd, wd, yd, xd16, wd16
     return out
 
 

@@ -307,6 +307,7 @@ struct KernelArgs {
     int total_pix;
     int n_tile, n_blocks, mt, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
     int fp16;         // 16-bit operands only: 1 = IEEE half, 0 = bf16
+    int helpers;      // 1: warps 8-15 share the write-back of a block's last item (operand-swap layout only)
     int pair;         // 16-bit operands only: producers load two adjacent pixels per 32-bit word (needs H*W even)
     int cbg, groups;        // channel blocks per activation stage, number of such groups
     int resident;           // filters loaded once per thread block instead of streamed
@@ -453,7 +454,8 @@ general_tc_kernel(const KernelArgs a)
     uint64_t* b_empty = b_full + kMaxBStages;              // [kMaxBStages]
     uint64_t* acc_full = b_empty + kMaxBStages;            // [2]
     uint64_t* acc_empty = acc_full + 2;                    // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* tail_full = acc_empty + 2;                   // [1] the block's last item is complete (for warps 8-15)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail_full + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -462,6 +464,7 @@ general_tc_kernel(const KernelArgs a)
         for (int i = 0; i < a.a_stages; ++i) { mbar_init(&a_full[i], kProducers); mbar_init(&a_empty[i], 1); }
         for (int i = 0; i < a.b_stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpilogueWarps); }
+        mbar_init(tail_full, 1);
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -621,6 +624,7 @@ general_tc_kernel(const KernelArgs a)
                     if (++as == a.a_stages) { as = 0; a_phase ^= 1u; }
                 }
                 if (alive) mma_commit(&acc_full[buf]);
+                if (alive && item + (int)gridDim.x >= a.items) mma_commit(tail_full);
                 if (buf) acc_phase1 ^= 1u; else acc_phase0 ^= 1u;
                 if (++buf == a.nbuf) buf = 0;
                 ++n_items;
@@ -632,7 +636,8 @@ general_tc_kernel(const KernelArgs a)
                 a.status[5] = (unsigned)n_items;
             }
         }
-    } else if (producer_index(warp) >= 0) {
+    } else {
+    if (producer_index(warp) >= 0) {
         // ---------------- producers: stage activations, running ahead across item boundaries
         const int wtid = producer_index(warp) * 32 + lane;
         bool alive = true;
@@ -660,23 +665,35 @@ general_tc_kernel(const KernelArgs a)
                 if (++as == a.a_stages) { as = 0; a_phase ^= 1u; }
             }
         }
-    } else if (warp >= 4 && warp < 4 + kEpilogueWarps) {
+    }
+    if (warp >= 4 && (warp < 4 + kEpilogueWarps || a.helpers)) {
         // ---------------- epilogue: drain finished accumulator sets (lane = pixel)
+        // Warps 4-7 drain every item.  The write-back of a block's LAST item cannot hide behind any later
+        // MMAs, so there the eight warps 8-15 (producers that have finished staging, and the two spare
+        // warps) join in: each lane quarter is then drained by three warps that take every third 32-pixel
+        // block.  Their transposition tiles reuse the activation ring, which is idle by then.
         const int quarter = warp & 3;                       // tensor-memory lanes this warp may read
+        const bool helper = warp >= 4 + kEpilogueWarps;
+        const int share = helper ? 1 + ((warp - 8) >> 2) : 0;
         const size_t plane = (size_t)a.P * a.Q;
         const int chunks_per_tile = a.n_tile / 16;
         const int total_chunks = a.mt * chunks_per_tile;
-        int buf = 0;
-        uint32_t acc_phase0 = 0, acc_phase1 = 0;
+        const int n_local = ((int)blockIdx.x < a.items) ? (a.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
         bool alive = true;
-        for (int item = blockIdx.x; item < a.items; item += gridDim.x) {
+        for (int li = helper ? n_local - 1 : 0; li >= 0 && li < n_local; ++li) {
+            const int item = (int)blockIdx.x + li * (int)gridDim.x;
+            const int buf = li % a.nbuf;
+            const uint32_t acc_phase = (uint32_t)(li / a.nbuf) & 1u;
+            const bool split = a.helpers && li == n_local - 1;
             const ItemInfo ii = decode_item(a, item);
             const int j0 = ii.supertile * a.mt * kTileM;
             const int nb = ii.nb;
             const bool add = a.ksplit > 1;                   // partial sums: add into the zeroed output
             // tcgen05.ld is warp-collective: take the decision for the whole warp
-            const uint32_t acc_phase = buf ? acc_phase1 : acc_phase0;
-            alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag, a.max_polls));
+            // (warps 8-15 come late and only for the last item: they wait on a barrier of its own, whose
+            // phase they cannot have missed)
+            alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(helper ? tail_full : &acc_full[buf],
+                                                                       helper ? 0u : acc_phase, abort_flag, a.max_polls));
             if (!alive) break;
             tc_fence_after_sync();
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * acc_cols);
@@ -685,7 +702,9 @@ general_tc_kernel(const KernelArgs a)
                 // Lanes are filters, columns pixels: this thread holds adjacent pixels of ONE map.  A
                 // warp-private shared-memory tile turns a 32-filter x 32-pixel block around so that each
                 // store instruction again writes 32 adjacent pixels of one map.
-                float* tile = xpose + (size_t)(warp - 4) * 32 * kXposePitch;
+                float* tile = helper ? reinterpret_cast<float*>(a_smem) + (size_t)(warp - 8) * 32 * kXposePitch
+                                     : xpose + (size_t)(warp - 4) * 32 * kXposePitch;
+                const int b_step = split ? 3 : 1;
                 const int rpq = a.n_tile / 4;      // filter rows per lane quarter: 32 (M = 128) or 16 (M = 64, lanes 0-15)
                 const int blocks = a.mt * kTileM / 32;
                 auto load_block = [&](uint32_t (&v0)[16], uint32_t (&v1)[16], int b) {
@@ -745,24 +764,22 @@ general_tc_kernel(const KernelArgs a)
                     }
                 };
                 uint32_t va0[16], va1[16], vb0[16], vb1[16];
-                int b = 0;
-                load_block(va0, va1, b);
+                int b = split ? share : 0;
+                if (b < blocks) load_block(va0, va1, b);
                 while (b < blocks) {
                     tmem_ld_wait();
-                    if (b + 1 < blocks) load_block(vb0, vb1, b + 1);
+                    if (b + b_step < blocks) load_block(vb0, vb1, b + b_step);
                     store_block(va0, va1, b);
-                    if (++b >= blocks) break;
+                    if ((b += b_step) >= blocks) break;
                     tmem_ld_wait();
-                    if (b + 1 < blocks) load_block(va0, va1, b + 1);
+                    if (b + b_step < blocks) load_block(va0, va1, b + b_step);
                     store_block(vb0, vb1, b);
-                    ++b;
+                    b += b_step;
                 }
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                if (lane == 0 && !helper) mbar_arrive(&acc_empty[buf]);
                 if (blockIdx.x == 0 && warp == 4 && lane == 0) a.status[6] = (unsigned)(clock_now() - t_epi);
-                if (buf) acc_phase1 ^= 1u; else acc_phase0 ^= 1u;
-                if (++buf == a.nbuf) buf = 0;
                 continue;
             }
             int cur_m = -1;
@@ -813,9 +830,8 @@ general_tc_kernel(const KernelArgs a)
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
-            if (buf) acc_phase1 ^= 1u; else acc_phase0 ^= 1u;
-            if (++buf == a.nbuf) buf = 0;
         }
+    }
     }
 
     tc_fence_before_sync();
@@ -895,6 +911,8 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     for (int v = 4; v >= 2; v >>= 1)
         if (sh.W % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
+    a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * p.npix * 4 >= 2 * kXposeBytes &&
+                 env_int("CONV2D_B200_TF32_HELPERS", 1) != 0) ? 1 : 0;
     a.fp16 = fp16 ? 1 : 0;
     a.pair = (b16 && (sh.H * sh.W) % 2 == 0 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
     a.items = p.supertiles * p.n_blocks * p.ksplit;
