@@ -86,7 +86,9 @@ constexpr size_t kXposeBytes = (size_t)kEpilogueWarps * 32 * kXposePitch * 4;
 struct Plan {
     int n_tile;       // filters per work item (UMMA N), multiple of 16
     int n_blocks;     // work-item columns over the filters
-    int mt;           // accumulator tiles per work item
+    int mt;           // accumulator tiles per work item (pixels-as-M layout; informative otherwise)
+    int tile_px;      // pixels per work item: mt * 128, or any multiple of 32 up to 512 in the operand-swap layout
+    int px_groups;    // operand-swap layout: MMAs per K step (each covers n_mma = tile_px / px_groups pixels)
     int nbuf;         // accumulator sets in tensor memory (2: write-back overlaps the next item)
     int npix;         // staged pixel rows per channel chunk
     int cblks;        // channel blocks
@@ -153,7 +155,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
 
     const int forced_mt = env_int("CONV2D_B200_TF32_MT", 0);      // benchmark ablations only
     const size_t wbytes = (size_t)p.cblks * p.taps * chunk;        // re-ordered filters of one filter block
-    auto npix_of = [&](int mt) { return (int)(((long long)mt * kTileM + halo + 7) / 8 * 8); };
+    auto npix_of = [&](int tile_px) { return (int)(((long long)tile_px + halo + 7) / 8 * 8); };
 
     // Light problems (1x1-like: few taps x channel blocks) with a small filter bank keep it resident in
     // shared memory: nothing is streamed, items are small (finest balance over the SMs, two accumulator
@@ -166,10 +168,11 @@ Plan make_plan(const Shape& sh, bool b16 = false)
     if (resident_mode != 0 && p.n_blocks == 1 && wbytes <= 152 * 1024 &&
         ((long long)p.taps * p.cblks <= 16 || resident_mode == 2)) {
         const int mt = forced_mt ? forced_mt : (p.swap ? 2 : 1);
-        const int npix = npix_of(mt);
+        const int npix = npix_of(mt * kTileM);
         if (mt * set_cols <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * npix * 4 + 512 <= kSmemLimit) {
             p.resident = 1;
             p.mt = mt;
+            p.tile_px = mt * kTileM;
             p.npix = npix;
             p.cbg = 1;
             p.a_stages = 2;
@@ -189,29 +192,54 @@ Plan make_plan(const Shape& sh, bool b16 = false)
         // reused by several tiles.  More tiles per item (mt) amortise that; fewer tiles leave room for a
         // second accumulator set (hidden write-back) and balance better.  Cost in units of one tile's MMA
         // time: rounds x mt x (1 + stage cost / MMA time) + exposed write-back.
-        const double mma_cycles = p.swap ? 64 : (p.n_tile > 128 ? p.n_tile / 2 : 90);   // per 128-pixel tile and K step
-        const double tile_cycles = (double)p.taps * p.cblks * 2 * mma_cycles;
-        int best_mt = 0;
-        double best_cost = 0;
         const size_t kLimit = kSmemLimit - extra;
-        for (int mt = 4; mt >= 1; mt >>= 1) {
-            if (forced_mt && mt != forced_mt) continue;
-            if (p.swap && mt < 2) continue;
-            if (mt * set_cols > 512) continue;
-            const int npix = npix_of(mt);
-            if (npix > 16000) continue;
-            if (smem_need(2, npix, p.n_tile, 2, 1, 1) > kLimit) continue;
-            const long long items = (tiles + mt - 1) / mt * p.n_blocks;
-            const long long rounds = (items + sms - 1) / sms;
-            const int nbuf = (2 * mt * set_cols <= 512) ? 2 : 1;
-            const double stream = 1.0 + (chunk / 66.0) / (mt * 2 * mma_cycles);
-            const double writeback = (nbuf == 1 ? 1.0 : 0.15) * mt * (3000.0 * p.n_tile / 128.0) / tile_cycles;
-            const double cost = rounds * (mt * stream + 0.5 * writeback);
-            if (best_mt == 0 || cost < best_cost) { best_mt = mt; best_cost = cost; }
+        const double stage_cycles = chunk / 66.0;           // one (tap, channel block) of filters through L2
+        const int forced_px = env_int("CONV2D_B200_TF32_TILE_PX", 0);
+        const bool ksplit_allowed = env_int("CONV2D_B200_TF32_KSPLIT", 1) != 0;
+        int best_px = 0;
+        double best_cost = 0;
+        if (p.swap) {
+            // Any multiple of 32 pixels per item: the item size follows from the pixel count and the 148 SMs
+            // (64 x 32 x 32 pixels: 448 per item = 147 items in one round, where 512 would occupy 128 SMs).
+            // One or two MMAs of equal width cover the item per K step; an MMA narrower than 128 pixels is
+            // bound by its ~64-cycle issue cost.
+            for (int px = 512; px >= 64; px -= 32) {
+                if (forced_px ? px != forced_px : (forced_mt && px != forced_mt * kTileM)) continue;
+                const int groups = (px + 255) / 256;
+                if (px % (16 * groups)) continue;
+                const int npix = npix_of(px);
+                if (npix > 16000 || smem_need(2, npix, p.n_tile, 2, 1, 1) > kLimit) continue;
+                const long long items = (total_pix + px - 1) / px * p.n_blocks;
+                const long long rounds = (items + sms - 1) / sms;
+                const int nbuf = 2 * px <= 512 ? 2 : 1;
+                const double mma_step = groups * ((px / groups) / 2.0 > 64.0 ? (px / groups) / 2.0 : 64.0);
+                const double tile_time = (double)p.taps * p.cblks * (2 * mma_step + stage_cycles);
+                const double writeback = (nbuf == 1 ? 1.0 : 0.15) * (px / 128.0) * (3000.0 * p.n_tile / 128.0);
+                double cost = rounds * (tile_time + 0.5 * writeback);
+                // (items that leave half of the SMs idle are split in two along the channels further down)
+                if (items * 2 <= sms && p.cblks >= 2 && ksplit_allowed) cost = 0.5 * tile_time + writeback;
+                if (best_px == 0 || cost < best_cost) { best_px = px; best_cost = cost; }
+            }
+        } else {
+            const double mma_cycles = p.n_tile > 128 ? p.n_tile / 2 : 90;   // per 128-pixel tile and K step
+            for (int mt = 4; mt >= 1; mt >>= 1) {
+                if (forced_mt && mt != forced_mt) continue;
+                if (mt * set_cols > 512) continue;
+                const int npix = npix_of(mt * kTileM);
+                if (npix > 16000 || smem_need(2, npix, p.n_tile, 2, 1, 1) > kLimit) continue;
+                const long long items = (tiles + mt - 1) / mt * p.n_blocks;
+                const long long rounds = (items + sms - 1) / sms;
+                const int nbuf = (2 * mt * set_cols <= 512) ? 2 : 1;
+                const double tile_time = (double)p.taps * p.cblks * (mt * 2 * mma_cycles + stage_cycles);
+                const double writeback = (nbuf == 1 ? 1.0 : 0.15) * mt * (3000.0 * p.n_tile / 128.0);
+                const double cost = rounds * (tile_time + 0.5 * writeback);
+                if (best_px == 0 || cost < best_cost) { best_px = mt * kTileM; best_cost = cost; }
+            }
         }
-        if (best_mt == 0) return p;
-        p.mt = best_mt;
-        p.npix = npix_of(p.mt);
+        if (best_px == 0) return p;
+        p.tile_px = best_px;
+        p.mt = (best_px + kTileM - 1) / kTileM;
+        p.npix = npix_of(p.tile_px);
         // Filter stages: several taps per stage (up to 32 KB) so that the single MMA-issuing thread pays
         // its per-stage bookkeeping (barrier wait, commit) once per 16-32 MMAs; the ring should hold
         // 64-128 KB in flight to cover the L2 latency.
@@ -230,8 +258,10 @@ Plan make_plan(const Shape& sh, bool b16 = false)
         p.smem_bytes = smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg) + extra;
     }
 
-    p.nbuf = (2 * p.mt * set_cols <= 512) ? 2 : 1;
-    p.supertiles = (int)((tiles + p.mt - 1) / p.mt);
+    const int item_cols = p.swap ? p.tile_px : p.mt * p.n_tile;     // tensor-memory columns of one accumulator set
+    p.px_groups = p.swap ? (p.tile_px + 255) / 256 : p.mt;
+    p.nbuf = (2 * item_cols <= 512) ? 2 : 1;
+    p.supertiles = (int)((total_pix + p.tile_px - 1) / p.tile_px);
     // Too few tiles for the machine (e.g. 14 x 14 images): two work items per tile, each contracting half of
     // the channel-block groups and adding into a zeroed output.
     const int n_groups = (p.cblks + p.cbg - 1) / p.cbg;
@@ -240,7 +270,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
     const long long items = (long long)p.supertiles * p.n_blocks * p.ksplit;
     if (items > 0x7fffffffLL) return p;
     p.grid = (int)(items < sms ? items : sms);
-    int cols = p.nbuf * p.mt * set_cols;
+    int cols = p.nbuf * item_cols;
     p.tmem_cols = 32;
     while (p.tmem_cols < cols) p.tmem_cols <<= 1;
     p.ok = true;
@@ -305,7 +335,7 @@ struct KernelArgs {
     int N, C, H, W, K, R, S, P, Q;
     int HW;
     int total_pix;
-    int n_tile, n_blocks, mt, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
+    int n_tile, n_blocks, mt, tile_px, px_groups, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
     int fp16;         // 16-bit operands only: 1 = IEEE half, 0 = bf16
     int helpers;      // 1: warps 8-15 share the write-back of a block's last item (operand-swap layout only)
     int pair;         // 16-bit operands only: producers load two adjacent pixels per 32-bit word (needs H*W even)
@@ -477,7 +507,7 @@ general_tc_kernel(const KernelArgs a)
 
     // Work item -> (supertile, filter block); blocks rotate the order of the channel-block groups by the
     // item number, so that at any moment they stream different parts of the filter bank.
-    const int acc_cols = a.mt * (a.swap ? kTileM : a.n_tile);   // tensor-memory columns of one accumulator set
+    const int acc_cols = a.swap ? a.tile_px : a.mt * a.n_tile;   // tensor-memory columns of one accumulator set
 
     if (warp == 0) {
         // ---------------- filters: global -> shared by bulk copy, up to `tps` taps of one channel block per stage
@@ -539,7 +569,8 @@ general_tc_kernel(const KernelArgs a)
             // that does not change is folded into a_lo_fixed / b_lo_fixed / desc_hi beforehand, because a
             // single thread issuing ~40 dependent integer instructions per MMA was slower than the MMA.
             const uint32_t m_rows = a.swap ? (uint32_t)a.n_tile : (uint32_t)kTileM;
-            const uint32_t n_cols = a.swap ? 256u : (uint32_t)a.n_tile;
+            const uint32_t n_mma = (uint32_t)(a.tile_px / a.px_groups);          // operand-swap layout: pixels per MMA
+            const uint32_t n_cols = a.swap ? n_mma : (uint32_t)a.n_tile;
             const uint32_t idesc = B16 ? idesc_b16(m_rows, n_cols, a.fp16 != 0) : idesc_tf32(m_rows, n_cols);
             auto mma = [](uint32_t d, uint64_t ad, uint64_t bd, uint32_t id, bool acc) {
                 if (B16) mma_b16(d, ad, bd, id, acc); else mma_tf32(d, ad, bd, id, acc);
@@ -598,8 +629,8 @@ general_tc_kernel(const KernelArgs a)
                                 uint32_t a_lo = a_lo_block + row_shift + (uint32_t)sx;
                                 uint32_t d = d0;
                                 if (a.swap) {
-                                    // M operand = the 128 filters of this stage, N operand = 256 staged pixels
-                                    for (int m = 0; m < a.mt; m += 2, a_lo += 2 * kTileM, d += 2 * kTileM) {
+                                    // M operand = the 128 filters of this stage, N operand = n_mma staged pixels
+                                    for (int m = 0; m < a.px_groups; ++m, a_lo += n_mma, d += n_mma) {
                                         mma(d, ((uint64_t)desc_hi << 32) | b_lo, ((uint64_t)desc_hi << 32) | a_lo, idesc, accumulate != 0);
                                         mma(d, ((uint64_t)desc_hi << 32) | (b_lo + b_kstep),
                                                  ((uint64_t)desc_hi << 32) | (a_lo + a_kstep), idesc, true);
@@ -646,7 +677,7 @@ general_tc_kernel(const KernelArgs a)
         const int units = a.npix * a.cbg;
         for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
             const ItemInfo ii = decode_item(a, item);
-            const int j0 = ii.supertile * a.mt * kTileM;                 // first flat pixel of the item
+            const int j0 = ii.supertile * a.tile_px;                     // first flat pixel of the item
             // One stage = cbg consecutive channel blocks.  All loads of a pass (kUnitsPerThread units of
             // 16 channels per thread) are issued before its first store: a pass costs one memory round trip.
             for (int grp = 0; grp < ii.n_groups && alive; ++grp) {
@@ -686,7 +717,7 @@ general_tc_kernel(const KernelArgs a)
             const uint32_t acc_phase = (uint32_t)(li / a.nbuf) & 1u;
             const bool split = a.helpers && li == n_local - 1;
             const ItemInfo ii = decode_item(a, item);
-            const int j0 = ii.supertile * a.mt * kTileM;
+            const int j0 = ii.supertile * a.tile_px;
             const int nb = ii.nb;
             const bool add = a.ksplit > 1;                   // partial sums: add into the zeroed output
             // tcgen05.ld is warp-collective: take the decision for the whole warp
@@ -698,15 +729,13 @@ general_tc_kernel(const KernelArgs a)
             tc_fence_after_sync();
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * acc_cols);
             if (a.swap) {
-                const long long t_epi = clock_now();
                 // Lanes are filters, columns pixels: this thread holds adjacent pixels of ONE map.  A
                 // warp-private shared-memory tile turns a 32-filter x 32-pixel block around so that each
                 // store instruction again writes 32 adjacent pixels of one map.
                 float* tile = helper ? reinterpret_cast<float*>(a_smem) + (size_t)(warp - 8) * 32 * kXposePitch
                                      : xpose + (size_t)(warp - 4) * 32 * kXposePitch;
-                const int b_step = split ? 3 : 1;
                 const int rpq = a.n_tile / 4;      // filter rows per lane quarter: 32 (M = 128) or 16 (M = 64, lanes 0-15)
-                const int blocks = a.mt * kTileM / 32;
+                const int blocks = a.tile_px / 32;
                 auto load_block = [&](uint32_t (&v0)[16], uint32_t (&v1)[16], int b) {
                     tmem_ld16(lane_base + (uint32_t)(b * 32), v0);
                     tmem_ld16(lane_base + (uint32_t)(b * 32 + 16), v1);
@@ -741,7 +770,7 @@ general_tc_kernel(const KernelArgs a)
                         const int kmax = min(rpq, a.K - nb * a.n_tile - quarter * rpq);   // maps of this quarter that exist
                         const float* src = tile + row_sub * kXposePitch + pg * vec;
                         if (vec == 4) {
-#pragma unroll
+#pragma unroll 4
                             for (int r = 0; r < 32; r += 4, o += 4 * plane, src += 4 * kXposePitch)
                                 if (r + row_sub < kmax) {
                                     const float4 t = *reinterpret_cast<const float4*>(src);
@@ -764,6 +793,7 @@ general_tc_kernel(const KernelArgs a)
                     }
                 };
                 uint32_t va0[16], va1[16], vb0[16], vb1[16];
+                const int b_step = split ? 3 : 1;
                 int b = split ? share : 0;
                 if (b < blocks) load_block(va0, va1, b);
                 while (b < blocks) {
@@ -779,7 +809,6 @@ general_tc_kernel(const KernelArgs a)
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0 && !helper) mbar_arrive(&acc_empty[buf]);
-                if (blockIdx.x == 0 && warp == 4 && lane == 0) a.status[6] = (unsigned)(clock_now() - t_epi);
                 continue;
             }
             int cur_m = -1;
@@ -903,7 +932,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     a.N = sh.N; a.C = sh.C; a.H = sh.H; a.W = sh.W; a.K = sh.K; a.R = sh.R; a.S = sh.S; a.P = sh.P; a.Q = sh.Q;
     a.HW = sh.H * sh.W;
     a.total_pix = sh.N * sh.H * sh.W;
-    a.n_tile = p.n_tile; a.n_blocks = p.n_blocks; a.mt = p.mt; a.nbuf = p.nbuf; a.npix = p.npix;
+    a.n_tile = p.n_tile; a.n_blocks = p.n_blocks; a.mt = p.mt; a.tile_px = p.tile_px; a.px_groups = p.px_groups; a.nbuf = p.nbuf; a.npix = p.npix;
     a.cblks = p.cblks; a.taps = p.taps;
     a.a_stages = p.a_stages; a.b_stages = p.b_stages; a.tps = p.tps;
     a.cbg = p.cbg; a.groups = (p.cblks + p.cbg - 1) / p.cbg; a.resident = p.resident; a.swap = p.swap;

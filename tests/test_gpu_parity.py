@@ -235,3 +235,18 @@ def test_relu_zero_windows_give_exact_zero(oracle):
     for algo in (ALGO_FFMA, ALGO_AUTO):
         y = run_library(x, w, entry="general", algo=algo)
         assert np.all(y[yabs == 0] == 0)
+
+
+@pytest.mark.parametrize("tile_px", [64, 96, 160, 224, 288, 352, 448, 512])
+def test_general_tf32_every_item_size(oracle, monkeypatch, tile_px):
+    """Work items of any multiple of 32 pixels (one or two MMAs per K step, ragged last item, images and rows
+    changing inside an item) give the same parity as the planner's own choice."""
+    dims = (3, 24, 19, 23, 200, 3, 3)              # 1311 pixels, two filter blocks, filters streamed
+    N, C, H, W, K, R, S = dims
+    monkeypatch.setenv("CONV2D_B200_TF32_TILE_PX", str(tile_px))
+    x, w = uniform((N, C, H, W), 421), uniform((K, C, R, S), 422)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, f"tile_px {tile_px}")
+    xi, wi = small_integers((N, C, H, W), 423), small_integers((K, C, R, S), 424)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry="general", algo=ALGO_TF32).astype(np.float64), yi_ref)
