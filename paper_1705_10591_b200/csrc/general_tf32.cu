@@ -91,7 +91,8 @@ struct Plan {
     int px_groups;    // operand-swap layout: MMAs per K step (each covers n_mma = tile_px / px_groups pixels)
     int nbuf;         // accumulator sets in tensor memory (2: write-back overlaps the next item)
     int npix;         // staged pixel rows per channel chunk
-    int cblks;        // channel blocks
+    int cblks;        // channel blocks (of the folded channels, see fold_r/fold_s)
+    int fold_r, fold_s;  // taps folded into the channel dimension: 1 or R rows, 1 or S columns
     int taps;
     int a_stages;
     int b_stages;
@@ -145,10 +146,32 @@ Plan make_plan(const Shape& sh, bool b16 = false)
     }
     const int set_cols = p.swap ? kTileM : p.n_tile;      // tensor-memory columns of one 128-pixel tile
     const int cbc = b16 ? 2 * kCB : kCB;                 // channels per staged block
-    p.cblks = (sh.C + cbc - 1) / cbc;
-    p.taps = sh.R * sh.S;
+    // Few input channels (first layers, the bridge between the one-channel and the many-channel case) would
+    // leave most of a staged channel block as zero padding.  Then taps are folded into the channel dimension:
+    // "channel" (c, r, s) of pixel j is x[c] at pixel j + r*W + s, so the contraction runs over C*fold_r*fold_s
+    // channels and only the remaining R/fold_r x S/fold_s taps are descriptor shifts.  The fold with the
+    // fewest MMAs (remaining taps x channel blocks) wins; ties keep more taps as shifts (fewer loads).
+    // Every folded tap multiplies the producers' loads, so by default only 1-3 channels are folded (measured:
+    // 3 channels 7 x 7 on 224 x 224: 0.91 ms folded, 1.06 ms not; 1 channel 5 x 5: 0.32 vs 0.40 ms; but
+    // 8 channels 3 x 3 on 112 x 112: 0.175 vs 0.093 ms).  CONV2D_B200_TF32_FOLD = 2 folds whenever C < 16.
+    p.fold_r = p.fold_s = 1;
+    const int fold_mode = env_int("CONV2D_B200_TF32_FOLD", 1);
+    if (sh.C < cbc && (fold_mode == 2 || (fold_mode == 1 && sh.C <= 3))) {
+        long long best = (long long)sh.R * sh.S * ((sh.C + cbc - 1) / cbc);
+        const int cand[3][2] = {{1, sh.S}, {sh.R, 1}, {sh.R, sh.S}};
+        for (const auto& f : cand) {
+            const long long ceff = (long long)sh.C * f[0] * f[1];
+            if (ceff > 4096) continue;
+            const long long mmas = (long long)(sh.R / f[0]) * (sh.S / f[1]) * ((ceff + cbc - 1) / cbc);
+            if (mmas < best) { best = mmas; p.fold_r = f[0]; p.fold_s = f[1]; }
+        }
+    }
+    const int c_eff = sh.C * p.fold_r * p.fold_s;
+    const int r_eff = sh.R / p.fold_r, s_eff = sh.S / p.fold_s;
+    p.cblks = (c_eff + cbc - 1) / cbc;
+    p.taps = r_eff * s_eff;
     const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
-    const long long halo = (long long)(sh.R - 1) * sh.W + (sh.S - 1);
+    const long long halo = (long long)(r_eff - 1) * sh.W + (s_eff - 1);     // shifts left to the descriptors
     const long long tiles = (total_pix + kTileM - 1) / kTileM;
     const int chunk = kCB * p.n_tile * 4;
     const int sms = 148;
@@ -260,7 +283,11 @@ Plan make_plan(const Shape& sh, bool b16 = false)
 
     const int item_cols = p.swap ? p.tile_px : p.mt * p.n_tile;     // tensor-memory columns of one accumulator set
     p.px_groups = p.swap ? (p.tile_px + 255) / 256 : p.mt;
-    p.nbuf = (2 * item_cols <= 512) ? 2 : 1;
+    {
+        const int want = env_int("CONV2D_B200_TF32_PX_GROUPS", 0);
+        if (p.swap && want > 0 && want <= 2 && p.tile_px % (16 * want) == 0 && p.tile_px / want <= 256) p.px_groups = want;
+    }
+    p.nbuf = (2 * item_cols <= 512 && env_int("CONV2D_B200_TF32_NBUF", 2) != 1) ? 2 : 1;
     p.supertiles = (int)((total_pix + p.tile_px - 1) / p.tile_px);
     // Too few tiles for the machine (e.g. 14 x 14 images): two work items per tile, each contracting half of
     // the channel-block groups and adding into a zeroed output.
@@ -284,8 +311,25 @@ size_t packed_floats(const Plan& p)
 
 // ---------------------------------------------------------------- filter re-ordering
 // wp[nb][cb][t][chunk][f][e] = tf32(w[nb*n_tile + f][cb*kCB + 4*chunk + e][t]), zero outside K, C.
+// With folded taps, channel index vc = (c*fold_r + r_in)*fold_s + s_in and tap index t = r_out*(S/fold_s) + s_out
+// stand for filter element w[k][c][r_out*fold_r + r_in][s_out*fold_s + s_in].
+struct FoldedFilter {
+    int C, R, S, fold_r, fold_s;
+    // offset of that element inside filter k's C*R*S block, or -1 for channel padding
+    __device__ __forceinline__ int offset(int vc, int t) const
+    {
+        const int frs = fold_r * fold_s;
+        const int c = vc / frs, rem = vc - c * frs;
+        if (c >= C) return -1;
+        const int r_in = rem / fold_s, s_in = rem - r_in * fold_s;
+        const int s_eff = S / fold_s;
+        const int r_out = t / s_eff, s_out = t - r_out * s_eff;
+        return (c * R + r_out * fold_r + r_in) * S + s_out * fold_s + s_in;
+    }
+};
+
 __global__ void repack_filters_kernel(const float* __restrict__ w, float* __restrict__ wp, unsigned* __restrict__ status,
-                                      int K, int C, int taps, int n_tile, int cblks, long long total)
+                                      int K, FoldedFilter ff, int taps, int n_tile, int cblks, long long total)
 {
     // the status block in front of the filters starts every (non-prepacked) call cleared
     if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
@@ -298,17 +342,18 @@ __global__ void repack_filters_kernel(const float* __restrict__ w, float* __rest
         const int t = (int)(r % taps); r /= taps;
         const int cb = (int)(r % cblks); r /= cblks;
         const int nb = (int)r;
-        const int k = nb * n_tile + f, c = cb * kCB + 4 * chunk + e;
+        const int k = nb * n_tile + f;
+        const int o = ff.offset(cb * kCB + 4 * chunk + e, t);
         float v = 0.f;
-        if (k < K && c < C) v = to_tf32_rna(__ldg(w + ((size_t)k * C + c) * taps + t));
+        if (k < K && o >= 0) v = to_tf32_rna(__ldg(w + (size_t)k * ff.C * ff.R * ff.S + o));
         wp[i] = v;
     }
 }
 
 // 16-bit variant: wp[nb][cb][t][chunk][f][e] = w[nb*n_tile + f][cb*32 + 8*chunk + e][t] (16-bit elements).
 __global__ void repack_filters_b16_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ wp,
-                                           unsigned* __restrict__ status, int K, int C, int taps, int n_tile, int cblks,
-                                           long long total)
+                                           unsigned* __restrict__ status, int K, FoldedFilter ff, int taps, int n_tile,
+                                           int cblks, long long total)
 {
     if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -320,9 +365,10 @@ __global__ void repack_filters_b16_kernel(const unsigned short* __restrict__ w, 
         const int t = (int)(r % taps); r /= taps;
         const int cb = (int)(r % cblks); r /= cblks;
         const int nb = (int)r;
-        const int k = nb * n_tile + f, c = cb * 2 * kCB + 8 * chunk + e;
+        const int k = nb * n_tile + f;
+        const int o = ff.offset(cb * 2 * kCB + 8 * chunk + e, t);
         unsigned short v = 0;
-        if (k < K && c < C) v = __ldg(w + ((size_t)k * C + c) * taps + t);
+        if (k < K && o >= 0) v = __ldg(w + (size_t)k * ff.C * ff.R * ff.S + o);
         wp[i] = v;
     }
 }
@@ -337,7 +383,10 @@ struct KernelArgs {
     int total_pix;
     int n_tile, n_blocks, mt, tile_px, px_groups, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
     int fp16;         // 16-bit operands only: 1 = IEEE half, 0 = bf16
+    int fold_r, fold_s;  // taps folded into the channel dimension (1, 1: none); R, S below are what is left as shifts
     int helpers;      // 1: warps 8-15 share the write-back of a block's last item (operand-swap layout only)
+    int pgroups;      // producer groups (1, 2 or 4): stage k is filled by group k % pgroups
+    int quad;         // fp32 operands only: producers load four adjacent pixels per 128-bit word (needs H*W % 4 == 0)
     int pair;         // 16-bit operands only: producers load two adjacent pixels per 32-bit word (needs H*W even)
     int cbg, groups;        // channel blocks per activation stage, number of such groups
     int resident;           // filters loaded once per thread block instead of streamed
@@ -354,19 +403,45 @@ struct KernelArgs {
 // [channel block][chunk][pixel] in 16-byte units.  A work unit is (channel block g, pixel jj), numbered
 // i = g * npix + jj; thread t of the 256 producers owns units first + t, first + t + 256, ...  Consecutive
 // lanes read consecutive pixels of one channel (coalesced) and write consecutive 16-byte units.
-template <bool B16, int CNT>
-__device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArgs& a, int j0, int cb0, int first, int wtid)
+template <bool B16, bool FOLD, int CNT>
+__device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArgs& a, int j0, int cb0, int first, int wtid, int nthr)
 {
     const int units = a.npix * a.cbg;
 #pragma unroll
     for (int u = 0; u < CNT; ++u) {
-        const int i = first + u * kProducers + wtid;
+        const int i = first + u * nthr + wtid;
 #pragma unroll
         for (int e = 0; e < kCB; ++e) v[u][e] = 0.f;
         if (i < units) {
             const int g = i / a.npix, jj = i - g * a.npix;
             const int j = j0 + jj;
-            if (B16 && a.pair) {
+            if (FOLD) {
+                // Folded taps: staged channel vc = (c, r, s) of pixel j is x[c] at pixel j + r*W + s (zero beyond
+                // the image: such windows belong to outputs that are dropped anyway).
+                constexpr int kPer = B16 ? 2 * kCB : kCB;             // channels per 64-byte unit
+                if (j < a.total_pix) {
+                    const int n = j / a.HW, off = j - n * a.HW;
+                    const int frs = a.fold_r * a.fold_s;
+                    const int vc0 = (cb0 + g) * kPer;
+                    int c = vc0 / frs, rem = vc0 - c * frs;
+                    int r = rem / a.fold_s, sft = rem - r * a.fold_s;
+                    const size_t base = (size_t)n * a.C * a.HW + off;
+#pragma unroll
+                    for (int e = 0; e < kPer; ++e) {
+                        const int shift = r * a.W + sft;
+                        const bool in = c < a.C && off + shift < a.HW;
+                        if (B16) {
+                            unsigned h = 0;
+                            if (in) h = __ldg(reinterpret_cast<const unsigned short*>(a.x) + base + (size_t)c * a.HW + shift);
+                            const unsigned prev = __float_as_uint(v[u][e >> 1]);
+                            v[u][e >> 1] = __uint_as_float((e & 1) ? (prev | (h << 16)) : h);
+                        } else {
+                            if (in) v[u][e] = __ldg(a.x + base + (size_t)c * a.HW + shift);
+                        }
+                        if (++sft == a.fold_s) { sft = 0; if (++r == a.fold_r) { r = 0; ++c; } }
+                    }
+                }
+            } else if (B16 && !FOLD && a.pair) {
                 // Unit = 2 adjacent pixels x 16 channels: every load is one aligned 32-bit word holding the
                 // two pixels of one channel (H*W even keeps pairs aligned and inside one image).
                 const int half_n = a.npix >> 1;
@@ -409,12 +484,12 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
 }
 
 template <bool B16, int CNT>
-__device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* dst, const KernelArgs& a, int first, int wtid)
+__device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* dst, const KernelArgs& a, int first, int wtid, int nthr)
 {
     const int units = a.npix * a.cbg;
 #pragma unroll
     for (int u = 0; u < CNT; ++u) {
-        const int i = first + u * kProducers + wtid;
+        const int i = first + u * nthr + wtid;
         if (i < units) {
             const int g = i / a.npix, jj = i - g * a.npix;
             if (B16 && a.pair) {
@@ -464,7 +539,7 @@ __device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
     return it;
 }
 
-template <bool B16>
+template <bool B16, bool FOLD>
 __global__ void __launch_bounds__(kThreads, 1)
 general_tc_kernel(const KernelArgs a)
 {
@@ -489,9 +564,11 @@ general_tc_kernel(const KernelArgs a)
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile unsigned long long* t_entry = reinterpret_cast<volatile unsigned long long*>(tmem_slot + 2);
+    if (tid == 0) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); *t_entry = t; }
 
     if (tid == 0) {
-        for (int i = 0; i < a.a_stages; ++i) { mbar_init(&a_full[i], kProducers); mbar_init(&a_empty[i], 1); }
+        for (int i = 0; i < a.a_stages; ++i) { mbar_init(&a_full[i], kProducers / a.pgroups); mbar_init(&a_empty[i], 1); }
         for (int i = 0; i < a.b_stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpilogueWarps); }
         mbar_init(tail_full, 1);
@@ -572,6 +649,11 @@ general_tc_kernel(const KernelArgs a)
             const uint32_t n_mma = (uint32_t)(a.tile_px / a.px_groups);          // operand-swap layout: pixels per MMA
             const uint32_t n_cols = a.swap ? n_mma : (uint32_t)a.n_tile;
             const uint32_t idesc = B16 ? idesc_b16(m_rows, n_cols, a.fp16 != 0) : idesc_tf32(m_rows, n_cols);
+            auto pack64 = [](uint32_t lo, uint32_t hi) {
+                uint64_t r;
+                asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+                return r;
+            };
             auto mma = [](uint32_t d, uint64_t ad, uint64_t bd, uint32_t id, bool acc) {
                 if (B16) mma_b16(d, ad, bd, id, acc); else mma_tf32(d, ad, bd, id, acc);
             };
@@ -585,8 +667,12 @@ general_tc_kernel(const KernelArgs a)
             uint32_t a_phase = 0, b_phase = 0, acc_phase0 = 0, acc_phase1 = 0;
             // diagnostics of block 0 (status words 2..5): cycles this thread waited for activations and for a
             // free accumulator set, its total cycles, its item count
-            long long wait_a = 0, wait_acc = 0;
+            long long wait_a = 0, wait_acc = 0, issue_cycles = 0;
             const long long t_begin = clock_now();
+            if (blockIdx.x == 0) {
+                unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+                a.status[6] = (unsigned)(t - *t_entry);          // ns from kernel entry to the start of the MMA loop
+            }
             int n_items = 0;
             if (a.resident) {
                 if (!mbar_wait_bounded(&b_full[0], 0u, abort_flag, a.max_polls)) alive = false;
@@ -607,6 +693,7 @@ general_tc_kernel(const KernelArgs a)
                     if (!mbar_wait_bounded(&a_full[as], a_phase, abort_flag, a.max_polls)) { alive = false; break; }
                     tc_fence_after_sync();
                     wait_a += clock_now() - tw;
+                    const long long t_issue0 = clock_now();
                     int gr = grp + ii.rot;
                     if (gr >= ii.n_groups) gr -= ii.n_groups;
                     gr += ii.g_begin;
@@ -629,11 +716,16 @@ general_tc_kernel(const KernelArgs a)
                                 uint32_t a_lo = a_lo_block + row_shift + (uint32_t)sx;
                                 uint32_t d = d0;
                                 if (a.swap) {
-                                    // M operand = the 128 filters of this stage, N operand = n_mma staged pixels
-                                    for (int m = 0; m < a.px_groups; ++m, a_lo += n_mma, d += n_mma) {
-                                        mma(d, ((uint64_t)desc_hi << 32) | b_lo, ((uint64_t)desc_hi << 32) | a_lo, idesc, accumulate != 0);
-                                        mma(d, ((uint64_t)desc_hi << 32) | (b_lo + b_kstep),
-                                                 ((uint64_t)desc_hi << 32) | (a_lo + a_kstep), idesc, true);
+                                    // M operand = the 128 filters of this stage, N operand = n_mma staged pixels.
+                                    // Straight-line code: this one thread's instruction stream is what bounds
+                                    // the MMA rate (~130 cycles per MMA with loop and address arithmetic around
+                                    // each one), so nothing is computed here that can be shared or hoisted.
+                                    const uint64_t bd0 = pack64(b_lo, desc_hi), bd1 = pack64(b_lo + b_kstep, desc_hi);
+                                    mma(d, bd0, pack64(a_lo, desc_hi), idesc, accumulate != 0);
+                                    mma(d, bd1, pack64(a_lo + a_kstep, desc_hi), idesc, true);
+                                    if (a.px_groups == 2) {
+                                        mma(d + n_mma, bd0, pack64(a_lo + n_mma, desc_hi), idesc, accumulate != 0);
+                                        mma(d + n_mma, bd1, pack64(a_lo + n_mma + a_kstep, desc_hi), idesc, true);
                                     }
                                 } else {
                                     for (int m = 0; m < a.mt; ++m, a_lo += kTileM, d += (uint32_t)a.n_tile) {
@@ -651,6 +743,7 @@ general_tc_kernel(const KernelArgs a)
                             }
                         }
                     }
+                    issue_cycles += clock_now() - t_issue0;
                     if (alive) mma_commit(&a_empty[as]);
                     if (++as == a.a_stages) { as = 0; a_phase ^= 1u; }
                 }
@@ -665,35 +758,74 @@ general_tc_kernel(const KernelArgs a)
                 a.status[3] = (unsigned)wait_acc;
                 a.status[4] = (unsigned)(clock_now() - t_begin);
                 a.status[5] = (unsigned)n_items;
+                a.status[9] = (unsigned)issue_cycles;
+                unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+                a.status[7] = (unsigned)(t - *t_entry);          // ns from kernel entry to the last MMA issued
             }
         }
     } else {
     if (producer_index(warp) >= 0) {
         // ---------------- producers: stage activations, running ahead across item boundaries
-        const int wtid = producer_index(warp) * 32 + lane;
+        // The producer warps form `pgroups` groups; stage k of the block's stage sequence is filled by group
+        // k % pgroups, so that several stages' memory round trips are in flight at once (a stage of a light
+        // problem has fewer 16-channel units than there are producer threads).
+        const int nthr = kProducers / a.pgroups;
+        const int gid = (producer_index(warp) * 32 + lane) / nthr;
+        const int wtid = (producer_index(warp) * 32 + lane) - gid * nthr;
         bool alive = true;
-        int as = 0;
-        uint32_t a_phase = 0;
+        int kstage = 0;
         const int units = a.npix * a.cbg;
         for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
             const ItemInfo ii = decode_item(a, item);
             const int j0 = ii.supertile * a.tile_px;                     // first flat pixel of the item
             // One stage = cbg consecutive channel blocks.  All loads of a pass (kUnitsPerThread units of
             // 16 channels per thread) are issued before its first store: a pass costs one memory round trip.
-            for (int grp = 0; grp < ii.n_groups && alive; ++grp) {
+            for (int grp = 0; grp < ii.n_groups && alive; ++grp, ++kstage) {
+                if (kstage % a.pgroups != gid) continue;
+                const int as = kstage % a.a_stages;
+                const uint32_t a_phase = (uint32_t)(kstage / a.a_stages) & 1u;
                 if (!mbar_wait_bounded(&a_empty[as], a_phase ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                 float4* dst = reinterpret_cast<float4*>(a_smem + (size_t)as * a_stage_bytes);
                 int gr = grp + ii.rot;
                 if (gr >= ii.n_groups) gr -= ii.n_groups;
                 gr += ii.g_begin;
-                for (int first = 0; first < units; first += kProducers * kUnitsPerThread) {
+                if (!B16 && !FOLD && a.quad) {
+                    // H*W a multiple of 4: a thread fetches 4 adjacent pixels of each of the 16 channels with
+                    // 128-bit loads (a quarter of the load instructions, which otherwise crowd the SM's memory
+                    // pipeline that the MMA instructions pass through as well) and writes four 16-channel units.
+                    const int qn = a.npix >> 2;
+                    for (int i = wtid; i < qn * a.cbg; i += nthr) {
+                        const int g = i / qn, pq = i - g * qn;
+                        const int j = j0 + 4 * pq;
+                        const int c0 = (gr * a.cbg + g) * kCB;
+                        float4 v[kCB];
+#pragma unroll
+                        for (int e = 0; e < kCB; ++e) v[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (j < a.total_pix && c0 < a.C) {
+                            const int n = j / a.HW, off = j - n * a.HW;
+                            const float* src = a.x + ((size_t)n * a.C + c0) * a.HW + off;
+#pragma unroll
+                            for (int e = 0; e < kCB; ++e)
+                                if (c0 + e < a.C) v[e] = __ldg(reinterpret_cast<const float4*>(src + (size_t)e * a.HW));
+                        }
+                        float4* d = dst + (size_t)g * kChunks * a.npix + 4 * pq;
+#pragma unroll
+                        for (int ch = 0; ch < kChunks; ++ch) {
+                            float4* dc = d + ch * a.npix;
+                            dc[0] = make_float4(to_tf32_rna(v[4 * ch].x), to_tf32_rna(v[4 * ch + 1].x), to_tf32_rna(v[4 * ch + 2].x), to_tf32_rna(v[4 * ch + 3].x));
+                            dc[1] = make_float4(to_tf32_rna(v[4 * ch].y), to_tf32_rna(v[4 * ch + 1].y), to_tf32_rna(v[4 * ch + 2].y), to_tf32_rna(v[4 * ch + 3].y));
+                            dc[2] = make_float4(to_tf32_rna(v[4 * ch].z), to_tf32_rna(v[4 * ch + 1].z), to_tf32_rna(v[4 * ch + 2].z), to_tf32_rna(v[4 * ch + 3].z));
+                            dc[3] = make_float4(to_tf32_rna(v[4 * ch].w), to_tf32_rna(v[4 * ch + 1].w), to_tf32_rna(v[4 * ch + 2].w), to_tf32_rna(v[4 * ch + 3].w));
+                        }
+                    }
+                } else
+                for (int first = 0; first < units; first += nthr * kUnitsPerThread) {
                     float v[kUnitsPerThread][kCB];
-                    load_units<B16>(v, a, j0, gr * a.cbg, first, wtid);
-                    store_units<B16>(v, dst, a, first, wtid);
+                    load_units<B16, FOLD>(v, a, j0, gr * a.cbg, first, wtid, nthr);
+                    store_units<B16>(v, dst, a, first, wtid, nthr);
                 }
                 fence_proxy_async_smem();
                 mbar_arrive(&a_full[as]);
-                if (++as == a.a_stages) { as = 0; a_phase ^= 1u; }
             }
         }
     }
@@ -867,6 +999,10 @@ general_tc_kernel(const KernelArgs a)
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, a.tmem_cols);
     if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
+    if (tid == 0 && blockIdx.x == 0) {
+        unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        a.status[8] = (unsigned)(t - *t_entry);                  // ns from kernel entry to the block's end
+    }
 }
 
 }  // namespace
@@ -908,28 +1044,32 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
 
     if (!weights_packed) {
         const long long total = (long long)packed_floats(p);
+        const FoldedFilter ff{sh.C, sh.R, sh.S, p.fold_r, p.fold_s};
         long long blocks = (total + 255) / 256;
         if (blocks > 148 * 16) blocks = 148 * 16;
         if (b16)
             repack_filters_b16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
-                static_cast<const unsigned short*>(w_any), reinterpret_cast<unsigned short*>(wp), status, sh.K, sh.C,
+                static_cast<const unsigned short*>(w_any), reinterpret_cast<unsigned short*>(wp), status, sh.K, ff,
                 p.taps, p.n_tile, p.cblks, 2 * total);
         else
-            repack_filters_kernel<<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, sh.C, p.taps, p.n_tile, p.cblks, total);
+            repack_filters_kernel<<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, ff, p.taps, p.n_tile, p.cblks, total);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
     }
 
     static bool attr_set = false;   // per process; the attribute is per function and device-wide
     if (!attr_set) {
-        if (cudaFuncSetAttribute(general_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
-            cudaFuncSetAttribute(general_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
+        if (cudaFuncSetAttribute(general_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(general_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(general_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(general_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
             return CONV2D_ERR_CUDA;
         attr_set = true;
     }
     KernelArgs a{};
     a.x = x; a.wp = wp; a.y = y; a.status = status;
-    a.N = sh.N; a.C = sh.C; a.H = sh.H; a.W = sh.W; a.K = sh.K; a.R = sh.R; a.S = sh.S; a.P = sh.P; a.Q = sh.Q;
+    a.N = sh.N; a.C = sh.C; a.H = sh.H; a.W = sh.W; a.K = sh.K; a.P = sh.P; a.Q = sh.Q;
+    a.fold_r = p.fold_r; a.fold_s = p.fold_s; a.R = sh.R / p.fold_r; a.S = sh.S / p.fold_s;
     a.HW = sh.H * sh.W;
     a.total_pix = sh.N * sh.H * sh.W;
     a.n_tile = p.n_tile; a.n_blocks = p.n_blocks; a.mt = p.mt; a.tile_px = p.tile_px; a.px_groups = p.px_groups; a.nbuf = p.nbuf; a.npix = p.npix;
@@ -942,8 +1082,19 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
     a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * p.npix * 4 >= 2 * kXposeBytes &&
                  env_int("CONV2D_B200_TF32_HELPERS", 1) != 0) ? 1 : 0;
+    a.quad = (!b16 && (sh.H * sh.W) % 4 == 0 && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
+    {
+        // as many producer groups as can each still cover a stage in one pass (one memory round trip)
+        const long long per_pass = a.quad ? kProducers : (long long)kProducers * kUnitsPerThread;
+        const long long stage_work = (long long)(a.quad ? p.npix / 4 : p.npix) * p.cbg;
+        int g = 1;
+        while (g < 4 && g * 2 <= p.a_stages && stage_work * (g * 2) <= per_pass) g *= 2;
+        a.pgroups = env_int("CONV2D_B200_TF32_PGROUPS", g);
+        if (a.pgroups != 1 && a.pgroups != 2 && a.pgroups != 4) a.pgroups = 1;
+        while (a.pgroups > p.a_stages) a.pgroups /= 2;
+    }
     a.fp16 = fp16 ? 1 : 0;
-    a.pair = (b16 && (sh.H * sh.W) % 2 == 0 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
+    a.pair = (b16 && (sh.H * sh.W) % 2 == 0 && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
     a.items = p.supertiles * p.n_blocks * p.ksplit;
     a.ksplit = p.ksplit;
     // Failure-detection test hooks (host-side injection only): a short wait bound and one filter copy that is
@@ -954,10 +1105,11 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     if (p.ksplit > 1 &&
         cudaMemsetAsync(y, 0, (size_t)sh.N * sh.K * sh.P * sh.Q * sizeof(float), stream) != cudaSuccess)
         return CONV2D_ERR_CUDA;
-    if (b16)
-        general_tc_kernel<true><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
-    else
-        general_tc_kernel<false><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
+    const bool fold = p.fold_r * p.fold_s > 1;
+    if (b16 && fold) general_tc_kernel<true, true><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
+    else if (b16) general_tc_kernel<true, false><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
+    else if (fold) general_tc_kernel<false, true><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
+    else general_tc_kernel<false, false><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
 }

@@ -201,7 +201,7 @@ def test_full_size_configs(oracle, name, algo):
 def test_auto_falls_back_to_fp32_when_no_tensor_core_instance_fits(oracle):
     """A very wide image needs a staged halo beyond shared memory: AUTO must still give the right answer."""
     import paper_1705_10591_b200 as lib
-    dims = (1, 4, 6, 6000, 8, 5, 5)
+    dims = (1, 16, 6, 6000, 8, 5, 5)
     assert not _tf32_available(dims)
     with pytest.raises(lib.Conv2dError) as e:
         lib.conv2d_fwd_workspace_size(*dims, ALGO_TF32)
@@ -250,3 +250,37 @@ def test_general_tf32_every_item_size(oracle, monkeypatch, tile_px):
     xi, wi = small_integers((N, C, H, W), 423), small_integers((K, C, R, S), 424)
     yi_ref, _ = oracle.conv2d_oracle(xi, wi)
     np.testing.assert_array_equal(run_library(xi, wi, entry="general", algo=ALGO_TF32).astype(np.float64), yi_ref)
+
+
+FEW_CHANNEL_SHAPES = [
+    # N, C, H, W, K, R, S      (taps folded into the channel dimension of the tensor-core kernel)
+    (2, 1, 20, 24, 40, 3, 3),      # one channel through the general entry: 9 folded channels, no shifts left
+    (1, 1, 30, 33, 70, 7, 7),      # 49 folded channels: four channel blocks, the last one nearly empty
+    (2, 3, 21, 26, 64, 3, 3),      # RGB first layer: 27 folded channels
+    (1, 3, 40, 40, 96, 7, 7),      # 147 folded channels
+    (2, 2, 9, 50, 33, 1, 5),       # one row of taps
+    (2, 5, 18, 7, 20, 5, 1),       # one column of taps
+    (1, 12, 16, 18, 130, 3, 3),    # 12 of 16 channels: folding the columns only (36 channels, 3 row shifts) wins
+    (3, 15, 10, 10, 16, 2, 2),
+]
+
+
+@pytest.mark.parametrize("dims", FEW_CHANNEL_SHAPES)
+@pytest.mark.parametrize("entry", ["general", "bf16"])
+def test_few_channels_folded_taps(oracle, monkeypatch, dims, entry):
+    N, C, H, W, K, R, S = dims
+    monkeypatch.setenv("CONV2D_B200_TF32_FOLD", "2")           # fold whenever a channel block is not full
+    xi, wi = small_integers((N, C, H, W), 431), small_integers((K, C, R, S), 432)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry=entry, algo=ALGO_TF32).astype(np.float64), yi_ref)
+    x, w = uniform((N, C, H, W), 433), uniform((K, C, R, S), 434)
+    if entry == "bf16":
+        from helpers import bf16_values
+        x, w = bf16_values(x)[0], bf16_values(w)[0]
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    y = run_library(x, w, entry=entry, algo=ALGO_TF32)
+    assert_parity(y, y_ref, yabs, TF32_TOL if entry == "general" else 1e-5, f"folded {entry} {dims}")
+    monkeypatch.setenv("CONV2D_B200_TF32_FOLD", "0")          # same operands, contraction in another order
+    y_plain = run_library(x, w, entry=entry, algo=ALGO_TF32)
+    assert_parity(y_plain, y_ref, yabs, TF32_TOL if entry == "general" else 1e-5, f"unfolded {entry} {dims}")
+    assert_parity(y, y_plain.astype(np.float64), yabs, 2e-5, f"folded vs unfolded {entry} {dims}")
