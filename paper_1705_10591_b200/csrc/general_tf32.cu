@@ -331,6 +331,7 @@ struct FoldedFilter {
 __global__ void repack_filters_kernel(const float* __restrict__ w, float* __restrict__ wp, unsigned* __restrict__ status,
                                       int K, FoldedFilter ff, int taps, int n_tile, int cblks, long long total)
 {
+    grid_dep_launch();      // the convolution kernel may set itself up while this one runs
     // the status block in front of the filters starts every (non-prepacked) call cleared
     if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -355,6 +356,7 @@ __global__ void repack_filters_b16_kernel(const unsigned short* __restrict__ w, 
                                            unsigned* __restrict__ status, int K, FoldedFilter ff, int taps, int n_tile,
                                            int cblks, long long total)
 {
+    grid_dep_launch();
     if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
@@ -581,6 +583,11 @@ general_tc_kernel(const KernelArgs a)
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
+    // Everything above touched only this block's shared and tensor memory; it may overlap the tail of the
+    // preceding kernel on the stream (the filter re-ordering of this call, or the previous call).  From here
+    // on global memory is read and written.
+    grid_dep_launch();
+    grid_dep_wait();
 
     // Work item -> (supertile, filter block); blocks rotate the order of the channel-block groups by the
     // item number, so that at any moment they stream different parts of the filter bank.
@@ -1105,11 +1112,22 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     if (p.ksplit > 1 &&
         cudaMemsetAsync(y, 0, (size_t)sh.N * sh.K * sh.P * sh.Q * sizeof(float), stream) != cudaSuccess)
         return CONV2D_ERR_CUDA;
+    // Programmatic dependent launch: the kernel's set-up (barriers, tensor-memory allocation) overlaps the
+    // tail of whatever kernel precedes it on the stream; it waits for that kernel before it touches global memory.
     const bool fold = p.fold_r * p.fold_s > 1;
-    if (b16 && fold) general_tc_kernel<true, true><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
-    else if (b16) general_tc_kernel<true, false><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
-    else if (fold) general_tc_kernel<false, true><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
-    else general_tc_kernel<false, false><<<(unsigned)p.grid, kThreads, p.smem_bytes, stream>>>(a);
+    void (*kernel)(KernelArgs) = b16 ? (fold ? general_tc_kernel<true, true> : general_tc_kernel<true, false>)
+                                     : (fold ? general_tc_kernel<false, true> : general_tc_kernel<false, false>);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = p.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = env_int("CONV2D_B200_TF32_PDL", 1) != 0 ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, a) != cudaSuccess) return CONV2D_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
 }

@@ -53,6 +53,15 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     return false;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// grid_dep_launch: the next kernel on the stream (if it was launched with programmatic stream
+// serialization) may start to be scheduled now instead of when this grid has drained.
+// grid_dep_wait: returns when the preceding grid has completed and its memory operations are visible;
+// it must come before the first access to anything that grid may have written or may still be reading.
+// Both do nothing in a kernel that was launched the ordinary way.
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- proxies and bulk copies
 // Makes this thread's earlier shared-memory writes visible to the async proxy (TMA, tcgen05.mma).
 __device__ __forceinline__ void fence_proxy_async_smem()
