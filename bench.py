@@ -292,6 +292,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
     ap.add_argument("--no-general", action="store_true", help="skip the general-case configurations")
+    ap.add_argument("--operand", default="fp32", choices=["fp32", "bf16"],
+                    help="general-case workloads only: bf16 runs the 16-bit operand entry on the same values rounded to bf16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()
@@ -327,7 +329,11 @@ def main():
     w_host = torch.from_numpy(w).pin_memory()
     xd, wd = x_host.to(dev), w_host.to(dev)
     yd = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), device=dev, dtype=torch.float32)
-    algo = lib.ALGO_FFMA if single else lib.ALGO_AUTO
+    b16 = args.operand == "bf16" and not single
+    if b16:
+        xd16, wd16 = xd.to(torch.bfloat16).contiguous(), wd.to(torch.bfloat16).contiguous()
+        args.no_e2e = True            # the host-buffer entry takes fp32 tensors only
+    algo = lib.ALGO_FFMA if single else (lib.ALGO_16BIT if b16 else lib.ALGO_AUTO)
     ws_bytes = 0 if single else lib.conv2d_fwd_workspace_size(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, algo)
     ws = torch.zeros(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream().cuda_stream
@@ -337,6 +343,9 @@ def main():
         if single:
             lib.conv2d_fwd_single_channel(xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.H, cfg.W,
                                           cfg.K, cfg.R, cfg.S, 0, 0, 0, stream)
+        elif b16:
+            lib.conv2d_fwd_general_16bit(xd16.data_ptr(), wd16.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
+                                         cfg.K, cfg.R, cfg.S, lib.OPERAND_BF16, ws.data_ptr(), ws_bytes, 0, stream)
         else:
             lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
                                    cfg.K, cfg.R, cfg.S, algo, ws.data_ptr(), ws_bytes, 0, stream)
@@ -348,6 +357,7 @@ def main():
         torch.cuda.synchronize()
 
     working_set = cfg.compulsory_bytes
+    algorithmic_bytes = cfg.compulsory_bytes if not b16 else 2 * (x.size + w.size) + 4 * yd.numel()
     flush_between = working_set < 2 * 126 * 1024 * 1024
     for _ in range(args.warmup):
         step()
@@ -390,23 +400,23 @@ def main():
     # ---- roofline of the dominant kernel (per launch = one step)
     t_kernel_s = ms_per_step * 1e-3
     fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # TFLOP/s at max clock
-    t_hbm = cfg.compulsory_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_hbm = algorithmic_bytes / (peaks["hbm_gbs"] * 1e9)
     if single:
         t_pipe, pipe_name, pipe_peak = cfg.flops / (fp32_peak * 1e12), "alu", fp32_peak
     else:
-        pipe_peak = peaks["bf16_tflops"] / 2.0
+        pipe_peak = peaks["bf16_tflops"] if b16 else peaks["bf16_tflops"] / 2.0
         t_pipe, pipe_name = cfg.flops / (pipe_peak * 1e12), "tensor"
     if t_pipe >= t_hbm:
         roof = {"bound": pipe_name, "achieved": cfg.flops / t_kernel_s / 1e12, "peak": pipe_peak, "unit": "TFLOP/s"}
     else:
-        roof = {"bound": "hbm", "achieved": cfg.compulsory_bytes / t_kernel_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        roof = {"bound": "hbm", "achieved": algorithmic_bytes / t_kernel_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof.update({
         "traffic": None, "peaks": peaks["source"],
-        "algorithmic_bytes_per_launch": cfg.compulsory_bytes, "flops_per_launch": cfg.flops,
-        "hbm_gbs_achieved": cfg.compulsory_bytes / t_kernel_s / 1e9,
-        "hbm_frac_of_measured": cfg.compulsory_bytes / t_kernel_s / 1e9 / peaks["hbm_gbs"],
-        "hbm_frac_of_nominal_8tbs": cfg.compulsory_bytes / t_kernel_s / 1e9 / 8000.0,
+        "algorithmic_bytes_per_launch": algorithmic_bytes, "flops_per_launch": cfg.flops,
+        "hbm_gbs_achieved": algorithmic_bytes / t_kernel_s / 1e9,
+        "hbm_frac_of_measured": algorithmic_bytes / t_kernel_s / 1e9 / peaks["hbm_gbs"],
+        "hbm_frac_of_nominal_8tbs": algorithmic_bytes / t_kernel_s / 1e9 / 8000.0,
         "alu_tflops_achieved": cfg.flops / t_kernel_s / 1e12,
         "alu_frac_at_max_clock": cfg.flops / t_kernel_s / 1e12 / fp32_peak,
     })
@@ -420,8 +430,8 @@ def main():
     result = {
         "metric": "conv_fwd_gflops", "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": cfg.name, **cfg.as_dict(), "parallelism": f"replicas x{world}",
+        "vs_baseline": None, "dtype": "bf16" if b16 else ("f32" if single else "tf32"), "data": "synthetic",
+        "config": {"workload": cfg.name, "operand": args.operand if not single else "fp32", **cfg.as_dict(), "parallelism": f"replicas x{world}",
                    "l2": "flushed between timed steps" if flush_between else
                          "inputs+outputs per step (2.2 GB) exceed the 126 MB L2"},
         "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "power_w_max")},
