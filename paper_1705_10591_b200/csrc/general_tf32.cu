@@ -328,50 +328,77 @@ struct FoldedFilter {
     }
 };
 
-__global__ void repack_filters_kernel(const float* __restrict__ w, float* __restrict__ wp, unsigned* __restrict__ status,
-                                      int K, FoldedFilter ff, int taps, int n_tile, int cblks, long long total)
+// One thread per (filter block, channel block, 16-byte chunk, filter, element) walks over the taps: its reads
+// are the contiguous taps of one (filter, channel) pair (cached lines are reused from tap to tap), and for
+// each tap a warp writes 32 adjacent elements.  T = float (rounded to TF32) with 4 elements per chunk, or a
+// 16-bit pattern with 8.
+template <typename T, int EPC>
+__global__ void repack_filters_kernel(const T* __restrict__ w, T* __restrict__ wp, unsigned* __restrict__ status,
+                                      int K, FoldedFilter ff, int taps, int n_tile, int cblks, long long threads_total)
 {
     grid_dep_launch();      // the convolution kernel may set itself up while this one runs
     // the status block in front of the filters starts every (non-prepacked) call cleared
     if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
+    const bool folded = ff.fold_r * ff.fold_s > 1;
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < threads_total; i += stride) {
         long long r = i;
-        const int e = (int)(r % 4); r /= 4;
+        const int e = (int)(r % EPC); r /= EPC;
         const int f = (int)(r % n_tile); r /= n_tile;
         const int chunk = (int)(r % kChunks); r /= kChunks;
-        const int t = (int)(r % taps); r /= taps;
         const int cb = (int)(r % cblks); r /= cblks;
         const int nb = (int)r;
         const int k = nb * n_tile + f;
-        const int o = ff.offset(cb * kCB + 4 * chunk + e, t);
-        float v = 0.f;
-        if (k < K && o >= 0) v = to_tf32_rna(__ldg(w + (size_t)k * ff.C * ff.R * ff.S + o));
-        wp[i] = v;
+        const int vc = (cb * kChunks + chunk) * EPC + e;
+        const T* src = w + (size_t)k * ff.C * ff.R * ff.S;
+        T* dst = wp + ((((size_t)nb * cblks + cb) * taps * kChunks + chunk) * n_tile + f) * EPC + e;
+        const size_t tap_stride = (size_t)kChunks * n_tile * EPC;
+        const bool live = k < K && (folded ? vc < ff.C * ff.fold_r * ff.fold_s : vc < ff.C);
+        for (int t = 0; t < taps; ++t, dst += tap_stride) {
+            T v = T(0);
+            if (live) {
+                const int o = folded ? ff.offset(vc, t) : vc * taps + t;
+                v = __ldg(src + o);
+                if (sizeof(T) == 4) v = (T)to_tf32_rna((float)v);
+            }
+            *dst = v;
+        }
     }
 }
 
-// 16-bit variant: wp[nb][cb][t][chunk][f][e] = w[nb*n_tile + f][cb*32 + 8*chunk + e][t] (16-bit elements).
-__global__ void repack_filters_b16_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ wp,
-                                           unsigned* __restrict__ status, int K, FoldedFilter ff, int taps, int n_tile,
-                                           int cblks, long long total)
+// Re-ordering through shared memory for unfolded filters: a block takes 8 filters x one channel block x all
+// taps.  Its reads are runs of (channels per block) x taps contiguous elements per filter, its writes runs of
+// 8 filters x EPC elements (128 bytes with fp32) per (tap, chunk): both sides coalesced.
+template <typename T, int EPC>
+__global__ void repack_filters_tiled_kernel(const T* __restrict__ w, T* __restrict__ wp, unsigned* __restrict__ status,
+                                            int K, int C, int taps, int n_tile, int cblks)
 {
+    extern __shared__ __align__(16) unsigned char repack_smem[];
+    T* tile = reinterpret_cast<T*>(repack_smem);                 // [8][cpb * taps]
     grid_dep_launch();
-    if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-        long long r = i;
-        const int e = (int)(r % 8); r /= 8;
-        const int f = (int)(r % n_tile); r /= n_tile;
-        const int chunk = (int)(r % kChunks); r /= kChunks;
-        const int t = (int)(r % taps); r /= taps;
-        const int cb = (int)(r % cblks); r /= cblks;
-        const int nb = (int)r;
-        const int k = nb * n_tile + f;
-        const int o = ff.offset(cb * 2 * kCB + 8 * chunk + e, t);
-        unsigned short v = 0;
-        if (k < K && o >= 0) v = __ldg(w + (size_t)k * ff.C * ff.R * ff.S + o);
-        wp[i] = v;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
+    constexpr int cpb = kChunks * EPC;                           // channels per block
+    const int cb = blockIdx.y, k0 = blockIdx.x * 8, c0 = cb * cpb;
+    const int row = cpb * taps;
+    const int c_live = min(cpb, C - c0) * taps;                  // elements of a filter's run that exist
+#pragma unroll 4
+    for (int idx = threadIdx.x; idx < 8 * row; idx += blockDim.x) {       // (independent loads: several in flight)
+        const int kk = idx / row, rem = idx - kk * row;
+        T v = T(0);
+        if (k0 + kk < K && rem < c_live) {
+            v = __ldg(w + ((size_t)(k0 + kk) * C + c0) * taps + rem);
+            if (sizeof(T) == 4) v = (T)to_tf32_rna((float)v);
+        }
+        tile[idx] = v;
+    }
+    __syncthreads();
+    const int nb = k0 / n_tile, f0 = k0 - nb * n_tile;
+    T* dst = wp + ((size_t)nb * cblks + cb) * taps * kChunks * n_tile * EPC;
+    for (int idx = threadIdx.x; idx < 8 * row; idx += blockDim.x) {
+        const int e = idx % EPC, kk = (idx / EPC) % 8;
+        const int rest = idx / (EPC * 8);
+        const int chunk = rest % kChunks, t = rest / kChunks;
+        dst[(((size_t)t * kChunks + chunk) * n_tile + f0 + kk) * EPC + e] = tile[kk * row + (chunk * EPC + e) * taps + t];
     }
 }
 
@@ -1039,6 +1066,24 @@ size_t b16_workspace_bytes(const Shape& sh)
 }
 
 namespace {
+// Launch with programmatic stream serialization: the kernel may be scheduled while the preceding kernel on the
+// stream drains; it calls grid_dep_wait() before it touches global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = env_int("CONV2D_B200_TF32_PDL", 1) != 0 ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* y, const Shape& sh, bool b16, bool fp16,
                                    void* workspace, bool weights_packed, cudaStream_t stream)
 {
@@ -1052,14 +1097,30 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     if (!weights_packed) {
         const long long total = (long long)packed_floats(p);
         const FoldedFilter ff{sh.C, sh.R, sh.S, p.fold_r, p.fold_s};
-        long long blocks = (total + 255) / 256;
+        const long long lanes = total / p.taps * (b16 ? 2 : 1);      // one thread per element of a tap's slice
+        long long blocks = (lanes + 255) / 256;
         if (blocks > 148 * 16) blocks = 148 * 16;
-        if (b16)
-            repack_filters_b16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+        const size_t tile_bytes = (size_t)8 * kCB * 4 * p.taps;       // 8 filters x one channel block x taps
+        if (p.fold_r * p.fold_s == 1 && tile_bytes <= 48 * 1024 && p.n_tile % 8 == 0) {
+            const dim3 grid((unsigned)(p.n_blocks * p.n_tile / 8), (unsigned)p.cblks);
+            int threads = (8 * kCB * p.taps / 4 + 31) / 32 * 32;          // about four elements per thread
+            threads = threads < 128 ? 128 : (threads > 1024 ? 1024 : threads);
+            // (launched the ordinary way: it starts only when the previous call's kernel, which may still
+            // be reading the workspace, has finished; measured no gain from overlapping its launch)
+            if (b16)
+                repack_filters_tiled_kernel<unsigned short, 8><<<grid, threads, tile_bytes, stream>>>(
+                    static_cast<const unsigned short*>(w_any), reinterpret_cast<unsigned short*>(wp), status, sh.K, sh.C,
+                    p.taps, p.n_tile, p.cblks);
+            else
+                repack_filters_tiled_kernel<float, 4><<<grid, threads, tile_bytes, stream>>>(w, wp, status, sh.K, sh.C, p.taps,
+                                                                                             p.n_tile, p.cblks);
+        } else if (b16)
+            repack_filters_kernel<unsigned short, 8><<<(unsigned)blocks, 256, 0, stream>>>(
                 static_cast<const unsigned short*>(w_any), reinterpret_cast<unsigned short*>(wp), status, sh.K, ff,
-                p.taps, p.n_tile, p.cblks, 2 * total);
+                p.taps, p.n_tile, p.cblks, lanes);
         else
-            repack_filters_kernel<<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, ff, p.taps, p.n_tile, p.cblks, total);
+            repack_filters_kernel<float, 4><<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, ff, p.taps,
+                                                                                  p.n_tile, p.cblks, lanes);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
     }
@@ -1117,17 +1178,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     const bool fold = p.fold_r * p.fold_s > 1;
     void (*kernel)(KernelArgs) = b16 ? (fold ? general_tc_kernel<true, true> : general_tc_kernel<true, false>)
                                      : (fold ? general_tc_kernel<false, true> : general_tc_kernel<false, false>);
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)p.grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = p.smem_bytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = env_int("CONV2D_B200_TF32_PDL", 1) != 0 ? 1 : 0;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kernel, a) != cudaSuccess) return CONV2D_ERR_CUDA;
+    if (launch_pdl(kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, stream, a) != cudaSuccess) return CONV2D_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
 }
