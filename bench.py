@@ -241,6 +241,7 @@ def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
             }
             if packed is not None:
                 entry["ms_warm_l2_weights_prepacked"] = packed
+                entry["roofline"]["pipe_frac_warm_weights_prepacked"] = t_pipe / packed
             out.append(entry)
         del xd, wd, yd, xd16, wd16
     return out
