@@ -93,6 +93,7 @@ struct Plan {
     int npix;         // staged pixel rows per channel chunk
     int cblks;        // channel blocks (of the folded channels, see fold_r/fold_s)
     int fold_r, fold_s;  // taps folded into the channel dimension: 1 or R rows, 1 or S columns
+    int patch_w, patch_tw, patch_rows, patch_cols;   // patch addressing (patch_w = 0: flat pixel run), see ItemGeom
     int taps;
     int a_stages;
     int b_stages;
@@ -171,7 +172,39 @@ Plan make_plan(const Shape& sh, bool b16 = false)
     p.cblks = (c_eff + cbc - 1) / cbc;
     p.taps = r_eff * s_eff;
     const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
-    const long long halo = (long long)(r_eff - 1) * sh.W + (s_eff - 1);     // shifts left to the descriptors
+    // Addressing mode.  In the flat pixel run the staged halo is (R-1) whole image rows; once that exceeds a
+    // 256-pixel item the item is cut as a rectangle of the image instead (patch_w columns wide, of which the
+    // first patch_tw produce outputs), whose halo is (R-1) patch rows.  The patch width with the least staged
+    // pixels per output wins.
+    p.patch_w = p.patch_tw = p.patch_rows = p.patch_cols = 0;
+    const long long flat_halo = (long long)(r_eff - 1) * sh.W + (s_eff - 1);
+    const int patch_mode = env_int("CONV2D_B200_TF32_PATCH", 1);       // 0 never, 1 when the flat halo is large, 2 always
+    if (p.swap && p.fold_r * p.fold_s == 1 && patch_mode != 0) {
+        double best_ratio = 0;
+        for (int wp = 32; wp <= 128; wp *= 2) {
+            const int tw = (wp - (s_eff - 1)) / 4 * 4;
+            if (tw < 4) continue;
+            const int th = 448 / wp > 0 ? 448 / wp : 1;                       // rows of a typical item
+            const long long rows_p = (sh.P + th - 1) / th, cols_p = (sh.Q + tw - 1) / tw;
+            const double ratio = (double)(rows_p * (th + r_eff - 1)) * wp * cols_p / ((double)sh.P * sh.Q);
+            if (p.patch_w == 0 || ratio < best_ratio) { best_ratio = ratio; p.patch_w = wp; p.patch_tw = tw; }
+        }
+        // staged pixels per output of the flat run, for a 448-pixel item.  Patches also cost extra work items at
+        // the ragged right edge and a narrower store run, so they must win clearly (measured: 3 x 3 on 224 x 224,
+        // ratio 2.0 flat vs 1.3 in patches, is 10 % faster flat; 3 x 3 on 512 x 512, 3.3 vs 1.3, 20 % faster in patches;
+        // 7 x 7 on 224 x 224, 4.2 vs 2.2, 20 % faster in patches).
+        const double flat_ratio = (448.0 + flat_halo) / 448.0 * ((double)sh.H * sh.W) / ((double)sh.P * sh.Q);
+        if (patch_mode == 1 && !(flat_ratio > 1.75 * best_ratio)) p.patch_w = p.patch_tw = 0;
+        if (p.patch_w) p.patch_cols = (sh.Q + p.patch_tw - 1) / p.patch_tw;
+    }
+    const long long halo = p.patch_w ? (long long)(r_eff - 1) * p.patch_w + (s_eff - 1) : flat_halo;
+    // work items along the pixels for an item of px pixels (0: px is not possible in this mode)
+    auto pixel_items = [&](int px) -> long long {
+        if (!p.patch_w) return (total_pix + px - 1) / px;
+        if (px % p.patch_w) return 0;
+        const int th = px / p.patch_w;
+        return (long long)sh.N * ((sh.P + th - 1) / th) * p.patch_cols;
+    };
     const long long tiles = (total_pix + kTileM - 1) / kTileM;
     const int chunk = kCB * p.n_tile * 4;
     const int sms = 148;
@@ -232,7 +265,8 @@ Plan make_plan(const Shape& sh, bool b16 = false)
                 if (px % (16 * groups)) continue;
                 const int npix = npix_of(px);
                 if (npix > 16000 || smem_need(2, npix, p.n_tile, 2, 1, 1) > kLimit) continue;
-                const long long items = (total_pix + px - 1) / px * p.n_blocks;
+                if (pixel_items(px) == 0) continue;
+                const long long items = pixel_items(px) * p.n_blocks;
                 const long long rounds = (items + sms - 1) / sms;
                 const int nbuf = 2 * px <= 512 ? 2 : 1;
                 const double mma_step = groups * ((px / groups) / 2.0 > 64.0 ? (px / groups) / 2.0 : 64.0);
@@ -288,7 +322,9 @@ Plan make_plan(const Shape& sh, bool b16 = false)
         if (p.swap && want > 0 && want <= 2 && p.tile_px % (16 * want) == 0 && p.tile_px / want <= 256) p.px_groups = want;
     }
     p.nbuf = (2 * item_cols <= 512 && env_int("CONV2D_B200_TF32_NBUF", 2) != 1) ? 2 : 1;
-    p.supertiles = (int)((total_pix + p.tile_px - 1) / p.tile_px);
+    if (p.patch_w) p.patch_rows = (sh.P + p.tile_px / p.patch_w - 1) / (p.tile_px / p.patch_w);
+    if (pixel_items(p.tile_px) <= 0 || pixel_items(p.tile_px) > 0x7fffffffLL) return p;
+    p.supertiles = (int)pixel_items(p.tile_px);
     // Too few tiles for the machine (e.g. 14 x 14 images): two work items per tile, each contracting half of
     // the channel-block groups and adding into a zeroed output.
     const int n_groups = (p.cblks + p.cbg - 1) / p.cbg;
@@ -411,6 +447,9 @@ struct KernelArgs {
     int HW;
     int total_pix;
     int n_tile, n_blocks, mt, tile_px, px_groups, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
+    int patch_w, patch_tw, patch_rows, patch_cols;   // patch addressing (PATCH kernels): staged row pitch, valid output
+                                                      // columns per patch row, patches per image down and across
+    int row_pitch;    // pixels between vertically adjacent taps in the staged sequence: W, or patch_w
     int fp16;         // 16-bit operands only: 1 = IEEE half, 0 = bf16
     int fold_r, fold_s;  // taps folded into the channel dimension (1, 1: none); R, S below are what is left as shifts
     int helpers;      // 1: warps 8-15 share the write-back of a block's last item (operand-swap layout only)
@@ -428,12 +467,59 @@ struct KernelArgs {
     unsigned tmem_cols;
 };
 
+// Where the staged pixel sequence of a work item lives in the image.
+//   flat  (PATCH = false): pixels of the whole batch numbered j = (n*H + h)*W + w; an item is the run
+//          [j0, j0 + tile_px) plus its halo; vertically adjacent taps are W pixels apart.
+//   patch (PATCH = true): an item is a rectangle of patch_rows... rows x patch_w columns of one image starting at
+//          (row0, col0), stored row after row with pitch patch_w (the staged halo adds R-1 rows); vertically adjacent
+//          taps are patch_w pixels apart.  Columns >= patch_tw of a patch row only feed outputs of the next patch and
+//          are dropped.  This keeps the halo small on wide images, for which the flat run would not fit on chip.
+struct ItemGeom {
+    int j0;             // flat: first pixel
+    int n, row0, col0;  // patch: image and top-left corner
+};
+// Staged pixel jj -> (image n, offset inside one H*W plane); false when the pixel lies outside the batch / the image.
+template <bool PATCH>
+__device__ __forceinline__ bool staged_pixel(const KernelArgs& a, const ItemGeom& g, int jj, int& n, int& off)
+{
+    if (PATCH) {
+        const int prow = jj / a.patch_w, pcol = jj - prow * a.patch_w;
+        const int h = g.row0 + prow, wc = g.col0 + pcol;
+        n = g.n;
+        off = h * a.W + wc;
+        return h < a.H && wc < a.W;
+    }
+    const int j = g.j0 + jj;
+    n = j / a.HW;
+    off = j - n * a.HW;
+    return j < a.total_pix;
+}
+// Accumulator column jj -> output (n, p, q); false when that output does not exist (window wraps over an edge).
+template <bool PATCH>
+__device__ __forceinline__ bool output_pixel(const KernelArgs& a, const ItemGeom& g, int jj, int& n, int& p, int& q)
+{
+    if (PATCH) {
+        const int prow = jj / a.patch_w, pcol = jj - prow * a.patch_w;
+        n = g.n;
+        p = g.row0 + prow;
+        q = g.col0 + pcol;
+        return pcol < a.patch_tw && p < a.P && q < a.Q;
+    }
+    const int j = g.j0 + jj;
+    if (j >= a.total_pix) return false;
+    n = j / a.HW;
+    const int off = j - n * a.HW;
+    p = off / a.W;
+    q = off - p * a.W;
+    return p < a.P && q < a.Q;
+}
+
 // Producer helpers.  A stage holds `cbg` channel blocks of kCB channels for npix pixels, laid out
 // [channel block][chunk][pixel] in 16-byte units.  A work unit is (channel block g, pixel jj), numbered
 // i = g * npix + jj; thread t of the 256 producers owns units first + t, first + t + 256, ...  Consecutive
 // lanes read consecutive pixels of one channel (coalesced) and write consecutive 16-byte units.
-template <bool B16, bool FOLD, int CNT>
-__device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArgs& a, int j0, int cb0, int first, int wtid, int nthr)
+template <bool B16, bool FOLD, bool PATCH, int CNT>
+__device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArgs& a, const ItemGeom& geom, int cb0, int first, int wtid, int nthr)
 {
     const int units = a.npix * a.cbg;
 #pragma unroll
@@ -443,13 +529,12 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
         for (int e = 0; e < kCB; ++e) v[u][e] = 0.f;
         if (i < units) {
             const int g = i / a.npix, jj = i - g * a.npix;
-            const int j = j0 + jj;
             if (FOLD) {
                 // Folded taps: staged channel vc = (c, r, s) of pixel j is x[c] at pixel j + r*W + s (zero beyond
                 // the image: such windows belong to outputs that are dropped anyway).
                 constexpr int kPer = B16 ? 2 * kCB : kCB;             // channels per 64-byte unit
-                if (j < a.total_pix) {
-                    const int n = j / a.HW, off = j - n * a.HW;
+                int n, off;
+                if (staged_pixel<false>(a, geom, jj, n, off)) {
                     const int frs = a.fold_r * a.fold_s;
                     const int vc0 = (cb0 + g) * kPer;
                     int c = vc0 / frs, rem = vc0 - c * frs;
@@ -475,10 +560,9 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
                 // two pixels of one channel (H*W even keeps pairs aligned and inside one image).
                 const int half_n = a.npix >> 1;
                 const int h = jj / half_n, pp = jj - h * half_n;
-                const int jp = j0 + 2 * pp;
                 const int c0 = (cb0 + g) * 2 * kCB + kCB * h;
-                if (jp < a.total_pix && c0 < a.C) {
-                    const int n = jp / a.HW, off = jp - n * a.HW;
+                int n, off;
+                if (staged_pixel<PATCH>(a, geom, 2 * pp, n, off) && c0 < a.C) {
                     const unsigned short* src = reinterpret_cast<const unsigned short*>(a.x) + ((size_t)n * a.C + c0) * a.HW + off;
 #pragma unroll
                     for (int e = 0; e < kCB; ++e)
@@ -487,8 +571,8 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
             } else if (B16) {
                 // 32 16-bit channels of this pixel, packed two per 32-bit word (lower channel in the low half)
                 const int c0 = (cb0 + g) * 2 * kCB;
-                if (j < a.total_pix && c0 < a.C) {
-                    const int n = j / a.HW, off = j - n * a.HW;
+                int n, off;
+                if (staged_pixel<PATCH>(a, geom, jj, n, off) && c0 < a.C) {
                     const unsigned short* src = reinterpret_cast<const unsigned short*>(a.x) + ((size_t)n * a.C + c0) * a.HW + off;
 #pragma unroll
                     for (int e = 0; e < kCB; ++e) {
@@ -500,8 +584,8 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
                 }
             } else {
                 const int c0 = (cb0 + g) * kCB;
-                if (j < a.total_pix && c0 < a.C) {
-                    const int n = j / a.HW, off = j - n * a.HW;
+                int n, off;
+                if (staged_pixel<PATCH>(a, geom, jj, n, off) && c0 < a.C) {
                     const float* src = a.x + ((size_t)n * a.C + c0) * a.HW + off;
 #pragma unroll
                     for (int e = 0; e < kCB; ++e)
@@ -554,6 +638,7 @@ __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* 
 // (zeroed beforehand); 0 + a + b does not depend on the order, so the result stays deterministic.
 struct ItemInfo {
     int supertile, nb, g_begin, n_groups, rot;
+    ItemGeom geom;
 };
 __device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
 {
@@ -565,10 +650,20 @@ __device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
     it.g_begin = part * a.groups / a.ksplit;
     it.n_groups = (part + 1) * a.groups / a.ksplit - it.g_begin;
     it.rot = rest % it.n_groups;        // blocks stream the filter bank in rotated order (see kernel)
+    it.geom.j0 = it.supertile * a.tile_px;
+    it.geom.n = it.geom.row0 = it.geom.col0 = 0;
+    if (a.patch_w) {
+        const int per_image = a.patch_rows * a.patch_cols;
+        it.geom.n = it.supertile / per_image;
+        const int rem = it.supertile - it.geom.n * per_image;
+        const int pr = rem / a.patch_cols;
+        it.geom.row0 = pr * (a.tile_px / a.patch_w);
+        it.geom.col0 = (rem - pr * a.patch_cols) * a.patch_tw;
+    }
     return it;
 }
 
-template <bool B16, bool FOLD>
+template <bool B16, bool FOLD, bool PATCH>
 __global__ void __launch_bounds__(kThreads, 1)
 general_tc_kernel(const KernelArgs a)
 {
@@ -769,7 +864,7 @@ general_tc_kernel(const KernelArgs a)
                                     }
                                 }
                                 accumulate = 1;
-                                if (++sx == a.S) { sx = 0; row_shift += (uint32_t)a.W; }
+                                if (++sx == a.S) { sx = 0; row_shift += (uint32_t)a.row_pitch; }
                             }
                             if (!a.resident) {
                                 mma_commit(&b_empty[bs]);   // frees the filter stage when these MMAs have read it
@@ -811,7 +906,6 @@ general_tc_kernel(const KernelArgs a)
         const int units = a.npix * a.cbg;
         for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
             const ItemInfo ii = decode_item(a, item);
-            const int j0 = ii.supertile * a.tile_px;                     // first flat pixel of the item
             // One stage = cbg consecutive channel blocks.  All loads of a pass (kUnitsPerThread units of
             // 16 channels per thread) are issued before its first store: a pass costs one memory round trip.
             for (int grp = 0; grp < ii.n_groups && alive; ++grp, ++kstage) {
@@ -830,13 +924,12 @@ general_tc_kernel(const KernelArgs a)
                     const int qn = a.npix >> 2;
                     for (int i = wtid; i < qn * a.cbg; i += nthr) {
                         const int g = i / qn, pq = i - g * qn;
-                        const int j = j0 + 4 * pq;
                         const int c0 = (gr * a.cbg + g) * kCB;
                         float4 v[kCB];
 #pragma unroll
                         for (int e = 0; e < kCB; ++e) v[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (j < a.total_pix && c0 < a.C) {
-                            const int n = j / a.HW, off = j - n * a.HW;
+                        int n, off;
+                        if (staged_pixel<PATCH>(a, ii.geom, 4 * pq, n, off) && c0 < a.C) {
                             const float* src = a.x + ((size_t)n * a.C + c0) * a.HW + off;
 #pragma unroll
                             for (int e = 0; e < kCB; ++e)
@@ -855,7 +948,7 @@ general_tc_kernel(const KernelArgs a)
                 } else
                 for (int first = 0; first < units; first += nthr * kUnitsPerThread) {
                     float v[kUnitsPerThread][kCB];
-                    load_units<B16, FOLD>(v, a, j0, gr * a.cbg, first, wtid, nthr);
+                    load_units<B16, FOLD, PATCH>(v, a, ii.geom, gr * a.cbg, first, wtid, nthr);
                     store_units<B16>(v, dst, a, first, wtid, nthr);
                 }
                 fence_proxy_async_smem();
@@ -883,7 +976,6 @@ general_tc_kernel(const KernelArgs a)
             const uint32_t acc_phase = (uint32_t)(li / a.nbuf) & 1u;
             const bool split = a.helpers && li == n_local - 1;
             const ItemInfo ii = decode_item(a, item);
-            const int j0 = ii.supertile * a.tile_px;
             const int nb = ii.nb;
             const bool add = a.ksplit > 1;                   // partial sums: add into the zeroed output
             // tcgen05.ld is warp-collective: take the decision for the whole warp
@@ -923,15 +1015,10 @@ general_tc_kernel(const KernelArgs a)
                     const int vec = a.vec;                          // 1, 2 or 4 (W, Q, P*Q multiples of vec)
                     const int lanes_per_row = 32 / vec;
                     const int row_sub = lane / lanes_per_row, pg = lane - row_sub * lanes_per_row;
-                    const int j = j0 + b * 32 + pg * vec;           // this lane's first pixel of the block
-                    bool ok = j < a.total_pix;
+                    int n, p, q;                                    // this lane's first pixel of the block
+                    const bool ok = output_pixel<PATCH>(a, ii.geom, b * 32 + pg * vec, n, p, q);
                     float* o = a.y;
-                    if (ok) {
-                        const int n = j / a.HW, off = j - n * a.HW;
-                        const int p = off / a.W, q = off - p * a.W;
-                        ok = (p < a.P) && (q < a.Q);
-                        o = a.y + (((size_t)n * a.K + nb * a.n_tile + quarter * rpq + row_sub) * a.P + p) * a.Q + q;
-                    }
+                    if (ok) o = a.y + (((size_t)n * a.K + nb * a.n_tile + quarter * rpq + row_sub) * a.P + p) * a.Q + q;
                     if (ok) {
                         const int kmax = min(rpq, a.K - nb * a.n_tile - quarter * rpq);   // maps of this quarter that exist
                         const float* src = tile + row_sub * kXposePitch + pg * vec;
@@ -990,14 +1077,9 @@ general_tc_kernel(const KernelArgs a)
                 const int m = c / chunks_per_tile, ch = c - m * chunks_per_tile;
                 if (m != cur_m) {
                     cur_m = m;
-                    const int j = j0 + m * kTileM + quarter * 32 + lane;
-                    ok = j < a.total_pix;
-                    if (ok) {
-                        const int n = j / a.HW, off = j - n * a.HW;
-                        const int p = off / a.W, q = off - p * a.W;
-                        ok = (p < a.P) && (q < a.Q);
-                        yb = a.y + ((size_t)n * a.K * a.P + p) * a.Q + q;
-                    }
+                    int n, p, q;
+                    ok = output_pixel<PATCH>(a, ii.geom, m * kTileM + quarter * 32 + lane, n, p, q);
+                    if (ok) yb = a.y + ((size_t)n * a.K * a.P + p) * a.Q + q;
                 }
                 const int k0 = nb * a.n_tile + ch * 16;
                 if (ok) {
@@ -1127,16 +1209,19 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
 
     static bool attr_set = false;   // per process; the attribute is per function and device-wide
     if (!attr_set) {
-        if (cudaFuncSetAttribute(general_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
-            cudaFuncSetAttribute(general_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
-            cudaFuncSetAttribute(general_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess ||
-            cudaFuncSetAttribute(general_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
+        void (*all[])(KernelArgs) = {general_tc_kernel<false, false, false>, general_tc_kernel<true, false, false>,
+                                     general_tc_kernel<false, true, false>,  general_tc_kernel<true, true, false>,
+                                     general_tc_kernel<false, false, true>,  general_tc_kernel<true, false, true>};
+        for (auto k : all)
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
             return CONV2D_ERR_CUDA;
         attr_set = true;
     }
     KernelArgs a{};
     a.x = x; a.wp = wp; a.y = y; a.status = status;
     a.N = sh.N; a.C = sh.C; a.H = sh.H; a.W = sh.W; a.K = sh.K; a.P = sh.P; a.Q = sh.Q;
+    a.patch_w = p.patch_w; a.patch_tw = p.patch_tw; a.patch_rows = p.patch_rows; a.patch_cols = p.patch_cols;
+    a.row_pitch = p.patch_w ? p.patch_w : sh.W;
     a.fold_r = p.fold_r; a.fold_s = p.fold_s; a.R = sh.R / p.fold_r; a.S = sh.S / p.fold_s;
     a.HW = sh.H * sh.W;
     a.total_pix = sh.N * sh.H * sh.W;
@@ -1145,12 +1230,12 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     a.a_stages = p.a_stages; a.b_stages = p.b_stages; a.tps = p.tps;
     a.cbg = p.cbg; a.groups = (p.cblks + p.cbg - 1) / p.cbg; a.resident = p.resident; a.swap = p.swap;
     a.vec = 1;
-    for (int v = 4; v >= 2; v >>= 1)
-        if (sh.W % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
+    for (int v = 4; v >= 2; v >>= 1)       // v adjacent accumulator columns must be v adjacent, aligned outputs of one row
+        if ((p.patch_w ? p.patch_tw : sh.W) % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
     a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * p.npix * 4 >= 2 * kXposeBytes &&
                  env_int("CONV2D_B200_TF32_HELPERS", 1) != 0) ? 1 : 0;
-    a.quad = (!b16 && (sh.H * sh.W) % 4 == 0 && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
+    a.quad = (!b16 && (p.patch_w ? sh.W % 4 == 0 : (sh.H * sh.W) % 4 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
     {
         // as many producer groups as can each still cover a stage in one pass (one memory round trip)
         const long long per_pass = a.quad ? kProducers : (long long)kProducers * kUnitsPerThread;
@@ -1162,7 +1247,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         while (a.pgroups > p.a_stages) a.pgroups /= 2;
     }
     a.fp16 = fp16 ? 1 : 0;
-    a.pair = (b16 && (sh.H * sh.W) % 2 == 0 && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
+    a.pair = (b16 && (p.patch_w ? sh.W % 2 == 0 : (sh.H * sh.W) % 2 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
     a.items = p.supertiles * p.n_blocks * p.ksplit;
     a.ksplit = p.ksplit;
     // Failure-detection test hooks (host-side injection only): a short wait bound and one filter copy that is
@@ -1176,8 +1261,10 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     // Programmatic dependent launch: the kernel's set-up (barriers, tensor-memory allocation) overlaps the
     // tail of whatever kernel precedes it on the stream; it waits for that kernel before it touches global memory.
     const bool fold = p.fold_r * p.fold_s > 1;
-    void (*kernel)(KernelArgs) = b16 ? (fold ? general_tc_kernel<true, true> : general_tc_kernel<true, false>)
-                                     : (fold ? general_tc_kernel<false, true> : general_tc_kernel<false, false>);
+    void (*kernel)(KernelArgs);
+    if (p.patch_w) kernel = b16 ? general_tc_kernel<true, false, true> : general_tc_kernel<false, false, true>;
+    else if (fold) kernel = b16 ? general_tc_kernel<true, true, false> : general_tc_kernel<false, true, false>;
+    else kernel = b16 ? general_tc_kernel<true, false, false> : general_tc_kernel<false, false, false>;
     if (launch_pdl(kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, stream, a) != cudaSuccess) return CONV2D_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;

@@ -198,9 +198,11 @@ def test_full_size_configs(oracle, name, algo):
     print(f"{name} algo={algo} max ratio {worst:.3e}")
 
 
-def test_auto_falls_back_to_fp32_when_no_tensor_core_instance_fits(oracle):
-    """A very wide image needs a staged halo beyond shared memory: AUTO must still give the right answer."""
+def test_auto_falls_back_to_fp32_when_no_tensor_core_instance_fits(oracle, monkeypatch):
+    """With the flat pixel run only, a very wide image needs a staged halo beyond shared memory: AUTO must still
+    give the right answer."""
     import paper_1705_10591_b200 as lib
+    monkeypatch.setenv("CONV2D_B200_TF32_PATCH", "0")
     dims = (1, 16, 6, 6000, 8, 5, 5)
     assert not _tf32_available(dims)
     with pytest.raises(lib.Conv2dError) as e:
@@ -284,3 +286,44 @@ def test_few_channels_folded_taps(oracle, monkeypatch, dims, entry):
     y_plain = run_library(x, w, entry=entry, algo=ALGO_TF32)
     assert_parity(y_plain, y_ref, yabs, TF32_TOL if entry == "general" else 1e-5, f"unfolded {entry} {dims}")
     assert_parity(y, y_plain.astype(np.float64), yabs, 2e-5, f"folded vs unfolded {entry} {dims}")
+
+
+WIDE_SHAPES = [
+    # N, C, H, W, K, R, S      (items cut as rectangles of the image: the flat run's halo would be (R-1) image rows)
+    (1, 16, 12, 600, 40, 3, 3),      # 128-bit producer loads, ragged last patch column
+    (2, 20, 9, 1100, 130, 5, 5),     # two filter blocks; the flat run has no instance at this width
+    (1, 8, 30, 260, 64, 7, 7),       # 7 x 7: three quarters of a 32-wide patch row are valid
+    (1, 8, 21, 303, 64, 3, 3),       # width not a multiple of 4: one pixel per load
+    (3, 33, 5, 520, 16, 1, 3),       # a single row of taps
+    (1, 16, 6, 6000, 8, 5, 5),       # extremely wide, few rows
+]
+
+
+@pytest.mark.parametrize("dims", WIDE_SHAPES)
+@pytest.mark.parametrize("entry", ["general", "bf16"])
+def test_wide_images_patch_addressing(oracle, dims, entry):
+    N, C, H, W, K, R, S = dims
+    xi, wi = small_integers((N, C, H, W), 451), small_integers((K, C, R, S), 452)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry=entry, algo=ALGO_TF32).astype(np.float64), yi_ref)
+    x, w = uniform((N, C, H, W), 453), uniform((K, C, R, S), 454)
+    if entry == "bf16":
+        from helpers import bf16_values
+        x, w = bf16_values(x)[0], bf16_values(w)[0]
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry=entry, algo=ALGO_TF32), y_ref, yabs,
+                  TF32_TOL if entry == "general" else 1e-5, f"patch {entry} {dims}")
+
+
+@pytest.mark.parametrize("dims", [(2, 17, 20, 21, 70, 3, 3), (1, 64, 14, 14, 96, 3, 3), (5, 33, 7, 9, 128, 3, 3),
+                                  (2, 48, 12, 12, 128, 1, 1), (1, 40, 16, 16, 130, 1, 7)])
+def test_patch_addressing_forced_on_narrow_images(oracle, monkeypatch, dims):
+    """The two addressing modes must agree (same operands, same contraction order per output)."""
+    N, C, H, W, K, R, S = dims
+    x, w = uniform((N, C, H, W), 455), uniform((K, C, R, S), 456)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    y_flat = run_library(x, w, entry="general", algo=ALGO_TF32)
+    monkeypatch.setenv("CONV2D_B200_TF32_PATCH", "2")
+    y_patch = run_library(x, w, entry="general", algo=ALGO_TF32)
+    assert_parity(y_patch, y_ref, yabs, TF32_TOL, f"patch {dims}")
+    assert_parity(y_patch, y_flat.astype(np.float64), yabs, 2e-5, f"patch vs flat {dims}")
