@@ -54,17 +54,25 @@ def run_point(torch, lib, peaks, flush, N, C, H, W, K, R, S, algo, label, extra=
     else:
         ws_bytes = lib.conv2d_fwd_workspace_size(N, C, H, W, K, R, S, algo)
         ws = torch.zeros(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+        if algo == lib.ALGO_16BIT:
+            x16, w16 = x.to(torch.bfloat16).contiguous(), w.to(torch.bfloat16).contiguous()
 
-        def fn():
-            lib.conv2d_fwd_general(x.data_ptr(), w.data_ptr(), y.data_ptr(), N, C, H, W, K, R, S, algo,
-                                   ws.data_ptr(), ws_bytes, 0, stream)
+            def fn():
+                lib.conv2d_fwd_general_16bit(x16.data_ptr(), w16.data_ptr(), y.data_ptr(), N, C, H, W, K, R, S,
+                                             lib.OPERAND_BF16, ws.data_ptr(), ws_bytes, 0, stream)
+        else:
+            def fn():
+                lib.conv2d_fwd_general(x.data_ptr(), w.data_ptr(), y.data_ptr(), N, C, H, W, K, R, S, algo,
+                                       ws.data_ptr(), ws_bytes, 0, stream)
     flops = 2 * N * K * C * R * S * P * Q
-    bytes_ = 4 * (N * C * H * W + K * C * R * S + N * K * P * Q)
+    in_bytes = 2 if (C > 1 and algo == lib.ALGO_16BIT) else 4
+    bytes_ = in_bytes * (N * C * H * W + K * C * R * S) + 4 * N * K * P * Q
     big = bytes_ > 2 * 126 * 1024 * 1024
     ms = time_call(torch, fn, None if big else flush)
     lib.conv2d_get_status(ws.data_ptr() if ws is not None else 0, stream)
     fp32_peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
-    pipe_peak = fp32_peak if (C == 1 or algo == lib.ALGO_FFMA) else peaks["bf16_tflops"] / 2
+    pipe_peak = fp32_peak if (C == 1 or algo == lib.ALGO_FFMA) else (
+        peaks["bf16_tflops"] if algo == lib.ALGO_16BIT else peaks["bf16_tflops"] / 2)
     t_roof = max(flops / (pipe_peak * 1e12), bytes_ / (peaks["hbm_gbs"] * 1e9)) * 1e3
     rec = {"sweep": label, "N": N, "C": C, "H": H, "W": W, "K": K, "R": R, "S": S, "ms": ms,
            "gflops": flops / ms / 1e6, "gbs": bytes_ / ms / 1e6, "roofline_frac": t_roof / ms,
@@ -91,11 +99,11 @@ def main():
                     run_point(torch, lib, peaks, flush, 1, 1, size, size, k, r, r, lib.ALGO_FFMA, "special")
     elif which == "general":
         for r in (3, 5, 7):
-            for size in (16, 32, 64):
+            for size in (16, 32, 64, 128, 256, 512):
                 for c in (64, 128):
                     for k in (64, 128, 256):
                         n = max(1, 65536 // (size * size))
-                        for algo, name in ((lib.ALGO_TF32, "tf32"), (lib.ALGO_FFMA, "fp32")):
+                        for algo, name in ((lib.ALGO_TF32, "tf32"), (lib.ALGO_16BIT, "bf16"), (lib.ALGO_FFMA, "fp32")):
                             run_point(torch, lib, peaks, flush, n, c, size, size, k, r, r, algo, "general", {"algo": name})
     elif which == "unit":
         for size in (2048, 4096):
