@@ -1,38 +1,50 @@
-// General case on the tcgen05 tensor cores: implicit-GEMM direct convolution, TF32 operands,
-// fp32 accumulators in tensor memory (the contraction of Section 4, Algorithm 2).
+// General case on the tcgen05 tensor cores: implicit-GEMM direct convolution with fp32 accumulators in
+// tensor memory (the contraction of Section 4, Algorithm 2).  fp32 inputs run as TF32 (kind::tf32, K = 8
+// per instruction), bf16 / fp16 inputs as kind::f16 (K = 16); a 64-byte staged unit is 16 fp32 or 32
+// 16-bit channels of one pixel, so both share every shared-memory layout and descriptor.
 //
 // Mapping of the paper's design onto B200
-//   * GEMM view: rows = output pixels, columns = filters, contraction over (channel, tap).
-//     The accumulator block rAcc[F_T][W_T] of Algorithm 2 becomes a 128-pixel x n_tile-filter
-//     fp32 tile in tensor memory; a work item is `mt` such tiles for adjacent pixels.
-//   * Pixels are numbered in one flat sequence j = (n*H + h)*W + w over the whole batch.  For tap
-//     (r,s) the input needed by output j is the pixel j + r*W + s of the same channel, a pure
-//     shift.  Per block of kCB channels ONE run of mt*128 + (R-1)*W + (S-1) pixels is staged
-//     ("block plus halo to the right and below", Section 3.1/4.1) and every tap reads it through
-//     a descriptor whose start address is shifted by r*W + s rows: the row reuse of Section 4.2
-//     (one staged input row serves all horizontal taps) extended to the vertical taps, with no
-//     im2col buffer.  Outputs whose window wraps over the right or bottom image edge are
-//     computed but not stored.
-//   * Shared-memory operand layout: K-major, no swizzle: [channel/4][row][4 channels], i.e. each
-//     row (pixel or filter) of a 4-channel chunk is one 16-byte unit and rows are 16 bytes apart.
-//     This is the transposed staging of Fig. 6 (adjacent units belong to adjacent rows) in the
-//     unit size the tensor core reads, and it is what makes a start address at any pixel legal.
+//   * GEMM view: M = a block of 128 (or 64) filters, N = the pixels of a work item, contraction over
+//     (channel, tap).  The accumulator block rAcc[F_T][W_T] of Algorithm 2 becomes a filters x pixels fp32
+//     tile in tensor memory (lanes = filters, columns = pixels); a work item is any multiple of 32 pixels
+//     up to 512, covered by one or two MMAs per K step.  (With the pixels as M a 128-filter problem needs
+//     twice as many instructions, and the single issuing thread is what limits the rate.)
+//   * Flat addressing: pixels are numbered in one sequence j = (n*H + h)*W + w over the whole batch.  For
+//     tap (r,s) the input needed by output j is pixel j + r*W + s of the same channel, a pure shift.  Per
+//     block of channels ONE run of tile_px + (R-1)*W + (S-1) pixels is staged ("block plus halo to the
+//     right and below", Section 3.1/4.1) and every tap reads it through a descriptor whose start address
+//     is shifted by r*W + s rows: the row reuse of Section 4.2 (one staged input row serves all
+//     horizontal taps) extended to the vertical taps, with no im2col buffer.  Outputs whose window wraps
+//     over the right or bottom image edge are computed but not stored.
+//   * Patch addressing (wide images): the item is a rectangle of one image, patch_w columns wide, staged
+//     row after row; the tap shift becomes r*patch_w + s and the halo (R-1) patch rows instead of (R-1)
+//     image rows.  See ItemGeom.
+//   * Few channels: taps are folded into the channel dimension (see make_plan), so that a staged channel
+//     block is not mostly padding.
+//   * Shared-memory operand layout: K-major, no swizzle: [channel/4][row][4 channels], i.e. each row
+//     (pixel or filter) of a chunk is one 16-byte unit and rows are 16 bytes apart.  This is the
+//     transposed staging of Fig. 6 (adjacent units belong to adjacent rows) in the unit size the tensor
+//     core reads, and it is what makes a start address at any pixel legal.
 //   * The filters are re-ordered once per call into exactly that layout in the workspace
-//     ([filter block][channel block][tap][channel/4][filter][4], rounded to TF32) and streamed
-//     with 1-D bulk (TMA) copies through an mbarrier ring.  Activations cannot be moved by TMA:
-//     NCHW has the pixels, not the channels, contiguous, and a tiled copy cannot transpose nor
-//     start at a 4-byte offset; eight producer warps gather them (coalesced along pixels),
-//     round to TF32 and write 16-byte units.
-//   * Persistent blocks, one per SM, walk over the work items round-robin.  Warp roles: warp 0
-//     streams filter stages, warp 1 (one thread) issues tcgen05.mma and owns the tensor-memory
-//     allocation, eight warps stage activations, four warps drain finished accumulators (lane =
-//     pixel, so a warp stores 32 adjacent outputs of one map: the coalesced write-back that
-//     Section 4.2 leaves out).  All rings run across item boundaries, so the loads of the next
-//     item proceed under the MMAs of the current one (the prefetch of Algorithm 2), and where two
-//     accumulator sets fit into the 512 tensor-memory columns the write-back of item i overlaps
-//     the MMAs of item i+1.
-//   * Every wait is bounded; on expiry the block raises a flag, stops storing, frees its tensor
-//     memory and the status word in the workspace becomes non-zero.
+//     ([filter block][channel block][tap][chunk][filter][unit], fp32 rounded to TF32) and either kept in
+//     shared memory for the life of the block or streamed with 1-D bulk (TMA) copies through an mbarrier
+//     ring.  Activations cannot be moved by TMA: NCHW has the pixels, not the channels, contiguous, and a
+//     tiled copy cannot transpose nor start at a 4-byte offset; eight producer warps gather them
+//     (coalesced along pixels, 128-bit loads where the alignment allows), round fp32 to TF32 and write
+//     16-byte units.
+//   * Persistent blocks, one per SM, walk over the work items round-robin.  Warp roles: warp 0 streams
+//     filter stages, warp 1 (one thread) issues tcgen05.mma and owns the tensor-memory allocation, eight
+//     warps stage activations (in up to four groups that fill different stages concurrently), four warps
+//     drain finished accumulators through a shared-memory transposition so that a store instruction
+//     writes adjacent outputs of one map (the coalesced write-back that Section 4.2 leaves out); for the
+//     block's last item the other eight warps join the drain.  All rings run across item boundaries, so
+//     the loads of the next item proceed under the MMAs of the current one (the prefetch of Algorithm 2),
+//     and where two accumulator sets fit into the 512 tensor-memory columns the write-back of item i
+//     overlaps the MMAs of item i+1.
+//   * The kernel is launched with programmatic stream serialization: everything before grid_dep_wait()
+//     touches only this block's shared and tensor memory and overlaps the preceding kernel's tail.
+//   * Every wait is bounded; on expiry the block raises a flag, stops storing, frees its tensor memory and
+//     the status word in the workspace becomes non-zero.
 #include <cstdlib>
 #include <mutex>
 
@@ -61,12 +73,13 @@ constexpr int kEpilogueWarps = 4;
 // Warp roles by warp index.  An SM has four warp schedulers and warp w is served by scheduler w % 4.  The
 // single thread that issues the MMAs (warp 1) must never wait for an issue slot behind arithmetic-heavy
 // warps -- measured: sharing its scheduler with two producer warps stretched each MMA issue from ~64 to
-// 120-180 cycles -- so scheduler 1 hosts only that warp, one epilogue warp and two warps that exit at once.
+// 120-180 cycles -- so scheduler 1 hosts only that warp, one epilogue warp and two warps that only wait.
 //   warp 0           filter copies (one thread)
 //   warp 1           MMA issue (one thread), owner of the tensor-memory allocation
 //   warps 4-7        epilogue, tensor-memory lane quarter = warp % 4
 //   warps 2,3,8,10,11,12,14,15   activation producers (schedulers 0, 2, 3)
-//   warps 9, 13      no work
+//   warps 9, 13      no work until the block's last item
+//   warps 8-15       help to drain the block's last item once their own work is done (quarter = warp % 4)
 constexpr int kThreads = 512;
 __device__ __forceinline__ int producer_index(int warp)     // 0..7 for producer warps, -1 otherwise
 {
@@ -84,7 +97,7 @@ constexpr int kXposePitch = 36;             // floats per row of the epilogue's 
 constexpr size_t kXposeBytes = (size_t)kEpilogueWarps * 32 * kXposePitch * 4;
 
 struct Plan {
-    int n_tile;       // filters per work item (UMMA N), multiple of 16
+    int n_tile;       // filters per work item: 64 or 128 rows of the M operand (with the pixels as M: UMMA N, a multiple of 16)
     int n_blocks;     // work-item columns over the filters
     int mt;           // accumulator tiles per work item (pixels-as-M layout; informative otherwise)
     int tile_px;      // pixels per work item: mt * 128, or any multiple of 32 up to 512 in the operand-swap layout
@@ -1218,7 +1231,12 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
     }
 
-    static bool attr_set = false;   // per process; the attribute is per function and device-wide
+    // The attribute belongs to a (function, device) pair: set once per device.  (A benign race: two threads
+    // may both set it.)
+    static bool attr_set_on[64] = {};
+    int dev_id = 0;
+    if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) return CONV2D_ERR_CUDA;
+    bool& attr_set = attr_set_on[dev_id];
     if (!attr_set) {
         void (*all[])(KernelArgs) = {general_tc_kernel<false, false, false>, general_tc_kernel<true, false, false>,
                                      general_tc_kernel<false, true, false>,  general_tc_kernel<true, true, false>,
