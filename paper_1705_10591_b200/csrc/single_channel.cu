@@ -860,21 +860,25 @@ conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shap
                                              : launch_unit<R, S, 4>(x, w, y, sh, tile_h, stream);
         if (st != CONV2D_ERR_UNSUPPORTED) return st;
     }
-    // Large images: the wide persistent kernel (needs 16-byte aligned input rows for the bulk copies).
-    const bool rows_ok = sh.W % 4 == 0 && sh.Q >= 1024 && reinterpret_cast<uintptr_t>(x) % 16 == 0;
+    // Large images: the wide persistent kernels (they need 16-byte aligned input rows for the bulk copies).
+    const bool rows_ok = sh.W % 4 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0;
     if (rows_ok && env_int("CONV2D_B200_SC_WIDE", 1) != 0) {
         int band_h = env_int("CONV2D_B200_SC_BAND_H", 8);
         if (band_h < 1) band_h = 1;
         if (band_h > 16) band_h = 16;
-        // rows that are only 8-byte aligned: the variant that shifts odd rows by two columns
-        if (sh.Q % 4 == 2 && ((long long)sh.P * sh.Q) % 4 == 0 && reinterpret_cast<uintptr_t>(y) % 16 == 0 &&
+        // Rows that are only 8-byte aligned: the variant that shifts odd rows by two columns.  Its aligned
+        // 128-bit stores beat the tile kernel's 64-bit pairs already on mid-size images (3 x 3, 32 filters,
+        // 1024 x 1024: 75 -> 41 us; 512 x 512: 26 -> 20 us), although half of its 2048 columns are idle there.
+        if (sh.Q >= 384 && sh.Q % 4 == 2 && ((long long)sh.P * sh.Q) % 4 == 0 && reinterpret_cast<uintptr_t>(y) % 16 == 0 &&
             env_int("CONV2D_B200_SC_SHIFT", 1) != 0) {
             const conv2d_status_t st = try_rows_shift<R, S>(x, w, y, sh, band_h, stream);
             if (st != CONV2D_ERR_UNSUPPORTED) return st;
         }
-        const conv2d_status_t st = (tr == 1 || R >= 7) ? launch_rows<R, S, 1>(x, w, y, sh, band_h, stream)
-                                                       : launch_rows<R, S, 2>(x, w, y, sh, band_h, stream);
-        if (st != CONV2D_ERR_UNSUPPORTED) return st;
+        if (sh.Q >= env_int("CONV2D_B200_SC_WIDE_MINQ", 1024)) {
+            const conv2d_status_t st = (tr == 1 || R >= 7) ? launch_rows<R, S, 1>(x, w, y, sh, band_h, stream)
+                                                           : launch_rows<R, S, 2>(x, w, y, sh, band_h, stream);
+            if (st != CONV2D_ERR_UNSUPPORTED) return st;
+        }
     }
     if (env_int("CONV2D_B200_SC_PACKED", 1) != 0 &&
         (size_t)((sh.K + 1) / 2) * RS2 * sizeof(float4) <= 96 * 1024) {

@@ -32,6 +32,8 @@ SINGLE_SHAPES = [
     (1, 9, 1028, 2, 7, 7),       # wide kernel, 7 x 7, band taller than the image's output rows
     (1, 14, 1040, 4, 1, 1),      # wide kernel, 1 x 1
     (1, 12, 1032, 3, 3, 3),      # shifted wide kernel: Q = 1030 (8-byte aligned rows), odd filter count
+    (1, 10, 388, 3, 3, 3),       # shifted wide kernel on a narrow image: Q = 386, most of the 2048 columns idle
+    (2, 14, 520, 5, 3, 3),       # shifted wide kernel: Q = 518, two images, two bands
     (2, 20, 2100, 5, 3, 3),      # shifted wide kernel: Q = 2098, two column tiles, three bands
     (1, 14, 1040, 4, 7, 7),      # wide kernel, 7 x 7, Q = 1034: 64-bit stores
 ]
