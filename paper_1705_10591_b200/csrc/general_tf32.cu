@@ -441,24 +441,57 @@ __global__ void repack_filters_tiled_kernel(const T* __restrict__ w, T* __restri
     const int cb = blockIdx.y, k0 = blockIdx.x * 8, c0 = cb * cpb;
     const int row = cpb * taps;
     const int c_live = min(cpb, C - c0) * taps;                  // elements of a filter's run that exist
+    // Load: whole 16-byte words where a filter's run is full and 16-byte aligned, single elements otherwise.
+    constexpr int kVec = 16 / (int)sizeof(T);
+    const bool vec_ok = c_live == row && row % kVec == 0 && ((size_t)C * taps) % kVec == 0 &&
+                        reinterpret_cast<uintptr_t>(w) % 16 == 0;
+    if (vec_ok) {
+        const int row_v = row / kVec;
 #pragma unroll 4
-    for (int idx = threadIdx.x; idx < 8 * row; idx += blockDim.x) {       // (independent loads: several in flight)
-        const int kk = idx / row, rem = idx - kk * row;
-        T v = T(0);
-        if (k0 + kk < K && rem < c_live) {
-            v = __ldg(w + ((size_t)(k0 + kk) * C + c0) * taps + rem);
-            if (sizeof(T) == 4) v = (T)to_tf32_rna((float)v);
+        for (int idx = threadIdx.x; idx < 8 * row_v; idx += blockDim.x) {       // (independent loads: several in flight)
+            const int kk = idx / row_v, rem = idx - kk * row_v;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (k0 + kk < K) {
+                v = __ldg(reinterpret_cast<const uint4*>(w + ((size_t)(k0 + kk) * C + c0) * taps) + rem);
+                if (sizeof(T) == 4) {
+                    v.x = __float_as_uint(to_tf32_rna(__uint_as_float(v.x))); v.y = __float_as_uint(to_tf32_rna(__uint_as_float(v.y)));
+                    v.z = __float_as_uint(to_tf32_rna(__uint_as_float(v.z))); v.w = __float_as_uint(to_tf32_rna(__uint_as_float(v.w)));
+                }
+            }
+            reinterpret_cast<uint4*>(tile)[idx] = v;
         }
-        tile[idx] = v;
+    } else {
+#pragma unroll 4
+        for (int idx = threadIdx.x; idx < 8 * row; idx += blockDim.x) {
+            const int kk = idx / row, rem = idx - kk * row;
+            T v = T(0);
+            if (k0 + kk < K && rem < c_live) {
+                v = __ldg(w + ((size_t)(k0 + kk) * C + c0) * taps + rem);
+                if (sizeof(T) == 4) v = (T)to_tf32_rna((float)v);
+            }
+            tile[idx] = v;
+        }
     }
     __syncthreads();
+    // Store: one 16-byte unit (EPC channels of one filter and tap) per thread and step.
     const int nb = k0 / n_tile, f0 = k0 - nb * n_tile;
     T* dst = wp + ((size_t)nb * cblks + cb) * taps * kChunks * n_tile * EPC;
-    for (int idx = threadIdx.x; idx < 8 * row; idx += blockDim.x) {
-        const int e = idx % EPC, kk = (idx / EPC) % 8;
-        const int rest = idx / (EPC * 8);
+    for (int idx = threadIdx.x; idx < 8 * kChunks * taps; idx += blockDim.x) {
+        const int kk = idx % 8;
+        const int rest = idx / 8;
         const int chunk = rest % kChunks, t = rest / kChunks;
-        dst[(((size_t)t * kChunks + chunk) * n_tile + f0 + kk) * EPC + e] = tile[kk * row + (chunk * EPC + e) * taps + t];
+        const T* src = tile + kk * row + (chunk * EPC) * taps + t;
+        T u[EPC];
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) u[e] = src[e * taps];
+        uint4 v;
+        if (sizeof(T) == 4) {
+            v = make_uint4(__float_as_uint((float)u[0]), __float_as_uint((float)u[1]), __float_as_uint((float)u[2]), __float_as_uint((float)u[3]));
+        } else {
+            v = make_uint4((unsigned)u[0] | ((unsigned)u[1] << 16), (unsigned)u[2 % EPC] | ((unsigned)u[3 % EPC] << 16),
+                           (unsigned)u[4 % EPC] | ((unsigned)u[5 % EPC] << 16), (unsigned)u[6 % EPC] | ((unsigned)u[7 % EPC] << 16));
+        }
+        *reinterpret_cast<uint4*>(dst + (((size_t)t * kChunks + chunk) * n_tile + f0 + kk) * EPC) = v;
     }
 }
 
@@ -1209,7 +1242,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         const size_t tile_bytes = (size_t)8 * kCB * 4 * p.taps;       // 8 filters x one channel block x taps
         if (p.fold_r * p.fold_s == 1 && tile_bytes <= 48 * 1024 && p.n_tile % 8 == 0) {
             const dim3 grid((unsigned)(p.n_blocks * p.n_tile / 8), (unsigned)p.cblks);
-            int threads = (8 * kCB * p.taps / 4 + 31) / 32 * 32;          // about four elements per thread
+            int threads = (8 * kChunks * p.taps + 31) / 32 * 32;          // one 16-byte unit per thread in the store phase
             threads = threads < 128 ? 128 : (threads > 1024 ? 1024 : threads);
             // (launched the ordinary way: it starts only when the previous call's kernel, which may still
             // be reading the workspace, has finished; measured no gain from overlapping its launch)
