@@ -321,12 +321,13 @@ Plan make_plan(const Shape& sh, bool b16 = false)
         p.tile_px = best_px;
         p.mt = (best_px + kTileM - 1) / kTileM;
         p.npix = npix_of(p.tile_px);
-        // Filter stages: several taps per stage (up to 32 KB) so that the single MMA-issuing thread pays
-        // its per-stage bookkeeping (barrier wait, commit) once per 16-32 MMAs; the ring should hold
+        // Filter stages: several taps per stage (up to 48 KB, trimmed below until three stages fit) so that the
+        // single MMA-issuing thread pays its per-stage bookkeeping (barrier wait, commit: ~90 cycles, measured
+        // by varying the stage size) once per 16-48 MMAs; the ring should hold
         // 64-128 KB in flight to cover the L2 latency.
         p.a_stages = 2;
         p.cbg = 1;
-        p.tps = 32 * 1024 / chunk;
+        p.tps = env_int("CONV2D_B200_TF32_STAGE_KB", 48) * 1024 / chunk;
         if (p.tps < 1) p.tps = 1;
         if (p.tps > p.taps) p.tps = p.taps;
         p.b_stages = 2;
