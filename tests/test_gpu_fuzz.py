@@ -1,0 +1,69 @@
+"""Seeded random shapes through every general-case path: the planner has many branches (operand roles, item size,
+flat or patch addressing, folded taps, resident or streamed filters, split contraction), and each shape below lands in
+some combination of them.  Every output element is compared with the oracle.
+"""
+import numpy as np
+import pytest
+
+from helpers import FFMA_TOL, TF32_TOL, assert_parity, bf16_values, run_library
+from workloads import uniform
+
+pytestmark = pytest.mark.gpu
+
+ALGO_FFMA, ALGO_TF32 = 1, 2
+
+
+def _draw(seed):
+    """One shape from a seeded stream of uniforms; sizes are log-distributed and the work is capped."""
+    u = uniform((16,), 9000 + seed, 0.0, 1.0)
+
+    def log_int(t, lo, hi):
+        return int(round(lo * (hi / lo) ** float(t)))
+
+    taps = (1, 2, 3, 5, 7)
+    R, S = taps[int(u[0] * 5) % 5], taps[int(u[1] * 5) % 5]
+    N = log_int(u[2], 1, 5)
+    C = log_int(u[3], 1, 200)
+    H = max(R, log_int(u[4], 3, 48))
+    W = max(S, log_int(u[5], 3, 900))
+    K = log_int(u[6], 1, 320)
+    while N * K * C * R * S * (H - R + 1) * (W - S + 1) > 6e8 and K > 1:      # keep the oracle under a second
+        K = max(1, K // 2)
+    while N * K * C * R * S * (H - R + 1) * (W - S + 1) > 6e8 and C > 1:
+        C = max(1, C // 2)
+    return N, C, H, W, K, R, S
+
+
+SHAPES = sorted({_draw(s) for s in range(72)})
+
+
+def _tc_available(dims, algo):
+    import paper_1705_10591_b200 as lib
+    try:
+        return lib.conv2d_fwd_workspace_size(*dims, algo) > 0
+    except lib.Conv2dError:
+        return False
+
+
+@pytest.mark.parametrize("dims", SHAPES)
+def test_random_shape_all_paths(oracle, dims):
+    N, C, H, W, K, R, S = dims
+    x, w = uniform((N, C, H, W), 461), uniform((K, C, R, S), 462)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_FFMA), y_ref, yabs, FFMA_TOL, f"fp32 {dims}")
+    if _tc_available(dims, ALGO_TF32):
+        assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, f"tf32 {dims}")
+    if _tc_available(dims, 3):
+        xb, wb = bf16_values(x)[0], bf16_values(w)[0]
+        yb_ref, yb_abs = oracle.conv2d_oracle(xb, wb)
+        assert_parity(run_library(xb, wb, entry="bf16"), yb_ref, yb_abs, 1e-5, f"bf16 {dims}")
+
+
+def test_the_random_shapes_reach_the_planner_branches():
+    """The stream above must contain wide images, few-channel shapes, many-channel shapes, many-filter shapes, 1 x 1 taps."""
+    assert any(W >= 400 for (_, _, _, W, _, _, _) in SHAPES)
+    assert any(C <= 3 for (_, C, _, _, _, _, _) in SHAPES)
+    assert any(K > 128 for (_, _, _, _, K, _, _) in SHAPES)
+    assert any(R == 1 and S == 1 for (*_, R, S) in SHAPES)
+    assert any(C >= 64 for (_, C, _, _, _, _, _) in SHAPES)
+    assert len(SHAPES) >= 60
