@@ -93,6 +93,8 @@ constexpr int kMaxBStages = 16;
 constexpr int kMaxAStages = 4;
 constexpr int kUnitsPerThread = 3;          // (pixel, channel block) units a producer thread keeps in flight per pass
 constexpr size_t kSmemLimit = 227 * 1024;
+constexpr int kMaxTaps = 256;                // taps left as descriptor shifts (after folding)
+constexpr size_t kBookBytes = 512 + kMaxTaps * 4;    // barriers, tensor-memory slot, flags + the table of tap shifts
 constexpr int kXposePitch = 36;             // floats per row of the epilogue's transposition tile (16-byte aligned, conflict-free)
 constexpr size_t kXposeBytes = (size_t)kEpilogueWarps * 32 * kXposePitch * 4;
 
@@ -125,7 +127,7 @@ struct Plan {
 // b_stages counts filter stages of `tps` taps each; an activation stage holds `cbg` channel blocks.
 size_t smem_need(int a_stages, int npix, int n_tile, int b_stages, int tps, int cbg)
 {
-    return (size_t)a_stages * cbg * kCB * npix * 4 + (size_t)b_stages * tps * kCB * n_tile * 4 + 512;
+    return (size_t)a_stages * cbg * kCB * npix * 4 + (size_t)b_stages * tps * kCB * n_tile * 4 + kBookBytes;
 }
 
 int env_int(const char* name, int dflt)
@@ -184,6 +186,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
     const int r_eff = sh.R / p.fold_r, s_eff = sh.S / p.fold_s;
     p.cblks = (c_eff + cbc - 1) / cbc;
     p.taps = r_eff * s_eff;
+    if (p.taps > kMaxTaps) return p;
     const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
     // Addressing mode.  In the flat pixel run the staged halo is (R-1) whole image rows; once that exceeds a
     // 256-pixel item the item is cut as a rectangle of the image instead (patch_w columns wide, of which the
@@ -249,7 +252,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
             if (p.swap && want >= 64 && want <= 512 && want % 32 == 0 && pixel_items(want) > 0) res_px = want;
         }
         const int npix = npix_of(res_px);
-        if ((p.swap ? res_px : mt * set_cols) <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * npix * 4 + 512 <= kSmemLimit) {
+        if ((p.swap ? res_px : mt * set_cols) <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * npix * 4 + kBookBytes <= kSmemLimit) {
             p.resident = 1;
             p.mt = p.swap ? (res_px + kTileM - 1) / kTileM : mt;
             p.tile_px = res_px;
@@ -258,7 +261,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
             p.a_stages = 2;
             p.b_stages = 1;
             p.tps = p.taps;
-            auto need = [&](int a_stages, int cbg) { return wbytes + extra + (size_t)a_stages * cbg * kCB * npix * 4 + 512; };
+            auto need = [&](int a_stages, int cbg) { return wbytes + extra + (size_t)a_stages * cbg * kCB * npix * 4 + kBookBytes; };
             while (p.cbg * 2 <= p.cblks && npix * p.cbg * 2 <= kProducers * kUnitsPerThread &&
                    need(p.a_stages, p.cbg * 2) <= kSmemLimit) p.cbg *= 2;
             while (p.a_stages < kMaxAStages && need(p.a_stages + 1, p.cbg) <= kSmemLimit) ++p.a_stages;
@@ -721,6 +724,36 @@ __device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
     return it;
 }
 
+// All MMAs of one tap of one channel block in the filters-as-M layout: K steps 0 and 1 for GROUPS pixel groups
+// of n_mma pixels.  d: accumulator column of group 0; px_lo / flt_lo: low words of the pixel and filter
+// descriptors of K step 0 (the K step and the group add constants to the start-address field); acc = 0 only
+// for the very first tap of an item.
+template <bool B16, int GROUPS>
+__device__ __forceinline__ void issue_tap(uint32_t d, uint32_t px_lo, uint32_t flt_lo, uint32_t px_kstep, uint32_t flt_kstep,
+                                          uint32_t n_mma, uint32_t desc_hi, uint32_t idesc, uint32_t acc)
+{
+#define CONV2D_TAP_MMA(KIND)                                                                                  \
+    asm volatile(                                                                                             \
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 f0, f1, x;\n\t.reg .b32 t, dd;\n\t"                                 \
+        "setp.ne.b32 p, %8, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"                                                   \
+        "mov.b64 f0, {%2, %6};\n\tadd.u32 t, %2, %4;\n\tmov.b64 f1, {t, %6};\n\t"                             \
+        "mov.b64 x, {%1, %6};\n\t"                                                                            \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], f0, x, %7, p;\n\t"                                      \
+        "add.u32 t, %1, %3;\n\tmov.b64 x, {t, %6};\n\t"                                                      \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], f1, x, %7, q;\n\t"                                      \
+        "setp.ne.b32 q, %9, 0;\n\t"                                                                           \
+        "@!q bra DONE_%=;\n\t"                                                                                \
+        "add.u32 dd, %0, %5;\n\tadd.u32 t, %1, %5;\n\tmov.b64 x, {t, %6};\n\t"                               \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [dd], f0, x, %7, p;\n\t"                                      \
+        "add.u32 t, t, %3;\n\tmov.b64 x, {t, %6};\n\t"                                                       \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [dd], f1, x, %7, q;\n\t"                                      \
+        "DONE_%=:\n\t}"                                                                                       \
+        ::"r"(d), "r"(px_lo), "r"(flt_lo), "r"(px_kstep), "r"(flt_kstep), "r"(n_mma), "r"(desc_hi), "r"(idesc), \
+          "r"(acc), "n"(GROUPS == 2 ? 1 : 0) : "memory")
+    if (B16) CONV2D_TAP_MMA("f16"); else CONV2D_TAP_MMA("tf32");
+#undef CONV2D_TAP_MMA
+}
+
 template <bool B16, bool FOLD, bool PATCH>
 __global__ void __launch_bounds__(kThreads, 1)
 general_tc_kernel(const KernelArgs a)
@@ -747,6 +780,8 @@ general_tc_kernel(const KernelArgs a)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile unsigned long long* t_entry = reinterpret_cast<volatile unsigned long long*>(tmem_slot + 2);
+    uint32_t* tap_shift = tmem_slot + 4;                   // [taps] r * row_pitch + s of every tap, in staged pixels
+    for (int t = tid; t < a.taps; t += kThreads) tap_shift[t] = (uint32_t)((t / a.S) * a.row_pitch + t % a.S);
     if (tid == 0) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); *t_entry = t; }
 
     if (tid == 0) {
@@ -887,7 +922,7 @@ general_tc_kernel(const KernelArgs a)
                     uint32_t a_lo_block = a_lo_fixed | (smem_u32(a_smem + (size_t)as * a_stage_bytes) >> 4);
                     for (int g = 0; g < a.cbg && alive; ++g, a_lo_block += a_block_bytes >> 4) {
                         if (gr * a.cbg + g >= a.cblks) break;
-                        uint32_t row_shift = 0;                                  // r * W, in pixels (= 16-byte units)
+                        uint32_t row_shift = 0;                                  // r * row pitch, in pixels (= 16-byte units)
                         int sx = 0;
                         for (int t0 = 0; t0 < a.taps; t0 += a.tps) {
                             const int nt = min(a.tps, a.taps - t0);
@@ -899,30 +934,42 @@ general_tc_kernel(const KernelArgs a)
                                 tc_fence_after_sync();
                                 b_lo = b_lo_fixed | (smem_u32(b_smem + (size_t)bs * b_stage_bytes) >> 4);
                             }
-                            for (int t = 0; t < nt; ++t, b_lo += b_chunk_bytes >> 4) {
-                                uint32_t a_lo = a_lo_block + row_shift + (uint32_t)sx;
-                                uint32_t d = d0;
-                                if (a.swap) {
-                                    // M operand = the 128 filters of this stage, N operand = n_mma staged pixels.
-                                    // Straight-line code: this one thread's instruction stream is what bounds
-                                    // the MMA rate (~130 cycles per MMA with loop and address arithmetic around
-                                    // each one), so nothing is computed here that can be shared or hoisted.
-                                    const uint64_t bd0 = pack64(b_lo, desc_hi), bd1 = pack64(b_lo + b_kstep, desc_hi);
-                                    mma(d, bd0, pack64(a_lo, desc_hi), idesc, accumulate != 0);
-                                    mma(d, bd1, pack64(a_lo + a_kstep, desc_hi), idesc, true);
-                                    if (a.px_groups == 2) {
+                            if (a.swap && a.px_groups == 1) {
+                                // M operand = the 128 filters of this stage, N operand = n_mma staged pixels.
+                                // One MMA pair per tap carries less tensor-pipe work than this one thread needs to
+                                // issue it with loop and address arithmetic around it (~230 cycles per MMA that
+                                // way), so a tap is one block of straight-line code and its shift comes from a
+                                // table, fetched one tap ahead.
+                                const uint32_t* shift = tap_shift + t0;
+                                uint32_t cur = shift[0];
+                                for (int t = 0; t < nt; ++t, b_lo += b_chunk_bytes >> 4) {
+                                    const uint32_t a_lo = a_lo_block + cur;
+                                    cur = shift[t + 1 < nt ? t + 1 : t];
+                                    issue_tap<B16, 1>(d0, a_lo, b_lo, a_kstep, b_kstep, n_mma, desc_hi, idesc, accumulate);
+                                    accumulate = 1;
+                                }
+                            } else {
+                                for (int t = 0; t < nt; ++t, b_lo += b_chunk_bytes >> 4) {
+                                    uint32_t a_lo = a_lo_block + row_shift + (uint32_t)sx;
+                                    uint32_t d = d0;
+                                    if (a.swap) {
+                                        // two pixel groups: four MMAs per tap keep the pipe busy (measured faster
+                                        // when the compiler schedules the address arithmetic between them)
+                                        const uint64_t bd0 = pack64(b_lo, desc_hi), bd1 = pack64(b_lo + b_kstep, desc_hi);
+                                        mma(d, bd0, pack64(a_lo, desc_hi), idesc, accumulate != 0);
+                                        mma(d, bd1, pack64(a_lo + a_kstep, desc_hi), idesc, true);
                                         mma(d + n_mma, bd0, pack64(a_lo + n_mma, desc_hi), idesc, accumulate != 0);
                                         mma(d + n_mma, bd1, pack64(a_lo + n_mma + a_kstep, desc_hi), idesc, true);
+                                    } else {
+                                        for (int m = 0; m < a.mt; ++m, a_lo += kTileM, d += (uint32_t)a.n_tile) {
+                                            mma(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, accumulate != 0);
+                                            mma(d, ((uint64_t)desc_hi << 32) | (a_lo + a_kstep),
+                                                     ((uint64_t)desc_hi << 32) | (b_lo + b_kstep), idesc, true);
+                                        }
                                     }
-                                } else {
-                                    for (int m = 0; m < a.mt; ++m, a_lo += kTileM, d += (uint32_t)a.n_tile) {
-                                        mma(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, accumulate != 0);
-                                        mma(d, ((uint64_t)desc_hi << 32) | (a_lo + a_kstep),
-                                                 ((uint64_t)desc_hi << 32) | (b_lo + b_kstep), idesc, true);
-                                    }
+                                    accumulate = 1;
+                                    if (++sx == a.S) { sx = 0; row_shift += (uint32_t)a.row_pitch; }
                                 }
-                                accumulate = 1;
-                                if (++sx == a.S) { sx = 0; row_shift += (uint32_t)a.row_pitch; }
                             }
                             if (!a.resident) {
                                 mma_commit(&b_empty[bs]);   // frees the filter stage when these MMAs have read it
