@@ -942,6 +942,7 @@ general_tc_kernel(const KernelArgs a)
                                 // table, fetched one tap ahead.
                                 const uint32_t* shift = tap_shift + t0;
                                 uint32_t cur = shift[0];
+#pragma unroll 3
                                 for (int t = 0; t < nt; ++t, b_lo += b_chunk_bytes >> 4) {
                                     const uint32_t a_lo = a_lo_block + cur;
                                     cur = shift[t + 1 < nt ? t + 1 : t];
