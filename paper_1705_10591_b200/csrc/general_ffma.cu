@@ -19,38 +19,39 @@ namespace conv2d_b200 {
 namespace {
 
 constexpr int kTileK = 64;    // filters per thread block (the paper's F_TB)
-constexpr int kTileW = 32;    // output columns per thread block
-constexpr int kTileH = 8;     // output rows per thread block
 constexpr int kThrK = 8;      // filters per thread (F_T)
 constexpr int kThrQ = 8;      // adjacent outputs per thread (W_T)
-constexpr int kThreads = (kTileK / kThrK) * (kTileW * kTileH / kThrQ);   // 8 x 32 = 256
+constexpr int kThreads = 256; // (kTileK / kThrK) = 8 filter groups x 32 output segments of kThrQ pixels
 
-template <int R, int S, int CB>
+// Image tile TW x TH outputs (TW * TH = 256): 32 x 8 for ordinary images, 16 x 16 for images of at most 16
+// output columns (a 12 x 12 map fills 56 % of one square tile but 28 % of two wide ones: 492 -> 270 us on
+// 32 x 256 x 14 x 14 with 256 filters of 3 x 3).
+template <int R, int S, int CB, int TW, int TH>
 struct Smem {
-    static constexpr int kRows = kTileH + R - 1;
-    static constexpr int kPitch = (kTileW + S - 1 + 3 + 3) / 4 * 4;   // room for whole 128-bit reads past the halo
+    static constexpr int kRows = TH + R - 1;
+    static constexpr int kPitch = (TW + S - 1 + 3 + 3) / 4 * 4;   // room for whole 128-bit reads past the halo
     float img[CB][kRows][kPitch];
     float flt[CB][R * S][kTileK + 4];   // +4: transposed filter stores spread over banks, 128-bit reads stay aligned
 };
 
-template <int R, int S, int CB>
+template <int R, int S, int CB, int TW, int TH>
 __global__ void __launch_bounds__(kThreads, 2)
 general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
                     int C, int H, int W, int K, int P, int Q, int tiles_q, int vec_st)
 {
-    using SM = Smem<R, S, CB>;
+    using SM = Smem<R, S, CB, TW, TH>;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SM& sm = *reinterpret_cast<SM*>(smem_raw);
 
     const int tid = threadIdx.x;
     const int tx = tid % (kTileK / kThrK);            // filter group: adjacent threads, adjacent filter units
     const int ty = tid / (kTileK / kThrK);            // output segment
-    const int seg_row = ty / (kTileW / kThrQ);
-    const int seg_col = (ty % (kTileW / kThrQ)) * kThrQ;
+    const int seg_row = ty / (TW / kThrQ);
+    const int seg_col = (ty % (TW / kThrQ)) * kThrQ;
 
     const int k0 = blockIdx.y * kTileK;
     const int tq = blockIdx.x % tiles_q, tp = blockIdx.x / tiles_q;
-    const int p0 = tp * kTileH, q0 = tq * kTileW;
+    const int p0 = tp * TH, q0 = tq * TW;
     const int n = blockIdx.z;
     const float* xin = x + (size_t)n * C * H * W;
 
@@ -141,21 +142,28 @@ general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
     }
 }
 
-template <int R, int S, int CB>
-conv2d_status_t launch_instance(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
+template <int R, int S, int CB, int TW, int TH>
+conv2d_status_t launch_tile(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
 {
-    auto kern = general_ffma_kernel<R, S, CB>;
-    const size_t smem = sizeof(Smem<R, S, CB>);
+    auto kern = general_ffma_kernel<R, S, CB, TW, TH>;
+    const size_t smem = sizeof(Smem<R, S, CB, TW, TH>);
     if (smem > 48 * 1024) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return CONV2D_ERR_CUDA;
     }
-    const int tiles_q = (sh.Q + kTileW - 1) / kTileW, tiles_p = (sh.P + kTileH - 1) / kTileH;
+    const int tiles_q = (sh.Q + TW - 1) / TW, tiles_p = (sh.P + TH - 1) / TH;
     dim3 grid(tiles_q * tiles_p, (sh.K + kTileK - 1) / kTileK, sh.N);
     const int vec_st = (sh.Q % 4 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
     kern<<<grid, kThreads, smem, stream>>>(x, w, y, sh.C, sh.H, sh.W, sh.K, sh.P, sh.Q, tiles_q, vec_st);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
+template <int R, int S, int CB>
+conv2d_status_t launch_instance(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
+{
+    if (sh.Q <= 16) return launch_tile<R, S, CB, 16, 16>(x, w, y, sh, stream);
+    return launch_tile<R, S, CB, 32, 8>(x, w, y, sh, stream);
 }
 
 // One thread per output, loops over c, r, s in that order: correct for every shape, tuned for none.
