@@ -25,6 +25,27 @@ conv2d_status_t make_shape(int N, int C, int H, int W, int K, int R, int S, Shap
     return CONV2D_OK;
 }
 
+// Zero extension of every H x W plane by pad_h rows above and below and pad_w columns left and right.
+__global__ void pad_planes_kernel(const float* __restrict__ x, float* __restrict__ xp, long long planes,
+                                  int H, int W, int pad_h, int pad_w, unsigned* status_to_clear)
+{
+    // (the fp32 path has no kernel that clears the status block in front of the workspace)
+    if (status_to_clear && blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status_to_clear[threadIdx.x] = 0u;
+    const int Hp = H + 2 * pad_h, Wp = W + 2 * pad_w;
+    const long long total = planes * Hp * Wp;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int wc = (int)(i % Wp) - pad_w;
+        const int h = (int)((i / Wp) % Hp) - pad_h;
+        const long long plane = i / ((long long)Wp * Hp);
+        float v = 0.f;
+        if (h >= 0 && h < H && wc >= 0 && wc < W) v = __ldg(x + (plane * H + h) * W + wc);
+        xp[i] = v;
+    }
+}
+
+size_t round_up_256(size_t v) { return (v + 255) / 256 * 256; }
+
 conv2d_status_t check_device()
 {
     int dev = 0;
@@ -134,6 +155,48 @@ conv2d_status_t conv2d_fwd_general_16bit(const void* x16, const void* w16, float
     if (st != CONV2D_OK) return st;
     return launch_general_b16(x16, w16, y, sh, operand == CONV2D_OPERAND_FP16, workspace,
                               (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+conv2d_status_t conv2d_fwd_padded_workspace_size(int N, int C, int H, int W, int K, int R, int S, int pad_h, int pad_w,
+                                                 conv2d_algo_t algo, size_t* bytes)
+{
+    if (!bytes) return CONV2D_ERR_NULL;
+    *bytes = 0;
+    if (pad_h < 0 || pad_w < 0 || pad_h > 4096 || pad_w > 4096 || H <= 0 || W <= 0) return CONV2D_ERR_SHAPE;
+    size_t inner = 0;
+    const conv2d_status_t st = conv2d_fwd_workspace_size(N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, algo, &inner);
+    if (st != CONV2D_OK) return st;
+    if (inner < kStatusBytes) inner = kStatusBytes;      // the status block is there for every algorithm
+    *bytes = round_up_256(inner) + (size_t)N * C * (H + 2 * pad_h) * (W + 2 * pad_w) * sizeof(float);
+    return CONV2D_OK;
+}
+
+conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float* y,
+                                          int N, int C, int H, int W, int K, int R, int S, int pad_h, int pad_w,
+                                          conv2d_algo_t algo, void* workspace, size_t workspace_bytes,
+                                          unsigned flags, void* cuda_stream)
+{
+    if (!x || !w || !y || !workspace) return CONV2D_ERR_NULL;
+    size_t need = 0, inner = 0;
+    conv2d_status_t st = conv2d_fwd_padded_workspace_size(N, C, H, W, K, R, S, pad_h, pad_w, algo, &need);
+    if (st != CONV2D_OK) return st;
+    if (!aligned16(x) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (workspace_bytes < need) return CONV2D_ERR_WORKSPACE;
+    st = conv2d_fwd_workspace_size(N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, algo, &inner);
+    if (st != CONV2D_OK) return st;
+    st = check_device();
+    if (st != CONV2D_OK) return st;
+    const bool own_status = inner < kStatusBytes;          // fp32 path: no workspace of its own
+    float* xp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + round_up_256(own_status ? kStatusBytes : inner));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const long long total = (long long)N * C * (H + 2 * pad_h) * (W + 2 * pad_w);
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    pad_planes_kernel<<<(unsigned)blocks, 256, 0, stream>>>(x, xp, (long long)N * C, H, W, pad_h, pad_w,
+                                                            own_status ? static_cast<unsigned*>(workspace) : nullptr);
+    count_launch(1);
+    if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
+    return conv2d_fwd_general(xp, w, y, N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, algo, workspace, inner, flags, cuda_stream);
 }
 
 conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float* y,

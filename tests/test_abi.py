@@ -111,3 +111,17 @@ def test_workspace_query_over_many_shapes_is_consistent(lib):
         assert lib.conv2d_fwd_workspace_size(N, C, HW, HW, K, R, R, lib.ALGO_AUTO) == tf32
         assert lib.conv2d_fwd_workspace_size(N, C, HW, HW, K, R, R, lib.ALGO_FFMA) == 0
     assert seen > 100
+
+
+def test_padded_workspace_query(lib):
+    plain = lib.conv2d_fwd_workspace_size(2, 16, 22, 22, 32, 3, 3, lib.ALGO_TF32)
+    padded = lib.conv2d_fwd_padded_workspace_size(2, 16, 20, 20, 32, 3, 3, 1, 1, lib.ALGO_TF32)
+    assert padded >= plain + 2 * 16 * 22 * 22 * 4          # the general workspace of the extended image + that image
+    assert lib.conv2d_fwd_padded_workspace_size(2, 16, 20, 20, 32, 3, 3, 1, 1, lib.ALGO_FFMA) == 256 + 2 * 16 * 22 * 22 * 4
+    with pytest.raises(lib.Conv2dError) as e:
+        lib.conv2d_fwd_padded_workspace_size(2, 16, 20, 20, 32, 3, 3, -1, 0, lib.ALGO_FFMA)
+    assert e.value.status == 2
+    # a filter larger than the image becomes legal once the padding makes room for it
+    assert lib.conv2d_fwd_padded_workspace_size(1, 4, 3, 3, 8, 5, 5, 1, 1, lib.ALGO_FFMA) > 0
+    with pytest.raises(lib.Conv2dError):
+        lib.conv2d_fwd_padded_workspace_size(1, 4, 3, 3, 8, 7, 7, 1, 1, lib.ALGO_FFMA)
