@@ -163,6 +163,25 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
                                           unsigned flags, void* cuda_stream);
 
 /*
+ * General case with zero padding and a stride (not in the paper, which has stride 1):
+ *   y[n,k,p,q] = sum_{c,r,s} xz[n,c,stride*p+r-pad_h,stride*q+s-pad_w] * w[k,c,r,s],
+ *   P = (H + 2*pad_h - R) / stride + 1, Q = (W + 2*pad_w - S) / stride + 1 (integer division), y [N][K][P][Q].
+ * The call rewrites the problem as a stride-1 convolution over stride*stride times as many channels
+ * ("space to depth": channel (c,a,b) of the rewritten image holds the pixels whose row is a and whose column
+ * is b modulo the stride; the filters are split the same way) with two extra kernels into the workspace and
+ * then runs conv2d_fwd_general on it: the same multiply-adds as the definition plus zeros, every algorithm.
+ * 1 <= stride <= 8.  Workspace from conv2d_fwd_strided_workspace_size; required, 16-byte aligned, status
+ * block first.  With CONV2D_FLAG_WEIGHTS_PACKED the rewritten filters of the previous call are reused too.
+ */
+conv2d_status_t conv2d_fwd_strided_workspace_size(int N, int C, int H, int W, int K, int R, int S,
+                                                  int pad_h, int pad_w, int stride, conv2d_algo_t algo, size_t* bytes);
+conv2d_status_t conv2d_fwd_general_strided(const float* x, const float* w, float* y,
+                                           int N, int C, int H, int W, int K, int R, int S,
+                                           int pad_h, int pad_w, int stride, conv2d_algo_t algo,
+                                           void* workspace, size_t workspace_bytes,
+                                           unsigned flags, void* cuda_stream);
+
+/*
  * General case on the tensor cores for callers that cannot hand over scratch memory.
  * (The paper has no counterpart; this is a packaging variant of conv2d_fwd_general with
  * algo = CONV2D_ALGO_TF32, same kernels, same results.)

@@ -53,6 +53,10 @@ def load_library() -> ctypes.CDLL:
     lib.conv2d_fwd_padded_workspace_size.restype = i
     lib.conv2d_fwd_general_padded.argtypes = [vp, vp, vp] + [i] * 9 + [i, vp, sz, u, vp]
     lib.conv2d_fwd_general_padded.restype = i
+    lib.conv2d_fwd_strided_workspace_size.argtypes = [i] * 10 + [i, ctypes.POINTER(sz)]
+    lib.conv2d_fwd_strided_workspace_size.restype = i
+    lib.conv2d_fwd_general_strided.argtypes = [vp, vp, vp] + [i] * 10 + [i, vp, sz, u, vp]
+    lib.conv2d_fwd_general_strided.restype = i
     lib.conv2d_fwd_general_noalloc.argtypes = [vp, vp, vp] + [i] * 7 + [i, vp]
     lib.conv2d_fwd_general_noalloc.restype = i
     lib.conv2d_fwd_host.argtypes = [vp] * 6 + [i] * 7 + [i, vp, sz, vp]
@@ -122,6 +126,21 @@ def conv2d_fwd_general_padded(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, pad_h, p
     _check(load_library().conv2d_fwd_general_padded(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, pad_h, pad_w, algo,
                                                     workspace_ptr or None, workspace_bytes, flags, stream or None),
            "conv2d_fwd_general_padded")
+
+
+def conv2d_fwd_strided_workspace_size(N, C, H, W, K, R, S, pad_h, pad_w, stride, algo=ALGO_AUTO) -> int:
+    out = ctypes.c_size_t(0)
+    _check(load_library().conv2d_fwd_strided_workspace_size(N, C, H, W, K, R, S, pad_h, pad_w, stride, algo,
+                                                            ctypes.byref(out)), "conv2d_fwd_strided_workspace_size")
+    return int(out.value)
+
+
+def conv2d_fwd_general_strided(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, pad_h, pad_w, stride, algo=ALGO_AUTO,
+                               workspace_ptr=0, workspace_bytes=0, flags=0, stream=0) -> None:
+    """Zero padding and stride; y is [N, K, (H+2*pad_h-R)//stride+1, (W+2*pad_w-S)//stride+1]."""
+    _check(load_library().conv2d_fwd_general_strided(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, pad_h, pad_w, stride, algo,
+                                                     workspace_ptr or None, workspace_bytes, flags, stream or None),
+           "conv2d_fwd_general_strided")
 
 
 def conv2d_fwd_general_noalloc(x_ptr, w_ptr, y_ptr, N, C, H, W, K, R, S, wait=0, stream=0) -> None:

@@ -46,6 +46,66 @@ __global__ void pad_planes_kernel(const float* __restrict__ x, float* __restrict
 
 size_t round_up_256(size_t v) { return (v + 255) / 256 * 256; }
 
+// Strided convolution as a stride-1 convolution over stride*stride times as many channels ("space to depth"):
+//   x2[n][(c*st + a)*st + b][h2][w2] = xz[n][c][st*h2 + a][st*w2 + b]      (xz = zero-padded x, 0 outside)
+//   w2[k][(c*st + a)*st + b][r2][s2] = w[k][c][st*r2 + a][st*s2 + b]       (0 where st*r2 + a >= R or st*s2 + b >= S)
+// so that sum_{c,r,s} xz[c][st*p + r][st*q + s] w[k][c][r][s] = sum over (c,a,b),(r2,s2) of x2[..][p + r2][q + s2] w2[..].
+__global__ void space_to_depth_kernel(const float* __restrict__ x, float* __restrict__ x2, int N, int C, int H, int W,
+                                      int pad_h, int pad_w, int st, int H2, int W2, unsigned* status_to_clear)
+{
+    if (status_to_clear && blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status_to_clear[threadIdx.x] = 0u;
+    const long long total = (long long)N * C * st * st * H2 * W2;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        long long r = i;
+        const int w2 = (int)(r % W2); r /= W2;
+        const int h2 = (int)(r % H2); r /= H2;
+        const int b = (int)(r % st); r /= st;
+        const int a = (int)(r % st); r /= st;
+        const int c = (int)(r % C); r /= C;
+        const int n = (int)r;
+        const int h = st * h2 + a - pad_h, wc = st * w2 + b - pad_w;
+        float v = 0.f;
+        if (h >= 0 && h < H && wc >= 0 && wc < W) v = __ldg(x + (((size_t)n * C + c) * H + h) * W + wc);
+        x2[i] = v;
+    }
+}
+__global__ void filters_to_depth_kernel(const float* __restrict__ w, float* __restrict__ w2, int K, int C, int R, int S,
+                                        int st, int R2, int S2)
+{
+    const long long total = (long long)K * C * st * st * R2 * S2;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        long long r = i;
+        const int s2 = (int)(r % S2); r /= S2;
+        const int r2 = (int)(r % R2); r /= R2;
+        const int b = (int)(r % st); r /= st;
+        const int a = (int)(r % st); r /= st;
+        const int c = (int)(r % C); r /= C;
+        const int k = (int)r;
+        const int rr = st * r2 + a, ss = st * s2 + b;
+        w2[i] = (rr < R && ss < S) ? __ldg(w + (((size_t)k * C + c) * R + rr) * S + ss) : 0.f;
+    }
+}
+
+// Derived sizes of the strided problem; returns false on a bad argument.
+struct StridedGeom { int P, Q, C2, H2, W2, R2, S2; };
+bool strided_geom(int C, int H, int W, int R, int S, int pad_h, int pad_w, int st, StridedGeom* g)
+{
+    if (st < 1 || st > 8 || pad_h < 0 || pad_w < 0 || pad_h > 4096 || pad_w > 4096) return false;
+    if (C <= 0 || H <= 0 || W <= 0 || R <= 0 || S <= 0 || C > (1 << 20)) return false;
+    const int Hz = H + 2 * pad_h, Wz = W + 2 * pad_w;
+    if (R > Hz || S > Wz) return false;
+    g->P = (Hz - R) / st + 1;
+    g->Q = (Wz - S) / st + 1;
+    g->R2 = (R + st - 1) / st;
+    g->S2 = (S + st - 1) / st;
+    g->C2 = C * st * st;
+    g->H2 = g->P + g->R2 - 1;
+    g->W2 = g->Q + g->S2 - 1;
+    return true;
+}
+
 conv2d_status_t check_device()
 {
     int dev = 0;
@@ -197,6 +257,56 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
     count_launch(1);
     if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
     return conv2d_fwd_general(xp, w, y, N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, algo, workspace, inner, flags, cuda_stream);
+}
+
+conv2d_status_t conv2d_fwd_strided_workspace_size(int N, int C, int H, int W, int K, int R, int S, int pad_h, int pad_w,
+                                                  int stride, conv2d_algo_t algo, size_t* bytes)
+{
+    if (!bytes) return CONV2D_ERR_NULL;
+    *bytes = 0;
+    StridedGeom g;
+    if (N <= 0 || K <= 0 || !strided_geom(C, H, W, R, S, pad_h, pad_w, stride, &g)) return CONV2D_ERR_SHAPE;
+    size_t inner = 0;
+    const conv2d_status_t st = conv2d_fwd_workspace_size(N, g.C2, g.H2, g.W2, K, g.R2, g.S2, algo, &inner);
+    if (st != CONV2D_OK) return st;
+    if (inner < kStatusBytes) inner = kStatusBytes;
+    *bytes = round_up_256(inner) + round_up_256((size_t)N * g.C2 * g.H2 * g.W2 * sizeof(float))
+           + (size_t)K * g.C2 * g.R2 * g.S2 * sizeof(float);
+    return CONV2D_OK;
+}
+
+conv2d_status_t conv2d_fwd_general_strided(const float* x, const float* w, float* y,
+                                           int N, int C, int H, int W, int K, int R, int S, int pad_h, int pad_w, int stride,
+                                           conv2d_algo_t algo, void* workspace, size_t workspace_bytes,
+                                           unsigned flags, void* cuda_stream)
+{
+    if (!x || !w || !y || !workspace) return CONV2D_ERR_NULL;
+    size_t need = 0, inner = 0;
+    conv2d_status_t st = conv2d_fwd_strided_workspace_size(N, C, H, W, K, R, S, pad_h, pad_w, stride, algo, &need);
+    if (st != CONV2D_OK) return st;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (workspace_bytes < need) return CONV2D_ERR_WORKSPACE;
+    StridedGeom g;
+    strided_geom(C, H, W, R, S, pad_h, pad_w, stride, &g);
+    st = conv2d_fwd_workspace_size(N, g.C2, g.H2, g.W2, K, g.R2, g.S2, algo, &inner);
+    if (st != CONV2D_OK) return st;
+    st = check_device();
+    if (st != CONV2D_OK) return st;
+    const bool own_status = inner < kStatusBytes;
+    unsigned char* base = static_cast<unsigned char*>(workspace);
+    float* x2 = reinterpret_cast<float*>(base + round_up_256(own_status ? kStatusBytes : inner));
+    float* w2 = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(x2) + round_up_256((size_t)N * g.C2 * g.H2 * g.W2 * sizeof(float)));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    auto blocks_for = [](long long total) { long long b = (total + 255) / 256; return (unsigned)(b > 148 * 32 ? 148 * 32 : b); };
+    space_to_depth_kernel<<<blocks_for((long long)N * g.C2 * g.H2 * g.W2), 256, 0, stream>>>(
+        x, x2, N, C, H, W, pad_h, pad_w, stride, g.H2, g.W2, own_status ? static_cast<unsigned*>(workspace) : nullptr);
+    count_launch(1);
+    if (!(flags & CONV2D_FLAG_WEIGHTS_PACKED)) {
+        filters_to_depth_kernel<<<blocks_for((long long)K * g.C2 * g.R2 * g.S2), 256, 0, stream>>>(w, w2, K, C, R, S, stride, g.R2, g.S2);
+        count_launch(1);
+    }
+    if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
+    return conv2d_fwd_general(x2, w2, y, N, g.C2, g.H2, g.W2, K, g.R2, g.S2, algo, workspace, inner, flags, cuda_stream);
 }
 
 conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float* y,

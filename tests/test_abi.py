@@ -125,3 +125,13 @@ def test_padded_workspace_query(lib):
     assert lib.conv2d_fwd_padded_workspace_size(1, 4, 3, 3, 8, 5, 5, 1, 1, lib.ALGO_FFMA) > 0
     with pytest.raises(lib.Conv2dError):
         lib.conv2d_fwd_padded_workspace_size(1, 4, 3, 3, 8, 7, 7, 1, 1, lib.ALGO_FFMA)
+
+
+def test_strided_workspace_query(lib):
+    # 224 x 224 RGB, 7 x 7, pad 3, stride 2 -> 112 x 112 outputs; rewritten as 12 channels of 115 x 115 with 4 x 4 filters
+    n = lib.conv2d_fwd_strided_workspace_size(2, 3, 224, 224, 64, 7, 7, 3, 3, 2, lib.ALGO_FFMA)
+    assert n >= 256 + 2 * 12 * 115 * 115 * 4 + 64 * 12 * 4 * 4 * 4
+    for bad in (0, 9, -1):
+        with pytest.raises(lib.Conv2dError) as e:
+            lib.conv2d_fwd_strided_workspace_size(2, 3, 224, 224, 64, 7, 7, 3, 3, bad, lib.ALGO_FFMA)
+        assert e.value.status == 2
