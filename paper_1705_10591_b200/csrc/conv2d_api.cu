@@ -26,21 +26,20 @@ conv2d_status_t make_shape(int N, int C, int H, int W, int K, int R, int S, Shap
 }
 
 // Zero extension of every H x W plane by pad_h rows above and below and pad_w columns left and right.
-__global__ void pad_planes_kernel(const float* __restrict__ x, float* __restrict__ xp, long long planes,
-                                  int H, int W, int pad_h, int pad_w, unsigned* status_to_clear)
+// One block row (blockIdx.y) per plane, 32-bit arithmetic inside a plane.
+__global__ void pad_planes_kernel(const float* __restrict__ x, float* __restrict__ xp, int H, int W, int pad_h, int pad_w,
+                                  unsigned* status_to_clear)
 {
     // (the fp32 path has no kernel that clears the status block in front of the workspace)
-    if (status_to_clear && blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status_to_clear[threadIdx.x] = 0u;
+    if (status_to_clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned))
+        status_to_clear[threadIdx.x] = 0u;
     const int Hp = H + 2 * pad_h, Wp = W + 2 * pad_w;
-    const long long total = planes * Hp * Wp;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-        const int wc = (int)(i % Wp) - pad_w;
-        const int h = (int)((i / Wp) % Hp) - pad_h;
-        const long long plane = i / ((long long)Wp * Hp);
-        float v = 0.f;
-        if (h >= 0 && h < H && wc >= 0 && wc < W) v = __ldg(x + (plane * H + h) * W + wc);
-        xp[i] = v;
+    const float* src = x + (size_t)blockIdx.y * H * W;
+    float* dst = xp + (size_t)blockIdx.y * Hp * Wp;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < Hp * Wp; i += gridDim.x * blockDim.x) {
+        const int hp = i / Wp;
+        const int h = hp - pad_h, wc = i - hp * Wp - pad_w;
+        dst[i] = (h >= 0 && h < H && wc >= 0 && wc < W) ? __ldg(src + h * W + wc) : 0.f;
     }
 }
 
@@ -50,24 +49,21 @@ size_t round_up_256(size_t v) { return (v + 255) / 256 * 256; }
 //   x2[n][(c*st + a)*st + b][h2][w2] = xz[n][c][st*h2 + a][st*w2 + b]      (xz = zero-padded x, 0 outside)
 //   w2[k][(c*st + a)*st + b][r2][s2] = w[k][c][st*r2 + a][st*s2 + b]       (0 where st*r2 + a >= R or st*s2 + b >= S)
 // so that sum_{c,r,s} xz[c][st*p + r][st*q + s] w[k][c][r][s] = sum over (c,a,b),(r2,s2) of x2[..][p + r2][q + s2] w2[..].
-__global__ void space_to_depth_kernel(const float* __restrict__ x, float* __restrict__ x2, int N, int C, int H, int W,
+__global__ void space_to_depth_kernel(const float* __restrict__ x, float* __restrict__ x2, int H, int W,
                                       int pad_h, int pad_w, int st, int H2, int W2, unsigned* status_to_clear)
 {
-    if (status_to_clear && blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status_to_clear[threadIdx.x] = 0u;
-    const long long total = (long long)N * C * st * st * H2 * W2;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-        long long r = i;
-        const int w2 = (int)(r % W2); r /= W2;
-        const int h2 = (int)(r % H2); r /= H2;
-        const int b = (int)(r % st); r /= st;
-        const int a = (int)(r % st); r /= st;
-        const int c = (int)(r % C); r /= C;
-        const int n = (int)r;
+    if (status_to_clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned))
+        status_to_clear[threadIdx.x] = 0u;
+    // blockIdx.y = source plane (n, c); it produces the st*st planes (a, b) of the rewritten image
+    const float* src = x + (size_t)blockIdx.y * H * W;
+    float* dst = x2 + (size_t)blockIdx.y * st * st * H2 * W2;
+    const int per_plane = H2 * W2, total = st * st * per_plane;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const int ab = i / per_plane, rem = i - ab * per_plane;
+        const int a = ab / st, b = ab - a * st;
+        const int h2 = rem / W2, w2 = rem - h2 * W2;
         const int h = st * h2 + a - pad_h, wc = st * w2 + b - pad_w;
-        float v = 0.f;
-        if (h >= 0 && h < H && wc >= 0 && wc < W) v = __ldg(x + (((size_t)n * C + c) * H + h) * W + wc);
-        x2[i] = v;
+        dst[i] = (h >= 0 && h < H && wc >= 0 && wc < W) ? __ldg(src + h * W + wc) : 0.f;
     }
 }
 __global__ void filters_to_depth_kernel(const float* __restrict__ w, float* __restrict__ w2, int K, int C, int R, int S,
@@ -249,11 +245,10 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
     const bool own_status = inner < kStatusBytes;          // fp32 path: no workspace of its own
     float* xp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + round_up_256(own_status ? kStatusBytes : inner));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const long long total = (long long)N * C * (H + 2 * pad_h) * (W + 2 * pad_w);
-    long long blocks = (total + 255) / 256;
-    if (blocks > 148 * 32) blocks = 148 * 32;
-    pad_planes_kernel<<<(unsigned)blocks, 256, 0, stream>>>(x, xp, (long long)N * C, H, W, pad_h, pad_w,
-                                                            own_status ? static_cast<unsigned*>(workspace) : nullptr);
+    if ((long long)N * C > 65535) return CONV2D_ERR_UNSUPPORTED;
+    const int plane_p = (H + 2 * pad_h) * (W + 2 * pad_w);
+    const dim3 grid((unsigned)((plane_p + 1023) / 1024 > 64 ? 64 : (plane_p + 1023) / 1024), (unsigned)(N * C));
+    pad_planes_kernel<<<grid, 256, 0, stream>>>(x, xp, H, W, pad_h, pad_w, own_status ? static_cast<unsigned*>(workspace) : nullptr);
     count_launch(1);
     if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
     return conv2d_fwd_general(xp, w, y, N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, algo, workspace, inner, flags, cuda_stream);
@@ -298,8 +293,13 @@ conv2d_status_t conv2d_fwd_general_strided(const float* x, const float* w, float
     float* w2 = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(x2) + round_up_256((size_t)N * g.C2 * g.H2 * g.W2 * sizeof(float)));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     auto blocks_for = [](long long total) { long long b = (total + 255) / 256; return (unsigned)(b > 148 * 32 ? 148 * 32 : b); };
-    space_to_depth_kernel<<<blocks_for((long long)N * g.C2 * g.H2 * g.W2), 256, 0, stream>>>(
-        x, x2, N, C, H, W, pad_h, pad_w, stride, g.H2, g.W2, own_status ? static_cast<unsigned*>(workspace) : nullptr);
+    if ((long long)N * C > 65535) return CONV2D_ERR_UNSUPPORTED;
+    {
+        const int work = stride * stride * g.H2 * g.W2;
+        const dim3 grid((unsigned)((work + 1023) / 1024 > 64 ? 64 : (work + 1023) / 1024), (unsigned)(N * C));
+        space_to_depth_kernel<<<grid, 256, 0, stream>>>(x, x2, H, W, pad_h, pad_w, stride, g.H2, g.W2,
+                                                        own_status ? static_cast<unsigned*>(workspace) : nullptr);
+    }
     count_launch(1);
     if (!(flags & CONV2D_FLAG_WEIGHTS_PACKED)) {
         filters_to_depth_kernel<<<blocks_for((long long)K * g.C2 * g.R2 * g.S2), 256, 0, stream>>>(w, w2, K, C, R, S, stride, g.R2, g.S2);

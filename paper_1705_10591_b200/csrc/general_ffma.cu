@@ -204,7 +204,9 @@ conv2d_status_t launch_general_ffma(const float* x, const float* w, float* y, co
 {
     if (sh.N > 65535 || (sh.K + kTileK - 1) / kTileK > 65535) return launch_direct_fallback(x, w, y, sh, stream);
     if (sh.R == 1 && sh.S == 1) return launch_instance<1, 1, 16>(x, w, y, sh, stream);
+    if (sh.R == 2 && sh.S == 2) return launch_instance<2, 2, 8>(x, w, y, sh, stream);      // (stride-2 rewriting of 3 x 3)
     if (sh.R == 3 && sh.S == 3) return launch_instance<3, 3, 8>(x, w, y, sh, stream);
+    if (sh.R == 4 && sh.S == 4) return launch_instance<4, 4, 4>(x, w, y, sh, stream);      // (stride-2 rewriting of 7 x 7)
     if (sh.R == 5 && sh.S == 5) return launch_instance<5, 5, 4>(x, w, y, sh, stream);
     if (sh.R == 7 && sh.S == 7) return launch_instance<7, 7, 2>(x, w, y, sh, stream);
     return launch_direct_fallback(x, w, y, sh, stream);

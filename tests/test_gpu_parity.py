@@ -119,6 +119,8 @@ GENERAL_SHAPES = [
     (2, 6, 15, 44, 9, 7, 7),
     (3, 32, 9, 9, 16, 1, 1),
     (1, 4, 11, 10, 3, 2, 4),       # rectangular taps -> shape-agnostic kernel
+    (2, 12, 19, 21, 70, 2, 2),     # 2 x 2 and 4 x 4 taps: the filters a stride-2 rewriting produces
+    (1, 12, 23, 40, 33, 4, 4),
     (2, 5, 3, 3, 4, 3, 3),         # one output per map
     (1, 64, 14, 14, 96, 3, 3),     # 96 filters: operand-swap path with zero-padded filters
     (2, 20, 10, 12, 300, 3, 3),    # 300 filters: two filter blocks, partial last channel block
