@@ -148,8 +148,9 @@ conv2d_status_t conv2d_fwd_general_16bit(const void* x16, const void* w16, float
  * variant users of convolution layers ask for):
  *   y[n,k,p,q] = sum_{c,r,s} xz[n,c,p+r-pad_h,q+s-pad_w] * w[k,c,r,s],  xz = x inside the image, 0 outside,
  *   P = H + 2*pad_h - R + 1, Q = W + 2*pad_w - S + 1, y [N][K][P][Q].
- * The call zero-extends x into the workspace with one extra kernel and then runs conv2d_fwd_general on the
- * extended image, so every algorithm and every property of that entry applies.  The workspace size comes
+ * With the tensor-core algorithms the kernel applies the padding while it stages the image; otherwise the call
+ * zero-extends x into the workspace with one extra kernel and then runs conv2d_fwd_general on the extended
+ * image.  Every algorithm and every property of that entry applies.  The workspace size comes
  * from conv2d_fwd_padded_workspace_size (the general workspace for the extended image, then the extended
  * image itself); it is required for every algorithm, 16-byte aligned, and its first 256 bytes are the
  * status block as usual.  pad_h, pad_w >= 0.  CONV2D_FLAG_WEIGHTS_PACKED keeps its meaning.

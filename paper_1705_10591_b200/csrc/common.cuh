@@ -12,6 +12,7 @@ namespace conv2d_b200 {
 // Problem extents, library symbols (N images, C channels, H x W image, K filters, R x S taps).
 struct Shape {
     int N, C, H, W, K, R, S, P, Q;
+    int pad_h = 0, pad_w = 0;   // zero padding; only the tensor-core path with patch addressing takes it natively
 };
 
 // Capacity of the per-device constant-memory filter bank of the single-channel kernel, in floats.

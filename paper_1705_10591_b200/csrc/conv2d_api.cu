@@ -242,6 +242,17 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
     if (st != CONV2D_OK) return st;
     st = check_device();
     if (st != CONV2D_OK) return st;
+    // The tensor-core kernel takes the padding itself where it has an instance with patch addressing (no extra
+    // pass over x); its workspace is the front part of this call's workspace as usual.
+    if (algo != CONV2D_ALGO_FFMA && (pad_h || pad_w) && aligned16(w) && aligned16(y)) {
+        Shape shp;
+        if (make_shape(N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, &shp) == CONV2D_OK) {
+            shp.H = H; shp.W = W; shp.pad_h = pad_h; shp.pad_w = pad_w;       // P, Q are those of the extended image
+            if (tf32_supported(shp) && tf32_workspace_bytes(shp) <= workspace_bytes)
+                return launch_general_tf32(x, w, y, shp, workspace, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0,
+                                           static_cast<cudaStream_t>(cuda_stream));
+        }
+    }
     const bool own_status = inner < kStatusBytes;          // fp32 path: no workspace of its own
     float* xp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + round_up_256(own_status ? kStatusBytes : inner));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -281,6 +292,8 @@ conv2d_status_t conv2d_fwd_general_strided(const float* x, const float* w, float
     if (st != CONV2D_OK) return st;
     if (!aligned16(x) || !aligned16(w) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
     if (workspace_bytes < need) return CONV2D_ERR_WORKSPACE;
+    if (stride == 1)            // nothing to rewrite: the padded entry (its workspace is a prefix of this one's)
+        return conv2d_fwd_general_padded(x, w, y, N, C, H, W, K, R, S, pad_h, pad_w, algo, workspace, workspace_bytes, flags, cuda_stream);
     StridedGeom g;
     strided_geom(C, H, W, R, S, pad_h, pad_w, stride, &g);
     st = conv2d_fwd_workspace_size(N, g.C2, g.H2, g.W2, K, g.R2, g.S2, algo, &inner);

@@ -171,7 +171,9 @@ Plan make_plan(const Shape& sh, bool b16 = false)
     // 3 channels 7 x 7 on 224 x 224: 0.91 ms folded, 1.06 ms not; 1 channel 5 x 5: 0.32 vs 0.40 ms; but
     // 8 channels 3 x 3 on 112 x 112: 0.175 vs 0.093 ms).  CONV2D_B200_TF32_FOLD = 2 folds whenever C < 16.
     p.fold_r = p.fold_s = 1;
-    const int fold_mode = env_int("CONV2D_B200_TF32_FOLD", 1);
+    const bool padded = sh.pad_h != 0 || sh.pad_w != 0;      // needs patch addressing: no folding, filters as M
+    if (padded && !p.swap) return p;
+    const int fold_mode = padded ? 0 : env_int("CONV2D_B200_TF32_FOLD", 1);
     if (sh.C < cbc && (fold_mode == 2 || (fold_mode == 1 && sh.C <= 3))) {
         long long best = (long long)sh.R * sh.S * ((sh.C + cbc - 1) / cbc);
         const int cand[3][2] = {{1, sh.S}, {sh.R, 1}, {sh.R, sh.S}};
@@ -194,7 +196,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
     // pixels per output wins.
     p.patch_w = p.patch_tw = p.patch_rows = p.patch_cols = 0;
     const long long flat_halo = (long long)(r_eff - 1) * sh.W + (s_eff - 1);
-    const int patch_mode = env_int("CONV2D_B200_TF32_PATCH", 1);       // 0 never, 1 when the flat halo is large, 2 always
+    const int patch_mode = padded ? 2 : env_int("CONV2D_B200_TF32_PATCH", 1);       // 0 never, 1 when the flat halo is large, 2 always
     if (p.swap && p.fold_r * p.fold_s == 1 && patch_mode != 0) {
         double best_ratio = 0;
         for (int wp = 32; wp <= 128; wp *= 2) {
@@ -213,6 +215,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
         if (patch_mode == 1 && !(flat_ratio > 1.75 * best_ratio)) p.patch_w = p.patch_tw = 0;
         if (p.patch_w) p.patch_cols = (sh.Q + p.patch_tw - 1) / p.patch_tw;
     }
+    if (padded && !p.patch_w) return p;
     const long long halo = p.patch_w ? (long long)(r_eff - 1) * p.patch_w + (s_eff - 1) : flat_halo;
     // work items along the pixels for an item of px pixels (0: px is not possible in this mode)
     auto pixel_items = [&](int px) -> long long {
@@ -510,6 +513,7 @@ struct KernelArgs {
     int n_tile, n_blocks, mt, tile_px, px_groups, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
     int patch_w, patch_tw, patch_rows, patch_cols;   // patch addressing (PATCH kernels): staged row pitch, valid output
                                                       // columns per patch row, patches per image down and across
+    int pad_h, pad_w; // zero padding (patch addressing only): staged pixel (row, col) is image pixel (row - pad_h, col - pad_w)
     int row_pitch;    // pixels between vertically adjacent taps in the staged sequence: W, or patch_w
     int fp16;         // 16-bit operands only: 1 = IEEE half, 0 = bf16
     int fold_r, fold_s;  // taps folded into the channel dimension (1, 1: none); R, S below are what is left as shifts
@@ -545,10 +549,10 @@ __device__ __forceinline__ bool staged_pixel(const KernelArgs& a, const ItemGeom
 {
     if (PATCH) {
         const int prow = jj / a.patch_w, pcol = jj - prow * a.patch_w;
-        const int h = g.row0 + prow, wc = g.col0 + pcol;
+        const int h = g.row0 + prow - a.pad_h, wc = g.col0 + pcol - a.pad_w;
         n = g.n;
         off = h * a.W + wc;
-        return h < a.H && wc < a.W;
+        return (unsigned)h < (unsigned)a.H && (unsigned)wc < (unsigned)a.W;
     }
     const int j = g.j0 + jj;
     n = j / a.HW;
@@ -1333,6 +1337,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     a.N = sh.N; a.C = sh.C; a.H = sh.H; a.W = sh.W; a.K = sh.K; a.P = sh.P; a.Q = sh.Q;
     a.patch_w = p.patch_w; a.patch_tw = p.patch_tw; a.patch_rows = p.patch_rows; a.patch_cols = p.patch_cols;
     a.row_pitch = p.patch_w ? p.patch_w : sh.W;
+    a.pad_h = sh.pad_h; a.pad_w = sh.pad_w;
     a.fold_r = p.fold_r; a.fold_s = p.fold_s; a.R = sh.R / p.fold_r; a.S = sh.S / p.fold_s;
     a.HW = sh.H * sh.W;
     a.total_pix = sh.N * sh.H * sh.W;
@@ -1346,7 +1351,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
     a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * p.npix * 4 >= 2 * kXposeBytes &&
                  env_int("CONV2D_B200_TF32_HELPERS", 1) != 0) ? 1 : 0;
-    a.quad = (!b16 && (p.patch_w ? sh.W % 4 == 0 : (sh.H * sh.W) % 4 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
+    a.quad = (!b16 && (p.patch_w ? (sh.W % 4 == 0 && sh.pad_w % 4 == 0) : (sh.H * sh.W) % 4 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
     {
         // as many producer groups as can each still cover a stage in one pass (one memory round trip)
         const long long per_pass = a.quad ? kProducers : (long long)kProducers * kUnitsPerThread;
@@ -1358,7 +1363,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         while (a.pgroups > p.a_stages) a.pgroups /= 2;
     }
     a.fp16 = fp16 ? 1 : 0;
-    a.pair = (b16 && (p.patch_w ? sh.W % 2 == 0 : (sh.H * sh.W) % 2 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
+    a.pair = (b16 && (p.patch_w ? (sh.W % 2 == 0 && sh.pad_w % 2 == 0) : (sh.H * sh.W) % 2 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
     a.items = p.supertiles * p.n_blocks * p.ksplit;
     a.ksplit = p.ksplit;
     // Failure-detection test hooks (host-side injection only): a short wait bound and one filter copy that is
