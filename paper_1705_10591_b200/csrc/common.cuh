@@ -28,6 +28,20 @@ cudaError_t consume_device_timeout(bool* raised);
 // Every kernel launch goes through this so that conv2d_launch_count() is exact.
 void count_launch(int launches = 1);
 
+// Raises a kernel's dynamic shared-memory limit to `bytes` unless this call site already did so on the
+// current device (`done`: one static array per call site, i.e. per kernel instance).  The runtime call costs a
+// few microseconds, which matters for kernels that run for ten.
+inline cudaError_t raise_smem_limit(const void* kernel, size_t bytes, size_t (&done)[64])
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && done[dev] >= bytes) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = bytes;
+    return e;
+}
+
 // Launchers.  Each returns CONV2D_OK, CONV2D_ERR_UNSUPPORTED (no instance) or CONV2D_ERR_CUDA.
 conv2d_status_t launch_single_channel(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);
 conv2d_status_t launch_general_ffma(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);

@@ -147,10 +147,9 @@ conv2d_status_t launch_tile(const float* x, const float* w, float* y, const Shap
 {
     auto kern = general_ffma_kernel<R, S, CB, TW, TH>;
     const size_t smem = sizeof(Smem<R, S, CB, TW, TH>);
-    if (smem > 48 * 1024) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return CONV2D_ERR_CUDA;
-    }
+    static size_t smem_done[64] = {};
+    if (smem > 48 * 1024 && raise_smem_limit(reinterpret_cast<const void*>(kern), smem, smem_done) != cudaSuccess)
+        return CONV2D_ERR_CUDA;
     const int tiles_q = (sh.Q + TW - 1) / TW, tiles_p = (sh.P + TH - 1) / TH;
     dim3 grid(tiles_q * tiles_p, (sh.K + kTileK - 1) / kTileK, sh.N);
     const int vec_st = (sh.Q % 4 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);

@@ -255,7 +255,8 @@ conv2d_status_t launch_unit(const float* x, const float* w, float* y, const Shap
     const size_t smem = ((size_t)(tile_h + R - 1) * (TW + 8) + (size_t)sh.K * R * S) * sizeof(float);
     if (smem > 200 * 1024) return CONV2D_ERR_UNSUPPORTED;
     auto kern = single_channel_unit_kernel<R, S, UNIT>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return CONV2D_ERR_CUDA;
+    static size_t smem_done[64] = {};
+    if (raise_smem_limit(reinterpret_cast<const void*>(kern), smem, smem_done) != cudaSuccess) return CONV2D_ERR_CUDA;
     dim3 grid((sh.Q + TW - 1) / TW, (sh.P + tile_h - 1) / tile_h, sh.N);
     const int vec_st = (sh.Q % UNIT == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
     kern<<<grid, kThreads, smem, stream>>>(x, w, y, sh.H, sh.W, sh.K, sh.P, sh.Q, tile_h, vec_st);
@@ -410,10 +411,9 @@ conv2d_status_t launch_packed(const float* x, const float* w, float* y, const Sh
     constexpr int RS2 = (R * S + 1) / 2;
     const size_t smem = (size_t)(tile_h + R - 1) * kPitch * sizeof(float) + (size_t)((sh.K + 1) / 2) * RS2 * sizeof(float4);
     auto kern = single_channel_packed_kernel<R, S, TR>;
-    if (smem > 48 * 1024) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return CONV2D_ERR_CUDA;
-    }
+    static size_t smem_done[64] = {};
+    if (smem > 48 * 1024 && raise_smem_limit(reinterpret_cast<const void*>(kern), smem, smem_done) != cudaSuccess)
+        return CONV2D_ERR_CUDA;
     dim3 grid((sh.Q + kTileW - 1) / kTileW, (sh.P + tile_h - 1) / tile_h, sh.N);
     const int vec_ld = (sh.W % 4 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0);
     const int vec_st = (sh.Q % 4 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
@@ -429,10 +429,9 @@ conv2d_status_t launch_instance(const float* x, const float* w, float* y, const 
     size_t smem = (size_t)(tile_h + R - 1) * kPitch * sizeof(float);
     if (WSRC == 1) smem += (size_t)sh.K * RSP * sizeof(float);
     auto kern = single_channel_kernel<R, S, TR, WSRC>;
-    if (smem > 48 * 1024) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return CONV2D_ERR_CUDA;
-    }
+    static size_t smem_done[64] = {};
+    if (smem > 48 * 1024 && raise_smem_limit(reinterpret_cast<const void*>(kern), smem, smem_done) != cudaSuccess)
+        return CONV2D_ERR_CUDA;
     dim3 grid((sh.Q + kTileW - 1) / kTileW, (sh.P + tile_h - 1) / tile_h, sh.N);
     const int vec_ld = (sh.W % 4 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0);
     const int vec_st = (sh.Q % 4 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
@@ -619,7 +618,8 @@ conv2d_status_t launch_rows(const float* x, const float* w, float* y, const Shap
                       + (size_t)((sh.K + 1) / 2) * RS2 * sizeof(float4) + 64;
     if (smem > 227 * 1024) return CONV2D_ERR_UNSUPPORTED;
     auto kern = single_channel_rows_kernel<R, S, TR>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    static size_t smem_done[64] = {};
+    if (raise_smem_limit(reinterpret_cast<const void*>(kern), smem, smem_done) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     const int col_tiles = (sh.Q + kRowsW - 1) / kRowsW;
     const long long items = (long long)sh.N * ((sh.P + band_h - 1) / band_h) * col_tiles;
@@ -806,7 +806,8 @@ conv2d_status_t launch_rows_shift(const float* x, const float* w, float* y, cons
     const size_t smem = need(band_h);
     if (smem > 227 * 1024) return CONV2D_ERR_UNSUPPORTED;
     auto kern = single_channel_rows_shift_kernel<R, S>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    static size_t smem_done[64] = {};
+    if (raise_smem_limit(reinterpret_cast<const void*>(kern), smem, smem_done) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     const int col_tiles = (sh.Q + 2 + kRowsW - 1) / kRowsW;    // odd rows start two columns to the left
     const long long items = 2LL * sh.N * ((sh.P + band_h - 1) / band_h) * col_tiles;
