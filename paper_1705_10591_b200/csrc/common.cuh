@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libconv2d_b200.
 #pragma once
 
+#include <cstdlib>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -42,6 +43,17 @@ inline cudaError_t raise_smem_limit(const void* kernel, size_t bytes, size_t (&d
     return e;
 }
 
+// Tuning and test switches come from the environment, but only in a process that was started with
+// CONV2D_B200_TUNING set (looked up once): production calls never scan the environment, and stray variables
+// cannot change what the library does.
+inline int env_int(const char* name, int dflt)
+{
+    static const bool tuning = getenv("CONV2D_B200_TUNING") != nullptr;
+    if (!tuning) return dflt;
+    const char* v = getenv(name);
+    return (v && *v) ? atoi(v) : dflt;
+}
+
 // Launchers.  Each returns CONV2D_OK, CONV2D_ERR_UNSUPPORTED (no instance) or CONV2D_ERR_CUDA.
 conv2d_status_t launch_single_channel(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);
 conv2d_status_t launch_general_ffma(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);
@@ -50,14 +62,15 @@ conv2d_status_t launch_direct_fallback(const float* x, const float* w, float* y,
 // Tensor-core path.
 bool tf32_supported(const Shape& sh);
 size_t tf32_workspace_bytes(const Shape& sh);   // includes the status block
+// (returns CONV2D_ERR_UNSUPPORTED without an instance, CONV2D_ERR_WORKSPACE when workspace_bytes is too small)
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
-                                    void* workspace, bool weights_packed, cudaStream_t stream);
+                                    void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream);
 
 // Same kernel with 16-bit operands (x, w hold bf16 or fp16 elements in the same NCHW / KCRS order), fp32 output.
 bool b16_supported(const Shape& sh);
 size_t b16_workspace_bytes(const Shape& sh);
 conv2d_status_t launch_general_b16(const void* x, const void* w, float* y, const Shape& sh, bool fp16,
-                                   void* workspace, bool weights_packed, cudaStream_t stream);
+                                   void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream);
 
 // Variant of the tensor-core path whose scratch is a fixed array inside the library image.
 constexpr size_t kNoAllocScratchBytes = kStatusBytes + (size_t)8 * 1024 * 1024;

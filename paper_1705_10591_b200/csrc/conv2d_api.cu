@@ -175,21 +175,15 @@ conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
     if (flags & ~(unsigned)CONV2D_FLAG_WEIGHTS_PACKED) return CONV2D_ERR_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
-    bool use_tf32 = false;
-    if (algo == CONV2D_ALGO_TF32) {
-        if (!tf32_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
-        if (!workspace) return CONV2D_ERR_NULL;
-        if (workspace_bytes < tf32_workspace_bytes(sh)) return CONV2D_ERR_WORKSPACE;
-        use_tf32 = true;
-    } else if (algo == CONV2D_ALGO_AUTO) {
-        use_tf32 = tf32_supported(sh) && workspace && workspace_bytes >= tf32_workspace_bytes(sh);
-    } else if (algo != CONV2D_ALGO_FFMA) {
-        return CONV2D_ERR_UNSUPPORTED;
-    }
+    if (algo != CONV2D_ALGO_TF32 && algo != CONV2D_ALGO_AUTO && algo != CONV2D_ALGO_FFMA) return CONV2D_ERR_UNSUPPORTED;
+    if (algo == CONV2D_ALGO_TF32 && !workspace) return tf32_supported(sh) ? CONV2D_ERR_NULL : CONV2D_ERR_UNSUPPORTED;
     st = check_device();
     if (st != CONV2D_OK) return st;
-    if (use_tf32)
-        return launch_general_tf32(x, w, y, sh, workspace, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0, stream);
+    if (algo != CONV2D_ALGO_FFMA && workspace) {
+        // one planning pass: the launcher reports "no instance" or "workspace too small" itself
+        st = launch_general_tf32(x, w, y, sh, workspace, workspace_bytes, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0, stream);
+        if (algo == CONV2D_ALGO_TF32 || (st != CONV2D_ERR_UNSUPPORTED && st != CONV2D_ERR_WORKSPACE)) return st;
+    }
     return launch_general_ffma(x, w, y, sh, stream);
 }
 
@@ -205,11 +199,9 @@ conv2d_status_t conv2d_fwd_general_16bit(const void* x16, const void* w16, float
     if (!aligned16(x16) || !aligned16(w16) || !aligned16(y) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
     if (flags & ~(unsigned)CONV2D_FLAG_WEIGHTS_PACKED) return CONV2D_ERR_UNSUPPORTED;
     if (operand != CONV2D_OPERAND_BF16 && operand != CONV2D_OPERAND_FP16) return CONV2D_ERR_UNSUPPORTED;
-    if (!b16_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
-    if (workspace_bytes < b16_workspace_bytes(sh)) return CONV2D_ERR_WORKSPACE;
     st = check_device();
     if (st != CONV2D_OK) return st;
-    return launch_general_b16(x16, w16, y, sh, operand == CONV2D_OPERAND_FP16, workspace,
+    return launch_general_b16(x16, w16, y, sh, operand == CONV2D_OPERAND_FP16, workspace, workspace_bytes,
                               (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -248,9 +240,10 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
         Shape shp;
         if (make_shape(N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, &shp) == CONV2D_OK) {
             shp.H = H; shp.W = W; shp.pad_h = pad_h; shp.pad_w = pad_w;       // P, Q are those of the extended image
-            if (tf32_supported(shp) && tf32_workspace_bytes(shp) <= workspace_bytes)
-                return launch_general_tf32(x, w, y, shp, workspace, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0,
-                                           static_cast<cudaStream_t>(cuda_stream));
+            const conv2d_status_t native = launch_general_tf32(x, w, y, shp, workspace, workspace_bytes,
+                                                               (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0,
+                                                               static_cast<cudaStream_t>(cuda_stream));
+            if (native != CONV2D_ERR_UNSUPPORTED && native != CONV2D_ERR_WORKSPACE) return native;
         }
     }
     const bool own_status = inner < kStatusBytes;          // fp32 path: no workspace of its own
@@ -331,8 +324,6 @@ conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float
     conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
     if (st != CONV2D_OK) return st;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return CONV2D_ERR_ALIGN;
-    if (!tf32_supported(sh)) return CONV2D_ERR_UNSUPPORTED;
-    if (tf32_workspace_bytes(sh) > kNoAllocScratchBytes) return CONV2D_ERR_WORKSPACE;
     st = check_device();
     if (st != CONV2D_OK) return st;
     return launch_general_tf32_noalloc(x, w, y, sh, wait != 0, static_cast<cudaStream_t>(cuda_stream));

@@ -130,12 +130,6 @@ size_t smem_need(int a_stages, int npix, int n_tile, int b_stages, int tps, int 
     return (size_t)a_stages * cbg * kCB * npix * 4 + (size_t)b_stages * tps * kCB * n_tile * 4 + kBookBytes;
 }
 
-int env_int(const char* name, int dflt)
-{
-    const char* v = getenv(name);
-    return (v && *v) ? atoi(v) : dflt;
-}
-
 // b16: the operands are 16-bit floats, bf16 or fp16 (16-byte unit = 8 channels, 32 channels per staged block, K = 16 per MMA); the
 // byte layout of every stage is the same as for TF32 (16 channels of 4 bytes).
 Plan make_plan(const Shape& sh, bool b16 = false)
@@ -1276,13 +1270,16 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// workspace_bytes: checked against the plan's need here, so that a call plans only once (the planner reads two
+// dozen environment switches and costs ~2 us); SIZE_MAX = the caller has checked already.
 conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* y, const Shape& sh, bool b16, bool fp16,
-                                   void* workspace, bool weights_packed, cudaStream_t stream)
+                                   void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream)
 {
     const float* x = static_cast<const float*>(x_any);   // 16-bit operands: re-read as such inside the kernel
     const float* w = static_cast<const float*>(w_any);
     const Plan p = make_plan(sh, b16);
     if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
+    if (workspace_bytes < kStatusBytes + packed_floats(p) * sizeof(float)) return CONV2D_ERR_WORKSPACE;
     unsigned* status = static_cast<unsigned*>(workspace);
     float* wp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
 
@@ -1388,15 +1385,15 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
 }  // namespace
 
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
-                                    void* workspace, bool weights_packed, cudaStream_t stream)
+                                    void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream)
 {
-    return launch_tensor_core(x, w, y, sh, false, false, workspace, weights_packed, stream);
+    return launch_tensor_core(x, w, y, sh, false, false, workspace, workspace_bytes, weights_packed, stream);
 }
 
 conv2d_status_t launch_general_b16(const void* x, const void* w, float* y, const Shape& sh, bool fp16,
-                                   void* workspace, bool weights_packed, cudaStream_t stream)
+                                   void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream)
 {
-    return launch_tensor_core(x, w, y, sh, true, fp16, workspace, weights_packed, stream);
+    return launch_tensor_core(x, w, y, sh, true, fp16, workspace, workspace_bytes, weights_packed, stream);
 }
 
 // ---------------------------------------------------------------- variant without caller-provided scratch
@@ -1427,7 +1424,7 @@ conv2d_status_t launch_general_tf32_noalloc(const float* x, const float* w, floa
         }
         scratch = scratch_of_device[dev];
     }
-    conv2d_status_t st = launch_general_tf32(x, w, y, sh, scratch, /*weights_packed=*/false, stream);
+    conv2d_status_t st = launch_general_tf32(x, w, y, sh, scratch, kNoAllocScratchBytes, /*weights_packed=*/false, stream);
     if (st != CONV2D_OK || !wait) return st;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return CONV2D_ERR_CUDA;
     unsigned word = 0;

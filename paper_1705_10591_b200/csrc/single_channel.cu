@@ -831,12 +831,6 @@ conv2d_status_t try_rows_shift<3, 3>(const float* x, const float* w, float* y, c
     return launch_rows_shift<3, 3>(x, w, y, sh, band_h, stream);
 }
 
-int env_int(const char* name, int dflt)
-{
-    const char* v = getenv(name);
-    return (v && *v) ? atoi(v) : dflt;
-}
-
 template <int R, int S>
 conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
 {

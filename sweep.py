@@ -106,6 +106,7 @@ def main():
                         for algo, name in ((lib.ALGO_TF32, "tf32"), (lib.ALGO_16BIT, "bf16"), (lib.ALGO_FFMA, "fp32")):
                             run_point(torch, lib, peaks, flush, n, c, size, size, k, r, r, algo, "general", {"algo": name})
     elif which == "unit":
+        os.environ["CONV2D_B200_TUNING"] = "1"      # must be set before the library's first call
         for size in (2048, 4096):
             for k in (8, 32):
                 for unit in (1, 2, 4):
