@@ -513,7 +513,7 @@ struct KernelArgs {
     int fold_r, fold_s;  // taps folded into the channel dimension (1, 1: none); R, S below are what is left as shifts
     int helpers;      // 1: warps 8-15 share the write-back of a block's last item (operand-swap layout only)
     int pgroups;      // producer groups (1, 2 or 4): stage k is filled by group k % pgroups
-    int quad;         // fp32 operands only: producers load four adjacent pixels per 128-bit word (needs H*W % 4 == 0)
+    int quad;         // producers load four adjacent pixels per 128-bit (fp32) or 64-bit (16-bit operands) word (needs H*W % 4 == 0)
     int pair;         // 16-bit operands only: producers load two adjacent pixels per 32-bit word (needs H*W even)
     int cbg, groups;        // channel blocks per activation stage, number of such groups
     int resident;           // filters loaded once per thread block instead of streamed
@@ -1049,6 +1049,40 @@ general_tc_kernel(const KernelArgs a)
                             dc[3] = make_float4(to_tf32_rna(v[4 * ch].w), to_tf32_rna(v[4 * ch + 1].w), to_tf32_rna(v[4 * ch + 2].w), to_tf32_rna(v[4 * ch + 3].w));
                         }
                     }
+                } else if (B16 && !FOLD && a.quad) {
+                    // 16-bit operands, same idea: 64-bit loads of 4 adjacent pixels for each of the 32 channels of a
+                    // block, then the 4 x 32 block is turned around in registers into four 64-byte units.
+                    const int qn = a.npix >> 2;
+                    for (int i = wtid; i < qn * a.cbg; i += nthr) {
+                        const int g = i / qn, pq = i - g * qn;
+                        const int c0 = (gr * a.cbg + g) * 2 * kCB;
+                        uint2 v[2 * kCB];
+#pragma unroll
+                        for (int e = 0; e < 2 * kCB; ++e) v[e] = make_uint2(0u, 0u);
+                        int n, off;
+                        if (staged_pixel<PATCH>(a, ii.geom, 4 * pq, n, off) && c0 < a.C) {
+                            const unsigned short* src = reinterpret_cast<const unsigned short*>(a.x) + ((size_t)n * a.C + c0) * a.HW + off;
+#pragma unroll
+                            for (int e = 0; e < 2 * kCB; ++e)
+                                if (c0 + e < a.C) v[e] = __ldg(reinterpret_cast<const uint2*>(src + (size_t)e * a.HW));
+                        }
+                        float4* d = dst + (size_t)g * kChunks * a.npix + 4 * pq;
+#pragma unroll
+                        for (int ch = 0; ch < kChunks; ++ch) {        // 8 channels per 16-byte unit; word k = channels 2k, 2k+1
+                            float4* dc = d + ch * a.npix;
+                            unsigned p0[4], p1[4], p2[4], p3[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const uint2 lo = v[8 * ch + 2 * k], hi = v[8 * ch + 2 * k + 1];
+                                p0[k] = __byte_perm(lo.x, hi.x, 0x5410); p1[k] = __byte_perm(lo.x, hi.x, 0x7632);
+                                p2[k] = __byte_perm(lo.y, hi.y, 0x5410); p3[k] = __byte_perm(lo.y, hi.y, 0x7632);
+                            }
+                            dc[0] = make_float4(__uint_as_float(p0[0]), __uint_as_float(p0[1]), __uint_as_float(p0[2]), __uint_as_float(p0[3]));
+                            dc[1] = make_float4(__uint_as_float(p1[0]), __uint_as_float(p1[1]), __uint_as_float(p1[2]), __uint_as_float(p1[3]));
+                            dc[2] = make_float4(__uint_as_float(p2[0]), __uint_as_float(p2[1]), __uint_as_float(p2[2]), __uint_as_float(p2[3]));
+                            dc[3] = make_float4(__uint_as_float(p3[0]), __uint_as_float(p3[1]), __uint_as_float(p3[2]), __uint_as_float(p3[3]));
+                        }
+                    }
                 } else
                 for (int first = 0; first < units; first += nthr * kUnitsPerThread) {
                     float v[kUnitsPerThread][kCB];
@@ -1348,7 +1382,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
     a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * p.npix * 4 >= 2 * kXposeBytes &&
                  env_int("CONV2D_B200_TF32_HELPERS", 1) != 0) ? 1 : 0;
-    a.quad = (!b16 && (p.patch_w ? (sh.W % 4 == 0 && sh.pad_w % 4 == 0) : (sh.H * sh.W) % 4 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
+    a.quad = ((p.patch_w ? (sh.W % 4 == 0 && sh.pad_w % 4 == 0) : (sh.H * sh.W) % 4 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
     {
         // as many producer groups as can each still cover a stage in one pass (one memory round trip)
         const long long per_pass = a.quad ? kProducers : (long long)kProducers * kUnitsPerThread;
