@@ -496,6 +496,24 @@ __global__ void repack_filters_tiled_kernel(const T* __restrict__ w, T* __restri
     }
 }
 
+// Division of a non-negative int below 2^31 by a divisor fixed per launch, as a multiply-high, an add and a
+// shift (round-up method for invariant divisors): a plain 32-bit division is a ~35-instruction dependent chain,
+// and the pixel decoding below sits on the critical path of every producer unit and every epilogue block.
+struct FastDiv {
+    uint32_t mul, shift;
+    int d;
+    FastDiv() : mul(0), shift(0), d(1) {}
+    explicit FastDiv(int divisor) : d(divisor)
+    {
+        uint32_t l = 0;
+        while ((1ull << l) < (unsigned long long)divisor) ++l;
+        shift = l;
+        mul = (uint32_t)((((1ull << l) - (unsigned long long)divisor) << 32) / (unsigned long long)divisor + 1ull);
+    }
+    __device__ __forceinline__ int div(int n) const { return (int)((__umulhi((uint32_t)n, mul) + (uint32_t)n) >> shift); }
+    __device__ __forceinline__ int divmod(int n, int& rem) const { const int q = div(n); rem = n - q * d; return q; }
+};
+
 struct KernelArgs {
     const float* x;
     const float* wp;
@@ -504,6 +522,8 @@ struct KernelArgs {
     int N, C, H, W, K, R, S, P, Q;
     int HW;
     int total_pix;
+    FastDiv div_HW, div_W, div_npix, div_qn, div_patch_w;   // divisors of the pixel decoding (qn = npix / 4)
+    int vec_shift;    // log2(vec)
     int n_tile, n_blocks, mt, tile_px, px_groups, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
     int patch_w, patch_tw, patch_rows, patch_cols;   // patch addressing (PATCH kernels): staged row pitch, valid output
                                                       // columns per patch row, patches per image down and across
@@ -542,15 +562,15 @@ template <bool PATCH>
 __device__ __forceinline__ bool staged_pixel(const KernelArgs& a, const ItemGeom& g, int jj, int& n, int& off)
 {
     if (PATCH) {
-        const int prow = jj / a.patch_w, pcol = jj - prow * a.patch_w;
+        int pcol;
+        const int prow = a.div_patch_w.divmod(jj, pcol);
         const int h = g.row0 + prow - a.pad_h, wc = g.col0 + pcol - a.pad_w;
         n = g.n;
         off = h * a.W + wc;
         return (unsigned)h < (unsigned)a.H && (unsigned)wc < (unsigned)a.W;
     }
     const int j = g.j0 + jj;
-    n = j / a.HW;
-    off = j - n * a.HW;
+    n = a.div_HW.divmod(j, off);
     return j < a.total_pix;
 }
 // Accumulator column jj -> output (n, p, q); false when that output does not exist (window wraps over an edge).
@@ -558,7 +578,8 @@ template <bool PATCH>
 __device__ __forceinline__ bool output_pixel(const KernelArgs& a, const ItemGeom& g, int jj, int& n, int& p, int& q)
 {
     if (PATCH) {
-        const int prow = jj / a.patch_w, pcol = jj - prow * a.patch_w;
+        int pcol;
+        const int prow = a.div_patch_w.divmod(jj, pcol);
         n = g.n;
         p = g.row0 + prow;
         q = g.col0 + pcol;
@@ -566,10 +587,9 @@ __device__ __forceinline__ bool output_pixel(const KernelArgs& a, const ItemGeom
     }
     const int j = g.j0 + jj;
     if (j >= a.total_pix) return false;
-    n = j / a.HW;
-    const int off = j - n * a.HW;
-    p = off / a.W;
-    q = off - p * a.W;
+    int off;
+    n = a.div_HW.divmod(j, off);
+    p = a.div_W.divmod(off, q);
     return p < a.P && q < a.Q;
 }
 
@@ -587,7 +607,8 @@ __device__ __forceinline__ void load_units(float (&v)[CNT][kCB], const KernelArg
 #pragma unroll
         for (int e = 0; e < kCB; ++e) v[u][e] = 0.f;
         if (i < units) {
-            const int g = i / a.npix, jj = i - g * a.npix;
+            int jj;
+            const int g = a.div_npix.divmod(i, jj);
             if (FOLD) {
                 // Folded taps: staged channel vc = (c, r, s) of pixel j is x[c] at pixel j + r*W + s (zero beyond
                 // the image: such windows belong to outputs that are dropped anyway).
@@ -663,7 +684,8 @@ __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* 
     for (int u = 0; u < CNT; ++u) {
         const int i = first + u * nthr + wtid;
         if (i < units) {
-            const int g = i / a.npix, jj = i - g * a.npix;
+            int jj;
+            const int g = a.div_npix.divmod(i, jj);
             if (B16 && a.pair) {
                 const int half_n = a.npix >> 1;
                 const int h = jj / half_n, pp = jj - h * half_n;
@@ -1027,7 +1049,8 @@ general_tc_kernel(const KernelArgs a)
                     // pipeline that the MMA instructions pass through as well) and writes four 16-channel units.
                     const int qn = a.npix >> 2;
                     for (int i = wtid; i < qn * a.cbg; i += nthr) {
-                        const int g = i / qn, pq = i - g * qn;
+                        int pq;
+                        const int g = a.div_qn.divmod(i, pq);
                         const int c0 = (gr * a.cbg + g) * kCB;
                         float4 v[kCB];
 #pragma unroll
@@ -1054,7 +1077,8 @@ general_tc_kernel(const KernelArgs a)
                     // block, then the 4 x 32 block is turned around in registers into four 64-byte units.
                     const int qn = a.npix >> 2;
                     for (int i = wtid; i < qn * a.cbg; i += nthr) {
-                        const int g = i / qn, pq = i - g * qn;
+                        int pq;
+                        const int g = a.div_qn.divmod(i, pq);
                         const int c0 = (gr * a.cbg + g) * 2 * kCB;
                         uint2 v[2 * kCB];
 #pragma unroll
@@ -1151,8 +1175,8 @@ general_tc_kernel(const KernelArgs a)
                     // per-warp store throughput is bounded by instructions in flight, not bytes (measured
                     // ~2.7 B/clk per warp with 4-byte lanes), hence the widest unit the alignment allows.
                     const int vec = a.vec;                          // 1, 2 or 4 (W, Q, P*Q multiples of vec)
-                    const int lanes_per_row = 32 / vec;
-                    const int row_sub = lane / lanes_per_row, pg = lane - row_sub * lanes_per_row;
+                    const int lanes_per_row = 32 >> a.vec_shift;
+                    const int row_sub = lane >> (5 - a.vec_shift), pg = lane & (lanes_per_row - 1);
                     int n, p, q;                                    // this lane's first pixel of the block
                     const bool ok = output_pixel<PATCH>(a, ii.geom, b * 32 + pg * vec, n, p, q);
                     float* o = a.y;
@@ -1380,6 +1404,9 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     for (int v = 4; v >= 2; v >>= 1)       // v adjacent accumulator columns must be v adjacent, aligned outputs of one row
         if ((p.patch_w ? p.patch_tw : sh.W) % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
+    a.vec_shift = a.vec == 4 ? 2 : (a.vec == 2 ? 1 : 0);
+    a.div_HW = FastDiv(a.HW); a.div_W = FastDiv(sh.W); a.div_npix = FastDiv(p.npix);
+    a.div_qn = FastDiv(p.npix / 4 > 0 ? p.npix / 4 : 1); a.div_patch_w = FastDiv(p.patch_w ? p.patch_w : 1);
     a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * p.npix * 4 >= 2 * kXposeBytes &&
                  env_int("CONV2D_B200_TF32_HELPERS", 1) != 0) ? 1 : 0;
     a.quad = ((p.patch_w ? (sh.W % 4 == 0 && sh.pad_w % 4 == 0) : (sh.H * sh.W) % 4 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
