@@ -1163,6 +1163,7 @@ general_tc_kernel(const KernelArgs a)
                 auto store_block = [&](const uint32_t (&v0)[16], const uint32_t (&v1)[16], int b) {
                     __syncwarp();                                   // the previous block has been read out
                     float4* row = reinterpret_cast<float4*>(tile + lane * kXposePitch);
+                    if (lane < rpq)                                 // M = 64: only lanes 0-15 of a quarter hold rows
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         row[i] = make_float4(__uint_as_float(v0[4 * i]), __uint_as_float(v0[4 * i + 1]),
