@@ -524,6 +524,8 @@ struct KernelArgs {
     int total_pix;
     FastDiv div_HW, div_W, div_npix, div_qn, div_patch_w;   // divisors of the pixel decoding (qn = npix / 4)
     int vec_shift;    // log2(vec)
+    FastDiv div_ksplit, div_n_blocks, div_groups_lo, div_groups_hi, div_per_image, div_patch_cols;   // divisors of the item decoding
+    int patch_item_rows;   // patch addressing: output rows of one item (tile_px / patch_w)
     int n_tile, n_blocks, mt, tile_px, px_groups, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
     int patch_w, patch_tw, patch_rows, patch_cols;   // patch addressing (PATCH kernels): staged row pitch, valid output
                                                       // columns per patch row, patches per image down and across
@@ -724,22 +726,22 @@ struct ItemInfo {
 __device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
 {
     ItemInfo it;
-    const int part = item % a.ksplit;
-    const int rest = item / a.ksplit;
-    it.nb = rest % a.n_blocks;
-    it.supertile = rest / a.n_blocks;
-    it.g_begin = part * a.groups / a.ksplit;
-    it.n_groups = (part + 1) * a.groups / a.ksplit - it.g_begin;
-    it.rot = rest % it.n_groups;        // blocks stream the filter bank in rotated order (see kernel)
+    // (multiply-high divisions: this runs at the head of every item on the MMA thread and on the producers)
+    int part;
+    const int rest = a.div_ksplit.divmod(item, part);
+    it.supertile = a.div_n_blocks.divmod(rest, it.nb);
+    it.g_begin = a.div_ksplit.div(part * a.groups);
+    it.n_groups = a.div_ksplit.div((part + 1) * a.groups) - it.g_begin;
+    // blocks stream the filter bank in rotated order (see kernel); n_groups is floor or ceil of groups / ksplit
+    (it.n_groups == a.div_groups_lo.d ? a.div_groups_lo : a.div_groups_hi).divmod(rest, it.rot);
     it.geom.j0 = it.supertile * a.tile_px;
     it.geom.n = it.geom.row0 = it.geom.col0 = 0;
     if (a.patch_w) {
-        const int per_image = a.patch_rows * a.patch_cols;
-        it.geom.n = it.supertile / per_image;
-        const int rem = it.supertile - it.geom.n * per_image;
-        const int pr = rem / a.patch_cols;
-        it.geom.row0 = pr * (a.tile_px / a.patch_w);
-        it.geom.col0 = (rem - pr * a.patch_cols) * a.patch_tw;
+        int rem, pc;
+        it.geom.n = a.div_per_image.divmod(it.supertile, rem);
+        const int pr = a.div_patch_cols.divmod(rem, pc);
+        it.geom.row0 = pr * a.patch_item_rows;
+        it.geom.col0 = pc * a.patch_tw;
     }
     return it;
 }
@@ -1425,6 +1427,11 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     a.pair = (b16 && (p.patch_w ? (sh.W % 2 == 0 && sh.pad_w % 2 == 0) : (sh.H * sh.W) % 2 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_B16_PAIR", 1) != 0) ? 1 : 0;
     a.items = p.supertiles * p.n_blocks * p.ksplit;
     a.ksplit = p.ksplit;
+    a.div_ksplit = FastDiv(p.ksplit); a.div_n_blocks = FastDiv(p.n_blocks);
+    a.div_groups_lo = FastDiv(a.groups / p.ksplit > 0 ? a.groups / p.ksplit : 1);
+    a.div_groups_hi = FastDiv((a.groups + p.ksplit - 1) / p.ksplit);
+    a.div_per_image = FastDiv(p.patch_w ? p.patch_rows * p.patch_cols : 1); a.div_patch_cols = FastDiv(p.patch_w ? p.patch_cols : 1);
+    a.patch_item_rows = p.patch_w ? p.tile_px / p.patch_w : 0;
     // Failure-detection test hooks (host-side injection only): a short wait bound and one filter copy that is
     // never issued, so that a bounded wait expires and the time-out path can be checked without hanging anything.
     a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
