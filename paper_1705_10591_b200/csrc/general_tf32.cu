@@ -69,6 +69,7 @@ constexpr int kCB = 16;                     // channels per staged block (two UM
 constexpr int kChunks = kCB / 4;            // 16-byte channel chunks per block
 constexpr int kProducerWarps = 8;
 constexpr int kProducers = kProducerWarps * 32;
+static_assert(kProducers == 256, "the producer group arithmetic assumes 256 producer threads");
 constexpr int kEpilogueWarps = 4;
 // Warp roles by warp index.  An SM has four warp schedulers and warp w is served by scheduler w % 4.  The
 // single thread that issues the MMAs (warp 1) must never wait for an issue slot behind arithmetic-heavy
@@ -1026,20 +1027,24 @@ general_tc_kernel(const KernelArgs a)
         // The producer warps form `pgroups` groups; stage k of the block's stage sequence is filled by group
         // k % pgroups, so that several stages' memory round trips are in flight at once (a stage of a light
         // problem has fewer 16-channel units than there are producer threads).
-        const int nthr = kProducers / a.pgroups;
-        const int gid = (producer_index(warp) * 32 + lane) / nthr;
+        const int nthr_shift = a.pgroups == 4 ? 6 : (a.pgroups == 2 ? 7 : 8);     // kProducers = 256 threads; no divisions here:
+        const int nthr = 1 << nthr_shift;                                         // this is on the path to the first load
+        const int gid = (producer_index(warp) * 32 + lane) >> nthr_shift;
         const int wtid = (producer_index(warp) * 32 + lane) - gid * nthr;
         bool alive = true;
         int kstage = 0;
+        int next_as = 0;                 // ring slot and phase of stage `kstage`, advanced without divisions
+        uint32_t next_phase = 0;
         const int units = a.npix * a.cbg;
         for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
             const ItemInfo ii = decode_item(a, item);
             // One stage = cbg consecutive channel blocks.  All loads of a pass (kUnitsPerThread units of
             // 16 channels per thread) are issued before its first store: a pass costs one memory round trip.
             for (int grp = 0; grp < ii.n_groups && alive; ++grp, ++kstage) {
-                if (kstage % a.pgroups != gid) continue;
-                const int as = kstage % a.a_stages;
-                const uint32_t a_phase = (uint32_t)(kstage / a.a_stages) & 1u;
+                const int as = next_as;
+                const uint32_t a_phase = next_phase;
+                if (++next_as == a.a_stages) { next_as = 0; next_phase ^= 1u; }
+                if ((kstage & (a.pgroups - 1)) != gid) continue;         // pgroups is 1, 2 or 4
                 if (!mbar_wait_bounded(&a_empty[as], a_phase ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                 float4* dst = reinterpret_cast<float4*>(a_smem + (size_t)as * a_stage_bytes);
                 int gr = grp + ii.rot;
@@ -1136,8 +1141,8 @@ general_tc_kernel(const KernelArgs a)
         bool alive = true;
         for (int li = helper ? n_local - 1 : 0; li >= 0 && li < n_local; ++li) {
             const int item = (int)blockIdx.x + li * (int)gridDim.x;
-            const int buf = li % a.nbuf;
-            const uint32_t acc_phase = (uint32_t)(li / a.nbuf) & 1u;
+            const int buf = a.nbuf == 2 ? (li & 1) : 0;                              // nbuf is 1 or 2
+            const uint32_t acc_phase = (uint32_t)(a.nbuf == 2 ? li >> 1 : li) & 1u;
             const bool split = a.helpers && li == n_local - 1;
             const ItemInfo ii = decode_item(a, item);
             const int nb = ii.nb;
