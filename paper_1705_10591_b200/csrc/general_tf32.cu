@@ -125,10 +125,17 @@ struct Plan {
     bool ok;
 };
 
+// Distance between the 4-channel chunks of a staged channel block, in 16-byte units: the pixel count plus one, so
+// that it is odd.  A producer lane writes four adjacent pixels (64 bytes) per chunk; with lanes 64 bytes apart a
+// 128-bit store instruction would hit only two of the eight 16-byte bank groups (4-way conflict, ~1 M conflict
+// cycles per launch in the profiles).  With an odd chunk stride, lanes that would collide write different chunks
+// at the same time (each lane rotates its chunk order), and the eight lanes of a store phase cover all banks.
+inline int chunk_stride(int npix) { return npix + 1; }
+
 // b_stages counts filter stages of `tps` taps each; an activation stage holds `cbg` channel blocks.
 size_t smem_need(int a_stages, int npix, int n_tile, int b_stages, int tps, int cbg)
 {
-    return (size_t)a_stages * cbg * kCB * npix * 4 + (size_t)b_stages * tps * kCB * n_tile * 4 + kBookBytes;
+    return (size_t)a_stages * cbg * kCB * chunk_stride(npix) * 4 + (size_t)b_stages * tps * kCB * n_tile * 4 + kBookBytes;
 }
 
 // b16: the operands are 16-bit floats, bf16 or fp16 (16-byte unit = 8 channels, 32 channels per staged block, K = 16 per MMA); the
@@ -250,7 +257,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
             if (p.swap && want >= 64 && want <= 512 && want % 32 == 0 && pixel_items(want) > 0) res_px = want;
         }
         const int npix = npix_of(res_px);
-        if ((p.swap ? res_px : mt * set_cols) <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * npix * 4 + kBookBytes <= kSmemLimit) {
+        if ((p.swap ? res_px : mt * set_cols) <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * chunk_stride(npix) * 4 + kBookBytes <= kSmemLimit) {
             p.resident = 1;
             p.mt = p.swap ? (res_px + kTileM - 1) / kTileM : mt;
             p.tile_px = res_px;
@@ -259,7 +266,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
             p.a_stages = 2;
             p.b_stages = 1;
             p.tps = p.taps;
-            auto need = [&](int a_stages, int cbg) { return wbytes + extra + (size_t)a_stages * cbg * kCB * npix * 4 + kBookBytes; };
+            auto need = [&](int a_stages, int cbg) { return wbytes + extra + (size_t)a_stages * cbg * kCB * chunk_stride(npix) * 4 + kBookBytes; };
             while (p.cbg * 2 <= p.cblks && npix * p.cbg * 2 <= kProducers * kUnitsPerThread &&
                    need(p.a_stages, p.cbg * 2) <= kSmemLimit) p.cbg *= 2;
             while (p.a_stages < kMaxAStages && need(p.a_stages + 1, p.cbg) <= kSmemLimit) ++p.a_stages;
@@ -528,6 +535,8 @@ struct KernelArgs {
     FastDiv div_ksplit, div_n_blocks, div_groups_lo, div_groups_hi, div_per_image, div_patch_cols;   // divisors of the item decoding
     int patch_item_rows;   // patch addressing: output rows of one item (tile_px / patch_w)
     int n_tile, n_blocks, mt, tile_px, px_groups, nbuf, npix, cblks, taps, a_stages, b_stages, tps;
+    int rot;          // quad producers rotate their chunk order per lane (see there)
+    int cstride;      // 16-byte units between the 4-channel chunks of a staged channel block (npix + 1: odd)
     int patch_w, patch_tw, patch_rows, patch_cols;   // patch addressing (PATCH kernels): staged row pitch, valid output
                                                       // columns per patch row, patches per image down and across
     int pad_h, pad_w; // zero padding (patch addressing only): staged pixel (row, col) is image pixel (row - pad_h, col - pad_w)
@@ -692,7 +701,7 @@ __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* 
             if (B16 && a.pair) {
                 const int half_n = a.npix >> 1;
                 const int h = jj / half_n, pp = jj - h * half_n;
-                float4* d = dst + ((size_t)g * kChunks + 2 * h) * a.npix + 2 * pp;
+                float4* d = dst + ((size_t)g * kChunks + 2 * h) * a.cstride + 2 * pp;
 #pragma unroll
                 for (int m = 0; m < 2; ++m) {       // 8 channels per 16-byte unit; word k = channels 2k, 2k+1
                     unsigned lo[4], hi[4];
@@ -702,15 +711,15 @@ __device__ __forceinline__ void store_units(const float (&v)[CNT][kCB], float4* 
                         lo[k] = __byte_perm(w0, w1, 0x5410);     // first pixel: low halves
                         hi[k] = __byte_perm(w0, w1, 0x7632);     // second pixel: high halves
                     }
-                    d[m * a.npix] = make_float4(__uint_as_float(lo[0]), __uint_as_float(lo[1]), __uint_as_float(lo[2]), __uint_as_float(lo[3]));
-                    d[m * a.npix + 1] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(hi[2]), __uint_as_float(hi[3]));
+                    d[m * a.cstride] = make_float4(__uint_as_float(lo[0]), __uint_as_float(lo[1]), __uint_as_float(lo[2]), __uint_as_float(lo[3]));
+                    d[m * a.cstride + 1] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(hi[2]), __uint_as_float(hi[3]));
                 }
                 continue;
             }
-            float4* d = dst + (size_t)g * kChunks * a.npix + jj;
+            float4* d = dst + (size_t)g * kChunks * a.cstride + jj;
 #pragma unroll
             for (int ch = 0; ch < kChunks; ++ch)
-                d[ch * a.npix] = B16 ? make_float4(v[u][4 * ch], v[u][4 * ch + 1], v[u][4 * ch + 2], v[u][4 * ch + 3])
+                d[ch * a.cstride] = B16 ? make_float4(v[u][4 * ch], v[u][4 * ch + 1], v[u][4 * ch + 2], v[u][4 * ch + 3])
                                       : make_float4(to_tf32_rna(v[u][4 * ch]), to_tf32_rna(v[u][4 * ch + 1]),
                                                     to_tf32_rna(v[u][4 * ch + 2]), to_tf32_rna(v[u][4 * ch + 3]));
         }
@@ -782,7 +791,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 general_tc_kernel(const KernelArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    const uint32_t a_block_bytes = (uint32_t)kCB * a.npix * 4;          // one channel block of a stage
+    const uint32_t a_block_bytes = (uint32_t)kCB * a.cstride * 4;       // one channel block of a stage
     const uint32_t a_stage_bytes = a_block_bytes * (uint32_t)a.cbg;
     const uint32_t b_chunk_bytes = (uint32_t)kCB * a.n_tile * 4;        // one (channel block, tap)
     const uint32_t b_stage_bytes = b_chunk_bytes * (uint32_t)a.tps;
@@ -903,9 +912,9 @@ general_tc_kernel(const KernelArgs a)
                 if (B16) mma_b16(d, ad, bd, id, acc); else mma_tf32(d, ad, bd, id, acc);
             };
             const uint32_t desc_hi = (128u >> 4) | (1u << 14);                  // SBO = 128 B, descriptor version 1
-            const uint32_t a_lo_fixed = ((uint32_t)a.npix & 0x3FFFu) << 16;     // LBO = npix * 16 B
+            const uint32_t a_lo_fixed = ((uint32_t)a.cstride & 0x3FFFu) << 16;  // LBO = chunk stride * 16 B
             const uint32_t b_lo_fixed = ((uint32_t)a.n_tile & 0x3FFFu) << 16;   // LBO = n_tile * 16 B
-            const uint32_t a_kstep = 2u * (uint32_t)a.npix;                     // 8 channels further, in 16-byte units
+            const uint32_t a_kstep = 2u * (uint32_t)a.cstride;                  // 8 channels further, in 16-byte units
             const uint32_t b_kstep = 2u * (uint32_t)a.n_tile;
             bool alive = true;
             int as = 0, bs = 0, buf = 0;
@@ -1059,6 +1068,11 @@ general_tc_kernel(const KernelArgs a)
                         int pq;
                         const int g = a.div_qn.divmod(i, pq);
                         const int c0 = (gr * a.cbg + g) * kCB;
+                        // Register group ch of this lane holds chunk (ch + rot) & 3: lanes whose 64-byte pieces
+                        // would fall on the same banks write different chunks in the same instruction.  Measured:
+                        // a gain with 16-bit operands (below) only; with fp32 inputs the rotation is left out,
+                        // as it splits every 512-byte load instruction over four channel planes (slower from DRAM).
+                        const int rot = a.rot ? (pq >> 1) & 3 : 0;
                         float4 v[kCB];
 #pragma unroll
                         for (int e = 0; e < kCB; ++e) v[e] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1066,13 +1080,19 @@ general_tc_kernel(const KernelArgs a)
                         if (staged_pixel<PATCH>(a, ii.geom, 4 * pq, n, off) && c0 < a.C) {
                             const float* src = a.x + ((size_t)n * a.C + c0) * a.HW + off;
 #pragma unroll
-                            for (int e = 0; e < kCB; ++e)
-                                if (c0 + e < a.C) v[e] = __ldg(reinterpret_cast<const float4*>(src + (size_t)e * a.HW));
+                            for (int ch = 0; ch < kChunks; ++ch) {
+                                const int cc = ((ch + rot) & 3) << 2;                 // first channel of this register group
+                                const float* sc = src + (size_t)cc * a.HW;
+                                const int left = a.C - c0 - cc;                       // channels that exist from there on
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    if (j < left) v[4 * ch + j] = __ldg(reinterpret_cast<const float4*>(sc + (size_t)j * a.HW));
+                            }
                         }
-                        float4* d = dst + (size_t)g * kChunks * a.npix + 4 * pq;
+                        float4* d = dst + (size_t)g * kChunks * a.cstride + 4 * pq;
 #pragma unroll
                         for (int ch = 0; ch < kChunks; ++ch) {
-                            float4* dc = d + ch * a.npix;
+                            float4* dc = d + ((ch + rot) & 3) * a.cstride;
                             dc[0] = make_float4(to_tf32_rna(v[4 * ch].x), to_tf32_rna(v[4 * ch + 1].x), to_tf32_rna(v[4 * ch + 2].x), to_tf32_rna(v[4 * ch + 3].x));
                             dc[1] = make_float4(to_tf32_rna(v[4 * ch].y), to_tf32_rna(v[4 * ch + 1].y), to_tf32_rna(v[4 * ch + 2].y), to_tf32_rna(v[4 * ch + 3].y));
                             dc[2] = make_float4(to_tf32_rna(v[4 * ch].z), to_tf32_rna(v[4 * ch + 1].z), to_tf32_rna(v[4 * ch + 2].z), to_tf32_rna(v[4 * ch + 3].z));
@@ -1087,6 +1107,7 @@ general_tc_kernel(const KernelArgs a)
                         int pq;
                         const int g = a.div_qn.divmod(i, pq);
                         const int c0 = (gr * a.cbg + g) * 2 * kCB;
+                        const int rot = a.rot ? (pq >> 1) & 3 : 0;    // chunk rotation of this lane, as above
                         uint2 v[2 * kCB];
 #pragma unroll
                         for (int e = 0; e < 2 * kCB; ++e) v[e] = make_uint2(0u, 0u);
@@ -1094,13 +1115,19 @@ general_tc_kernel(const KernelArgs a)
                         if (staged_pixel<PATCH>(a, ii.geom, 4 * pq, n, off) && c0 < a.C) {
                             const unsigned short* src = reinterpret_cast<const unsigned short*>(a.x) + ((size_t)n * a.C + c0) * a.HW + off;
 #pragma unroll
-                            for (int e = 0; e < 2 * kCB; ++e)
-                                if (c0 + e < a.C) v[e] = __ldg(reinterpret_cast<const uint2*>(src + (size_t)e * a.HW));
+                            for (int ch = 0; ch < kChunks; ++ch) {
+                                const int cc = ((ch + rot) & 3) << 3;
+                                const unsigned short* sc = src + (size_t)cc * a.HW;
+                                const int left = a.C - c0 - cc;
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    if (j < left) v[8 * ch + j] = __ldg(reinterpret_cast<const uint2*>(sc + (size_t)j * a.HW));
+                            }
                         }
-                        float4* d = dst + (size_t)g * kChunks * a.npix + 4 * pq;
+                        float4* d = dst + (size_t)g * kChunks * a.cstride + 4 * pq;
 #pragma unroll
                         for (int ch = 0; ch < kChunks; ++ch) {        // 8 channels per 16-byte unit; word k = channels 2k, 2k+1
-                            float4* dc = d + ch * a.npix;
+                            float4* dc = d + ((ch + rot) & 3) * a.cstride;
                             unsigned p0[4], p1[4], p2[4], p3[4];
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {
@@ -1404,7 +1431,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     a.fold_r = p.fold_r; a.fold_s = p.fold_s; a.R = sh.R / p.fold_r; a.S = sh.S / p.fold_s;
     a.HW = sh.H * sh.W;
     a.total_pix = sh.N * sh.H * sh.W;
-    a.n_tile = p.n_tile; a.n_blocks = p.n_blocks; a.mt = p.mt; a.tile_px = p.tile_px; a.px_groups = p.px_groups; a.nbuf = p.nbuf; a.npix = p.npix;
+    a.n_tile = p.n_tile; a.n_blocks = p.n_blocks; a.mt = p.mt; a.tile_px = p.tile_px; a.px_groups = p.px_groups; a.nbuf = p.nbuf; a.npix = p.npix; a.cstride = chunk_stride(p.npix);
     a.cblks = p.cblks; a.taps = p.taps;
     a.a_stages = p.a_stages; a.b_stages = p.b_stages; a.tps = p.tps;
     a.cbg = p.cbg; a.groups = (p.cblks + p.cbg - 1) / p.cbg; a.resident = p.resident; a.swap = p.swap;
@@ -1415,7 +1442,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     a.vec_shift = a.vec == 4 ? 2 : (a.vec == 2 ? 1 : 0);
     a.div_HW = FastDiv(a.HW); a.div_W = FastDiv(sh.W); a.div_npix = FastDiv(p.npix);
     a.div_qn = FastDiv(p.npix / 4 > 0 ? p.npix / 4 : 1); a.div_patch_w = FastDiv(p.patch_w ? p.patch_w : 1);
-    a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * p.npix * 4 >= 2 * kXposeBytes &&
+    a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * chunk_stride(p.npix) * 4 >= 2 * kXposeBytes &&
                  env_int("CONV2D_B200_TF32_HELPERS", 1) != 0) ? 1 : 0;
     a.quad = ((p.patch_w ? (sh.W % 4 == 0 && sh.pad_w % 4 == 0) : (sh.H * sh.W) % 4 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
     {
@@ -1440,6 +1467,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     // Failure-detection test hooks (host-side injection only): a short wait bound and one filter copy that is
     // never issued, so that a bounded wait expires and the time-out path can be checked without hanging anything.
     a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
+    a.rot = env_int("CONV2D_B200_TF32_ROT", b16 ? 1 : 0) != 0 ? 1 : 0;
     a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
     a.tmem_cols = (unsigned)p.tmem_cols;
     if (p.ksplit > 1 &&
