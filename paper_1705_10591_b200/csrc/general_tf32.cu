@@ -117,6 +117,9 @@ struct Plan {
     int cbg;          // channel blocks per activation stage
     int resident;     // 1: the whole filter block stays in shared memory for the life of the thread block
     int swap;         // 1: filters are the MMA's M operand, 256 pixels its N operand (K <= 128)
+    int pair_taps;    // 1: at most 64 filters, horizontally adjacent taps stacked in one M = 128 operand (see make_plan)
+    int s_slots;      // shift-table entries per filter row: S, or ceil(S / 2) with stacked taps
+    int ovl;          // pixels by which consecutive flat items overlap (4 with stacked taps, else 0)
     int ksplit;       // 2: the channel blocks of a tile are shared by two work items that add into y
     int tmem_cols;    // power of two >= 32
     int supertiles;   // work-item rows over the flat pixel sequence
@@ -189,7 +192,25 @@ Plan make_plan(const Shape& sh, bool b16 = false)
     const int c_eff = sh.C * p.fold_r * p.fold_s;
     const int r_eff = sh.R / p.fold_r, s_eff = sh.S / p.fold_s;
     p.cblks = (c_eff + cbc - 1) / cbc;
-    p.taps = r_eff * s_eff;
+    // Stacked taps.  With at most 64 filters an M = 64 instruction runs the tensor pipe at half its rate.  Instead
+    // half of the rows of an M = 128 operand hold the filters' tap (r, s) and the other half their tap (r, s + 1),
+    // both multiplied with the pixels shifted for (r, s): the accumulator row of tap (r, s + 1), column j + 1, then
+    // holds what that tap contributes to output j, and the epilogue adds the two rows of a map one column apart
+    // (rows are ordered so that both lie in the lane quarter of one epilogue warp).  A row of
+    // S taps takes ceil(S / 2) instructions instead of S (an odd last tap has zeros in the upper half).  In the
+    // flat pixel run the last column of an item has no right neighbour, so consecutive items overlap by 4 pixels.
+    // It pays when the MMAs dominate an item: the stacked operand doubles the filter bytes per instruction (a bank
+    // that was resident in shared memory may have to be streamed) and every block of the write-back reads two tile
+    // rows per map.  Measured with 64 filters: 128 channels 5 x 5 on 32 x 32: 63.9 -> 46.8 us, 7 x 7: 110.5 ->
+    // 74.4 us, 3 x 3: 31.7 -> 28.6 us; 64 channels 5 x 5 on 64 x 64 in bf16 (50 pairs of tap and channel block):
+    // 24.3 -> 20.8 us; 64 channels 3 x 3 on 56 x 56 (36 pairs): 27.6 -> 30.6 us.  Hence from 48 (tap, channel block)
+    // pairs on.  CONV2D_B200_TF32_PAIR_TAPS = 0 / 2: never / whenever possible.
+    const int pair_mode = env_int("CONV2D_B200_TF32_PAIR_TAPS", 1);
+    p.pair_taps = (p.swap && kp16 <= 64 && p.fold_r * p.fold_s == 1 && s_eff >= 2 && pair_mode != 0 &&
+                   (pair_mode == 2 || (long long)r_eff * s_eff * p.cblks >= 48)) ? 1 : 0;
+    if (p.pair_taps) p.n_tile = 128;
+    p.s_slots = p.pair_taps ? (s_eff + 1) / 2 : s_eff;
+    p.taps = r_eff * p.s_slots;
     if (p.taps > kMaxTaps) return p;
     const size_t extra = p.swap ? kXposeBytes : 0;       // epilogue transposition tile
     // Addressing mode.  In the flat pixel run the staged halo is (R-1) whole image rows; once that exceeds a
@@ -218,10 +239,11 @@ Plan make_plan(const Shape& sh, bool b16 = false)
         if (p.patch_w) p.patch_cols = (sh.Q + p.patch_tw - 1) / p.patch_tw;
     }
     if (padded && !p.patch_w) return p;
+    p.ovl = (p.pair_taps && !p.patch_w) ? 4 : 0;
     const long long halo = p.patch_w ? (long long)(r_eff - 1) * p.patch_w + (s_eff - 1) : flat_halo;
     // work items along the pixels for an item of px pixels (0: px is not possible in this mode)
     auto pixel_items = [&](int px) -> long long {
-        if (!p.patch_w) return (total_pix + px - 1) / px;
+        if (!p.patch_w) return px > p.ovl ? (total_pix + (px - p.ovl) - 1) / (px - p.ovl) : 0;
         if (px % p.patch_w) return 0;
         const int th = px / p.patch_w;
         return (long long)sh.N * ((sh.P + th - 1) / th) * p.patch_cols;
@@ -249,7 +271,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
         if (p.swap && !p.patch_w && !forced_mt) {
             // When all pixels fit in one round of items of at most 512 pixels, one item per block is the better
             // cut (64 x 32 x 32 pixels with 1 x 1 filters: 448 pixels per item 19.9 us, 256 per item 22.1 us).
-            const long long one_round = ((total_pix + sms - 1) / sms + 31) / 32 * 32;
+            const long long one_round = ((total_pix + sms - 1) / sms + p.ovl + 31) / 32 * 32;
             if (one_round >= 64 && one_round <= 512) res_px = (int)one_round;
         }
         {
@@ -401,9 +423,12 @@ struct FoldedFilter {
 // are the contiguous taps of one (filter, channel) pair (cached lines are reused from tap to tap), and for
 // each tap a warp writes 32 adjacent elements.  T = float (rounded to TF32) with 4 elements per chunk, or a
 // 16-bit pattern with 8.
+// stacked = 1: half of the rows of the 128-row block are the filters' tap (r, 2u), the other half their tap
+// (r, 2u + 1) (zeros where S is odd and 2u + 1 = S); tap index t = r * ceil(S / 2) + u.
 template <typename T, int EPC>
 __global__ void repack_filters_kernel(const T* __restrict__ w, T* __restrict__ wp, unsigned* __restrict__ status,
-                                      int K, FoldedFilter ff, int taps, int n_tile, int cblks, long long threads_total)
+                                      int K, FoldedFilter ff, int taps, int n_tile, int cblks, long long threads_total,
+                                      int stacked)
 {
     grid_dep_launch();      // the convolution kernel may set itself up while this one runs
     // the status block in front of the filters starts every (non-prepacked) call cleared
@@ -417,7 +442,12 @@ __global__ void repack_filters_kernel(const T* __restrict__ w, T* __restrict__ w
         const int chunk = (int)(r % kChunks); r /= kChunks;
         const int cb = (int)(r % cblks); r /= cblks;
         const int nb = (int)r;
-        const int k = nb * n_tile + f;
+        // stacked taps: rows 32q .. 32q+15 are maps 16q .. 16q+15 with the left-hand tap of a pair, rows 32q+16 .. 32q+31
+        // the same maps with the right-hand tap, so that both halves of a map lie in the same quarter of the
+        // accumulator lanes (the quarter one epilogue warp can read)
+        const int k = stacked ? ((f >> 5) << 4) + (f & 15) : nb * n_tile + f;
+        const int upper = stacked ? (f >> 4) & 1 : 0;
+        const int s_slots = (ff.S + 1) / 2;
         const int vc = (cb * kChunks + chunk) * EPC + e;
         const T* src = w + (size_t)k * ff.C * ff.R * ff.S;
         T* dst = wp + ((((size_t)nb * cblks + cb) * taps * kChunks + chunk) * n_tile + f) * EPC + e;
@@ -426,9 +456,15 @@ __global__ void repack_filters_kernel(const T* __restrict__ w, T* __restrict__ w
         for (int t = 0; t < taps; ++t, dst += tap_stride) {
             T v = T(0);
             if (live) {
-                const int o = folded ? ff.offset(vc, t) : vc * taps + t;
-                v = __ldg(src + o);
-                if (sizeof(T) == 4) v = (T)to_tf32_rna((float)v);
+                int o = folded ? ff.offset(vc, t) : vc * taps + t;
+                if (stacked) {
+                    const int r = t / s_slots, sx = 2 * (t - r * s_slots) + upper;
+                    o = sx < ff.S ? (vc * ff.R + r) * ff.S + sx : -1;
+                }
+                if (o >= 0) {
+                    v = __ldg(src + o);
+                    if (sizeof(T) == 4) v = (T)to_tf32_rna((float)v);
+                }
             }
             *dst = v;
         }
@@ -551,6 +587,9 @@ struct KernelArgs {
     int resident;           // filters loaded once per thread block instead of streamed
     int swap;               // operand roles swapped: accumulator lanes = filters, columns = pixels
     int vec;                // swap mode: adjacent pixels a lane stores as one unit (1, 2 or 4)
+    int pair_taps;          // stacked taps: accumulator lanes 64-127 hold the right-hand tap of each pair, one column to the right
+    int s_slots, s_step;    // shift-table entries per filter row and the horizontal shift between them (2 with stacked taps)
+    int item_stride;        // flat addressing: pixels between the starts of consecutive items (tile_px minus the overlap)
     int ksplit;             // items per output tile (split of the contraction): 1 or 2
     unsigned max_polls;     // bound of every barrier wait
     int test_drop_stage;    // test hook: the filter copy with this ordinal is armed but never issued (-1: none)
@@ -598,7 +637,7 @@ __device__ __forceinline__ bool output_pixel(const KernelArgs& a, const ItemGeom
         return pcol < a.patch_tw && p < a.P && q < a.Q;
     }
     const int j = g.j0 + jj;
-    if (j >= a.total_pix) return false;
+    if (j >= a.total_pix || jj >= a.item_stride) return false;       // (columns past the stride belong to the next item)
     int off;
     n = a.div_HW.divmod(j, off);
     p = a.div_W.divmod(off, q);
@@ -744,7 +783,7 @@ __device__ __forceinline__ ItemInfo decode_item(const KernelArgs& a, int item)
     it.n_groups = a.div_ksplit.div((part + 1) * a.groups) - it.g_begin;
     // blocks stream the filter bank in rotated order (see kernel); n_groups is floor or ceil of groups / ksplit
     (it.n_groups == a.div_groups_lo.d ? a.div_groups_lo : a.div_groups_hi).divmod(rest, it.rot);
-    it.geom.j0 = it.supertile * a.tile_px;
+    it.geom.j0 = it.supertile * a.item_stride;
     it.geom.n = it.geom.row0 = it.geom.col0 = 0;
     if (a.patch_w) {
         int rem, pc;
@@ -786,7 +825,7 @@ __device__ __forceinline__ void issue_tap(uint32_t d, uint32_t px_lo, uint32_t f
 #undef CONV2D_TAP_MMA
 }
 
-template <bool B16, bool FOLD, bool PATCH>
+template <bool B16, bool FOLD, bool PATCH, bool STACK>
 __global__ void __launch_bounds__(kThreads, 1)
 general_tc_kernel(const KernelArgs a)
 {
@@ -813,7 +852,7 @@ general_tc_kernel(const KernelArgs a)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile unsigned long long* t_entry = reinterpret_cast<volatile unsigned long long*>(tmem_slot + 2);
     uint32_t* tap_shift = tmem_slot + 4;                   // [taps] r * row_pitch + s of every tap, in staged pixels
-    for (int t = tid; t < a.taps; t += kThreads) tap_shift[t] = (uint32_t)((t / a.S) * a.row_pitch + t % a.S);
+    for (int t = tid; t < a.taps; t += kThreads) tap_shift[t] = (uint32_t)((t / a.s_slots) * a.row_pitch + (t % a.s_slots) * a.s_step);
     if (tid == 0) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); *t_entry = t; }
 
     if (tid == 0) {
@@ -955,7 +994,7 @@ general_tc_kernel(const KernelArgs a)
                     for (int g = 0; g < a.cbg && alive; ++g, a_lo_block += a_block_bytes >> 4) {
                         if (gr * a.cbg + g >= a.cblks) break;
                         uint32_t row_shift = 0;                                  // r * row pitch, in pixels (= 16-byte units)
-                        int sx = 0;
+                        int sx = 0, sc = 0;
                         for (int t0 = 0; t0 < a.taps; t0 += a.tps) {
                             const int nt = min(a.tps, a.taps - t0);
                             uint32_t b_lo;
@@ -1001,7 +1040,8 @@ general_tc_kernel(const KernelArgs a)
                                         }
                                     }
                                     accumulate = 1;
-                                    if (++sx == a.S) { sx = 0; row_shift += (uint32_t)a.row_pitch; }
+                                    sx += a.s_step;
+                                    if (++sc == a.s_slots) { sc = 0; sx = 0; row_shift += (uint32_t)a.row_pitch; }
                                 }
                             }
                             if (!a.resident) {
@@ -1188,22 +1228,39 @@ general_tc_kernel(const KernelArgs a)
                 // store instruction again writes 32 adjacent pixels of one map.
                 float* tile = helper ? reinterpret_cast<float*>(a_smem) + (size_t)(warp - 8) * 32 * kXposePitch
                                      : xpose + (size_t)(warp - 4) * 32 * kXposePitch;
-                const int rpq = a.n_tile / 4;      // filter rows per lane quarter: 32 (M = 128) or 16 (M = 64, lanes 0-15)
+                // Stacked taps: lanes 0-15 of the quarter hold 16 maps summed over the left-hand taps, lanes 16-31 the
+                // same maps over the right-hand taps, one column to the right: those lanes write their row shifted
+                // by one column (with the first column of the next block), and a map is the sum of two tile rows.
+                constexpr bool stacked = STACK;         // (a template parameter: as a run-time flag it slowed the ordinary epilogue by 15 %)
+                const int rpq = stacked ? 16 : a.n_tile / 4;    // maps per lane quarter: 32 (M = 128) or 16 (M = 64: lanes 0-15; stacked taps)
                 const int blocks = a.tile_px / 32;
-                auto load_block = [&](uint32_t (&v0)[16], uint32_t (&v1)[16], int b) {
+                auto load_block = [&](uint32_t (&v0)[16], uint32_t (&v1)[16], uint32_t (&vx)[1], int b) {
                     tmem_ld16(lane_base + (uint32_t)(b * 32), v0);
                     tmem_ld16(lane_base + (uint32_t)(b * 32 + 16), v1);
+                    vx[0] = 0u;
+                    if (stacked && b + 1 < blocks) tmem_ld1(lane_base + (uint32_t)(b * 32 + 32), vx);
                 };
-                auto store_block = [&](const uint32_t (&v0)[16], const uint32_t (&v1)[16], int b) {
+                auto store_block = [&](const uint32_t (&v0)[16], const uint32_t (&v1)[16], const uint32_t (&vx)[1], int b) {
                     __syncwarp();                                   // the previous block has been read out
                     float4* row = reinterpret_cast<float4*>(tile + lane * kXposePitch);
-                    if (lane < rpq)                                 // M = 64: only lanes 0-15 of a quarter hold rows
+                    if (stacked) {
+                        const bool up = lane >= 16;
+                        auto sel = [&](uint32_t lo, uint32_t hi) { return __uint_as_float(up ? hi : lo); };
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        row[i] = make_float4(__uint_as_float(v0[4 * i]), __uint_as_float(v0[4 * i + 1]),
-                                             __uint_as_float(v0[4 * i + 2]), __uint_as_float(v0[4 * i + 3]));
-                        row[4 + i] = make_float4(__uint_as_float(v1[4 * i]), __uint_as_float(v1[4 * i + 1]),
-                                                 __uint_as_float(v1[4 * i + 2]), __uint_as_float(v1[4 * i + 3]));
+                        for (int i = 0; i < 4; ++i) {
+                            row[i] = make_float4(sel(v0[4 * i], v0[4 * i + 1]), sel(v0[4 * i + 1], v0[4 * i + 2]),
+                                                 sel(v0[4 * i + 2], v0[4 * i + 3]), sel(v0[4 * i + 3], i < 3 ? v0[(4 * i + 4) & 15] : v1[0]));
+                            row[4 + i] = make_float4(sel(v1[4 * i], v1[4 * i + 1]), sel(v1[4 * i + 1], v1[4 * i + 2]),
+                                                     sel(v1[4 * i + 2], v1[4 * i + 3]), sel(v1[4 * i + 3], i < 3 ? v1[(4 * i + 4) & 15] : vx[0]));
+                        }
+                    } else if (lane < rpq) {                        // M = 64: only lanes 0-15 of a quarter hold rows
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            row[i] = make_float4(__uint_as_float(v0[4 * i]), __uint_as_float(v0[4 * i + 1]),
+                                                 __uint_as_float(v0[4 * i + 2]), __uint_as_float(v0[4 * i + 3]));
+                            row[4 + i] = make_float4(__uint_as_float(v1[4 * i]), __uint_as_float(v1[4 * i + 1]),
+                                                     __uint_as_float(v1[4 * i + 2]), __uint_as_float(v1[4 * i + 3]));
+                        }
                     }
                     __syncwarp();
                     // Each lane stores `vec` adjacent pixels of one map, so one instruction covers `vec` maps:
@@ -1223,7 +1280,11 @@ general_tc_kernel(const KernelArgs a)
 #pragma unroll 4
                             for (int r = 0; r < 32; r += 4, o += 4 * plane, src += 4 * kXposePitch)
                                 if (r + row_sub < kmax) {
-                                    const float4 t = *reinterpret_cast<const float4*>(src);
+                                    float4 t = *reinterpret_cast<const float4*>(src);
+                                    if (stacked) {
+                                        const float4 u = *reinterpret_cast<const float4*>(src + 16 * kXposePitch);
+                                        t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+                                    }
                                     if (add) { atomicAdd(o, t.x); atomicAdd(o + 1, t.y); atomicAdd(o + 2, t.z); atomicAdd(o + 3, t.w); }
                                     else *reinterpret_cast<float4*>(o) = t;
                                 }
@@ -1231,29 +1292,36 @@ general_tc_kernel(const KernelArgs a)
 #pragma unroll 8
                             for (int r = 0; r < 32; r += 2, o += 2 * plane, src += 2 * kXposePitch)
                                 if (r + row_sub < kmax) {
-                                    const float2 t = *reinterpret_cast<const float2*>(src);
+                                    float2 t = *reinterpret_cast<const float2*>(src);
+                                    if (stacked) {
+                                        const float2 u = *reinterpret_cast<const float2*>(src + 16 * kXposePitch);
+                                        t.x += u.x; t.y += u.y;
+                                    }
                                     if (add) { atomicAdd(o, t.x); atomicAdd(o + 1, t.y); }
                                     else *reinterpret_cast<float2*>(o) = t;
                                 }
                         } else {
 #pragma unroll 8
                             for (int r = 0; r < 32; ++r, o += plane, src += kXposePitch)
-                                if (r < kmax) { if (add) atomicAdd(o, *src); else *o = *src; }
+                                if (r < kmax) {
+                                    const float t = stacked ? src[0] + src[16 * kXposePitch] : src[0];
+                                    if (add) atomicAdd(o, t); else *o = t;
+                                }
                         }
                     }
                 };
-                uint32_t va0[16], va1[16], vb0[16], vb1[16];
+                uint32_t va0[16], va1[16], vb0[16], vb1[16], vax[1], vbx[1];
                 const int b_step = split ? 3 : 1;
                 int b = split ? share : 0;
-                if (b < blocks) load_block(va0, va1, b);
+                if (b < blocks) load_block(va0, va1, vax, b);
                 while (b < blocks) {
                     tmem_ld_wait();
-                    if (b + b_step < blocks) load_block(vb0, vb1, b + b_step);
-                    store_block(va0, va1, b);
+                    if (b + b_step < blocks) load_block(vb0, vb1, vbx, b + b_step);
+                    store_block(va0, va1, vax, b);
                     if ((b += b_step) >= blocks) break;
                     tmem_ld_wait();
-                    if (b + b_step < blocks) load_block(va0, va1, b + b_step);
-                    store_block(vb0, vb1, b);
+                    if (b + b_step < blocks) load_block(va0, va1, vax, b + b_step);
+                    store_block(vb0, vb1, vbx, b);
                     b += b_step;
                 }
                 tc_fence_before_sync();
@@ -1383,7 +1451,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         long long blocks = (lanes + 255) / 256;
         if (blocks > 148 * 16) blocks = 148 * 16;
         const size_t tile_bytes = (size_t)8 * kCB * 4 * p.taps;       // 8 filters x one channel block x taps
-        if (p.fold_r * p.fold_s == 1 && tile_bytes <= 48 * 1024 && p.n_tile % 8 == 0) {
+        if (p.fold_r * p.fold_s == 1 && tile_bytes <= 48 * 1024 && p.n_tile % 8 == 0 && !p.pair_taps) {
             const dim3 grid((unsigned)(p.n_blocks * p.n_tile / 8), (unsigned)p.cblks);
             int threads = (8 * kChunks * p.taps + 31) / 32 * 32;          // one 16-byte unit per thread in the store phase
             threads = threads < 128 ? 128 : (threads > 1024 ? 1024 : threads);
@@ -1399,10 +1467,10 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         } else if (b16)
             repack_filters_kernel<unsigned short, 8><<<(unsigned)blocks, 256, 0, stream>>>(
                 static_cast<const unsigned short*>(w_any), reinterpret_cast<unsigned short*>(wp), status, sh.K, ff,
-                p.taps, p.n_tile, p.cblks, lanes);
+                p.taps, p.n_tile, p.cblks, lanes, p.pair_taps);
         else
             repack_filters_kernel<float, 4><<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, ff, p.taps,
-                                                                                  p.n_tile, p.cblks, lanes);
+                                                                                  p.n_tile, p.cblks, lanes, p.pair_taps);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
     }
@@ -1414,9 +1482,11 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) return CONV2D_ERR_CUDA;
     bool& attr_set = attr_set_on[dev_id];
     if (!attr_set) {
-        void (*all[])(KernelArgs) = {general_tc_kernel<false, false, false>, general_tc_kernel<true, false, false>,
-                                     general_tc_kernel<false, true, false>,  general_tc_kernel<true, true, false>,
-                                     general_tc_kernel<false, false, true>,  general_tc_kernel<true, false, true>};
+        void (*all[])(KernelArgs) = {general_tc_kernel<false, false, false, false>, general_tc_kernel<true, false, false, false>,
+                                     general_tc_kernel<false, true, false, false>,  general_tc_kernel<true, true, false, false>,
+                                     general_tc_kernel<false, false, true, false>,  general_tc_kernel<true, false, true, false>,
+                                     general_tc_kernel<false, false, false, true>,  general_tc_kernel<true, false, false, true>,
+                                     general_tc_kernel<false, false, true, true>,   general_tc_kernel<true, false, true, true>};
         for (auto k : all)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
             return CONV2D_ERR_CUDA;
@@ -1440,6 +1510,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         if ((p.patch_w ? p.patch_tw : sh.W) % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
     a.vec_shift = a.vec == 4 ? 2 : (a.vec == 2 ? 1 : 0);
+    a.pair_taps = p.pair_taps; a.s_slots = p.s_slots; a.s_step = p.pair_taps ? 2 : 1; a.item_stride = p.tile_px - p.ovl;
     a.div_HW = FastDiv(a.HW); a.div_W = FastDiv(sh.W); a.div_npix = FastDiv(p.npix);
     a.div_qn = FastDiv(p.npix / 4 > 0 ? p.npix / 4 : 1); a.div_patch_w = FastDiv(p.patch_w ? p.patch_w : 1);
     a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * chunk_stride(p.npix) * 4 >= 2 * kXposeBytes &&
@@ -1477,9 +1548,11 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     // tail of whatever kernel precedes it on the stream; it waits for that kernel before it touches global memory.
     const bool fold = p.fold_r * p.fold_s > 1;
     void (*kernel)(KernelArgs);
-    if (p.patch_w) kernel = b16 ? general_tc_kernel<true, false, true> : general_tc_kernel<false, false, true>;
-    else if (fold) kernel = b16 ? general_tc_kernel<true, true, false> : general_tc_kernel<false, true, false>;
-    else kernel = b16 ? general_tc_kernel<true, false, false> : general_tc_kernel<false, false, false>;
+    if (p.pair_taps && p.patch_w) kernel = b16 ? general_tc_kernel<true, false, true, true> : general_tc_kernel<false, false, true, true>;
+    else if (p.pair_taps) kernel = b16 ? general_tc_kernel<true, false, false, true> : general_tc_kernel<false, false, false, true>;
+    else if (p.patch_w) kernel = b16 ? general_tc_kernel<true, false, true, false> : general_tc_kernel<false, false, true, false>;
+    else if (fold) kernel = b16 ? general_tc_kernel<true, true, false, false> : general_tc_kernel<false, true, false, false>;
+    else kernel = b16 ? general_tc_kernel<true, false, false, false> : general_tc_kernel<false, false, false, false>;
     if (launch_pdl(kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, stream, a) != cudaSuccess) return CONV2D_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;

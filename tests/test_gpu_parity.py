@@ -331,3 +331,38 @@ def test_patch_addressing_forced_on_narrow_images(oracle, monkeypatch, dims):
     y_patch = run_library(x, w, entry="general", algo=ALGO_TF32)
     assert_parity(y_patch, y_ref, yabs, TF32_TOL, f"patch {dims}")
     assert_parity(y_patch, y_flat.astype(np.float64), yabs, 2e-5, f"patch vs flat {dims}")
+
+
+STACKED_TAP_SHAPES = [
+    # N, C, H, W, K, R, S      (at most 64 filters: horizontally adjacent taps share one 128-row operand)
+    (3, 64, 20, 22, 64, 3, 3),       # odd tap count per row: the last tap of a row has an empty upper half
+    (2, 40, 17, 19, 50, 5, 5),       # filter count not a multiple of 16; odd image width (one pixel per store)
+    (1, 72, 12, 30, 33, 2, 2),       # even taps per row: no empty halves
+    (2, 16, 9, 44, 7, 7, 7),         # fewer filters than one lane quarter holds
+    (1, 130, 6, 10, 64, 3, 4),       # too few pixels for the machine: split contraction, partial sums added
+    (1, 24, 14, 640, 48, 3, 3),      # wide image: items are rectangles, no overlap between items
+    (4, 32, 33, 36, 64, 1, 6),       # a single row of taps; several items per block
+]
+
+
+@pytest.mark.parametrize("dims", STACKED_TAP_SHAPES)
+@pytest.mark.parametrize("entry", ["general", "bf16"])
+def test_stacked_taps_for_few_filters(oracle, monkeypatch, dims, entry):
+    """Exact on integers and within tolerance, forced on, and equal to the unstacked kernel's result."""
+    N, C, H, W, K, R, S = dims
+    monkeypatch.setenv("CONV2D_B200_TF32_PAIR_TAPS", "2")
+    xi, wi = small_integers((N, C, H, W), 471), small_integers((K, C, R, S), 472)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry=entry, algo=ALGO_TF32).astype(np.float64), yi_ref)
+    x, w = uniform((N, C, H, W), 473), uniform((K, C, R, S), 474)
+    if entry == "bf16":
+        from helpers import bf16_values
+        x, w = bf16_values(x)[0], bf16_values(w)[0]
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    tol = TF32_TOL if entry == "general" else 1e-5
+    y_stacked = run_library(x, w, entry=entry, algo=ALGO_TF32)
+    assert_parity(y_stacked, y_ref, yabs, tol, f"stacked taps {entry} {dims}")
+    monkeypatch.setenv("CONV2D_B200_TF32_PAIR_TAPS", "0")
+    y_plain = run_library(x, w, entry=entry, algo=ALGO_TF32)
+    assert_parity(y_plain, y_ref, yabs, tol, f"unstacked {entry} {dims}")
+    assert_parity(y_stacked, y_plain.astype(np.float64), yabs, 2e-5, f"stacked vs unstacked {entry} {dims}")
