@@ -10,8 +10,12 @@
 //     keeps one input row segment of kThrQ+S-1 pixels in registers and reuses it for the S
 //     horizontal taps (Section 4.2); filter values are read as 128-bit units, image pixels are
 //     broadcast to the threads that differ only in their filter group.
+//   * the next channel block is fetched while the current one is multiplied (Algorithm 2's prefetch): here
+//     by asynchronous copies (cp.async) into a second image buffer and a raw filter buffer, so no thread
+//     holds the prefetched data in registers.
 // Changed for B200: register tile 8 x 8 with 128-bit shared-memory reads on both operands and packed
-// two-filter FMAs;
+// two-filter FMAs; the filters arrive as they lie in memory ([filter][channel][tap], 16-byte pieces) and are
+// turned around shared memory -> shared memory once per channel block;
 // the output is written with 128-bit stores per filter row segment where alignment allows.
 #include "common.cuh"
 
@@ -30,11 +34,25 @@ template <int R, int S, int CB, int TW, int TH>
 struct Smem {
     static constexpr int kRows = TH + R - 1;
     static constexpr int kPitch = (TW + S - 1 + 3 + 3) / 4 * 4;   // room for whole 128-bit reads past the halo
-    float img[CB][kRows][kPitch];
+    static constexpr int kRaw = CB * R * S;                      // floats of one filter in a channel block, as in memory
+    static constexpr int kRawPitch = (kRaw + 3) / 4 * 4;
+    float img[2][CB][kRows][kPitch];    // double buffer: channel block i + 1 lands while block i is multiplied
+    float raw[kTileK][kRawPitch];       // filters of the coming block as they lie in memory
     float flt[CB][R * S][kTileK + 4];   // +4: transposed filter stores spread over banks, 128-bit reads stay aligned
 };
 
-template <int R, int S, int CB, int TW, int TH>
+// Asynchronous global -> shared copy of `bytes` (4, 8 or 16); only the first src_bytes are read, the rest is zero.
+template <int BYTES>
+__device__ __forceinline__ void cp_async(void* dst_smem, const void* src, int src_bytes)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(dst_smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;" ::"r"(d), "l"(src), "n"(BYTES), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// XV / WV: floats per asynchronous copy of the image rows / of the filters (4, 2 or 1, by alignment).
+template <int R, int S, int CB, int TW, int TH, int XV, int WV>
 __global__ void __launch_bounds__(kThreads, 2)
 general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
                     int C, int H, int W, int K, int P, int Q, int tiles_q, int vec_st)
@@ -65,35 +83,52 @@ general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
 
     constexpr int NV = (kThrQ + S - 1 + 3) / 4;       // 128-bit reads per input row segment
 
-    for (int c0 = 0; c0 < C; c0 += CB) {
-        // ---- stage CB channels: image block with halo, filters transposed to [tap][filter] ----
-        for (int idx = tid; idx < CB * SM::kRows * SM::kPitch; idx += kThreads) {
-            const int col = idx % SM::kPitch;
-            const int row = (idx / SM::kPitch) % SM::kRows;
-            const int cc = idx / (SM::kPitch * SM::kRows);
-            const int c = c0 + cc, h = p0 + row, ww = q0 + col;
-            float v = 0.f;
-            if (c < C && h < H && ww < W) v = __ldg(xin + ((size_t)c * H + h) * W + ww);
-            sm.img[cc][row][col] = v;
+    // Issues the copies of the channel block that starts at c0: image rows with their halo into img[buf], the
+    // filters' runs of CB x R x S floats into raw.  Pieces outside the tensors are filled with zeros.
+    auto issue = [&](int c0, int buf) {
+        constexpr int kPieces = SM::kPitch / XV;
+        for (int idx = tid; idx < CB * SM::kRows * kPieces; idx += kThreads) {
+            const int v = idx % kPieces;
+            const int row = (idx / kPieces) % SM::kRows;
+            const int cc = idx / (kPieces * SM::kRows);
+            const int c = c0 + cc, h = p0 + row, col = q0 + v * XV;
+            const bool in = c < C && h < H && col < W;
+            const int left = in ? min(XV, W - col) * 4 : 0;
+            const float* src = in ? xin + ((size_t)c * H + h) * W + col : x;
+            cp_async<4 * XV>(&sm.img[buf][cc][row][v * XV], src, left);
         }
-        for (int idx = tid; idx < CB * R * S * kTileK; idx += kThreads) {
-            // consecutive threads walk the taps of one filter (contiguous in memory), then the channels
-            const int t = idx % (R * S);
-            const int cc = (idx / (R * S)) % CB;
-            const int kk = idx / (R * S * CB);
-            const int c = c0 + cc, k = k0 + kk;
-            float v = 0.f;
-            if (c < C && k < K) v = __ldg(w + ((size_t)k * C + c) * (R * S) + t);
-            sm.flt[cc][t][kk] = v;
+        constexpr int kRuns = SM::kRaw / WV;
+        const int live = (C - c0) * (R * S);                    // floats of a filter's run that exist
+        for (int idx = tid; idx < kTileK * kRuns; idx += kThreads) {
+            const int v = idx % kRuns, kk = idx / kRuns;
+            const int e = v * WV;
+            const bool in = k0 + kk < K && e < live;
+            const int left = in ? min(WV, live - e) * 4 : 0;
+            const float* src = in ? w + ((size_t)(k0 + kk) * C + c0) * (R * S) + e : w;
+            cp_async<4 * WV>(&sm.raw[kk][e], src, left);
+        }
+        cp_async_commit();
+    };
+
+    issue(0, 0);
+    for (int c0 = 0, it = 0; c0 < C; c0 += CB, ++it) {
+        const int buf = it & 1;
+        cp_async_wait_all();
+        __syncthreads();                 // this block has landed; everyone is done with the previous one
+        // filters: [filter][channel][tap] -> [channel][tap][filter]
+        for (int idx = tid; idx < kTileK * SM::kRaw; idx += kThreads) {
+            const int e = idx % SM::kRaw, kk = idx / SM::kRaw;
+            sm.flt[e / (R * S)][e % (R * S)][kk] = sm.raw[kk][e];
         }
         __syncthreads();
+        if (c0 + CB < C) issue(c0 + CB, buf ^ 1);      // the next block arrives under the multiplications below
 
 #pragma unroll 1
         for (int cc = 0; cc < CB; ++cc) {
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 float2 img[4 * NV];                              // (x, x)
-                const float4* src = reinterpret_cast<const float4*>(&sm.img[cc][seg_row + r][seg_col]);
+                const float4* src = reinterpret_cast<const float4*>(&sm.img[buf][cc][seg_row + r][seg_col]);
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     const float4 t = src[v];
@@ -116,7 +151,6 @@ general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
                 }
             }
         }
-        __syncthreads();
     }
 
     // ---- write the register tile ----
@@ -142,10 +176,10 @@ general_ffma_kernel(const float* __restrict__ x, const float* __restrict__ w, fl
     }
 }
 
-template <int R, int S, int CB, int TW, int TH>
-conv2d_status_t launch_tile(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
+template <int R, int S, int CB, int TW, int TH, int XV, int WV>
+conv2d_status_t launch_tile_v(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
 {
-    auto kern = general_ffma_kernel<R, S, CB, TW, TH>;
+    auto kern = general_ffma_kernel<R, S, CB, TW, TH, XV, WV>;
     const size_t smem = sizeof(Smem<R, S, CB, TW, TH>);
     static size_t smem_done[64] = {};
     if (smem > 48 * 1024 && raise_smem_limit(reinterpret_cast<const void*>(kern), smem, smem_done) != cudaSuccess)
@@ -156,6 +190,26 @@ conv2d_status_t launch_tile(const float* x, const float* w, float* y, const Shap
     kern<<<grid, kThreads, smem, stream>>>(x, w, y, sh.C, sh.H, sh.W, sh.K, sh.P, sh.Q, tiles_q, vec_st);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
+// Width of the asynchronous copies: whole 16-byte pieces where every piece starts on 16 bytes (image: W a multiple
+// of 4; filters: C*R*S and CB*R*S multiples of 4), else 8- or 4-byte pieces.
+template <int R, int S, int CB, int TW, int TH>
+conv2d_status_t launch_tile(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream)
+{
+    constexpr int kRaw = CB * R * S;
+    const bool x4 = sh.W % 4 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0;
+    const long long crs = (long long)sh.C * R * S;
+    const int wv = (kRaw % 4 == 0 && crs % 4 == 0 && reinterpret_cast<uintptr_t>(w) % 16 == 0) ? 4
+                 : (kRaw % 2 == 0 && crs % 2 == 0 && reinterpret_cast<uintptr_t>(w) % 8 == 0) ? 2 : 1;
+    if (x4) {
+        if (wv == 4) return launch_tile_v<R, S, CB, TW, TH, 4, (kRaw % 4 == 0 ? 4 : 1)>(x, w, y, sh, stream);
+        if (wv == 2) return launch_tile_v<R, S, CB, TW, TH, 4, (kRaw % 2 == 0 ? 2 : 1)>(x, w, y, sh, stream);
+        return launch_tile_v<R, S, CB, TW, TH, 4, 1>(x, w, y, sh, stream);
+    }
+    if (wv == 4) return launch_tile_v<R, S, CB, TW, TH, 1, (kRaw % 4 == 0 ? 4 : 1)>(x, w, y, sh, stream);
+    if (wv == 2) return launch_tile_v<R, S, CB, TW, TH, 1, (kRaw % 2 == 0 ? 2 : 1)>(x, w, y, sh, stream);
+    return launch_tile_v<R, S, CB, TW, TH, 1, 1>(x, w, y, sh, stream);
 }
 
 template <int R, int S, int CB>
