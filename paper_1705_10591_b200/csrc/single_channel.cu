@@ -858,7 +858,30 @@ conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shap
     // Large images: the wide persistent kernels (they need 16-byte aligned input rows for the bulk copies).
     const bool rows_ok = sh.W % 4 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0;
     if (rows_ok && env_int("CONV2D_B200_SC_WIDE", 1) != 0) {
-        int band_h = env_int("CONV2D_B200_SC_BAND_H", 8);
+        // Rows per work item: 8, or another height (4..16, as far as the double buffer fits) when that fills the last
+        // round of work items over the SMs clearly better (2048 x 2048, 1 x 1: 256 items of 8 rows are 1.73 rounds
+        // on 148 SMs, 146 items of 14 rows one round).  Every row below 8 costs a little (more halo rows, more
+        // per-item set-up), hence the 1.5 % per row.
+        // (Heights are multiples of the rows a step produces: an odd height would compute its last row twice.)
+        auto pick_band = [&](int step, int item_factor, size_t pitch_bytes) {
+            int sms = 148, dev = 0;
+            if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            const long long col_tiles = (sh.Q + kRowsW - 1) / kRowsW;
+            const size_t filter_bytes = (size_t)((sh.K + 1) / 2) * RS2 * sizeof(float4) + 64;
+            int best = 8;
+            double best_score = 0, score8 = 0;
+            for (int bh = 16; bh >= 4; bh -= step) {
+                if (bh % step || 2 * (size_t)(bh + R - 1) * pitch_bytes + filter_bytes > 227 * 1024) continue;
+                const long long items = (long long)item_factor * sh.N * ((sh.P + bh - 1) / bh) * col_tiles;
+                const long long rounds = (items + sms - 1) / sms;
+                const double score = (double)items / (double)(rounds * sms) * (1.0 - 0.015 * (8 - bh > 0 ? 8 - bh : 0));
+                if (bh == 8) score8 = score;
+                if (score > best_score) { best_score = score; best = bh; }
+            }
+            return score8 >= best_score - 0.02 ? 8 : best;       // 8 rows unless another height is clearly better
+        };
+        const int forced_band = env_int("CONV2D_B200_SC_BAND_H", 0);
+        int band_h = forced_band > 0 ? forced_band : pick_band((tr == 1 || R >= 7) ? 1 : 2, 1, kRowsPitch * sizeof(float));
         if (band_h < 1) band_h = 1;
         if (band_h > 16) band_h = 16;
         // Rows that are only 8-byte aligned: the variant that shifts odd rows by two columns.  Its aligned
@@ -866,7 +889,7 @@ conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shap
         // 1024 x 1024: 75 -> 41 us; 512 x 512: 26 -> 20 us), although half of its 2048 columns are idle there.
         if (sh.Q >= 384 && sh.Q % 4 == 2 && ((long long)sh.P * sh.Q) % 4 == 0 && reinterpret_cast<uintptr_t>(y) % 16 == 0 &&
             env_int("CONV2D_B200_SC_SHIFT", 1) != 0) {
-            const conv2d_status_t st = try_rows_shift<R, S>(x, w, y, sh, band_h, stream);
+            const conv2d_status_t st = try_rows_shift<R, S>(x, w, y, sh, forced_band > 0 ? band_h : pick_band(2, 2, kShiftPitch * sizeof(float)), stream);
             if (st != CONV2D_ERR_UNSUPPORTED) return st;
         }
         if (sh.Q >= env_int("CONV2D_B200_SC_WIDE_MINQ", 1024)) {
