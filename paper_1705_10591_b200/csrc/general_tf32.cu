@@ -45,6 +45,7 @@
 //     touches only this block's shared and tensor memory and overlaps the preceding kernel's tail.
 //   * Every wait is bounded; on expiry the block raises a flag, stops storing, frees its tensor memory and
 //     the status word in the workspace becomes non-zero.
+#include <cstdio>
 #include <cstdlib>
 #include <mutex>
 
@@ -109,6 +110,13 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     const float* w = static_cast<const float*>(w_any);
     const Plan p = make_plan(sh, b16);
     if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
+    if (env_int("CONV2D_B200_TF32_VERBOSE", 0) != 0)
+        fprintf(stderr, "conv2d plan: n_tile %d n_blocks %d tile_px %d groups %d nbuf %d npix %d cblks %d taps %d stacked %d "
+                "fold %dx%d patch_w %d tw %d rows %d cols %d a_stages %d cbg %d b_stages %d tps %d resident %d ksplit %d "
+                "items %lld grid %d smem %zu\n",
+                p.n_tile, p.n_blocks, p.tile_px, p.px_groups, p.nbuf, p.npix, p.cblks, p.taps, p.pair_taps, p.fold_r, p.fold_s,
+                p.patch_w, p.patch_tw, p.patch_rows, p.patch_cols, p.a_stages, p.cbg, p.b_stages, p.tps, p.resident, p.ksplit,
+                (long long)p.supertiles * p.n_blocks * p.ksplit, p.grid, p.smem_bytes);
     if (workspace_bytes < kStatusBytes + packed_floats(p) * sizeof(float)) return CONV2D_ERR_WORKSPACE;
     unsigned* status = static_cast<unsigned*>(workspace);
     float* wp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
