@@ -308,6 +308,12 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
         if (p.tps > p.taps) p.tps = p.taps;
         p.b_stages = 2;
         while (p.tps > 1 && smem_need(p.a_stages, p.npix, p.n_tile, 3, p.tps, 1) > kLimit) --p.tps;
+        // equal stages: 6 taps as 3 + 3 instead of 5 + 1 (the short stage's MMAs would end long before the next
+        // long stage has arrived)
+        {
+            const int per_block = (p.taps + p.tps - 1) / p.tps;
+            p.tps = (p.taps + per_block - 1) / per_block;
+        }
         while (p.b_stages < 4 && smem_need(p.a_stages, p.npix, p.n_tile, p.b_stages + 1, p.tps, 1) <= kLimit) ++p.b_stages;
         while (p.a_stages < kMaxAStages && p.taps <= 3 &&
                smem_need(p.a_stages + 1, p.npix, p.n_tile, p.b_stages, p.tps, p.cbg) <= kLimit - 32 * 1024) ++p.a_stages;
