@@ -128,6 +128,9 @@ GENERAL_SHAPES = [
     (5, 33, 7, 9, 128, 3, 3),      # batch*H*W = 315 pixels: ragged last tile, images change inside a tile
     (1, 16, 6, 70, 72, 5, 3),      # wide rows: horizontal wrap inside a tile
     (2, 48, 12, 12, 128, 1, 1),    # 1 x 1 with resident filters
+    (1, 24, 9, 10, 1000, 3, 3),    # 1000 filters: eight filter blocks, the last one partial
+    (1, 200, 8, 8, 24, 5, 5),      # long contraction, few filters and pixels: stacked taps with a split contraction
+    (3, 7, 33, 31, 64, 3, 2),      # odd image width, even tap count per row
 ]
 
 
