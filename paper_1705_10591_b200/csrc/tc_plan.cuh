@@ -273,6 +273,12 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
                 const double tile_time = (double)p.taps * p.cblks * (2 * mma_step + stage_cycles);
                 const double writeback = (nbuf == 1 ? 1.0 : 0.15) * (px / 128.0) * (3000.0 * p.n_tile / 128.0);
                 double cost = rounds * (tile_time + 0.5 * writeback);
+                // With one accumulator set the MMAs of an item wait for the whole write-back of the item before it
+                // (four warps, measured ~2000 cycles per 32-pixel block of 128 maps, ~1200 of 64); from the third round
+                // of items on that outweighs the wider MMAs (64 x 64 x 56 x 56 -> 128 maps, 3 x 3: 480-pixel items
+                // 69.1 us, 256-pixel items with two accumulator sets 64.6 us).
+                if (nbuf == 1 && rounds >= 3)
+                    cost += (double)(rounds - 2) * 0.75 * (px / 32.0) * (p.n_tile >= 128 ? 2000.0 : 1200.0);
                 // (items that leave half of the SMs idle are split in two along the channels further down)
                 if (items * 2 <= sms && p.cblks >= 2 && ksplit_allowed) cost = 0.5 * tile_time + writeback;
                 if (best_px == 0 || cost < best_cost) { best_px = px; best_cost = cost; }
