@@ -293,8 +293,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
     ap.add_argument("--no-general", action="store_true", help="skip the general-case configurations")
-    ap.add_argument("--operand", default="fp32", choices=["fp32", "bf16"],
-                    help="general-case workloads only: bf16 runs the 16-bit operand entry on the same values rounded to bf16")
+    ap.add_argument("--operand", default="fp32", choices=["fp32", "bf16", "fp32-exact"],
+                    help="general-case workloads only: bf16 runs the 16-bit operand entry on the same values rounded to "
+                         "bf16; fp32-exact runs the fp32 FMA kernel (1e-5 tolerance) instead of the tensor cores")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()
@@ -334,7 +335,8 @@ def main():
     if b16:
         xd16, wd16 = xd.to(torch.bfloat16).contiguous(), wd.to(torch.bfloat16).contiguous()
         args.no_e2e = True            # the host-buffer entry takes fp32 tensors only
-    algo = lib.ALGO_FFMA if single else (lib.ALGO_16BIT if b16 else lib.ALGO_AUTO)
+    ffma = args.operand == "fp32-exact" and not single
+    algo = lib.ALGO_FFMA if (single or ffma) else (lib.ALGO_16BIT if b16 else lib.ALGO_AUTO)
     ws_bytes = 0 if single else lib.conv2d_fwd_workspace_size(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, algo)
     ws = torch.zeros(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream().cuda_stream
@@ -402,7 +404,7 @@ def main():
     t_kernel_s = ms_per_step * 1e-3
     fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # TFLOP/s at max clock
     t_hbm = algorithmic_bytes / (peaks["hbm_gbs"] * 1e9)
-    if single:
+    if single or ffma:
         t_pipe, pipe_name, pipe_peak = cfg.flops / (fp32_peak * 1e12), "alu", fp32_peak
     else:
         pipe_peak = peaks["bf16_tflops"] if b16 else peaks["bf16_tflops"] / 2.0
@@ -431,7 +433,7 @@ def main():
     result = {
         "metric": "conv_fwd_gflops", "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16" if b16 else ("f32" if single else "tf32"), "data": "synthetic",
+        "vs_baseline": None, "dtype": "bf16" if b16 else ("f32" if (single or ffma) else "tf32"), "data": "synthetic",
         "config": {"workload": cfg.name, "operand": args.operand if not single else "fp32", **cfg.as_dict(), "parallelism": f"replicas x{world}",
                    "l2": "flushed between timed steps" if flush_between else
                          "inputs+outputs per step (2.2 GB) exceed the 126 MB L2"},
