@@ -154,6 +154,8 @@ conv2d_status_t conv2d_fwd_general_16bit(const void* x16, const void* w16, float
  * from conv2d_fwd_padded_workspace_size (the general workspace for the extended image, then the extended
  * image itself); it is required for every algorithm, 16-byte aligned, and its first 256 bytes are the
  * status block as usual.  pad_h, pad_w >= 0.  CONV2D_FLAG_WEIGHTS_PACKED keeps its meaning.
+ * algo is AUTO, FFMA or TF32.  N * C must not exceed 65535 (CONV2D_ERR_UNSUPPORTED otherwise, as for an unknown
+ * flag or algorithm; all of these are checked before anything is enqueued).
  */
 conv2d_status_t conv2d_fwd_padded_workspace_size(int N, int C, int H, int W, int K, int R, int S,
                                                  int pad_h, int pad_w, conv2d_algo_t algo, size_t* bytes);
@@ -173,6 +175,8 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
  * then runs conv2d_fwd_general on it: the same multiply-adds as the definition plus zeros, every algorithm.
  * 1 <= stride <= 8.  Workspace from conv2d_fwd_strided_workspace_size; required, 16-byte aligned, status
  * block first.  With CONV2D_FLAG_WEIGHTS_PACKED the rewritten filters of the previous call are reused too.
+ * algo is AUTO, FFMA or TF32; N * C must not exceed 65535 (CONV2D_ERR_UNSUPPORTED otherwise, checked before
+ * anything is enqueued).
  */
 conv2d_status_t conv2d_fwd_strided_workspace_size(int N, int C, int H, int W, int K, int R, int S,
                                                   int pad_h, int pad_w, int stride, conv2d_algo_t algo, size_t* bytes);
@@ -211,7 +215,9 @@ conv2d_status_t conv2d_fwd_general_strided(const float* x, const float* w, float
  *
  * x, w, y: device pointers as for conv2d_fwd_general.  wait = 0: enqueue and return;
  * wait != 0: also wait for the stream and return CONV2D_ERR_DEVICE_TIMEOUT if a bounded
- * on-device wait expired.
+ * on-device wait expired.  After a wait = 0 call, conv2d_get_status(NULL, cuda_stream) on the
+ * same device reports such a time-out (the array's status word stays set until the next call
+ * of this entry point clears it).
  */
 conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float* y,
                                            int N, int C, int H, int W, int K, int R, int S,
@@ -223,7 +229,11 @@ conv2d_status_t conv2d_fwd_general_noalloc(const float* x, const float* w, float
  * convolution runs (single-channel kernel when C == 1, else conv2d_fwd_general
  * with `algo`), y is copied back into y_host and the stream is synchronised.
  * Host buffers should be page-locked for the copies to run at full speed.
- * Returns the first error met, or the device status after synchronising.
+ * Returns the first error met, or the device status after synchronising
+ * (CONV2D_ERR_DEVICE_TIMEOUT if a bounded on-device wait expired).  The
+ * workspace is the one conv2d_fwd_general would need for `algo`; it may be
+ * NULL / 0 bytes when no tensor-core kernel can run (C == 1, algo = FFMA), and
+ * it is only read for a status when the tensor-core kernel ran.
  */
 conv2d_status_t conv2d_fwd_host(const float* x_host, const float* w_host, float* y_host,
                                 float* x, float* w, float* y,
@@ -232,10 +242,12 @@ conv2d_status_t conv2d_fwd_host(const float* x_host, const float* w_host, float*
                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Waits for `cuda_stream`, then reads the status block at the start of
- * `workspace` (NULL workspace: only waits).  Returns CONV2D_OK,
- * CONV2D_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded wait, or
- * CONV2D_ERR_CUDA if the stream reported an error.
+ * Waits for `cuda_stream`, then reads the device's time-out words: the one the
+ * single-channel kernels raise (read and cleared), the status word of the fixed
+ * array of conv2d_fwd_general_noalloc if that entry has run on the current
+ * device, and the status block at the start of `workspace` unless it is NULL.
+ * Returns CONV2D_OK, CONV2D_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded
+ * wait, or CONV2D_ERR_CUDA if the stream reported an error.
  */
 conv2d_status_t conv2d_get_status(const void* workspace, void* cuda_stream);
 

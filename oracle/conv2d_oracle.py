@@ -45,7 +45,7 @@ def _load():
         fp = ctypes.POINTER(ctypes.c_float)
         dp = ctypes.POINTER(ctypes.c_double)
         i = ctypes.c_int
-        lib.conv2d_oracle_range.argtypes = [fp, fp, dp, fp, dp] + [i] * 7 + [i] * 6 + [i, i]
+        lib.conv2d_oracle_range.argtypes = [fp, fp, dp, dp] + [i] * 7 + [i] * 6 + [i]
         lib.conv2d_oracle_range.restype = i
         lib.conv2d_oracle_threads.argtypes = []
         lib.conv2d_oracle_threads.restype = i
@@ -85,8 +85,8 @@ def conv2d_oracle_range(x, w, n_range=None, k_range=None, p_range=None, mode=MOD
     dp = ctypes.POINTER(ctypes.c_double)
     rc = _load().conv2d_oracle_range(
         x.ctypes.data_as(fp), w.ctypes.data_as(fp),
-        y64.ctypes.data_as(dp), None, yabs.ctypes.data_as(dp),
-        N, C, H, W, K, R, S, n0, n1, k0, k1, p0, p1, 1, int(mode))
+        y64.ctypes.data_as(dp), yabs.ctypes.data_as(dp),
+        N, C, H, W, K, R, S, n0, n1, k0, k1, p0, p1, int(mode))
     if rc != 0:
         raise ValueError(f"oracle rejected its arguments (code {rc})")
     return y64, yabs

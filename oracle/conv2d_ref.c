@@ -66,16 +66,16 @@ int conv2d_oracle_threads(void)
 
 /*
  * Computes output rows p in [p_begin, p_end) of maps k in [k_begin, k_end) of
- * images n in [n_begin, n_end).  Results are written at their natural offsets
- * of full-size NKPQ arrays when `compact` is 0, or into a dense
- * [n_end-n_begin][k_end-k_begin][p_end-p_begin][Q] array when `compact` is 1.
- * y64, y32 and yabs may each be NULL.  Returns 0, or 1 on a bad argument.
+ * images n in [n_begin, n_end) into dense arrays
+ * [n_end-n_begin][k_end-k_begin][p_end-p_begin][Q]; the whole problem is the
+ * range [0,N) x [0,K) x [0,P).  y64 and yabs may each be NULL.
+ * Returns 0, or 1 on a bad argument.
  */
 int conv2d_oracle_range(const float *x, const float *w,
-                        double *y64, float *y32, double *yabs,
+                        double *y64, double *yabs,
                         int N, int C, int H, int W, int K, int R, int S,
                         int n_begin, int n_end, int k_begin, int k_end,
-                        int p_begin, int p_end, int compact, int mode)
+                        int p_begin, int p_end, int mode)
 {
     if (!x || !w) return 1;
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || R <= 0 || S <= 0) return 1;
@@ -106,25 +106,10 @@ int conv2d_oracle_range(const float *x, const float *w,
                     }
                 }
             }
-            size_t yi;
-            if (compact)
-                yi = (((size_t)(n - n_begin) * nk + (size_t)(k - k_begin)) * np + (size_t)(p - p_begin)) * Q + (size_t)q;
-            else
-                yi = (((size_t)n * K + k) * P + (size_t)p) * Q + (size_t)q;
+            const size_t yi = (((size_t)(n - n_begin) * nk + (size_t)(k - k_begin)) * np + (size_t)(p - p_begin)) * Q + (size_t)q;
             if (y64) y64[yi] = acc;
-            if (y32) y32[yi] = (float)acc;
             if (yabs) yabs[yi] = mag;
         }
     }
     return 0;
-}
-
-/* The whole problem. */
-int conv2d_oracle(const float *x, const float *w,
-                  double *y64, float *y32, double *yabs,
-                  int N, int C, int H, int W, int K, int R, int S, int mode)
-{
-    if (R > H || S > W || H <= 0 || R <= 0) return 1;
-    return conv2d_oracle_range(x, w, y64, y32, yabs, N, C, H, W, K, R, S,
-                               0, N, 0, K, 0, H - R + 1, 0, mode);
 }

@@ -24,23 +24,40 @@ def _stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> Path:
+    """Compiles every source to an object file (in parallel) and links the shared library."""
     if not force and not _stale():
         return LIB
-    cmd = [
+    from concurrent.futures import ThreadPoolExecutor
+    import tempfile
+
+    common = [
         "nvcc", "-std=c++17", "-O3", "-lineinfo",
         "-gencode", "arch=compute_100a,code=sm_100a",
-        "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
+        "-Xcompiler", "-fPIC",
         "-I", str(ROOT / "include"), "-I", str(CSRC),
         "-DCONV2D_B200_BUILD",
-        "-o", str(LIB),
-    ] + [str(CSRC / s) for s in SOURCES]
+    ]
     if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose:
-        sys.stderr.write(res.stderr)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        common.insert(1, "-Xptxas=-v")
+    with tempfile.TemporaryDirectory(prefix="conv2d_b200_build_") as tmp:
+        objs = [str(Path(tmp) / (Path(s).stem + ".o")) for s in SOURCES]
+
+        def compile_one(job):
+            src, obj = job
+            return subprocess.run(common + ["-c", str(CSRC / src), "-o", obj], capture_output=True, text=True)
+
+        with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
+            results = list(pool.map(compile_one, zip(SOURCES, objs)))
+        for res in results:
+            if verbose:
+                sys.stderr.write(res.stderr)
+            if res.returncode != 0:
+                raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        link = ["nvcc", "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a",
+                "-o", str(LIB)] + objs
+        res = subprocess.run(link, capture_output=True, text=True)
+        if res.returncode != 0:
+            raise RuntimeError("nvcc (link) failed:\n" + res.stdout + res.stderr)
     return LIB
 
 

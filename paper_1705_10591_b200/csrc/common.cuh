@@ -43,6 +43,20 @@ inline cudaError_t raise_smem_limit(const void* kernel, size_t bytes, size_t (&d
     return e;
 }
 
+// Multiprocessors of the current device (looked up once per device; 148 on B200, which is also the answer when
+// the query fails).  Planners size their grids and pick their tiles from it.
+inline int sm_count()
+{
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        cached[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+    }
+    return cached[dev];
+}
+
 // Tuning and test switches come from the environment, but only in a process that was started with
 // CONV2D_B200_TUNING set (looked up once): production calls never scan the environment, and stray variables
 // cannot change what the library does.
@@ -74,6 +88,8 @@ conv2d_status_t launch_general_b16(const void* x, const void* w, float* y, const
 
 // Variant of the tensor-core path whose scratch is a fixed array inside the library image.
 constexpr size_t kNoAllocScratchBytes = kStatusBytes + (size_t)8 * 1024 * 1024;
+// Status word of that array on the current device (false when no such call has run there); stream idle.
+cudaError_t noalloc_device_timeout(bool* raised);
 conv2d_status_t launch_general_tf32_noalloc(const float* x, const float* w, float* y, const Shape& sh,
                                             bool wait, cudaStream_t stream);
 

@@ -161,12 +161,15 @@ conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float*
     return launch_single_channel(x, w, y, sh, static_cast<cudaStream_t>(cuda_stream));
 }
 
-conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
-                                   int N, int C, int H, int W, int K, int R, int S,
-                                   conv2d_algo_t algo,
-                                   void* workspace, size_t workspace_bytes,
-                                   unsigned flags, void* cuda_stream)
+// The general entry; *status_in_workspace (optional) is set when the tensor-core launcher ran, i.e. when the
+// status block at the start of the workspace was cleared by this call and is the place to look for a time-out.
+static conv2d_status_t general_dispatch(const float* x, const float* w, float* y,
+                                        int N, int C, int H, int W, int K, int R, int S,
+                                        conv2d_algo_t algo,
+                                        void* workspace, size_t workspace_bytes,
+                                        unsigned flags, void* cuda_stream, bool* status_in_workspace)
 {
+    if (status_in_workspace) *status_in_workspace = false;
     if (!x || !w || !y) return CONV2D_ERR_NULL;
     Shape sh;
     conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
@@ -182,9 +185,19 @@ conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
     if (algo != CONV2D_ALGO_FFMA && workspace) {
         // one planning pass: the launcher reports "no instance" or "workspace too small" itself
         st = launch_general_tf32(x, w, y, sh, workspace, workspace_bytes, (flags & CONV2D_FLAG_WEIGHTS_PACKED) != 0, stream);
+        if (st == CONV2D_OK && status_in_workspace) *status_in_workspace = true;
         if (algo == CONV2D_ALGO_TF32 || (st != CONV2D_ERR_UNSUPPORTED && st != CONV2D_ERR_WORKSPACE)) return st;
     }
     return launch_general_ffma(x, w, y, sh, stream);
+}
+
+conv2d_status_t conv2d_fwd_general(const float* x, const float* w, float* y,
+                                   int N, int C, int H, int W, int K, int R, int S,
+                                   conv2d_algo_t algo,
+                                   void* workspace, size_t workspace_bytes,
+                                   unsigned flags, void* cuda_stream)
+{
+    return general_dispatch(x, w, y, N, C, H, W, K, R, S, algo, workspace, workspace_bytes, flags, cuda_stream, nullptr);
 }
 
 conv2d_status_t conv2d_fwd_general_16bit(const void* x16, const void* w16, float* y,
@@ -228,7 +241,10 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
     size_t need = 0, inner = 0;
     conv2d_status_t st = conv2d_fwd_padded_workspace_size(N, C, H, W, K, R, S, pad_h, pad_w, algo, &need);
     if (st != CONV2D_OK) return st;
-    if (!aligned16(x) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (flags & ~(unsigned)CONV2D_FLAG_WEIGHTS_PACKED) return CONV2D_ERR_UNSUPPORTED;
+    if (algo != CONV2D_ALGO_TF32 && algo != CONV2D_ALGO_AUTO && algo != CONV2D_ALGO_FFMA) return CONV2D_ERR_UNSUPPORTED;
+    if ((long long)N * C > 65535) return CONV2D_ERR_UNSUPPORTED;      // one block row of the extension kernel per plane
     if (workspace_bytes < need) return CONV2D_ERR_WORKSPACE;
     st = conv2d_fwd_workspace_size(N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, algo, &inner);
     if (st != CONV2D_OK) return st;
@@ -236,7 +252,7 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
     if (st != CONV2D_OK) return st;
     // The tensor-core kernel takes the padding itself where it has an instance with patch addressing (no extra
     // pass over x); its workspace is the front part of this call's workspace as usual.
-    if (algo != CONV2D_ALGO_FFMA && (pad_h || pad_w) && aligned16(w) && aligned16(y)) {
+    if (algo != CONV2D_ALGO_FFMA && (pad_h || pad_w)) {
         Shape shp;
         if (make_shape(N, C, H + 2 * pad_h, W + 2 * pad_w, K, R, S, &shp) == CONV2D_OK) {
             shp.H = H; shp.W = W; shp.pad_h = pad_h; shp.pad_w = pad_w;       // P, Q are those of the extended image
@@ -249,7 +265,6 @@ conv2d_status_t conv2d_fwd_general_padded(const float* x, const float* w, float*
     const bool own_status = inner < kStatusBytes;          // fp32 path: no workspace of its own
     float* xp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + round_up_256(own_status ? kStatusBytes : inner));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if ((long long)N * C > 65535) return CONV2D_ERR_UNSUPPORTED;
     const int plane_p = (H + 2 * pad_h) * (W + 2 * pad_w);
     const dim3 grid((unsigned)((plane_p + 1023) / 1024 > 64 ? 64 : (plane_p + 1023) / 1024), (unsigned)(N * C));
     pad_planes_kernel<<<grid, 256, 0, stream>>>(x, xp, H, W, pad_h, pad_w, own_status ? static_cast<unsigned*>(workspace) : nullptr);
@@ -283,7 +298,10 @@ conv2d_status_t conv2d_fwd_general_strided(const float* x, const float* w, float
     size_t need = 0, inner = 0;
     conv2d_status_t st = conv2d_fwd_strided_workspace_size(N, C, H, W, K, R, S, pad_h, pad_w, stride, algo, &need);
     if (st != CONV2D_OK) return st;
-    if (!aligned16(x) || !aligned16(w) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(workspace)) return CONV2D_ERR_ALIGN;
+    if (flags & ~(unsigned)CONV2D_FLAG_WEIGHTS_PACKED) return CONV2D_ERR_UNSUPPORTED;
+    if (algo != CONV2D_ALGO_TF32 && algo != CONV2D_ALGO_AUTO && algo != CONV2D_ALGO_FFMA) return CONV2D_ERR_UNSUPPORTED;
+    if ((long long)N * C > 65535) return CONV2D_ERR_UNSUPPORTED;      // one block row of the rewriting kernel per plane
     if (workspace_bytes < need) return CONV2D_ERR_WORKSPACE;
     if (stride == 1)            // nothing to rewrite: the padded entry (its workspace is a prefix of this one's)
         return conv2d_fwd_general_padded(x, w, y, N, C, H, W, K, R, S, pad_h, pad_w, algo, workspace, workspace_bytes, flags, cuda_stream);
@@ -298,8 +316,7 @@ conv2d_status_t conv2d_fwd_general_strided(const float* x, const float* w, float
     float* x2 = reinterpret_cast<float*>(base + round_up_256(own_status ? kStatusBytes : inner));
     float* w2 = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(x2) + round_up_256((size_t)N * g.C2 * g.H2 * g.W2 * sizeof(float)));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    auto blocks_for = [](long long total) { long long b = (total + 255) / 256; return (unsigned)(b > 148 * 32 ? 148 * 32 : b); };
-    if ((long long)N * C > 65535) return CONV2D_ERR_UNSUPPORTED;
+    auto blocks_for = [](long long total) { long long b = (total + 255) / 256; return (unsigned)(b > sm_count() * 32LL ? sm_count() * 32LL : b); };
     {
         const int work = stride * stride * g.H2 * g.W2;
         const dim3 grid((unsigned)((work + 1023) / 1024 > 64 ? 64 : (work + 1023) / 1024), (unsigned)(N * C));
@@ -345,13 +362,16 @@ conv2d_status_t conv2d_fwd_host(const float* x_host, const float* w_host, float*
     const size_t yb = (size_t)N * K * sh.P * sh.Q * sizeof(float);
     if (cudaMemcpyAsync(x, x_host, xb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CONV2D_ERR_CUDA;
     if (cudaMemcpyAsync(w, w_host, wb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CONV2D_ERR_CUDA;
+    // Only the tensor-core launcher clears and uses the status block in the workspace; after any other kernel the
+    // workspace (which may be NULL, of size 0, or never written) must not be read for a status.
+    bool status_in_workspace = false;
     if (C == 1 && algo != CONV2D_ALGO_TF32)
         st = conv2d_fwd_single_channel(x, w, y, N, H, W, K, R, S, nullptr, 0, 0, cuda_stream);
     else
-        st = conv2d_fwd_general(x, w, y, N, C, H, W, K, R, S, algo, workspace, workspace_bytes, 0, cuda_stream);
+        st = general_dispatch(x, w, y, N, C, H, W, K, R, S, algo, workspace, workspace_bytes, 0, cuda_stream, &status_in_workspace);
     if (st != CONV2D_OK) return st;
     if (cudaMemcpyAsync(y_host, y, yb, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return CONV2D_ERR_CUDA;
-    return conv2d_get_status(workspace, cuda_stream);
+    return conv2d_get_status(status_in_workspace ? workspace : nullptr, cuda_stream);
 }
 
 conv2d_status_t conv2d_get_status(const void* workspace, void* cuda_stream)
@@ -360,6 +380,9 @@ conv2d_status_t conv2d_get_status(const void* workspace, void* cuda_stream)
     if (cudaStreamSynchronize(stream) != cudaSuccess) return CONV2D_ERR_CUDA;
     bool raised = false;
     if (consume_device_timeout(&raised) != cudaSuccess) return CONV2D_ERR_CUDA;
+    if (raised) return CONV2D_ERR_DEVICE_TIMEOUT;
+    // the fixed array of conv2d_fwd_general_noalloc: its status word stays set until that entry's next call
+    if (noalloc_device_timeout(&raised) != cudaSuccess) return CONV2D_ERR_CUDA;
     if (raised) return CONV2D_ERR_DEVICE_TIMEOUT;
     if (!workspace) return CONV2D_OK;
     unsigned word = 0;

@@ -247,7 +247,7 @@ conv2d_status_t launch_direct_fallback(const float* x, const float* w, float* y,
     const long long total = (long long)sh.N * sh.K * sh.P * sh.Q;
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
-    if (blocks > 148LL * 64) blocks = 148LL * 64;
+    if (blocks > (long long)sm_count() * 64) blocks = (long long)sm_count() * 64;
     direct_kernel<<<(unsigned)blocks, threads, 0, stream>>>(x, w, y, sh.C, sh.H, sh.W, sh.K, sh.R, sh.S, sh.P, sh.Q, total);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;

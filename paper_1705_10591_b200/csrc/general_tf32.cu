@@ -126,7 +126,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         const FoldedFilter ff{sh.C, sh.R, sh.S, p.fold_r, p.fold_s};
         const long long lanes = total / p.taps * (b16 ? 2 : 1);      // one thread per element of a tap's slice
         long long blocks = (lanes + 255) / 256;
-        if (blocks > 148 * 16) blocks = 148 * 16;
+        if (blocks > sm_count() * 16LL) blocks = sm_count() * 16LL;
         const size_t tile_bytes = (size_t)8 * kCB * 4 * p.taps;       // 8 filters x one channel block x taps
         if (p.fold_r * p.fold_s == 1 && tile_bytes <= 48 * 1024 && p.n_tile % 8 == 0 && !p.pair_taps) {
             const dim3 grid((unsigned)(p.n_blocks * p.n_tile / 8), (unsigned)p.cblks);
@@ -253,6 +253,31 @@ conv2d_status_t launch_general_b16(const void* x, const void* w, float* y, const
 // device image, so every GPU that loads the library holds these bytes until the process exits.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mu;
+void* g_noalloc_scratch_of_device[kMaxDevices] = {};     // device address of the array, per device, once looked up
+}  // namespace
+
+// Reads the status word of the fixed array on the current device, if a call without caller scratch has run
+// there (otherwise the word cannot be set and nothing is read).  The stream must already be idle.
+cudaError_t noalloc_device_timeout(bool* raised)
+{
+    *raised = false;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaSuccess;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mu);
+        scratch = g_noalloc_scratch_of_device[dev];
+    }
+    if (!scratch) return cudaSuccess;
+    unsigned word = 0;
+    const cudaError_t e = cudaMemcpy(&word, scratch, sizeof word, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) *raised = word != 0;
+    return e;
+}
+
 conv2d_status_t launch_general_tf32_noalloc(const float* x, const float* w, float* y, const Shape& sh,
                                             bool wait, cudaStream_t stream)
 {
@@ -261,20 +286,17 @@ conv2d_status_t launch_general_tf32_noalloc(const float* x, const float* w, floa
 
     // In host code the array's name is only a handle; the device address has to be asked for, once per
     // device, with that device current.
-    constexpr int kMaxDevices = 64;
-    static std::mutex mu;
-    static void* scratch_of_device[kMaxDevices] = {};
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CONV2D_ERR_CUDA;
     void* scratch = nullptr;
     {
-        std::lock_guard<std::mutex> lock(mu);
-        if (!scratch_of_device[dev]) {
+        std::lock_guard<std::mutex> lock(g_noalloc_mu);
+        if (!g_noalloc_scratch_of_device[dev]) {
             void* p = nullptr;
             if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return CONV2D_ERR_CUDA;
-            scratch_of_device[dev] = p;
+            g_noalloc_scratch_of_device[dev] = p;
         }
-        scratch = scratch_of_device[dev];
+        scratch = g_noalloc_scratch_of_device[dev];
     }
     conv2d_status_t st = launch_general_tf32(x, w, y, sh, scratch, kNoAllocScratchBytes, /*weights_packed=*/false, stream);
     if (st != CONV2D_OK || !wait) return st;

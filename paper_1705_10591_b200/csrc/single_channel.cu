@@ -459,7 +459,8 @@ constexpr int kRowsPitch4 = kRowsPitch / 4;
 template <int R, int S, int TR>
 __global__ void __launch_bounds__(kRowsThreads, 1)
 single_channel_rows_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
-                           int N, int H, int W, int K, int P, int Q, int band_h, int col_tiles, int items, int unit)
+                           int N, int H, int W, int K, int P, int Q, int band_h, int col_tiles, int items, int unit,
+                           unsigned max_polls, int test_short_item)
 {
     constexpr int NV = (S + kVec - 1 + 3) / 4;
     constexpr int WC = 4 * NV;
@@ -496,6 +497,7 @@ single_channel_rows_kernel(const float* __restrict__ x, const float* __restrict_
 
     const int bands = (P + band_h - 1) / band_h;
     // item -> (image, band, column tile); the column tile varies fastest
+    uint32_t issued[2] = {0u, 0u};                        // copies armed per stage (thread 0)
     auto issue = [&](int item, int stage) {               // thread 0 only
         const int ct = item % col_tiles;
         const int band = (item / col_tiles) % bands;
@@ -504,7 +506,10 @@ single_channel_rows_kernel(const float* __restrict__ x, const float* __restrict_
         const int rows_in = min(band_h, P - row0) + R - 1;
         const int cols = min(kRowsPitch, W - col0);                   // multiple of 4 (W % 4 == 0)
         const uint32_t row_bytes = (uint32_t)cols * 4u;
-        ptx::mbar_arrive_expect_tx(&full[stage], row_bytes * (uint32_t)rows_in);
+        if (*abort_flag) return;                                      // a wait has run out: no further copies
+        ++issued[stage];
+        // (test hook: one item is armed for one row more than is copied, so that its wait runs out)
+        ptx::mbar_arrive_expect_tx(&full[stage], row_bytes * (uint32_t)(rows_in + (item == test_short_item ? 1 : 0)));
         const float* src = x + ((size_t)n * H + row0) * W + col0;
         float4* dst = tiles4 + (size_t)stage * stage_f4;
         for (int r = 0; r < rows_in; ++r)
@@ -519,7 +524,7 @@ single_channel_rows_kernel(const float* __restrict__ x, const float* __restrict_
         const int stage = local & 1;
         __syncthreads();                                              // everyone is done reading the other buffer
         if (tid == 0 && it + (int)gridDim.x < items) issue(it + gridDim.x, stage ^ 1);
-        if (alive && !ptx::mbar_wait_bounded(&full[stage], (uint32_t)(local >> 1) & 1u, abort_flag)) alive = false;
+        if (alive && !ptx::mbar_wait_bounded(&full[stage], (uint32_t)(local >> 1) & 1u, abort_flag, max_polls)) alive = false;
         if (!alive) continue;                                         // keep meeting the barriers, do no work
 
         const int ct = it % col_tiles;
@@ -602,10 +607,11 @@ single_channel_rows_kernel(const float* __restrict__ x, const float* __restrict_
     }
     __syncthreads();
     if (tid == 0 && *abort_flag) {
-        // a copy may still be in flight into this block's shared memory: give it a bounded time to land
+        // The last copy armed on each stage may still be in flight into this block's shared memory: give it a
+        // bounded time to land (a copy that completed long ago answers at the first poll).
         uint32_t dummy = 0;
-        ptx::mbar_wait_bounded(&full[0], 0u, &dummy, 1u << 12);
-        ptx::mbar_wait_bounded(&full[1], 0u, &dummy, 1u << 12);
+        for (int st = 0; st < 2; ++st)
+            if (issued[st]) ptx::mbar_wait_bounded(&full[st], (issued[st] - 1u) & 1u, &dummy, 1u << 12);
         atomicExch(&g_device_timeout, 1u);
     }
 }
@@ -624,11 +630,14 @@ conv2d_status_t launch_rows(const float* x, const float* w, float* y, const Shap
     const int col_tiles = (sh.Q + kRowsW - 1) / kRowsW;
     const long long items = (long long)sh.N * ((sh.P + band_h - 1) / band_h) * col_tiles;
     if (items > 0x7fffffffLL) return CONV2D_ERR_UNSUPPORTED;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int grid = (int)(items < sms ? items : sms);
     const int unit = (reinterpret_cast<uintptr_t>(y) % 16 != 0) ? 1 : (sh.Q % 4 == 0 ? 4 : (sh.Q % 2 == 0 ? 2 : 1));
-    kern<<<grid, kRowsThreads, smem, stream>>>(x, w, y, sh.N, sh.H, sh.W, sh.K, sh.P, sh.Q, band_h, col_tiles, (int)items, unit);
+    // Failure-detection test hooks (host-side injection only): a short wait bound and one item whose barrier
+    // expects a row that is never copied, so that the wait expires and the time-out path can be checked.
+    kern<<<grid, kRowsThreads, smem, stream>>>(x, w, y, sh.N, sh.H, sh.W, sh.K, sh.P, sh.Q, band_h, col_tiles, (int)items, unit,
+                                               (unsigned)env_int("CONV2D_B200_SC_MAX_POLLS", 1 << 22),
+                                               env_int("CONV2D_B200_SC_TEST_SHORT_ITEM", -1));
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
 }
@@ -648,7 +657,8 @@ constexpr int kShiftPitch2 = kShiftPitch / 2;
 template <int R, int S>
 __global__ void __launch_bounds__(kRowsThreads, 1)
 single_channel_rows_shift_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
-                                 int N, int H, int W, int K, int P, int Q, int band_h, int col_tiles, int items)
+                                 int N, int H, int W, int K, int P, int Q, int band_h, int col_tiles, int items,
+                                 unsigned max_polls, int test_short_item)
 {
     constexpr int WC = (S + kVec - 1 + 1) / 2 * 2;      // window columns, even
     constexpr int RS = R * S;
@@ -684,6 +694,7 @@ single_channel_rows_shift_kernel(const float* __restrict__ x, const float* __res
     const int bands = (P + band_h - 1) / band_h;
     // item -> (image, band, column tile, row class); the class varies fastest, then the column tile.
     // Staged column c of a row holds image column col0 - 4 + c.
+    uint32_t issued[2] = {0u, 0u};                        // copies armed per stage (thread 0)
     auto issue = [&](int item, int stage) {               // thread 0 only
         const int rest = item >> 1;
         const int ct = rest % col_tiles;
@@ -695,7 +706,10 @@ single_channel_rows_shift_kernel(const float* __restrict__ x, const float* __res
         const int dst_off = src_col - (col0 - 4);                     // 0 or 4 floats
         const int cols = min(kShiftPitch - dst_off, W - src_col);     // multiple of 4 (W % 4 == 0)
         const uint32_t row_bytes = (uint32_t)cols * 4u;
-        ptx::mbar_arrive_expect_tx(&full[stage], row_bytes * (uint32_t)rows_in);
+        if (*abort_flag) return;                                      // a wait has run out: no further copies
+        ++issued[stage];
+        // (test hook: one item is armed for one row more than is copied, so that its wait runs out)
+        ptx::mbar_arrive_expect_tx(&full[stage], row_bytes * (uint32_t)(rows_in + (item == test_short_item ? 1 : 0)));
         const float* src = x + ((size_t)n * H + row0) * W + src_col;
         float* dst = tiles + (size_t)stage * stage_f + dst_off;
         for (int r = 0; r < rows_in; ++r)
@@ -710,7 +724,7 @@ single_channel_rows_shift_kernel(const float* __restrict__ x, const float* __res
         const int stage = local & 1;
         __syncthreads();                                              // everyone is done reading the other buffer
         if (tid == 0 && it + (int)gridDim.x < items) issue(it + gridDim.x, stage ^ 1);
-        if (alive && !ptx::mbar_wait_bounded(&full[stage], (uint32_t)(local >> 1) & 1u, abort_flag)) alive = false;
+        if (alive && !ptx::mbar_wait_bounded(&full[stage], (uint32_t)(local >> 1) & 1u, abort_flag, max_polls)) alive = false;
         if (!alive) continue;                                         // keep meeting the barriers, do no work
 
         const int cls = it & 1;                                       // parity of the output rows of this item
@@ -786,9 +800,10 @@ single_channel_rows_shift_kernel(const float* __restrict__ x, const float* __res
     }
     __syncthreads();
     if (tid == 0 && *abort_flag) {
+        // as in the kernel above: wait (bounded) for the last copy armed on each stage
         uint32_t dummy = 0;
-        ptx::mbar_wait_bounded(&full[0], 0u, &dummy, 1u << 12);
-        ptx::mbar_wait_bounded(&full[1], 0u, &dummy, 1u << 12);
+        for (int st = 0; st < 2; ++st)
+            if (issued[st]) ptx::mbar_wait_bounded(&full[st], (issued[st] - 1u) & 1u, &dummy, 1u << 12);
         atomicExch(&g_device_timeout, 1u);
     }
 }
@@ -812,10 +827,11 @@ conv2d_status_t launch_rows_shift(const float* x, const float* w, float* y, cons
     const int col_tiles = (sh.Q + 2 + kRowsW - 1) / kRowsW;    // odd rows start two columns to the left
     const long long items = 2LL * sh.N * ((sh.P + band_h - 1) / band_h) * col_tiles;
     if (items > 0x7fffffffLL) return CONV2D_ERR_UNSUPPORTED;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int grid = (int)(items < sms ? items : sms);
-    kern<<<grid, kRowsThreads, smem, stream>>>(x, w, y, sh.N, sh.H, sh.W, sh.K, sh.P, sh.Q, band_h, col_tiles, (int)items);
+    kern<<<grid, kRowsThreads, smem, stream>>>(x, w, y, sh.N, sh.H, sh.W, sh.K, sh.P, sh.Q, band_h, col_tiles, (int)items,
+                                               (unsigned)env_int("CONV2D_B200_SC_MAX_POLLS", 1 << 22),
+                                               env_int("CONV2D_B200_SC_TEST_SHORT_ITEM", -1));
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
 }
@@ -841,7 +857,7 @@ conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shap
         // down to 2, aiming at four blocks per SM
         tile_h = 8;
         const long long col_tiles = (sh.Q + kTileW - 1) / kTileW;
-        while (tile_h > 2 && col_tiles * ((sh.P + tile_h - 1) / tile_h) * sh.N < 4 * 148) tile_h >>= 1;
+        while (tile_h > 2 && col_tiles * ((sh.P + tile_h - 1) / tile_h) * sh.N < 4 * sm_count()) tile_h >>= 1;
     }
     if (tile_h < 1) tile_h = 1;
     if (tile_h > 64) tile_h = 64;
@@ -864,8 +880,7 @@ conv2d_status_t dispatch_rs(const float* x, const float* w, float* y, const Shap
         // per-item set-up), hence the 1.5 % per row.
         // (Heights are multiples of the rows a step produces: an odd height would compute its last row twice.)
         auto pick_band = [&](int step, int item_factor, size_t pitch_bytes) {
-            int sms = 148, dev = 0;
-            if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            const int sms = sm_count();
             const long long col_tiles = (sh.Q + kRowsW - 1) / kRowsW;
             const size_t filter_bytes = (size_t)((sh.K + 1) / 2) * RS2 * sizeof(float4) + 64;
             int best = 8;

@@ -10,11 +10,25 @@ namespace {
 
 using namespace ptx;
 
-// Cycle counter read that the compiler may not move across memory operations or barriers.
+// Tuning builds (-DCONV2D_B200_TC_DIAGNOSTICS) make the MMA-issuing thread of block 0 count its cycles and leave
+// them in status words 2-9.  The product build contains none of it: that thread's instruction stream is what
+// bounds the heavy shapes, and a timer read with a memory clobber around every wait is not free.
+#ifdef CONV2D_B200_TC_DIAGNOSTICS
+constexpr bool kDiag = true;
+#else
+constexpr bool kDiag = false;
+#endif
+// Cycle counter read that the compiler may not move across memory operations or barriers (0 in product builds).
 __device__ __forceinline__ long long clock_now()
 {
-    long long t;
-    asm volatile("mov.u64 %0, %%clock64;" : "=l"(t) :: "memory");
+    long long t = 0;
+    if (kDiag) asm volatile("mov.u64 %0, %%clock64;" : "=l"(t) :: "memory");
+    return t;
+}
+__device__ __forceinline__ unsigned long long wall_ns()
+{
+    unsigned long long t = 0;
+    if (kDiag) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
 
@@ -324,20 +338,22 @@ general_tc_kernel(const KernelArgs a)
     uint64_t* acc_full = b_empty + kMaxBStages;            // [2]
     uint64_t* acc_empty = acc_full + 2;                    // [2]
     uint64_t* tail_full = acc_empty + 2;                   // [1] the block's last item is complete (for warps 8-15)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail_full + 1);
+    uint64_t* drain_bar = tail_full + 1;                   // [1] time-out path only: the MMAs issued so far have completed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile unsigned long long* t_entry = reinterpret_cast<volatile unsigned long long*>(tmem_slot + 2);
     uint32_t* tap_shift = tmem_slot + 4;                   // [taps] r * row_pitch + s of every tap, in staged pixels
     for (int t = tid; t < a.taps; t += kThreads) tap_shift[t] = (uint32_t)((t / a.s_slots) * a.row_pitch + (t % a.s_slots) * a.s_step);
-    if (tid == 0) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); *t_entry = t; }
+    if (kDiag && tid == 0) *t_entry = wall_ns();
 
     if (tid == 0) {
         for (int i = 0; i < a.a_stages; ++i) { mbar_init(&a_full[i], kProducers / a.pgroups); mbar_init(&a_empty[i], 1); }
         for (int i = 0; i < a.b_stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpilogueWarps); }
         mbar_init(tail_full, 1);
+        mbar_init(drain_bar, 1);
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -440,10 +456,7 @@ general_tc_kernel(const KernelArgs a)
             // free accumulator set, its total cycles, its item count
             long long wait_a = 0, wait_acc = 0, issue_cycles = 0;
             const long long t_begin = clock_now();
-            if (blockIdx.x == 0) {
-                unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-                a.status[6] = (unsigned)(t - *t_entry);          // ns from kernel entry to the start of the MMA loop
-            }
+            if (kDiag && blockIdx.x == 0) a.status[6] = (unsigned)(wall_ns() - *t_entry);   // ns from kernel entry to the start of the MMA loop
             int n_items = 0;
             if (a.resident) {
                 if (!mbar_wait_bounded(&b_full[0], 0u, abort_flag, a.max_polls)) alive = false;
@@ -538,14 +551,20 @@ general_tc_kernel(const KernelArgs a)
                 if (++buf == a.nbuf) buf = 0;
                 ++n_items;
             }
-            if (blockIdx.x == 0) {
+            if (!alive) {
+                // A wait ran out: MMAs issued before that may still be reading shared memory and writing tensor
+                // memory.  Let them finish (bounded) before the block frees its tensor memory and exits.
+                mma_commit(drain_bar);
+                uint32_t dummy = 0;
+                mbar_wait_bounded(drain_bar, 0u, &dummy, 1u << 16);
+            }
+            if (kDiag && blockIdx.x == 0) {
                 a.status[2] = (unsigned)wait_a;
                 a.status[3] = (unsigned)wait_acc;
                 a.status[4] = (unsigned)(clock_now() - t_begin);
                 a.status[5] = (unsigned)n_items;
                 a.status[9] = (unsigned)issue_cycles;
-                unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-                a.status[7] = (unsigned)(t - *t_entry);          // ns from kernel entry to the last MMA issued
+                a.status[7] = (unsigned)(wall_ns() - *t_entry);  // ns from kernel entry to the last MMA issued
             }
         }
     } else {
@@ -858,10 +877,7 @@ general_tc_kernel(const KernelArgs a)
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, a.tmem_cols);
     if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
-    if (tid == 0 && blockIdx.x == 0) {
-        unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        a.status[8] = (unsigned)(t - *t_entry);                  // ns from kernel entry to the block's end
-    }
+    if (kDiag && tid == 0 && blockIdx.x == 0) a.status[8] = (unsigned)(wall_ns() - *t_entry);   // ns from kernel entry to the block's end
 }
 
 }  // namespace

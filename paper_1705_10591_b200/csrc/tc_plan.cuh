@@ -196,7 +196,7 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
     };
     const long long tiles = (total_pix + kTileM - 1) / kTileM;
     const int chunk = kCB * p.n_tile * 4;
-    const int sms = 148;
+    const int sms = sm_count();
 
     const int forced_mt = env_int("CONV2D_B200_TF32_MT", 0);      // benchmark ablations only
     const size_t wbytes = (size_t)p.cblks * p.taps * chunk;        // re-ordered filters of one filter block
