@@ -134,7 +134,7 @@ def time_oracle_sample(cfg, target_seconds: float):
     oracle.conv2d_oracle_range(x, w, k_range=(1, 1 + maps))
     t = time.perf_counter() - t0
     return dict(value=flops_per_map * maps / t / 1e9, unit="GFLOP/s", cores=oracle.oracle_threads(),
-                kind="oracle", sample=f"{cfg.name}: all outputs of {maps} of {cfg.K} maps, {t:.1f} s, {cpu_model()}")
+                kind="oracle", sample=f"{cfg.name}: all outputs of {maps}/{cfg.K} maps, {t:.1f} s")
 
 
 def run_reference(args, rank: int):
@@ -176,22 +176,58 @@ def event_ms(fn, torch, iters=1):
     return start.elapsed_time(stop) / iters
 
 
-def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
-    """Times every general-case configuration, tensor-core and fp32 variants, cold and warm L2."""
-    out = []
+def sig(v, digits=4):
+    """Rounds a float to `digits` significant digits (the JSON line has to stay short)."""
+    if v is None or isinstance(v, (int, str, bool)):
+        return v
+    if v == 0 or v != v or v in (float("inf"), float("-inf")):
+        return v
+    from math import floor, log10
+    return round(v, digits - 1 - int(floor(log10(abs(v)))))
+
+
+def sustained_ms(fn, torch, sampler, seconds=1.0):
+    """Back-to-back calls for at least `seconds`: mean time per call, with the SM clock sampled during the loop."""
+    ms1 = max(event_ms(fn, torch, iters=5), 1e-3)
+    iters = int(max(20, seconds * 1e3 / ms1))
+    torch.cuda.synchronize()
+    n0 = len(sampler.samples)
+    sampler.begin()
+    ms = event_ms(fn, torch, iters=iters)
+    sampler.end()
+    clocks = sampler.samples[n0:]
+    mhz = statistics.median(clocks) if clocks else None
+    return ms, mhz, iters
+
+
+GENERAL_COLS = ["us_cold_full_call", "us_warm", "us_warm_prepacked", "frac_cold_full_call", "frac_warm_prepacked",
+                "frac_cold_of_nominal_peak", "us_sustained_1s", "sm_mhz_sustained", "frac_sustained_of_sustained_peak",
+                "mma_useful_px", "mma_useful_flops"]
+
+
+def bench_general(torch, lib, peaks, flush, sampler, detail):
+    """Times every general-case configuration: tensor cores on fp32 (TF32) and bf16 inputs, and the fp32 kernel.
+
+    Per (configuration, algorithm) one row of GENERAL_COLS: a complete call from cold L2 (filter re-ordering
+    included; `frac` is the roofline fraction of that), warm L2, warm L2 with the filters already re-ordered,
+    and a loop of at least one second of back-to-back complete calls with the SM clock sampled during it.
+    """
+    rows = {}
     dev = torch.device("cuda")
     stream = torch.cuda.current_stream().cuda_stream
+    fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
     for name in ["cfg3", "cfg4", "cfg5_r1", "cfg5_r3", "cfg5_r5", "cfg5_r7"]:
         cfg = CONFIGS[name]
         x, w = make_inputs(cfg)
         xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
         yd = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), device=dev, dtype=torch.float32)
         xd16 = wd16 = None
+        rows[name] = {}
         for algo_name, algo in (("tf32", lib.ALGO_TF32), ("bf16", lib.ALGO_16BIT), ("ffma", lib.ALGO_FFMA)):
             try:
                 ws_bytes = lib.conv2d_fwd_workspace_size(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, algo)
             except lib.Conv2dError:
-                out.append({"workload": name, "algo": algo_name, "unavailable": "no instance"})
+                rows[name][algo_name] = None
                 continue
             ws = torch.zeros(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
 
@@ -216,35 +252,62 @@ def bench_general(torch, lib, peaks, flush, sm_mhz_hint):
                 cold.append(event_ms(call, torch))
             warm = event_ms(call, torch, iters=20)
             packed = event_ms(lambda: call(lib.FLAG_WEIGHTS_PACKED), torch, iters=20) if tensor_core else None
+            sust, sust_mhz, sust_iters = sustained_ms(call, torch, sampler, 1.0 if algo_name != "ffma" else 0.3)
             lib.conv2d_get_status(ws.data_ptr(), stream)
-            t_cold, t_warm = statistics.median(cold), warm
+            t_cold = statistics.median(cold)
             nbytes = cfg.compulsory_bytes
             if algo == lib.ALGO_TF32:
-                pipe_peak = peaks["bf16_tflops"] / 2.0     # TF32 dense rate is half of bf16 per clock
-                bound = "tensor"
+                pipe_peak, pipe_sustained, pipe_nominal = peaks["bf16_tflops"] / 2.0, peaks["bf16_tflops_sustained"] / 2.0, NOMINAL_TF32_TFLOPS
             elif algo == lib.ALGO_16BIT:
-                pipe_peak = peaks["bf16_tflops"]
-                bound = "tensor"
+                pipe_peak, pipe_sustained, pipe_nominal = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"], NOMINAL_BF16_TFLOPS
                 nbytes = 2 * (x.size + w.size) + 4 * yd.numel()     # 2-byte operands, fp32 output
             else:
-                pipe_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
-                bound = "alu"
-            t_pipe = cfg.flops / (pipe_peak * 1e12) * 1e3
+                pipe_peak = pipe_sustained = pipe_nominal = fp32_peak
             t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9) * 1e3
-            entry = {
-                "workload": name, "algo": algo_name, "ms_cold_l2": t_cold, "ms_warm_l2": t_warm,
-                "gflops_cold": cfg.flops / t_cold / 1e6, "gflops_warm": cfg.flops / t_warm / 1e6,
-                "roofline": {"bound": bound if t_pipe >= t_hbm else "hbm",
-                             "pipe_peak_tflops": pipe_peak, "pipe_frac_warm": t_pipe / t_warm,
-                             "pipe_frac_cold": t_pipe / t_cold, "hbm_frac_cold": t_hbm / t_cold,
-                             "frac": max(t_pipe, t_hbm) / t_cold, "peaks": peaks["source"]},
-            }
-            if packed is not None:
-                entry["ms_warm_l2_weights_prepacked"] = packed
-                entry["roofline"]["pipe_frac_warm_weights_prepacked"] = t_pipe / packed
-            out.append(entry)
+            t_hbm_nominal = nbytes / 8000e9 * 1e3
+
+            def roof_ms(peak_tflops, hbm_ms=t_hbm):
+                return max(cfg.flops / (peak_tflops * 1e12) * 1e3, hbm_ms)
+            plan = {}
+            if tensor_core:
+                plan = lib.conv2d_fwd_plan_describe(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, algo)
+            bound = ("tensor" if tensor_core else "alu") if cfg.flops / (pipe_peak * 1e12) * 1e3 >= t_hbm else "hbm"
+            row = [t_cold * 1e3, warm * 1e3, packed * 1e3 if packed else None,
+                   roof_ms(pipe_peak) / t_cold, roof_ms(pipe_peak) / packed if packed else None,
+                   roof_ms(pipe_nominal, t_hbm_nominal) / t_cold, sust * 1e3, sust_mhz, roof_ms(pipe_sustained) / sust,
+                   plan.get("mma_useful_px"), plan.get("mma_useful_flops")]
+            rows[name][algo_name] = [sig(v) for v in row]
+            detail.append({"workload": name, "algo": algo_name, "bound": bound, "cold_us_all": [sig(c * 1e3) for c in cold],
+                           "sustained_iters": sust_iters, "pipe_peak_tflops": pipe_peak, "pipe_nominal_tflops": pipe_nominal,
+                           "pipe_sustained_tflops": pipe_sustained, "t_hbm_us": sig(t_hbm * 1e3), "plan": plan,
+                           "gflops_cold": sig(cfg.flops / t_cold / 1e6)})
         del xd, wd, yd, xd16, wd16
-    return out
+    return {"cols": GENERAL_COLS, "rows": rows,
+            "peaks": {"tf32": "bf16 burst/2", "bf16": "bf16 burst", "ffma": "148x128x2x1.965GHz", "hbm": peaks["hbm_gbs"],
+                      "nominal": "1125 tf32 / 2250 bf16 TFLOP/s, 8 TB/s", "sustained": "bf16_tflops_sustained (/2 for tf32)",
+                      "source": peaks["source"]}}
+
+
+def bench_cfg1(torch, lib):
+    """cfg1 (64 x 64 image, 8 filters of 3 x 3) is bound by launch latency: time of a single launch and of
+    back-to-back launches, in microseconds."""
+    cfg = CONFIGS["cfg1"]
+    dev = torch.device("cuda")
+    x, w = make_inputs(cfg)
+    xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
+    yd = torch.empty((cfg.N, cfg.K, cfg.P, cfg.Q), device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        lib.conv2d_fwd_single_channel(xd.data_ptr(), wd.data_ptr(), yd.data_ptr(), cfg.N, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S,
+                                      0, 0, 0, stream)
+    for _ in range(5):
+        call()
+    single = []
+    for _ in range(20):
+        torch.cuda.synchronize()
+        single.append(event_ms(call, torch))
+    return {"us_single_launch": sig(statistics.median(single) * 1e3), "us_back_to_back": sig(event_ms(call, torch, iters=200) * 1e3)}
 
 
 def reduce_max(value: float, device=None) -> float:
@@ -423,6 +486,9 @@ def main():
         "alu_tflops_achieved": cfg.flops / t_kernel_s / 1e12,
         "alu_frac_at_max_clock": cfg.flops / t_kernel_s / 1e12 / fp32_peak,
     })
+    if not (single or ffma):
+        nominal = NOMINAL_BF16_TFLOPS if b16 else NOMINAL_TF32_TFLOPS
+        roof["pipe_frac_of_nominal"] = cfg.flops / t_kernel_s / 1e12 / nominal
     traffic_file = ROOT / "profiles" / "traffic.json"
     if traffic_file.exists():
         roof["traffic"] = json.loads(traffic_file.read_text()).get(args.workload)
@@ -435,19 +501,42 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if b16 else ("f32" if (single or ffma) else "tf32"), "data": "synthetic",
         "config": {"workload": cfg.name, "operand": args.operand if not single else "fp32", **cfg.as_dict(), "parallelism": f"replicas x{world}",
-                   "l2": "flushed between timed steps" if flush_between else
-                         "inputs+outputs per step (2.2 GB) exceed the 126 MB L2"},
+                   "l2": "flushed between steps" if flush_between else "step moves 2.2 GB > 126 MB L2"},
         "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "power_w_max")},
         "e2e": e2e, "gpu_launches": int(launches), "roofline": roof,
     }
 
+    detail = []
     if rank == 0 and world == 1:
+        sampler2 = ClockSampler(local_rank)
+        sampler2.start()
+        # a sustained leg of the headline workload: at least one second of back-to-back steps
+        sust, sust_mhz, sust_iters = sustained_ms(step, torch, sampler2, 1.0)
+        fp32_at = (lambda mhz: SM_COUNT * FP32_LANES_PER_SM * 2 * mhz * 1e6 / 1e12)
+        result["sustained"] = {"ms_per_step": sust, "steps": sust_iters, "sm_mhz": sust_mhz,
+                               "ms_x_mhz": sust * sust_mhz if sust_mhz else None,
+                               "value": cfg.flops / sust / 1e6}
+        if single or ffma:
+            result["sustained"]["alu_frac_at_sampled_clock"] = cfg.flops / (sust * 1e-3) / 1e12 / fp32_at(sust_mhz) if sust_mhz else None
+            result["sustained"]["hbm_frac_of_measured"] = algorithmic_bytes / (sust * 1e-3) / 1e9 / peaks["hbm_gbs"]
         if not args.no_general:
-            result["general"] = bench_general(torch, lib, peaks, flush, clocks.get("sm_mhz"))
+            result["cfg1"] = bench_cfg1(torch, lib)
+            result["general"] = bench_general(torch, lib, peaks, flush, sampler2, detail)
+        sampler2.stop()
         if not args.no_cpu_baseline:
             result["cpu_baseline"] = time_oracle_sample(cfg, 12.0)
     if rank == 0:
-        print(json.dumps(result))
+        def compact(o):
+            if isinstance(o, float):
+                return sig(o)
+            if isinstance(o, dict):
+                return {k: compact(v) for k, v in o.items()}
+            if isinstance(o, list):
+                return [compact(v) for v in o]
+            return o
+        if detail:
+            sys.stderr.write("general-case detail: " + json.dumps(detail) + "\n")
+        print(json.dumps(compact(result), separators=(",", ":")))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()

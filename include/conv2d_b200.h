@@ -85,6 +85,19 @@ conv2d_status_t conv2d_fwd_workspace_size(int N, int C, int H, int W, int K, int
                                           conv2d_algo_t algo, size_t* bytes);
 
 /*
+ * Plan query (host only, touches no device; no counterpart in the paper, whose tilings are fixed per filter
+ * size in its Table 1).  Writes into `text` one NUL-terminated line of space-separated key=value pairs that
+ * describe how the tensor-core path (algo = TF32, AUTO or 16BIT) would cut this shape into work items:
+ * addressing mode, rows of the M operand, pixels per item, item and grid counts, and which part of the
+ * tensor-core work ends up in stored outputs (mma_useful_px: stored pixels / accumulator columns computed;
+ * mma_useful_flops: 2*N*K*C*R*S*P*Q / flops of all MMAs issued).  "tensor_core=0" when no instance fits.
+ * Returns CONV2D_ERR_WORKSPACE when text_bytes is too small (512 is enough), CONV2D_ERR_UNSUPPORTED for
+ * algo = FFMA.
+ */
+conv2d_status_t conv2d_fwd_plan_describe(int N, int C, int H, int W, int K, int R, int S,
+                                         conv2d_algo_t algo, char* text, size_t text_bytes);
+
+/*
  * Special case, one input channel (Section 3, Algorithm 1).
  *   x [N][1][H][W], w [K][1][R][S], y [N][K][P][Q]; fp32 FMA arithmetic.
  * The filters are small in this case (Section 3.2) and are kept on chip for the

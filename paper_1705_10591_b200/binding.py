@@ -43,6 +43,8 @@ def load_library() -> ctypes.CDLL:
     vp, i, sz, u = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_uint
     lib.conv2d_fwd_workspace_size.argtypes = [i] * 7 + [i, ctypes.POINTER(sz)]
     lib.conv2d_fwd_workspace_size.restype = i
+    lib.conv2d_fwd_plan_describe.argtypes = [i] * 7 + [i, ctypes.c_char_p, sz]
+    lib.conv2d_fwd_plan_describe.restype = i
     lib.conv2d_fwd_single_channel.argtypes = [vp, vp, vp] + [i] * 6 + [vp, sz, u, vp]
     lib.conv2d_fwd_single_channel.restype = i
     lib.conv2d_fwd_general.argtypes = [vp, vp, vp] + [i] * 7 + [i, vp, sz, u, vp]
@@ -89,6 +91,23 @@ def conv2d_fwd_workspace_size(N, C, H, W, K, R, S, algo=ALGO_AUTO) -> int:
     _check(load_library().conv2d_fwd_workspace_size(N, C, H, W, K, R, S, algo, ctypes.byref(out)),
            "conv2d_fwd_workspace_size")
     return int(out.value)
+
+
+def conv2d_fwd_plan_describe(N, C, H, W, K, R, S, algo=ALGO_AUTO) -> dict:
+    """The library's description of its tensor-core plan for a shape, as a dict of its key=value pairs."""
+    buf = ctypes.create_string_buffer(1024)
+    _check(load_library().conv2d_fwd_plan_describe(N, C, H, W, K, R, S, algo, buf, len(buf)), "conv2d_fwd_plan_describe")
+    out = {}
+    for pair in buf.value.decode().split():
+        key, _, val = pair.partition("=")
+        try:
+            out[key] = int(val)
+        except ValueError:
+            try:
+                out[key] = float(val)
+            except ValueError:
+                out[key] = val
+    return out
 
 
 def conv2d_fwd_single_channel(x_ptr, w_ptr, y_ptr, N, H, W, K, R, S,

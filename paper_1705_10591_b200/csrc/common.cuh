@@ -80,6 +80,9 @@ size_t tf32_workspace_bytes(const Shape& sh);   // includes the status block
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
                                     void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream);
 
+// Text description of the tensor-core plan of a shape (snprintf semantics: returns the length it needs).
+int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text_bytes);
+
 // Same kernel with 16-bit operands (x, w hold bf16 or fp16 elements in the same NCHW / KCRS order), fp32 output.
 bool b16_supported(const Shape& sh);
 size_t b16_workspace_bytes(const Shape& sh);

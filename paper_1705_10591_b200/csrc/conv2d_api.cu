@@ -143,6 +143,19 @@ conv2d_status_t conv2d_fwd_workspace_size(int N, int C, int H, int W, int K, int
     }
 }
 
+conv2d_status_t conv2d_fwd_plan_describe(int N, int C, int H, int W, int K, int R, int S,
+                                         conv2d_algo_t algo, char* text, size_t text_bytes)
+{
+    if (!text || text_bytes == 0) return CONV2D_ERR_NULL;
+    text[0] = 0;
+    Shape sh;
+    conv2d_status_t st = make_shape(N, C, H, W, K, R, S, &sh);
+    if (st != CONV2D_OK) return st;
+    if (algo != CONV2D_ALGO_TF32 && algo != CONV2D_ALGO_AUTO && algo != CONV2D_ALGO_16BIT) return CONV2D_ERR_UNSUPPORTED;
+    const int need = describe_tensor_core_plan(sh, algo == CONV2D_ALGO_16BIT, text, text_bytes);
+    return (need < 0 || (size_t)need >= text_bytes) ? CONV2D_ERR_WORKSPACE : CONV2D_OK;
+}
+
 conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float* y,
                                           int N, int H, int W, int K, int R, int S,
                                           void* workspace, size_t workspace_bytes,

@@ -82,6 +82,31 @@ size_t b16_workspace_bytes(const Shape& sh)
     return kStatusBytes + packed_floats(p) * sizeof(float);
 }
 
+// One line of text about the plan for `sh`: which addressing, item size, grid, and how much of the tensor-core work
+// is useful.  mma_useful_px = stored output pixels / accumulator columns computed (the flat run and the patches also
+// compute windows that wrap over an image edge); mma_useful_flops = 2*N*K*C*R*S*P*Q / flops of all MMAs issued
+// (this also counts filter rows, channels and stacked taps that are zero padding).
+int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text_bytes)
+{
+    const Plan p = make_plan(sh, b16);
+    if (!p.ok) return snprintf(text, text_bytes, "tensor_core=0");
+    const double out_px = (double)sh.N * sh.P * sh.Q;
+    const double cols = (double)p.supertiles * p.tile_px;
+    const double rows = p.swap ? p.n_tile : kTileM;                     // rows of the M operand
+    const double ncols = p.swap ? (double)p.supertiles * p.tile_px * p.n_blocks
+                                : (double)p.supertiles * p.mt * p.n_blocks * p.n_tile;
+    const double kdim = (double)p.cblks * (b16 ? 2 * kCB : kCB) * p.taps;
+    const double issued = 2.0 * rows * ncols * kdim * (p.swap ? 1.0 : 1.0);
+    const double useful = 2.0 * out_px * sh.K * sh.C * sh.R * sh.S;
+    return snprintf(text, text_bytes,
+                    "tensor_core=1 addressing=%s filters_as=%s m_rows=%d tile_px=%d px_groups=%d acc_sets=%d items=%lld grid=%d "
+                    "ksplit=%d resident_filters=%d stacked_taps=%d fold=%dx%d patch_w=%d smem_bytes=%zu "
+                    "mma_useful_px=%.4f mma_useful_flops=%.4f",
+                    p.patch_w ? "patch" : "flat", p.swap ? "M" : "N", (int)rows, p.tile_px, p.px_groups, p.nbuf,
+                    (long long)p.supertiles * p.n_blocks * p.ksplit, p.grid, p.ksplit, p.resident, p.pair_taps,
+                    p.fold_r, p.fold_s, p.patch_w, p.smem_bytes, out_px / cols, useful / issued);
+}
+
 namespace {
 // Launch with programmatic stream serialization: the kernel may be scheduled while the preceding kernel on the
 // stream drains; it calls grid_dep_wait() before it touches global memory.

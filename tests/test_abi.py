@@ -74,6 +74,25 @@ def test_argument_errors_come_before_any_device_work(lib):
     with pytest.raises(lib.Conv2dError) as e:      # unknown algorithm
         lib.conv2d_fwd_general(ok, ok, ok, 1, 3, 8, 8, 2, 3, 3, 7, 0, 0, 0, 0)
     assert e.value.status == 5
+    # The padded and strided entries launch a rewriting kernel of their own before the general entry: whatever
+    # that entry would reject (misaligned w or y, unknown flag, an algorithm it does not take, too many planes)
+    # must be rejected before that kernel.  The launch counter shows that nothing was enqueued.
+    big = 1 << 30
+    before = lib.conv2d_launch_count()
+    padded = [(dict(w=ok + 4), 3), (dict(y=ok + 8), 3), (dict(flags=2), 5), (dict(algo=lib.ALGO_16BIT), 5),
+              (dict(algo=7), 5), (dict(N=700, C=100), 5)]
+    for override, status in padded:
+        a = dict(x=ok, w=ok, y=ok, N=1, C=3, algo=lib.ALGO_FFMA, flags=0)
+        a.update(override)
+        with pytest.raises(lib.Conv2dError) as e:
+            lib.conv2d_fwd_general_padded(a["x"], a["w"], a["y"], a["N"], a["C"], 8, 8, 2, 3, 3, 1, 1, a["algo"],
+                                          ok, big, a["flags"], 0)
+        assert e.value.status == status, ("padded", override, e.value.status)
+        with pytest.raises(lib.Conv2dError) as e:
+            lib.conv2d_fwd_general_strided(a["x"], a["w"], a["y"], a["N"], a["C"], 8, 8, 2, 3, 3, 1, 1, 2, a["algo"],
+                                           ok, big, a["flags"], 0)
+        assert e.value.status == status, ("strided", override, e.value.status)
+    assert lib.conv2d_launch_count() == before
 
 
 def test_no_silent_fallback_without_a_gpu(lib):

@@ -65,16 +65,10 @@ def test_16bit_within_tolerance(oracle, dims, kind):
     print(f"{kind} {dims} max ratio {r:.3e}")
 
 
-def _sampled_planes(cfg, count, seed):
-    n = (uniform((count,), seed, 0, 1) * cfg.N).astype(np.int64)
-    k = (uniform((count,), seed + 1, 0, 1) * cfg.K).astype(np.int64)
-    return sorted({(0, 0), (cfg.N - 1, cfg.K - 1)} | set(zip(n.tolist(), k.tolist())))
-
-
 @pytest.mark.parametrize("name", ["cfg3", "cfg4", "cfg5_r1", "cfg5_r3", "cfg5_r5", "cfg5_r7"])
 @pytest.mark.parametrize("kind", TYPES)
 def test_16bit_full_size_configs(oracle, name, kind):
-    """Benchmark shapes at full size with the inputs rounded to the 16-bit type; sampled (image, map) planes are checked."""
+    """Benchmark shapes at full size with the inputs rounded to the 16-bit type; every output element is checked."""
     cfg = CONFIGS[name]
     dims = (cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S)
     if not _available(dims):
@@ -82,12 +76,9 @@ def test_16bit_full_size_configs(oracle, name, kind):
     x, w = make_inputs(cfg)
     x, w = ROUND[kind](x)[0], ROUND[kind](w)[0]
     y = run_library(x, w, entry=kind)
-    worst = 0.0
-    for n, k in _sampled_planes(cfg, 32, 600 + cfg.seed):
-        y_ref, yabs = oracle.conv2d_oracle_range(x, w, n_range=(n, n + 1), k_range=(k, k + 1))
-        worst = max(worst, assert_parity(y[n:n + 1, k:k + 1], y_ref, yabs, B16_TOL, f"{name} plane {(n, k)}"))
-    assert np.isfinite(y).all()
-    print(f"{name} {kind} max ratio {worst:.3e}")
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    worst = assert_parity(y, y_ref, yabs, B16_TOL, f"{name} {kind}")
+    print(f"{name} {kind} max ratio over all {y.size} outputs {worst:.3e}")
 
 
 def test_16bit_prepacked_filters_flag(oracle):

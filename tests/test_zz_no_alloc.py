@@ -6,7 +6,8 @@ a real-time loop that must stay away from the allocator.  For them the library k
 of the tensor-core path in a fixed device array of its own.  This test calls that entry point
 through the C ABI twice in a row, with different shapes and filters so that whatever the first call
 left in the shared array would corrupt the second if it were reused, and checks each result
-against the regular entry point (conv2d_fwd_general with a caller-provided workspace).
+against the oracle (tensor-core tolerance) and against the regular entry point (conv2d_fwd_general
+with a caller-provided workspace), with which it must agree bit for bit: same kernels, same plan.
 
 Collected last on purpose (file name), so a run that stops at the first failure has already
 run every other test; it does not depend on any other test having run.
@@ -14,7 +15,7 @@ run every other test; it does not depend on any other test having run.
 import numpy as np
 import pytest
 
-from helpers import TF32_TOL
+from helpers import TF32_TOL, assert_parity
 from workloads import uniform
 
 ALGO_TF32 = 2
@@ -53,10 +54,38 @@ def test_noalloc_entry_matches_workspace_entry_on_two_calls_in_a_row(oracle):
         x, w = uniform((N, C, H, W), 900 + call), uniform((K, C, R, S), 910 + call)
         y_new = _device_run(True, x, w)
         y_old = _device_run(False, x, w)
-        _, yabs = oracle.conv2d_oracle(x, w)
-        assert np.isfinite(y_new).all()
-        excess = np.abs(y_new.astype(np.float64) - y_old.astype(np.float64)) - TF32_TOL * yabs
-        assert excess.max() <= 0.0, f"call {call}: differs from the workspace entry point by more than the tolerance"
+        y_ref, yabs = oracle.conv2d_oracle(x, w)
+        assert_parity(y_new, y_ref, yabs, TF32_TOL, f"call {call}: entry without caller scratch vs the oracle")
+        np.testing.assert_array_equal(y_new, y_old, err_msg=f"call {call}: differs from the workspace entry point")
+
+
+@pytest.mark.gpu
+def test_noalloc_entry_timeout_is_visible_after_an_asynchronous_call(oracle, monkeypatch):
+    """wait = 0 returns before the kernels have run, so an expired on-device wait cannot come back from the call
+    itself: conv2d_get_status(NULL, stream) reports it, and the next call of the entry clears it.  The fault is
+    injected on the host (one filter copy armed but never issued, short wait bound); nothing hangs or traps."""
+    import torch
+    import paper_1705_10591_b200 as lib
+
+    N, C, H, W, K, R, S = 2, 64, 16, 16, 128, 3, 3
+    x, w = uniform((N, C, H, W), 920), uniform((K, C, R, S), 921)
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.current_stream().cuda_stream
+    xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
+    y = torch.zeros((N, K, H - R + 1, W - S + 1), device=dev)
+    monkeypatch.setenv("CONV2D_B200_TF32_MAX_POLLS", "2048")
+    monkeypatch.setenv("CONV2D_B200_TF32_TEST_DROP_STAGE", "1")
+    lib.conv2d_fwd_general_noalloc(xd.data_ptr(), wd.data_ptr(), y.data_ptr(), N, C, H, W, K, R, S, 0, stream)
+    with pytest.raises(lib.Conv2dError) as e:
+        lib.conv2d_get_status(0, stream)
+    assert e.value.status == 8                       # CONV2D_ERR_DEVICE_TIMEOUT
+    torch.cuda.synchronize()                         # the context is intact
+    monkeypatch.delenv("CONV2D_B200_TF32_MAX_POLLS")
+    monkeypatch.delenv("CONV2D_B200_TF32_TEST_DROP_STAGE")
+    y_new = _device_run(True, x, w)                  # wait = 1: would raise on a time-out; clears the status word
+    lib.conv2d_get_status(0, stream)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(y_new, y_ref, yabs, TF32_TOL, "after a time-out")
 
 
 @pytest.mark.gpu
