@@ -12,7 +12,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libconv2d_b200.so"
-SOURCES = ["conv2d_api.cu", "single_channel.cu", "general_ffma.cu", "general_tf32.cu"]
+SOURCES = ["conv2d_api.cu", "single_channel.cu", "general_ffma.cu", "general_tf32.cu", "pointwise_tma.cu"]
 
 
 def _stale() -> bool:

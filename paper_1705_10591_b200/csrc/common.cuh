@@ -68,6 +68,24 @@ inline int env_int(const char* name, int dflt)
     return (v && *v) ? atoi(v) : dflt;
 }
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while the preceding kernel on the
+// stream drains; it calls grid_dep_wait() before it touches global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = env_int("CONV2D_B200_TF32_PDL", 1) != 0 ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Launchers.  Each returns CONV2D_OK, CONV2D_ERR_UNSUPPORTED (no instance) or CONV2D_ERR_CUDA.
 conv2d_status_t launch_single_channel(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);
 conv2d_status_t launch_general_ffma(const float* x, const float* w, float* y, const Shape& sh, cudaStream_t stream);
@@ -79,6 +97,13 @@ size_t tf32_workspace_bytes(const Shape& sh);   // includes the status block
 // (returns CONV2D_ERR_UNSUPPORTED without an instance, CONV2D_ERR_WORKSPACE when workspace_bytes is too small)
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
                                     void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream);
+
+// 1 x 1 filters with every operand moved by tensor-map (TMA) copies; `workspace` only holds the status block.
+// CONV2D_ERR_UNSUPPORTED when the shape or its alignment has no such instance (the caller then takes the general kernel).
+bool pointwise_tma_supported(const Shape& sh);
+conv2d_status_t launch_pointwise_tma(const float* x, const float* w, float* y, const Shape& sh,
+                                     void* workspace, size_t workspace_bytes, cudaStream_t stream);
+int describe_pointwise_tma_plan(const Shape& sh, char* text, size_t text_bytes);   // -1: no such instance
 
 // Text description of the tensor-core plan of a shape (snprintf semantics: returns the length it needs).
 int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text_bytes);

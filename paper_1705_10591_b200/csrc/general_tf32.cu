@@ -60,7 +60,7 @@ namespace conv2d_b200 {
 
 bool tf32_supported(const Shape& sh)
 {
-    return make_plan(sh).ok;
+    return make_plan(sh).ok || pointwise_tma_supported(sh);
 }
 
 size_t tf32_workspace_bytes(const Shape& sh)
@@ -88,6 +88,10 @@ size_t b16_workspace_bytes(const Shape& sh)
 // (this also counts filter rows, channels and stacked taps that are zero padding).
 int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text_bytes)
 {
+    if (!b16) {
+        const int n = describe_pointwise_tma_plan(sh, text, text_bytes);
+        if (n >= 0) return n;
+    }
     const Plan p = make_plan(sh, b16);
     if (!p.ok) return snprintf(text, text_bytes, "tensor_core=0");
     const double out_px = (double)sh.N * sh.P * sh.Q;
@@ -99,7 +103,7 @@ int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text
     const double issued = 2.0 * rows * ncols * kdim * (p.swap ? 1.0 : 1.0);
     const double useful = 2.0 * out_px * sh.K * sh.C * sh.R * sh.S;
     return snprintf(text, text_bytes,
-                    "tensor_core=1 addressing=%s filters_as=%s m_rows=%d tile_px=%d px_groups=%d acc_sets=%d items=%lld grid=%d "
+                    "tensor_core=1 kernel=general_tc addressing=%s filters_as=%s m_rows=%d tile_px=%d px_groups=%d acc_sets=%d items=%lld grid=%d "
                     "ksplit=%d resident_filters=%d stacked_taps=%d fold=%dx%d patch_w=%d smem_bytes=%zu "
                     "mma_useful_px=%.4f mma_useful_flops=%.4f",
                     p.patch_w ? "patch" : "flat", p.swap ? "M" : "N", (int)rows, p.tile_px, p.px_groups, p.nbuf,
@@ -108,24 +112,6 @@ int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text
 }
 
 namespace {
-// Launch with programmatic stream serialization: the kernel may be scheduled while the preceding kernel on the
-// stream drains; it calls grid_dep_wait() before it touches global memory.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)
-{
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = env_int("CONV2D_B200_TF32_PDL", 1) != 0 ? 1 : 0;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
 // workspace_bytes: checked against the plan's need here, so that a call plans only once (the planner reads two
 // dozen environment switches and costs ~2 us); SIZE_MAX = the caller has checked already.
 conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* y, const Shape& sh, bool b16, bool fp16,
@@ -133,6 +119,11 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
 {
     const float* x = static_cast<const float*>(x_any);   // 16-bit operands: re-read as such inside the kernel
     const float* w = static_cast<const float*>(w_any);
+    if (!b16) {
+        // 1 x 1 filters on suitably aligned tensors: the kernel whose operands and output all move by tensor-map copies
+        const conv2d_status_t st = launch_pointwise_tma(x, w, y, sh, workspace, workspace_bytes, stream);
+        if (st != CONV2D_ERR_UNSUPPORTED) return st;
+    }
     const Plan p = make_plan(sh, b16);
     if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
     if (env_int("CONV2D_B200_TF32_VERBOSE", 0) != 0)

@@ -1,0 +1,430 @@
+// General case with 1 x 1 filters on the tcgen05 tensor cores, every operand and the output moved by tiled TMA
+// copies (the staging and the prefetch of Algorithm 2, lines 4-5 and 8-9, done by the copy engine; its write-back,
+// line 20, as well).
+//
+// With one tap per filter the convolution of image n is the matrix product
+//     Y[n] (K x HW) = Wmat (K x C) * X[n] (C x HW),
+// and both operands already lie in memory the way the tensor core can read them, so nothing has to be turned
+// around by threads:
+//   * Filters, the M operand: w[k][c] has the channels contiguous = K-major.  A tensor-map copy with a 32-channel
+//     (128-byte) inner box and 128-byte swizzle writes exactly the 8-row x 128-byte atoms the MMA reads; the whole
+//     bank of a filter block (up to 128 filters x 256 channels) stays in shared memory for the life of the block
+//     (Section 3.2: the filters are small, keep them on chip).
+//   * Pixels, the N operand: NCHW has the pixels of a channel contiguous = MN-major, which kind::tf32 accepts in one
+//     layout only: 128-byte rows (32 pixels of one channel) whose 32-byte chunks are swizzled over groups of 4
+//     channel rows, as a tensor-map copy with SWIZZLE_128B_ATOM_32B writes them.  One box of 32 pixels x 32 channels
+//     serves four K steps of 8 channels; an MMA covers up to 8 such boxes (N <= 256) that lie 32 * 128 bytes apart.
+//     A stage of the mbarrier ring holds 32 channels of all pixels of a work item.
+//   * Output: accumulators (lanes = filters, columns = pixels) go tensor memory -> registers -> a swizzled
+//     32-filter x 32-pixel shared-memory tile per warp -> one tensor-map store per tile.  Out-of-range rows and
+//     pixels are clipped by the copy engine, so ragged images and filter counts need no predicates.
+// The tensor core reads fp32 bits as TF32 by dropping the low 13 mantissa bits, so on this path both operands are
+// truncated, not rounded: |error| <= (2^-10 + 2^-10 + 2^-20) * sum|x*w| plus fp32 accumulation over at most 256
+// channels, (C + 1) * 2^-24 * sum|x*w|: below 1.97e-3 * sum|x*w|, inside the 2e-3 bound of CONV2D_ALGO_TF32.
+//
+// Persistent blocks, one per SM: warp 0 (one thread) issues the loads, warp 1 (one thread) the MMAs, warps 2-9
+// drain the accumulators, two per tensor-memory lane quarter.  Two accumulator sets: the write-back of item i runs
+// under the loads and MMAs of item i + 1, which is what an operation bound by memory traffic needs.
+// Work items are runs of `a_item` 32-pixel atoms of the flat atom sequence (image-major; an image has
+// ceil(HW / 32) atoms, the last one may be ragged and is zero-filled on load and clipped on store).
+// Every wait is bounded; on expiry the block stops, frees its tensor memory and raises the status word.
+#include <cstdio>
+#include <cuda.h>
+
+#include "common.cuh"
+#include "fastdiv.cuh"
+#include "ptx.cuh"
+
+namespace conv2d_b200 {
+namespace {
+
+using namespace ptx;
+
+constexpr int kPwThreads = 320;           // warp 0: loads, warp 1: MMAs, warps 2-9: write-back
+constexpr int kPwEpiWarps = 8;
+constexpr int kAtomPx = 32;               // pixels per 128-byte row of a swizzle atom
+constexpr int kStageCh = 32;              // channels per activation stage: four K steps of 8
+constexpr int kAtomBytes = kAtomPx * kStageCh * 4;     // one box of 32 pixels x 32 channels
+constexpr int kMaxAtoms = 8;              // atoms per work item: N <= 256 columns per MMA
+constexpr int kPwMaxStages = 8;
+constexpr int kAccCols = 256;             // tensor-memory columns of one accumulator set
+constexpr int kMaxChannels = 256;         // the filter bank of a block must stay resident
+constexpr size_t kPwSmemLimit = 227 * 1024;
+constexpr size_t kPwBookBytes = 256;      // barriers, tensor-memory slot, abort flag
+
+struct PwArgs {
+    unsigned* status;
+    int K;
+    int apb;             // atoms per image: ceil(HW / 32)
+    int total_atoms;     // N * apb
+    int a_item;          // atoms per work item
+    int tiles;           // work items along the pixels
+    int n_blocks;        // filter blocks of m_rows filters
+    int m_rows;          // rows of the M operand: 64 (at most 64 filters) or 128
+    int items;           // tiles * n_blocks, numbered filter block-major
+    int cchunks;         // 32-channel chunks: ceil(C / 32)
+    int ksteps;          // K steps of 8 channels: ceil(C / 8)
+    int stages;          // activation ring depth
+    unsigned max_polls;  // bound of every barrier wait
+    int test_drop_stage; // test hook: the activation stage with this ordinal is armed but never copied (-1: none)
+    FastDiv div_apb, div_tiles;
+};
+
+__global__ void __launch_bounds__(kPwThreads, 1)
+pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+                     const __grid_constant__ CUtensorMap map_y, const PwArgs a)
+{
+    extern __shared__ unsigned char smem_raw[];
+    // swizzle atoms must start on 1024 bytes
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const uint32_t a_chunk_bytes = (uint32_t)a.m_rows * 128u;                 // filters x 32 channels
+    const uint32_t b_stage_bytes = (uint32_t)a.a_item * kAtomBytes;
+    unsigned char* a_smem = smem;
+    unsigned char* b_smem = a_smem + (size_t)a.cchunks * a_chunk_bytes;
+    unsigned char* o_smem = b_smem + (size_t)a.stages * b_stage_bytes;      // [kPwEpiWarps][32 rows x 128 bytes]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(o_smem + (size_t)kPwEpiWarps * 4096);
+    uint64_t* a_full = bars;                       // [1] the filter bank of the current block has landed
+    uint64_t* a_empty = a_full + 1;                // [1] all MMAs that read it have completed
+    uint64_t* b_full = a_empty + 1;                // [kPwMaxStages]
+    uint64_t* b_empty = b_full + kPwMaxStages;     // [kPwMaxStages]
+    uint64_t* acc_full = b_empty + kPwMaxStages;   // [2]
+    uint64_t* acc_empty = acc_full + 2;            // [2]
+    uint64_t* drain_bar = acc_empty + 2;           // [1] time-out path: the MMAs issued so far have completed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        prefetch_tensormap(&map_w);
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_y);
+        mbar_init(a_full, 1);
+        mbar_init(a_empty, 1);
+        for (int i = 0; i < a.stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kPwEpiWarps); }
+        mbar_init(drain_bar, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (warp == 1) { tmem_alloc(tmem_slot, 2 * kAccCols); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    // Everything above touched only this block's shared and tensor memory and may overlap the tail of the
+    // preceding kernel on the stream; global memory is read and written from here on.
+    grid_dep_launch();
+    grid_dep_wait();
+    if (blockIdx.x == 0 && tid == 0) *a.status = 0u;       // (a block that gives up raises it at its very end)
+
+    // item -> (filter block, first atom, atoms): filter block-major, so that a block rarely changes its bank
+    auto decode = [&](int item, int& nb, int& first, int& atoms) {
+        int tile;
+        nb = a.div_tiles.divmod(item, tile);
+        first = tile * a.a_item;
+        atoms = min(a.a_item, a.total_atoms - first);
+    };
+
+    if (warp == 0) {
+        // ---------------- loads (one thread)
+        if (lane == 0) {
+            int cur_nb = -1, slot = 0, issued = 0;
+            uint32_t ph = 0, a_loads = 0;
+            bool alive = true;
+            for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
+                int nb, first, atoms;
+                decode(item, nb, first, atoms);
+                if (nb != cur_nb) {
+                    // the bank of another filter block: wait until the MMAs on the old one are done
+                    if (a_loads && !mbar_wait_bounded(a_empty, (a_loads - 1u) & 1u, abort_flag, a.max_polls)) { alive = false; break; }
+                    mbar_arrive_expect_tx(a_full, a_chunk_bytes * (uint32_t)a.cchunks);
+                    for (int cb = 0; cb < a.cchunks; ++cb)
+                        tma_load_2d(a_smem + (size_t)cb * a_chunk_bytes, &map_w, cb * kStageCh, nb * a.m_rows, a_full);
+                    cur_nb = nb;
+                    ++a_loads;
+                }
+                for (int st = 0; st < a.cchunks; ++st) {
+                    if (!mbar_wait_bounded(&b_empty[slot], ph ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
+                    mbar_arrive_expect_tx(&b_full[slot], (uint32_t)atoms * kAtomBytes);
+                    if (issued != a.test_drop_stage) {
+                        unsigned char* dst = b_smem + (size_t)slot * b_stage_bytes;
+                        int blk;
+                        int n = a.div_apb.divmod(first, blk);
+                        for (int i = 0; i < atoms; ++i, dst += kAtomBytes) {
+                            tma_load_3d(dst, &map_x, blk * kAtomPx, st * kStageCh, n, &b_full[slot]);
+                            if (++blk == a.apb) { blk = 0; ++n; }
+                        }
+                    }
+                    ++issued;
+                    if (++slot == a.stages) { slot = 0; ph ^= 1u; }
+                }
+            }
+            if (*abort_flag) {
+                // let copies already in flight land before the block's shared memory is released
+                uint32_t dummy = 0;
+                if (a_loads) mbar_wait_bounded(a_full, (a_loads - 1u) & 1u, &dummy, 1u << 14);
+                const int pending = issued < a.stages ? issued : a.stages;
+                for (int i = 0; i < pending; ++i) {
+                    const int it = issued - 1 - i;
+                    mbar_wait_bounded(&b_full[it % a.stages], (uint32_t)(it / a.stages) & 1u, &dummy, 1u << 14);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issue (one thread)
+        if (lane == 0) {
+            const uint32_t a_base = smem_u32(a_smem), b_base = smem_u32(b_smem);
+            int cur_nb = -1, slot = 0, buf = 0;
+            uint32_t ph = 0, a_waits = 0, acc_phase[2] = {0u, 0u};
+            bool alive = true;
+            for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
+                int nb, first, atoms;
+                decode(item, nb, first, atoms);
+                if (nb != cur_nb) {
+                    if (!mbar_wait_bounded(a_full, a_waits & 1u, abort_flag, a.max_polls)) { alive = false; break; }
+                    ++a_waits;
+                    cur_nb = nb;
+                }
+                if (!mbar_wait_bounded(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
+                tc_fence_after_sync();
+                const uint32_t idesc = idesc_tf32((uint32_t)a.m_rows, (uint32_t)(atoms * kAtomPx)) | kIdescBMajorMN;
+                const uint32_t d = tmem + (uint32_t)(buf * kAccCols);
+                bool accumulate = false;
+                for (int st = 0; st < a.cchunks && alive; ++st) {
+                    if (!mbar_wait_bounded(&b_full[slot], ph, abort_flag, a.max_polls)) { alive = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_chunk = a_base + (uint32_t)st * a_chunk_bytes;
+                    const uint32_t b_stage = b_base + (uint32_t)slot * b_stage_bytes;
+                    const int ks = min(kStageCh / 8, a.ksteps - st * (kStageCh / 8));
+                    for (int kk = 0; kk < ks; ++kk) {
+                        // filters: 32 bytes further inside the 128-byte rows; pixels: the next atom of 8 channel rows
+                        mma_tf32(d, smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u),
+                                 smem_desc_mn_sw128_32b(b_stage + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u), idesc, accumulate);
+                        accumulate = true;
+                    }
+                    mma_commit(&b_empty[slot]);
+                    if (++slot == a.stages) { slot = 0; ph ^= 1u; }
+                }
+                if (!alive) break;
+                mma_commit(&acc_full[buf]);
+                // the next item of this block uses another filter block: tell the loader when this bank is free
+                const int next = item + (int)gridDim.x;
+                if (next < a.items && a.div_tiles.div(next) != nb) mma_commit(a_empty);
+                acc_phase[buf] ^= 1u;
+                buf ^= 1;
+            }
+            if (!alive) {
+                mma_commit(drain_bar);
+                uint32_t dummy = 0;
+                mbar_wait_bounded(drain_bar, 0u, &dummy, 1u << 16);
+            }
+        }
+    } else {
+        // ---------------- write-back: tensor memory -> registers -> swizzled tile -> tensor-map store
+        const int ew = warp - 2;
+        const int quarter = warp & 3;                       // tensor-memory lanes this warp may read
+        const int half = ew >> 2;                           // the two warps of a quarter take alternate atoms
+        unsigned char* tile = o_smem + (size_t)ew * 4096;
+        const int rows_q = a.m_rows / 4;                    // filters per lane quarter: 32, or 16 (M = 64: lanes 0-15)
+        bool alive = true;
+        int li = 0;
+        for (int item = blockIdx.x; item < a.items; item += gridDim.x, ++li) {
+            int nb, first, atoms;
+            decode(item, nb, first, atoms);
+            const int buf = li & 1;
+            const uint32_t acc_phase = (uint32_t)(li >> 1) & 1u;
+            alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag, a.max_polls));
+            if (!alive) break;
+            tc_fence_after_sync();
+            const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccCols);
+            const int k0 = nb * a.m_rows + quarter * rows_q;
+            for (int i = half; i < atoms; i += 2) {
+                uint32_t v[32];
+                tmem_ld32(lane_base + (uint32_t)(i * kAtomPx), v);
+                tmem_ld_wait();
+                if (lane == 0) bulk_wait_group_read<0>();       // the previous store has read the tile
+                __syncwarp();
+                if (lane < rows_q) {
+                    // row = this lane's filter, 32 pixels = eight 16-byte chunks, chunk c stored at c ^ (row & 7)
+                    unsigned char* row = tile + lane * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4*>(row + ((c ^ (lane & 7)) << 4)) = make_uint4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && k0 < a.K) {
+                    int blk;
+                    const int n = a.div_apb.divmod(first + i, blk);
+                    tma_store_3d(&map_y, blk * kAtomPx, k0, n, tile);
+                    bulk_commit_group();
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+        if (lane == 0) bulk_wait_group<0>();                 // this thread's stores are complete
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 2 * kAccCols);
+    if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
+}
+
+// ---------------------------------------------------------------- host side
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime so that the library does not link against the
+// driver (it must load on machines without one).
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// fp32 tensor of `rank` dimensions (innermost first), zeros for out-of-range elements.  `swizzle`: 128-byte rows
+// with 16-byte chunks swizzled (K-major operands, output tiles) or with 32-byte chunks (the MN-major TF32 operand).
+bool encode_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+                const cuuint32_t* box, CUtensorMapSwizzle swizzle)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint32_t ones[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, ones,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct PwPlan {
+    bool ok;
+    int m_rows, n_blocks, apb, a_item, tiles, cchunks, stages, grid;
+    long long total_atoms;
+    size_t smem_bytes;
+};
+
+PwPlan make_pw_plan(const Shape& sh)
+{
+    PwPlan p{};
+    p.ok = false;
+    if (sh.R != 1 || sh.S != 1 || sh.pad_h || sh.pad_w) return p;
+    const long long HW = (long long)sh.H * sh.W;
+    // tensor-map strides are multiples of 16 bytes; the filter bank of a block stays in shared memory
+    if (HW % 4 != 0 || sh.C % 4 != 0 || sh.C > kMaxChannels) return p;
+    if (env_int("CONV2D_B200_TF32_TMA", 1) == 0) return p;
+    p.m_rows = sh.K <= 64 ? 64 : 128;
+    p.n_blocks = (sh.K + p.m_rows - 1) / p.m_rows;
+    p.apb = (int)((HW + kAtomPx - 1) / kAtomPx);
+    p.total_atoms = (long long)sh.N * p.apb;
+    if (p.total_atoms > 0x3fffffffLL) return p;
+    p.cchunks = (sh.C + kStageCh - 1) / kStageCh;
+    const int sms = sm_count();
+    // Atoms per item: the fewest rounds of items over the SMs, counted in atoms, plus half an atom of fixed cost per
+    // item; ties go to the larger item (wider MMAs).  64 x 32 x 32 pixels = 2048 atoms: 7 per item = 293 items = two
+    // rounds of 7, where 8 per item would be two rounds of 8.
+    double best = 0;
+    p.a_item = 0;
+    const int forced = env_int("CONV2D_B200_TMA_ATOMS", 0);
+    for (int at = kMaxAtoms; at >= 1; --at) {
+        if (forced ? at != forced : false) continue;
+        const long long tiles = (p.total_atoms + at - 1) / at;
+        const long long rounds = (tiles * p.n_blocks + sms - 1) / sms;
+        const double cost = (double)rounds * (at + 0.5);
+        if (p.a_item == 0 || cost < best - 1e-9) { best = cost; p.a_item = at; }
+    }
+    if (p.a_item == 0) return p;
+    p.tiles = (int)((p.total_atoms + p.a_item - 1) / p.a_item);
+    const long long items = (long long)p.tiles * p.n_blocks;
+    if (items > 0x7fffffffLL) return p;
+    const size_t fixed = (size_t)p.cchunks * p.m_rows * 128 + (size_t)kPwEpiWarps * 4096 + kPwBookBytes + 1024;
+    const size_t stage = (size_t)p.a_item * kAtomBytes;
+    if (fixed + 2 * stage > kPwSmemLimit) return p;
+    p.stages = (int)((kPwSmemLimit - fixed) / stage);
+    if (p.stages > kPwMaxStages) p.stages = kPwMaxStages;
+    p.smem_bytes = fixed + (size_t)p.stages * stage;
+    // more than half of an SM's shared memory, so that two of these blocks, which both want all 512 tensor-memory
+    // columns, never share an SM
+    if (p.smem_bytes < 116 * 1024) p.smem_bytes = 116 * 1024;
+    p.grid = (int)(items < sms ? items : sms);
+    p.ok = true;
+    return p;
+}
+
+}  // namespace
+
+bool pointwise_tma_supported(const Shape& sh) { return make_pw_plan(sh).ok; }
+
+int describe_pointwise_tma_plan(const Shape& sh, char* text, size_t text_bytes)
+{
+    const PwPlan p = make_pw_plan(sh);
+    if (!p.ok) return -1;
+    const double px = (double)sh.N * sh.H * sh.W;
+    const double cols = (double)p.total_atoms * kAtomPx;
+    const double issued = 2.0 * p.m_rows * p.n_blocks * cols * ((sh.C + 7) / 8 * 8);
+    return snprintf(text, text_bytes,
+                    "tensor_core=1 kernel=pointwise_tma addressing=atoms filters_as=M m_rows=%d tile_px=%d acc_sets=2 items=%lld "
+                    "grid=%d stages=%d resident_filters=1 smem_bytes=%zu mma_useful_px=%.4f mma_useful_flops=%.4f",
+                    p.m_rows, p.a_item * kAtomPx, (long long)p.tiles * p.n_blocks, p.grid, p.stages, p.smem_bytes,
+                    px / cols, 2.0 * px * sh.K * sh.C / issued);
+}
+
+conv2d_status_t launch_pointwise_tma(const float* x, const float* w, float* y, const Shape& sh,
+                                     void* workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    const PwPlan p = make_pw_plan(sh);
+    if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < kStatusBytes) return CONV2D_ERR_WORKSPACE;
+    const cuuint64_t HW = (cuuint64_t)sh.H * sh.W;
+    CUtensorMap map_w, map_x, map_y;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)sh.C, (cuuint64_t)sh.K};
+        const cuuint64_t strides[1] = {(cuuint64_t)sh.C * 4};
+        const cuuint32_t box[2] = {(cuuint32_t)kStageCh, (cuuint32_t)p.m_rows};
+        if (!encode_map(&map_w, w, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return CONV2D_ERR_UNSUPPORTED;
+    }
+    {
+        const cuuint64_t dims[3] = {HW, (cuuint64_t)sh.C, (cuuint64_t)sh.N};
+        const cuuint64_t strides[2] = {HW * 4, HW * 4 * (cuuint64_t)sh.C};
+        const cuuint32_t box[3] = {(cuuint32_t)kAtomPx, (cuuint32_t)kStageCh, 1};
+        if (!encode_map(&map_x, x, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) return CONV2D_ERR_UNSUPPORTED;
+    }
+    {
+        const cuuint64_t dims[3] = {HW, (cuuint64_t)sh.K, (cuuint64_t)sh.N};
+        const cuuint64_t strides[2] = {HW * 4, HW * 4 * (cuuint64_t)sh.K};
+        const cuuint32_t box[3] = {(cuuint32_t)kAtomPx, (cuuint32_t)(p.m_rows / 4), 1};
+        if (!encode_map(&map_y, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return CONV2D_ERR_UNSUPPORTED;
+    }
+    static size_t smem_done[64] = {};
+    if (raise_smem_limit(reinterpret_cast<const void*>(pointwise_tma_kernel), p.smem_bytes, smem_done) != cudaSuccess)
+        return CONV2D_ERR_CUDA;
+    PwArgs a{};
+    a.status = static_cast<unsigned*>(workspace);
+    a.K = sh.K;
+    a.apb = p.apb; a.total_atoms = (int)p.total_atoms; a.a_item = p.a_item; a.tiles = p.tiles;
+    a.n_blocks = p.n_blocks; a.m_rows = p.m_rows; a.items = p.tiles * p.n_blocks;
+    a.cchunks = p.cchunks; a.ksteps = (sh.C + 7) / 8; a.stages = p.stages;
+    a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
+    a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
+    a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles);
+    if (env_int("CONV2D_B200_TF32_VERBOSE", 0) != 0)
+        fprintf(stderr, "conv2d plan: pointwise_tma m_rows %d n_blocks %d atoms/item %d tiles %d stages %d grid %d smem %zu\n",
+                p.m_rows, p.n_blocks, p.a_item, p.tiles, p.stages, p.grid, p.smem_bytes);
+    if (launch_pdl(pointwise_tma_kernel, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
+                   map_w, map_x, map_y, a) != cudaSuccess)
+        return CONV2D_ERR_CUDA;
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
+}  // namespace conv2d_b200

@@ -76,6 +76,38 @@ __device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gmem_src, u
                  ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// Tiled (tensor-map) TMA copies.  `map` points to a CUtensorMap in kernel-parameter (grid-constant) space.
+// Loads signal `bar` with the box's byte count (out-of-range elements are written as zeros and still counted);
+// the innermost coordinate times the element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* map, int c0, int c1, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const void* map, int c0, int c1, int c2, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
+}
+// Store of one box shared -> global (elements outside the tensor are dropped); completion is tracked per thread
+// in bulk groups.
+__device__ __forceinline__ void tma_store_3d(const void* map, int c0, int c1, int c2, const void* smem_src)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(smem_src)) : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all but the newest `N` groups of this thread have finished READING their shared-memory source
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+// all but the newest `N` groups of this thread are complete (their global writes are done)
+template <int N>
+__device__ __forceinline__ void bulk_wait_group() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void prefetch_tensormap(const void* map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
 // ---------------------------------------------------------------- tensor memory
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t columns)   // whole warp; columns: power of 2 >= 32
 {
@@ -124,6 +156,18 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
           "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
         : "r"(taddr) : "memory");
 }
+// 32 lanes x 32 consecutive columns
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t (&v)[1])
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v[0]) : "r"(taddr) : "memory");
@@ -143,6 +187,36 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor_noswizzle(uint32_t smem_add
          | ((uint64_t)((row_group_bytes >> 4) & 0x3FFFu) << 32)
          | (1ull << 46);                       // descriptor version of sm_100
 }
+// Shared-memory matrix descriptor for a 128-byte-swizzled operand, as a tiled TMA copy with SWIZZLE_128B and a
+// 128-byte inner box writes it: 1024-byte atoms of 8 rows x 128 bytes whose 16-byte chunks are XOR-ed with the row
+// number (atoms must start on 1024 bytes).
+//   K-major  (a row = one M/N index, 32 consecutive K elements of 4 bytes): `stride_bytes` = distance between
+//            groups of 8 rows; a K step of 8 elements advances the start address by 32 bytes inside the row.
+//   MN-major (a row = one K index, 32 consecutive M/N elements): `leading_bytes` = distance between atoms that are
+//            adjacent along M/N, `stride_bytes` = distance between groups of 8 K rows.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t leading_bytes, uint32_t stride_bytes)
+{
+    return (uint64_t)((smem_addr >> 4) & 0x3FFFu)
+         | ((uint64_t)((leading_bytes >> 4) & 0x3FFFu) << 16)
+         | ((uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32)
+         | (1ull << 46)                        // descriptor version of sm_100
+         | (2ull << 61);                       // layout type: 128-byte swizzle
+}
+// MN-major operand of 4-byte elements (TF32): the one layout the tensor core takes for it swizzles 32-byte chunks
+// inside 128-byte rows (chunk index XOR row number mod 4; tensor-map copies write it with SWIZZLE_128B_ATOM_32B).
+// Atom = 4 K rows x 128 bytes (32 consecutive M/N elements per row).  `leading_bytes` = distance between atoms
+// adjacent along M/N, `stride_bytes` = distance between groups of 4 K rows (an MMA of K = 8 reads two groups).
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128_32b(uint32_t smem_addr, uint32_t leading_bytes, uint32_t stride_bytes)
+{
+    return (uint64_t)((smem_addr >> 4) & 0x3FFFu)
+         | ((uint64_t)((leading_bytes >> 4) & 0x3FFFu) << 16)
+         | ((uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32)
+         | (1ull << 46)                        // descriptor version of sm_100
+         | (1ull << 61);                       // layout type: 128-byte swizzle with 32-byte atoms
+}
+// Bit of the instruction descriptor that declares the B operand MN-major (its M/N index contiguous in memory).
+constexpr uint32_t kIdescBMajorMN = 1u << 16;
+
 // Instruction descriptor: TF32 x TF32 -> fp32, both operands K-major, M x N tile.
 __host__ __device__ constexpr uint32_t idesc_tf32(uint32_t m, uint32_t n)
 {

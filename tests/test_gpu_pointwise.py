@@ -1,0 +1,107 @@
+"""1 x 1 filters on the tensor cores with every operand moved by tensor-map (TMA) copies, against the oracle.
+
+Shapes are chosen so that the library takes that kernel (the plan query says which one it is) and so that its
+edges are met: an image whose last 32-pixel atom is ragged, a channel count that is not a multiple of the
+32-channel stage or of the 8-channel MMA step, filter counts below and above one 128-filter block, the 64-row
+variant, more work items than SMs, items that straddle two images.
+"""
+import numpy as np
+import pytest
+
+from helpers import TF32_TOL, assert_parity, run_library
+from workloads import small_integers, uniform
+
+pytestmark = pytest.mark.gpu
+ALGO_TF32 = 2
+
+SHAPES = [
+    # N, C, H, W, K
+    (2, 32, 8, 8, 16),          # two atoms per image, 64-row operand
+    (1, 8, 4, 4, 8),            # a single ragged atom (16 pixels), one MMA step
+    (1, 64, 12, 10, 200),       # HW = 120: last atom holds 24 pixels; two filter blocks, the second ragged
+    (2, 36, 6, 6, 70),          # C = 36: second stage holds 4 channels (half an MMA step: zero-filled rows)
+    (5, 100, 10, 10, 64),       # M = 64 rows, ragged atoms, C = 100
+    (4, 256, 14, 14, 300),      # most channels the resident bank takes; three filter blocks
+    (3, 128, 32, 32, 128),      # the benchmark's per-image shape; items straddle images
+    (40, 16, 20, 20, 24),       # 520 atoms: several rounds of items per block
+]
+
+
+def _takes_tma_kernel(dims):
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K = dims
+    return lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, ALGO_TF32).get("kernel") == "pointwise_tma"
+
+
+@pytest.mark.parametrize("dims", SHAPES)
+def test_pointwise_exact_on_integers(oracle, dims):
+    assert _takes_tma_kernel(dims)
+    N, C, H, W, K = dims
+    x, w = small_integers((N, C, H, W), 961), small_integers((K, C, 1, 1), 962)
+    y_ref, _ = oracle.conv2d_oracle(x, w)
+    np.testing.assert_array_equal(run_library(x, w, entry="general", algo=ALGO_TF32).astype(np.float64), y_ref)
+
+
+@pytest.mark.parametrize("dims", SHAPES)
+def test_pointwise_within_tolerance(oracle, dims):
+    from oracle.conv2d_oracle import MODE_TF32_TRUNC
+    N, C, H, W, K = dims
+    x, w = uniform((N, C, H, W), 963), uniform((K, C, 1, 1), 964)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    y = run_library(x, w, entry="general", algo=ALGO_TF32)
+    r = assert_parity(y, y_ref, yabs, TF32_TOL, f"pointwise {dims}")
+    # the tensor core truncates fp32 operands to TF32: against the oracle fed truncated operands only the order
+    # of the fp32 additions differs
+    y_t, yabs_t = oracle.conv2d_oracle(x, w, mode=MODE_TF32_TRUNC)
+    assert_parity(y, y_t, yabs_t, 2e-5, f"pointwise vs truncated-operand oracle {dims}")
+    print(f"pointwise {dims} max ratio {r:.3e}")
+
+
+def test_pointwise_item_sizes_agree(oracle, monkeypatch):
+    """Every item size (atoms per work item) must give the same bits on integer inputs."""
+    dims = (3, 40, 16, 12, 96)
+    N, C, H, W, K = dims
+    x, w = small_integers((N, C, H, W), 965), small_integers((K, C, 1, 1), 966)
+    y_ref, _ = oracle.conv2d_oracle(x, w)
+    for atoms in (1, 2, 3, 5, 8):
+        monkeypatch.setenv("CONV2D_B200_TMA_ATOMS", str(atoms))
+        np.testing.assert_array_equal(run_library(x, w, entry="general", algo=ALGO_TF32).astype(np.float64), y_ref)
+
+
+def test_pointwise_general_kernel_still_serves_the_shape(oracle, monkeypatch):
+    """With the tensor-map kernel switched off the general tensor-core kernel takes the same shape."""
+    dims = (2, 32, 8, 8, 16)
+    monkeypatch.setenv("CONV2D_B200_TF32_TMA", "0")
+    assert not _takes_tma_kernel(dims)
+    N, C, H, W, K = dims
+    x, w = small_integers((N, C, H, W), 967), small_integers((K, C, 1, 1), 968)
+    y_ref, _ = oracle.conv2d_oracle(x, w)
+    np.testing.assert_array_equal(run_library(x, w, entry="general", algo=ALGO_TF32).astype(np.float64), y_ref)
+
+
+def test_pointwise_expired_wait_is_reported(oracle, monkeypatch):
+    """Host-side injection: one activation stage is armed but never copied and the wait bound is short.  The block
+    gives up, frees its tensor memory and returns; the status word reports it and the next call is correct."""
+    import torch
+    import paper_1705_10591_b200 as lib
+
+    N, C, H, W, K = 2, 64, 16, 16, 128
+    x, w = uniform((N, C, H, W), 969), uniform((K, C, 1, 1), 970)
+    dev = torch.device("cuda:0")
+    xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
+    y = torch.zeros((N, K, H, W), device=dev)
+    ws_bytes = lib.conv2d_fwd_workspace_size(N, C, H, W, K, 1, 1, ALGO_TF32)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    monkeypatch.setenv("CONV2D_B200_TF32_MAX_POLLS", "2048")
+    monkeypatch.setenv("CONV2D_B200_TF32_TEST_DROP_STAGE", "1")
+    lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), y.data_ptr(), N, C, H, W, K, 1, 1, ALGO_TF32,
+                           ws.data_ptr(), ws_bytes, 0, stream)
+    with pytest.raises(lib.Conv2dError) as e:
+        lib.conv2d_get_status(ws.data_ptr(), stream)
+    assert e.value.status == 8                       # CONV2D_ERR_DEVICE_TIMEOUT
+    torch.cuda.synchronize()
+    monkeypatch.delenv("CONV2D_B200_TF32_MAX_POLLS")
+    monkeypatch.delenv("CONV2D_B200_TF32_TEST_DROP_STAGE")
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, "after a time-out")
