@@ -200,17 +200,25 @@ def sustained_ms(fn, torch, sampler, seconds=1.0):
     return ms, mhz, iters
 
 
-GENERAL_COLS = ["us_cold_full_call", "us_warm", "us_warm_prepacked", "frac_cold_full_call", "frac_warm_prepacked",
-                "frac_cold_of_nominal_peak", "us_sustained_1s", "sm_mhz_sustained", "frac_sustained_of_sustained_peak",
+GENERAL_COLS = ["us_cold", "us_cold_after_flush", "us_warm", "us_warm_prepacked", "frac_cold", "frac_warm_prepacked",
+                "frac_cold_of_nominal", "us_sustained_1s", "mhz_sustained", "frac_sustained",
                 "mma_useful_px", "mma_useful_flops"]
+L2_BYTES = 126 * 1024 * 1024
 
 
 def bench_general(torch, lib, peaks, flush, sampler, detail):
     """Times every general-case configuration: tensor cores on fp32 (TF32) and bf16 inputs, and the fp32 kernel.
 
-    Per (configuration, algorithm) one row of GENERAL_COLS: a complete call from cold L2 (filter re-ordering
-    included; `frac` is the roofline fraction of that), warm L2, warm L2 with the filters already re-ordered,
-    and a loop of at least one second of back-to-back complete calls with the SM clock sampled during it.
+    Per (configuration, algorithm) one row of GENERAL_COLS.  All times are complete calls (filter re-ordering
+    included) except the "prepacked" one.
+      us_cold            inputs and outputs larger than L2: the calls rotate over enough distinct (x, y) buffer sets
+                         to exceed twice the 126 MB L2, so no call finds its image in L2 and every call evicts an
+                         earlier call's output: DRAM traffic per call = the algorithmic bytes.  `frac_cold` is the
+                         roofline fraction of this time.
+      us_cold_after_flush  one call after a 256 MB fill: L2 then holds only dirty lines of the fill, so every line
+                         the call brings in also costs a write-back that is not the call's own traffic
+      us_warm, us_warm_prepacked   same buffers back to back (L2 resident); with the filters already re-ordered
+      us_sustained_1s    at least one second of back-to-back calls, SM clock sampled during the loop
     """
     rows = {}
     dev = torch.device("cuda")
@@ -250,11 +258,39 @@ def bench_general(torch, lib, peaks, flush, sampler, detail):
             for _ in range(10):
                 flush.zero_()
                 cold.append(event_ms(call, torch))
+            # rotating buffer sets: more than twice the L2 in distinct inputs and outputs
+            src, src16 = (xd16, None) if algo == lib.ALGO_16BIT else (xd, None)
+            per_set = src.numel() * src.element_size() + yd.numel() * 4
+            n_sets = int(2 * L2_BYTES // per_set) + 2
+            xs = [src.clone() for _ in range(n_sets)]
+            ys = [torch.empty_like(yd) for _ in range(n_sets)]
+
+            def call_set(i):
+                if algo == lib.ALGO_16BIT:
+                    lib.conv2d_fwd_general_16bit(xs[i].data_ptr(), wd16.data_ptr(), ys[i].data_ptr(), cfg.N, cfg.C, cfg.H,
+                                                 cfg.W, cfg.K, cfg.R, cfg.S, lib.OPERAND_BF16, ws.data_ptr(), ws_bytes,
+                                                 0, stream)
+                else:
+                    lib.conv2d_fwd_general(xs[i].data_ptr(), wd.data_ptr(), ys[i].data_ptr(), cfg.N, cfg.C, cfg.H, cfg.W,
+                                           cfg.K, cfg.R, cfg.S, algo, ws.data_ptr(), ws_bytes, 0, stream)
+            for i in range(n_sets):
+                call_set(i)
+            rounds = 3
+            start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            start.record()
+            for _ in range(rounds):
+                for i in range(n_sets):
+                    call_set(i)
+            stop.record()
+            stop.synchronize()
+            t_rot = start.elapsed_time(stop) / (rounds * n_sets)
+            del xs, ys
             warm = event_ms(call, torch, iters=20)
             packed = event_ms(lambda: call(lib.FLAG_WEIGHTS_PACKED), torch, iters=20) if tensor_core else None
             sust, sust_mhz, sust_iters = sustained_ms(call, torch, sampler, 1.0 if algo_name != "ffma" else 0.3)
             lib.conv2d_get_status(ws.data_ptr(), stream)
-            t_cold = statistics.median(cold)
+            t_flush = statistics.median(cold)
+            t_cold = t_rot
             nbytes = cfg.compulsory_bytes
             if algo == lib.ALGO_TF32:
                 pipe_peak, pipe_sustained, pipe_nominal = peaks["bf16_tflops"] / 2.0, peaks["bf16_tflops_sustained"] / 2.0, NOMINAL_TF32_TFLOPS
@@ -272,12 +308,12 @@ def bench_general(torch, lib, peaks, flush, sampler, detail):
             if tensor_core:
                 plan = lib.conv2d_fwd_plan_describe(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, algo)
             bound = ("tensor" if tensor_core else "alu") if cfg.flops / (pipe_peak * 1e12) * 1e3 >= t_hbm else "hbm"
-            row = [t_cold * 1e3, warm * 1e3, packed * 1e3 if packed else None,
+            row = [t_cold * 1e3, t_flush * 1e3, warm * 1e3, packed * 1e3 if packed else None,
                    roof_ms(pipe_peak) / t_cold, roof_ms(pipe_peak) / packed if packed else None,
                    roof_ms(pipe_nominal, t_hbm_nominal) / t_cold, sust * 1e3, sust_mhz, roof_ms(pipe_sustained) / sust,
                    plan.get("mma_useful_px"), plan.get("mma_useful_flops")]
             rows[name][algo_name] = [sig(v) for v in row]
-            detail.append({"workload": name, "algo": algo_name, "bound": bound, "cold_us_all": [sig(c * 1e3) for c in cold],
+            detail.append({"workload": name, "algo": algo_name, "bound": bound, "cold_after_flush_us_all": [sig(c * 1e3) for c in cold], "rotating_sets": n_sets,
                            "sustained_iters": sust_iters, "pipe_peak_tflops": pipe_peak, "pipe_nominal_tflops": pipe_nominal,
                            "pipe_sustained_tflops": pipe_sustained, "t_hbm_us": sig(t_hbm * 1e3), "plan": plan,
                            "gflops_cold": sig(cfg.flops / t_cold / 1e6)})
@@ -361,6 +397,7 @@ def main():
                          "bf16; fp32-exact runs the fp32 FMA kernel (1e-5 tolerance) instead of the tensor cores")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the one-second sustained leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -511,12 +548,13 @@ def main():
         sampler2 = ClockSampler(local_rank)
         sampler2.start()
         # a sustained leg of the headline workload: at least one second of back-to-back steps
-        sust, sust_mhz, sust_iters = sustained_ms(step, torch, sampler2, 1.0)
-        fp32_at = (lambda mhz: SM_COUNT * FP32_LANES_PER_SM * 2 * mhz * 1e6 / 1e12)
-        result["sustained"] = {"ms_per_step": sust, "steps": sust_iters, "sm_mhz": sust_mhz,
-                               "ms_x_mhz": sust * sust_mhz if sust_mhz else None,
-                               "value": cfg.flops / sust / 1e6}
-        if single or ffma:
+        if not args.no_sustained:
+            sust, sust_mhz, sust_iters = sustained_ms(step, torch, sampler2, 1.0)
+            fp32_at = (lambda mhz: SM_COUNT * FP32_LANES_PER_SM * 2 * mhz * 1e6 / 1e12)
+            result["sustained"] = {"ms_per_step": sust, "steps": sust_iters, "sm_mhz": sust_mhz,
+                                   "ms_x_mhz": sust * sust_mhz if sust_mhz else None,
+                                   "value": cfg.flops / sust / 1e6}
+        if (single or ffma) and not args.no_sustained:
             result["sustained"]["alu_frac_at_sampled_clock"] = cfg.flops / (sust * 1e-3) / 1e12 / fp32_at(sust_mhz) if sust_mhz else None
             result["sustained"]["hbm_frac_of_measured"] = algorithmic_bytes / (sust * 1e-3) / 1e9 / peaks["hbm_gbs"]
         if not args.no_general:

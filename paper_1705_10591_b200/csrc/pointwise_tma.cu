@@ -49,8 +49,9 @@ constexpr int kMaxAtoms = 8;              // atoms per work item: N <= 256 colum
 constexpr int kPwMaxStages = 8;
 constexpr int kAccCols = 256;             // tensor-memory columns of one accumulator set
 constexpr int kMaxChannels = 256;         // the filter bank of a block must stay resident
+constexpr int kMaxChunks = kMaxChannels / kStageCh;
 constexpr size_t kPwSmemLimit = 227 * 1024;
-constexpr size_t kPwBookBytes = 256;      // barriers, tensor-memory slot, abort flag
+constexpr size_t kPwBookBytes = 512;      // barriers, tensor-memory slot, abort flag
 
 struct PwArgs {
     unsigned* status;
@@ -83,8 +84,8 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     unsigned char* b_smem = a_smem + (size_t)a.cchunks * a_chunk_bytes;
     unsigned char* o_smem = b_smem + (size_t)a.stages * b_stage_bytes;      // [kPwEpiWarps][32 rows x 128 bytes]
     uint64_t* bars = reinterpret_cast<uint64_t*>(o_smem + (size_t)kPwEpiWarps * 4096);
-    uint64_t* a_full = bars;                       // [1] the filter bank of the current block has landed
-    uint64_t* a_empty = a_full + 1;                // [1] all MMAs that read it have completed
+    uint64_t* a_full = bars;                       // [kMaxChunks] 32-channel chunk i of the current filter block has landed
+    uint64_t* a_empty = a_full + kMaxChunks;       // [1] all MMAs that read the bank have completed
     uint64_t* b_full = a_empty + 1;                // [kPwMaxStages]
     uint64_t* b_empty = b_full + kPwMaxStages;     // [kPwMaxStages]
     uint64_t* acc_full = b_empty + kPwMaxStages;   // [2]
@@ -98,7 +99,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         prefetch_tensormap(&map_w);
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_y);
-        mbar_init(a_full, 1);
+        for (int i = 0; i < a.cchunks; ++i) mbar_init(&a_full[i], 1);
         mbar_init(a_empty, 1);
         for (int i = 0; i < a.stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kPwEpiWarps); }
@@ -135,16 +136,20 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
                 int nb, first, atoms;
                 decode(item, nb, first, atoms);
-                if (nb != cur_nb) {
+                const bool new_bank = nb != cur_nb;
+                if (new_bank) {
                     // the bank of another filter block: wait until the MMAs on the old one are done
                     if (a_loads && !mbar_wait_bounded(a_empty, (a_loads - 1u) & 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                    mbar_arrive_expect_tx(a_full, a_chunk_bytes * (uint32_t)a.cchunks);
-                    for (int cb = 0; cb < a.cchunks; ++cb)
-                        tma_load_2d(a_smem + (size_t)cb * a_chunk_bytes, &map_w, cb * kStageCh, nb * a.m_rows, a_full);
                     cur_nb = nb;
                     ++a_loads;
                 }
                 for (int st = 0; st < a.cchunks; ++st) {
+                    if (new_bank) {
+                        // chunk st of the bank goes out just ahead of the activation stage that needs it, so the
+                        // first MMA waits for 16 KB of filters, not for the whole bank
+                        mbar_arrive_expect_tx(&a_full[st], a_chunk_bytes);
+                        tma_load_2d(a_smem + (size_t)st * a_chunk_bytes, &map_w, st * kStageCh, nb * a.m_rows, &a_full[st]);
+                    }
                     if (!mbar_wait_bounded(&b_empty[slot], ph ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                     mbar_arrive_expect_tx(&b_full[slot], (uint32_t)atoms * kAtomBytes);
                     if (issued != a.test_drop_stage) {
@@ -163,7 +168,8 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             if (*abort_flag) {
                 // let copies already in flight land before the block's shared memory is released
                 uint32_t dummy = 0;
-                if (a_loads) mbar_wait_bounded(a_full, (a_loads - 1u) & 1u, &dummy, 1u << 14);
+                for (int cb = 0; cb < a.cchunks && a_loads; ++cb)
+                    mbar_wait_bounded(&a_full[cb], (a_loads - 1u) & 1u, &dummy, 1u << 14);
                 const int pending = issued < a.stages ? issued : a.stages;
                 for (int i = 0; i < pending; ++i) {
                     const int it = issued - 1 - i;
@@ -181,17 +187,15 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
                 int nb, first, atoms;
                 decode(item, nb, first, atoms);
-                if (nb != cur_nb) {
-                    if (!mbar_wait_bounded(a_full, a_waits & 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                    ++a_waits;
-                    cur_nb = nb;
-                }
+                const bool new_bank = nb != cur_nb;
+                cur_nb = nb;
                 if (!mbar_wait_bounded(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                 tc_fence_after_sync();
                 const uint32_t idesc = idesc_tf32((uint32_t)a.m_rows, (uint32_t)(atoms * kAtomPx)) | kIdescBMajorMN;
                 const uint32_t d = tmem + (uint32_t)(buf * kAccCols);
                 bool accumulate = false;
                 for (int st = 0; st < a.cchunks && alive; ++st) {
+                    if (new_bank && !mbar_wait_bounded(&a_full[st], a_waits & 1u, abort_flag, a.max_polls)) { alive = false; break; }
                     if (!mbar_wait_bounded(&b_full[slot], ph, abort_flag, a.max_polls)) { alive = false; break; }
                     tc_fence_after_sync();
                     const uint32_t a_chunk = a_base + (uint32_t)st * a_chunk_bytes;
@@ -207,6 +211,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     if (++slot == a.stages) { slot = 0; ph ^= 1u; }
                 }
                 if (!alive) break;
+                if (new_bank) ++a_waits;
                 mma_commit(&acc_full[buf]);
                 // the next item of this block uses another filter block: tell the loader when this bank is free
                 const int next = item + (int)gridDim.x;
