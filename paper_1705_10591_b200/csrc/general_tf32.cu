@@ -104,10 +104,10 @@ int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text
     const double useful = 2.0 * out_px * sh.K * sh.C * sh.R * sh.S;
     return snprintf(text, text_bytes,
                     "tensor_core=1 kernel=general_tc addressing=%s filters_as=%s m_rows=%d tile_px=%d px_groups=%d acc_sets=%d items=%lld grid=%d "
-                    "ksplit=%d resident_filters=%d stacked_taps=%d fold=%dx%d patch_w=%d smem_bytes=%zu "
+                    "ksplit=%d cluster=%d resident_filters=%d stacked_taps=%d fold=%dx%d patch_w=%d smem_bytes=%zu "
                     "mma_useful_px=%.4f mma_useful_flops=%.4f",
                     p.patch_w ? "patch" : "flat", p.swap ? "M" : "N", (int)rows, p.tile_px, p.px_groups, p.nbuf,
-                    (long long)p.supertiles * p.n_blocks * p.ksplit, p.grid, p.ksplit, p.resident, p.pair_taps,
+                    (long long)p.supertiles * p.n_blocks * p.ksplit, p.grid, p.ksplit, p.cluster, p.resident, p.pair_taps,
                     p.fold_r, p.fold_s, p.patch_w, p.smem_bytes, out_px / cols, useful / issued);
 }
 
@@ -179,7 +179,8 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
                                      general_tc_kernel<false, true, false, false>,  general_tc_kernel<true, true, false, false>,
                                      general_tc_kernel<false, false, true, false>,  general_tc_kernel<true, false, true, false>,
                                      general_tc_kernel<false, false, false, true>,  general_tc_kernel<true, false, false, true>,
-                                     general_tc_kernel<false, false, true, true>,   general_tc_kernel<true, false, true, true>};
+                                     general_tc_kernel<false, false, true, true>,   general_tc_kernel<true, false, true, true>,
+                                     general_tc_kernel<false, false, false, false, true>, general_tc_kernel<true, false, false, false, true>};
         for (auto k : all)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
             return CONV2D_ERR_CUDA;
@@ -206,7 +207,9 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     a.pair_taps = p.pair_taps; a.s_slots = p.s_slots; a.s_step = p.pair_taps ? 2 : 1; a.item_stride = p.tile_px - p.ovl;
     a.div_HW = FastDiv(a.HW); a.div_W = FastDiv(sh.W); a.div_npix = FastDiv(p.npix);
     a.div_qn = FastDiv(p.npix / 4 > 0 ? p.npix / 4 : 1); a.div_patch_w = FastDiv(p.patch_w ? p.patch_w : 1);
-    a.helpers = (p.swap && (size_t)p.a_stages * p.cbg * kCB * chunk_stride(p.npix) * 4 >= 2 * kXposeBytes &&
+    a.xchg_slots = p.xchg_slots;
+    a.xchg_bytes = (int)xchg_area_bytes(p.xchg_slots);
+    a.helpers = (p.swap && !p.cluster && (size_t)p.a_stages * p.cbg * kCB * chunk_stride(p.npix) * 4 >= 2 * kXposeBytes &&
                  env_int("CONV2D_B200_TF32_HELPERS", 1) != 0) ? 1 : 0;
     a.quad = ((p.patch_w ? (sh.W % 4 == 0 && sh.pad_w % 4 == 0) : (sh.H * sh.W) % 4 == 0) && p.fold_r * p.fold_s == 1 && env_int("CONV2D_B200_TF32_QUAD", 1) != 0) ? 1 : 0;
     {
@@ -234,7 +237,8 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     a.rot = env_int("CONV2D_B200_TF32_ROT", b16 ? 1 : 0) != 0 ? 1 : 0;
     a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
     a.tmem_cols = (unsigned)p.tmem_cols;
-    if (p.ksplit > 1 &&
+    a.early_x = (!weights_packed && (p.ksplit == 1 || p.cluster) && env_int("CONV2D_B200_TF32_EARLY_X", 1) != 0) ? 1 : 0;
+    if (p.ksplit > 1 && !p.cluster &&
         cudaMemsetAsync(y, 0, (size_t)sh.N * sh.K * sh.P * sh.Q * sizeof(float), stream) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     // Programmatic dependent launch: the kernel's set-up (barriers, tensor-memory allocation) overlaps the
@@ -246,7 +250,11 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     else if (p.patch_w) kernel = b16 ? general_tc_kernel<true, false, true, false> : general_tc_kernel<false, false, true, false>;
     else if (fold) kernel = b16 ? general_tc_kernel<true, true, false, false> : general_tc_kernel<false, true, false, false>;
     else kernel = b16 ? general_tc_kernel<true, false, false, false> : general_tc_kernel<false, false, false, false>;
-    if (launch_pdl(kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, stream, a) != cudaSuccess) return CONV2D_ERR_CUDA;
+    if (p.cluster) {
+        kernel = b16 ? general_tc_kernel<true, false, false, false, true> : general_tc_kernel<false, false, false, false, true>;
+        if (launch_pdl_cluster(kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, stream, 2u, a) != cudaSuccess)
+            return CONV2D_ERR_CUDA;
+    } else if (launch_pdl(kernel, dim3((unsigned)p.grid), dim3(kThreads), p.smem_bytes, stream, a) != cudaSuccess) return CONV2D_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
 }

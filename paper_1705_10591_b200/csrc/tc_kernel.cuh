@@ -66,8 +66,12 @@ struct KernelArgs {
     int s_slots, s_step;    // shift-table entries per filter row and the horizontal shift between them (2 with stacked taps)
     int item_stride;        // flat addressing: pixels between the starts of consecutive items (tile_px minus the overlap)
     int ksplit;             // items per output tile (split of the contraction): 1 or 2
+    int xchg_slots;         // cluster instances: 32-pixel blocks each block of a pair receives from its peer
+    int xchg_bytes;         // ... and the bytes of the exchange area (rows + barriers) behind the transposition tiles
     unsigned max_polls;     // bound of every barrier wait
     int test_drop_stage;    // test hook: the filter copy with this ordinal is armed but never issued (-1: none)
+    int early_x;            // 1: this call's filter re-ordering kernel directly precedes on the stream, so the image is
+                            // final already and the producers need not wait for that kernel
     int items;              // work items = supertiles x n_blocks
     unsigned tmem_cols;
 };
@@ -300,7 +304,12 @@ __device__ __forceinline__ void issue_tap(uint32_t d, uint32_t px_lo, uint32_t f
 #undef CONV2D_TAP_MMA
 }
 
-template <bool B16, bool FOLD, bool PATCH, bool STACK>
+// CLUSTER: the two work items of a split contraction (ksplit = 2) run as a two-block cluster, one item per block.
+// Each block stores every other 32-pixel block of the tile: it sends its partial sums of the peer's blocks into the
+// peer's shared memory (distributed shared memory, plain stores) and adds what the peer sent to its own
+// accumulators before the ordinary write-back.  No zero-fill of y, no atomic adds, and a + b = b + a keeps the
+// result independent of timing.
+template <bool B16, bool FOLD, bool PATCH, bool STACK, bool CLUSTER = false>
 __global__ void __launch_bounds__(kThreads, 1)
 general_tc_kernel(const KernelArgs a)
 {
@@ -313,7 +322,10 @@ general_tc_kernel(const KernelArgs a)
     unsigned char* b_smem = smem + (size_t)a.a_stages * a_stage_bytes;
     const size_t b_region_bytes = a.resident ? (size_t)a.cblks * a.taps * b_chunk_bytes : (size_t)a.b_stages * b_stage_bytes;
     float* xpose = reinterpret_cast<float*>(b_smem + b_region_bytes);            // only present (and used) when a.swap
-    uint64_t* bars = reinterpret_cast<uint64_t*>(b_smem + b_region_bytes + (a.swap ? kXposeBytes : 0));
+    unsigned char* after_xpose = b_smem + b_region_bytes + (a.swap ? kXposeBytes : 0);
+    float* xchg = reinterpret_cast<float*>(after_xpose);     // CLUSTER: [4 warps][xchg_slots][32 lanes][kXchgPitch] partial sums from the peer
+    uint64_t* xbar = reinterpret_cast<uint64_t*>(after_xpose + (size_t)kEpilogueWarps * a.xchg_slots * 32 * kXchgPitch * 4);   // [4][xchg_slots]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(after_xpose + (CLUSTER ? a.xchg_bytes : 0));
     uint64_t* a_full = bars;                               // [kMaxAStages]
     uint64_t* a_empty = a_full + kMaxAStages;              // [kMaxAStages]
     uint64_t* b_full = a_empty + kMaxAStages;              // [kMaxBStages]
@@ -337,10 +349,13 @@ general_tc_kernel(const KernelArgs a)
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpilogueWarps); }
         mbar_init(tail_full, 1);
         mbar_init(drain_bar, 1);
+        if (CLUSTER)
+            for (int i = 0; i < kEpilogueWarps * a.xchg_slots; ++i) mbar_init(&xbar[i], 32);
         *abort_flag = 0;
         fence_mbar_init();
     }
     __syncthreads();
+    if (CLUSTER) cluster_sync_all();        // the peer's barriers exist before anything can arrive on them
     if (warp == 1) { tmem_alloc(tmem_slot, a.tmem_cols); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
@@ -348,9 +363,12 @@ general_tc_kernel(const KernelArgs a)
     const uint32_t tmem = *tmem_slot;
     // Everything above touched only this block's shared and tensor memory; it may overlap the tail of the
     // preceding kernel on the stream (the filter re-ordering of this call, or the previous call).  From here
-    // on global memory is read and written.
+    // on global memory is read and written: every role waits for the preceding kernel first, except that the
+    // producers go ahead when that kernel is this call's own filter re-ordering.  It was launched the ordinary way,
+    // so everything before it on the stream had finished when it started, it does not touch the image, and the
+    // image is read only: the first activation stages are then in flight while the filters are still being written.
     grid_dep_launch();
-    grid_dep_wait();
+    if (!(a.early_x && producer_index(warp) >= 0)) grid_dep_wait();
 
     // Work item -> (supertile, filter block); blocks rotate the order of the channel-block groups by the
     // item number, so that at any moment they stream different parts of the filter bank.
@@ -427,6 +445,8 @@ general_tc_kernel(const KernelArgs a)
             auto mma = [](uint32_t d, uint64_t ad, uint64_t bd, uint32_t id, bool acc) {
                 if (B16) mma_b16(d, ad, bd, id, acc); else mma_tf32(d, ad, bd, id, acc);
             };
+            // (the start-address field of a descriptor holds bits 4-17 of the shared-memory address; the address of a
+            // block that is not the first of its cluster has bits above those set, which must not leak into LBO)
             const uint32_t desc_hi = (128u >> 4) | (1u << 14);                  // SBO = 128 B, descriptor version 1
             const uint32_t a_lo_fixed = ((uint32_t)a.cstride & 0x3FFFu) << 16;  // LBO = chunk stride * 16 B
             const uint32_t b_lo_fixed = ((uint32_t)a.n_tile & 0x3FFFu) << 16;   // LBO = n_tile * 16 B
@@ -464,7 +484,7 @@ general_tc_kernel(const KernelArgs a)
                     int gr = grp + ii.rot;
                     if (gr >= ii.n_groups) gr -= ii.n_groups;
                     gr += ii.g_begin;
-                    uint32_t a_lo_block = a_lo_fixed | (smem_u32(a_smem + (size_t)as * a_stage_bytes) >> 4);
+                    uint32_t a_lo_block = a_lo_fixed | ((smem_u32(a_smem + (size_t)as * a_stage_bytes) >> 4) & 0x3FFFu);
                     for (int g = 0; g < a.cbg && alive; ++g, a_lo_block += a_block_bytes >> 4) {
                         if (gr * a.cbg + g >= a.cblks) break;
                         uint32_t row_shift = 0;                                  // r * row pitch, in pixels (= 16-byte units)
@@ -473,11 +493,11 @@ general_tc_kernel(const KernelArgs a)
                             const int nt = min(a.tps, a.taps - t0);
                             uint32_t b_lo;
                             if (a.resident) {
-                                b_lo = b_lo_fixed | (smem_u32(b_smem + (size_t)(gr * a.cbg + g) * a.taps * b_chunk_bytes) >> 4);
+                                b_lo = b_lo_fixed | ((smem_u32(b_smem + (size_t)(gr * a.cbg + g) * a.taps * b_chunk_bytes) >> 4) & 0x3FFFu);
                             } else {
                                 if (!mbar_wait_bounded(&b_full[bs], b_phase, abort_flag, a.max_polls)) { alive = false; break; }
                                 tc_fence_after_sync();
-                                b_lo = b_lo_fixed | (smem_u32(b_smem + (size_t)bs * b_stage_bytes) >> 4);
+                                b_lo = b_lo_fixed | ((smem_u32(b_smem + (size_t)bs * b_stage_bytes) >> 4) & 0x3FFFu);
                             }
                             if (a.swap && a.px_groups == 1) {
                                 // M operand = the 128 filters of this stage, N operand = n_mma staged pixels.
@@ -693,7 +713,7 @@ general_tc_kernel(const KernelArgs a)
             const bool split = a.helpers && li == n_local - 1;
             const ItemInfo ii = decode_item(a, item);
             const int nb = ii.nb;
-            const bool add = a.ksplit > 1;                   // partial sums: add into the zeroed output
+            const bool add = !CLUSTER && a.ksplit > 1;       // partial sums: add into the zeroed output
             // tcgen05.ld is warp-collective: take the decision for the whole warp
             // (warps 8-15 come late and only for the last item: they wait on a barrier of its own, whose
             // phase they cannot have missed)
@@ -790,6 +810,58 @@ general_tc_kernel(const KernelArgs a)
                         }
                     }
                 };
+                if (CLUSTER) {
+                    const uint32_t rank = cluster_ctarank(), peer = rank ^ 1u;
+                    float* my_rows = xchg + (size_t)(warp - 4) * a.xchg_slots * 32 * kXchgPitch;
+                    uint64_t* my_bars = xbar + (warp - 4) * a.xchg_slots;
+                    uint32_t v0[16], v1[16], vx[1];
+                    vx[0] = 0u;
+                    // the blocks the peer stores: this block's partial sums go into the peer's shared memory, one
+                    // 144-byte row per accumulator lane (= filter), and every lane then arrives on the peer's barrier
+                    for (int b = (int)peer; b < blocks; b += 2) {
+                        tmem_ld16(lane_base + (uint32_t)(b * 32), v0);
+                        tmem_ld16(lane_base + (uint32_t)(b * 32 + 16), v1);
+                        tmem_ld_wait();
+                        const int slot = b >> 1;
+                        const uint32_t dst = map_to_cta(smem_u32(my_rows + ((size_t)slot * 32 + lane) * kXchgPitch), peer);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            st_cluster_v4(dst + 16u * i, __uint_as_float(v0[4 * i]), __uint_as_float(v0[4 * i + 1]),
+                                          __uint_as_float(v0[4 * i + 2]), __uint_as_float(v0[4 * i + 3]));
+                            st_cluster_v4(dst + 64u + 16u * i, __uint_as_float(v1[4 * i]), __uint_as_float(v1[4 * i + 1]),
+                                          __uint_as_float(v1[4 * i + 2]), __uint_as_float(v1[4 * i + 3]));
+                        }
+                        mbar_arrive_remote(map_to_cta(smem_u32(&my_bars[slot]), peer));
+                    }
+                    // this block's own blocks: accumulators + the peer's partial sums, then the ordinary write-back
+                    for (int b = (int)rank; b < blocks; b += 2) {
+                        tmem_ld16(lane_base + (uint32_t)(b * 32), v0);
+                        tmem_ld16(lane_base + (uint32_t)(b * 32 + 16), v1);
+                        tmem_ld_wait();
+                        const int slot = b >> 1;
+                        alive = __all_sync(0xffffffffu, mbar_wait_bounded_cluster(&my_bars[slot], 0u, abort_flag, a.max_polls));
+                        if (!alive) break;
+                        const float4* row = reinterpret_cast<const float4*>(my_rows + ((size_t)slot * 32 + lane) * kXchgPitch);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float4 t = row[i], u = row[4 + i];
+                            v0[4 * i] = __float_as_uint(__uint_as_float(v0[4 * i]) + t.x);
+                            v0[4 * i + 1] = __float_as_uint(__uint_as_float(v0[4 * i + 1]) + t.y);
+                            v0[4 * i + 2] = __float_as_uint(__uint_as_float(v0[4 * i + 2]) + t.z);
+                            v0[4 * i + 3] = __float_as_uint(__uint_as_float(v0[4 * i + 3]) + t.w);
+                            v1[4 * i] = __float_as_uint(__uint_as_float(v1[4 * i]) + u.x);
+                            v1[4 * i + 1] = __float_as_uint(__uint_as_float(v1[4 * i + 1]) + u.y);
+                            v1[4 * i + 2] = __float_as_uint(__uint_as_float(v1[4 * i + 2]) + u.z);
+                            v1[4 * i + 3] = __float_as_uint(__uint_as_float(v1[4 * i + 3]) + u.w);
+                        }
+                        store_block(v0, v1, vx, b);
+                    }
+                    if (!alive) break;
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                    continue;
+                }
                 uint32_t va0[16], va1[16], vb0[16], vb1[16], vax[1], vbx[1];
                 const int b_step = split ? 3 : 1;
                 int b = split ? share : 0;
@@ -858,6 +930,8 @@ general_tc_kernel(const KernelArgs a)
 
     tc_fence_before_sync();
     __syncthreads();
+    // (a block must not exit while its peer may still write into its shared memory or arrive on its barriers)
+    if (CLUSTER) cluster_sync_all();
     if (warp == 1) tmem_dealloc(tmem, a.tmem_cols);
     if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
     if (kDiag && tid == 0 && blockIdx.x == 0) a.status[8] = (unsigned)(wall_ns() - *t_entry);   // ns from kernel entry to the block's end

@@ -42,6 +42,9 @@ constexpr int kMaxTaps = 256;                // taps left as descriptor shifts (
 constexpr size_t kBookBytes = 512 + kMaxTaps * 4;    // barriers, tensor-memory slot, flags + the table of tap shifts
 constexpr int kXposePitch = 36;             // floats per row of the epilogue's transposition tile (16-byte aligned, conflict-free)
 constexpr size_t kXposeBytes = (size_t)kEpilogueWarps * 32 * kXposePitch * 4;
+constexpr int kXchgPitch = 36;              // floats per row of the exchange area of a two-block cluster (as above)
+// bytes of that area for `slots` 32-pixel blocks per epilogue warp: rows, then one barrier per (warp, slot)
+constexpr size_t xchg_area_bytes(int slots) { return (size_t)kEpilogueWarps * slots * (32 * kXchgPitch * 4 + 8); }
 
 struct Plan {
     int n_tile;       // filters per work item: 64 or 128 rows of the M operand (with the pixels as M: UMMA N, a multiple of 16)
@@ -65,6 +68,8 @@ struct Plan {
     int s_slots;      // shift-table entries per filter row: S, or ceil(S / 2) with stacked taps
     int ovl;          // pixels by which consecutive flat items overlap (4 with stacked taps, else 0)
     int ksplit;       // 2: the channel blocks of a tile are shared by two work items that add into y
+    int cluster;      // 1 (with ksplit = 2): the two items run as a two-block cluster and exchange partial sums on chip
+    int xchg_slots;   // ... 32-pixel blocks each of them receives
     int tmem_cols;    // power of two >= 32
     int supertiles;   // work-item rows over the flat pixel sequence
     int grid;
@@ -346,6 +351,23 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
     const long long items = (long long)p.supertiles * p.n_blocks * p.ksplit;
     if (items > 0x7fffffffLL) return p;
     p.grid = (int)(items < sms ? items : sms);
+    // The split contraction as a two-block cluster: needs room for the exchange area behind the transposition tiles
+    // (the filter ring gives up stages for it, down to two) and one item per block.
+    p.cluster = 0;
+    p.xchg_slots = 0;
+    if (p.ksplit == 2 && p.swap && !p.patch_w && !p.pair_taps && p.fold_r * p.fold_s == 1 && p.n_tile == 128 && !p.resident &&
+        items <= sms && env_int("CONV2D_B200_TF32_KSPLIT_CLUSTER", 1) != 0) {
+        const int slots = (p.tile_px / 32 + 1) / 2;
+        const size_t xb = xchg_area_bytes(slots);
+        int bs = p.b_stages;
+        while (bs > 2 && smem_need(p.a_stages, p.npix, p.n_tile, bs, p.tps, p.cbg) + extra + xb > kSmemLimit) --bs;
+        if (smem_need(p.a_stages, p.npix, p.n_tile, bs, p.tps, p.cbg) + extra + xb <= kSmemLimit) {
+            p.cluster = 1;
+            p.xchg_slots = slots;
+            p.b_stages = bs;
+            p.smem_bytes = smem_need(p.a_stages, p.npix, p.n_tile, bs, p.tps, p.cbg) + extra + xb;
+        }
+    }
     int cols = p.nbuf * item_cols;
     p.tmem_cols = 32;
     while (p.tmem_cols < cols) p.tmem_cols <<= 1;
