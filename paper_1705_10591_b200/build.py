@@ -4,6 +4,7 @@ Usage: python -m paper_1705_10591_b200.build [--force] [--verbose]
 """
 from __future__ import annotations
 
+import os
 import subprocess
 import sys
 from pathlib import Path
@@ -39,6 +40,9 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     ]
     if verbose:
         common.insert(1, "-Xptxas=-v")
+    if os.environ.get("CONV2D_B200_BUILD_DIAGNOSTICS"):
+        # tuning build: the tensor-core kernel's MMA thread counts its cycles into status words 2-9
+        common.append("-DCONV2D_B200_TC_DIAGNOSTICS")
     with tempfile.TemporaryDirectory(prefix="conv2d_b200_build_") as tmp:
         objs = [str(Path(tmp) / (Path(s).stem + ".o")) for s in SOURCES]
 

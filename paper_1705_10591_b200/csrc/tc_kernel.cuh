@@ -812,13 +812,17 @@ general_tc_kernel(const KernelArgs a)
                 };
                 if (CLUSTER) {
                     const uint32_t rank = cluster_ctarank(), peer = rank ^ 1u;
-                    float* my_rows = xchg + (size_t)(warp - 4) * a.xchg_slots * 32 * kXchgPitch;
-                    uint64_t* my_bars = xbar + (warp - 4) * a.xchg_slots;
+                    // rows and barriers belong to a (lane quarter, block) pair; with the helper warps a quarter is
+                    // drained by three warps, block b going to warp (b / 2) mod 3 of the quarter on both sides
+                    float* my_rows = xchg + (size_t)quarter * a.xchg_slots * 32 * kXchgPitch;
+                    uint64_t* my_bars = xbar + quarter * a.xchg_slots;
+                    const int nshare = a.helpers ? 3 : 1;
                     uint32_t v0[16], v1[16], vx[1];
                     vx[0] = 0u;
                     // the blocks the peer stores: this block's partial sums go into the peer's shared memory, one
                     // 144-byte row per accumulator lane (= filter), and every lane then arrives on the peer's barrier
                     for (int b = (int)peer; b < blocks; b += 2) {
+                        if ((b >> 1) % nshare != share) continue;
                         tmem_ld16(lane_base + (uint32_t)(b * 32), v0);
                         tmem_ld16(lane_base + (uint32_t)(b * 32 + 16), v1);
                         tmem_ld_wait();
@@ -835,6 +839,7 @@ general_tc_kernel(const KernelArgs a)
                     }
                     // this block's own blocks: accumulators + the peer's partial sums, then the ordinary write-back
                     for (int b = (int)rank; b < blocks; b += 2) {
+                        if ((b >> 1) % nshare != share) continue;
                         tmem_ld16(lane_base + (uint32_t)(b * 32), v0);
                         tmem_ld16(lane_base + (uint32_t)(b * 32 + 16), v1);
                         tmem_ld_wait();
@@ -859,7 +864,7 @@ general_tc_kernel(const KernelArgs a)
                     if (!alive) break;
                     tc_fence_before_sync();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                    if (lane == 0 && !helper) mbar_arrive(&acc_empty[buf]);
                     continue;
                 }
                 uint32_t va0[16], va1[16], vb0[16], vb1[16], vax[1], vbx[1];
