@@ -100,14 +100,15 @@ int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text
     const double ncols = p.swap ? (double)p.supertiles * p.tile_px * p.n_blocks
                                 : (double)p.supertiles * p.mt * p.n_blocks * p.n_tile;
     const double kdim = (double)p.cblks * (b16 ? 2 * kCB : kCB) * p.taps;
-    const double issued = 2.0 * rows * ncols * kdim * (p.swap ? 1.0 : 1.0);
+    double issued = 2.0 * rows * ncols * kdim;
+    if (p.pair_compact) issued *= (double)p.cb_bytes / ((double)p.taps * kCB * p.n_tile * 4);    // lone taps are 64-row MMAs
     const double useful = 2.0 * out_px * sh.K * sh.C * sh.R * sh.S;
     return snprintf(text, text_bytes,
                     "tensor_core=1 kernel=general_tc addressing=%s filters_as=%s m_rows=%d tile_px=%d px_groups=%d acc_sets=%d items=%lld grid=%d "
-                    "ksplit=%d cluster=%d resident_filters=%d stacked_taps=%d fold=%dx%d patch_w=%d smem_bytes=%zu "
+                    "ksplit=%d cluster=%d resident_filters=%d stacked_taps=%d stacked_compact=%d fold=%dx%d patch_w=%d smem_bytes=%zu "
                     "mma_useful_px=%.4f mma_useful_flops=%.4f",
                     p.patch_w ? "patch" : "flat", p.swap ? "M" : "N", (int)rows, p.tile_px, p.px_groups, p.nbuf,
-                    (long long)p.supertiles * p.n_blocks * p.ksplit, p.grid, p.ksplit, p.cluster, p.resident, p.pair_taps,
+                    (long long)p.supertiles * p.n_blocks * p.ksplit, p.grid, p.ksplit, p.cluster, p.resident, p.pair_taps, p.pair_compact,
                     p.fold_r, p.fold_s, p.patch_w, p.smem_bytes, out_px / cols, useful / issued);
 }
 
@@ -140,7 +141,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     if (!weights_packed) {
         const long long total = (long long)packed_floats(p);
         const FoldedFilter ff{sh.C, sh.R, sh.S, p.fold_r, p.fold_s};
-        const long long lanes = total / p.taps * (b16 ? 2 : 1);      // one thread per element of a tap's slice
+        const long long lanes = (long long)p.n_blocks * p.cblks * kChunks * p.n_tile * (b16 ? 8 : 4);   // one thread per element of a tap's slice
         long long blocks = (lanes + 255) / 256;
         if (blocks > sm_count() * 16LL) blocks = sm_count() * 16LL;
         const size_t tile_bytes = (size_t)8 * kCB * 4 * p.taps;       // 8 filters x one channel block x taps
@@ -160,10 +161,10 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         } else if (b16)
             repack_filters_kernel<unsigned short, 8><<<(unsigned)blocks, 256, 0, stream>>>(
                 static_cast<const unsigned short*>(w_any), reinterpret_cast<unsigned short*>(wp), status, sh.K, ff,
-                p.taps, p.n_tile, p.cblks, lanes, p.pair_taps);
+                p.taps, p.n_tile, p.cblks, lanes, p.pair_taps + p.pair_compact);
         else
             repack_filters_kernel<float, 4><<<(unsigned)blocks, 256, 0, stream>>>(w, wp, status, sh.K, ff, p.taps,
-                                                                                  p.n_tile, p.cblks, lanes, p.pair_taps);
+                                                                                  p.n_tile, p.cblks, lanes, p.pair_taps + p.pair_compact);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return CONV2D_ERR_CUDA;
     }
@@ -204,6 +205,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
         if ((p.patch_w ? p.patch_tw : sh.W) % v == 0 && sh.Q % v == 0 && ((long long)sh.P * sh.Q) % v == 0 &&
             reinterpret_cast<uintptr_t>(y) % (4 * v) == 0) { a.vec = v; break; }
     a.vec_shift = a.vec == 4 ? 2 : (a.vec == 2 ? 1 : 0);
+    a.pair_compact = p.pair_compact; a.cb_bytes = (int)p.cb_bytes;
     a.pair_taps = p.pair_taps; a.s_slots = p.s_slots; a.s_step = p.pair_taps ? 2 : 1; a.item_stride = p.tile_px - p.ovl;
     a.div_HW = FastDiv(a.HW); a.div_W = FastDiv(sh.W); a.div_npix = FastDiv(p.npix);
     a.div_qn = FastDiv(p.npix / 4 > 0 ? p.npix / 4 : 1); a.div_patch_w = FastDiv(p.patch_w ? p.patch_w : 1);

@@ -64,6 +64,9 @@ struct KernelArgs {
     int vec;                // swap mode: adjacent pixels a lane stores as one unit (1, 2 or 4)
     int pair_taps;          // stacked taps: accumulator lanes 64-127 hold the right-hand tap of each pair, one column to the right
     int s_slots, s_step;    // shift-table entries per filter row and the horizontal shift between them (2 with stacked taps)
+    int pair_compact;       // stacked taps, resident bank: the odd last tap of a filter row is a 64-row slice of its own,
+                            // issued as an M = 64 MMA onto the same accumulator lanes (no zero-padded upper half)
+    int cb_bytes;           // resident filters: bytes of one channel block of the bank (all taps)
     int item_stride;        // flat addressing: pixels between the starts of consecutive items (tile_px minus the overlap)
     int ksplit;             // items per output tile (split of the contraction): 1 or 2
     int xchg_slots;         // cluster instances: 32-pixel blocks each block of a pair receives from its peer
@@ -320,7 +323,7 @@ general_tc_kernel(const KernelArgs a)
     const uint32_t b_stage_bytes = b_chunk_bytes * (uint32_t)a.tps;
     unsigned char* a_smem = smem;
     unsigned char* b_smem = smem + (size_t)a.a_stages * a_stage_bytes;
-    const size_t b_region_bytes = a.resident ? (size_t)a.cblks * a.taps * b_chunk_bytes : (size_t)a.b_stages * b_stage_bytes;
+    const size_t b_region_bytes = a.resident ? (size_t)a.cblks * a.cb_bytes : (size_t)a.b_stages * b_stage_bytes;
     float* xpose = reinterpret_cast<float*>(b_smem + b_region_bytes);            // only present (and used) when a.swap
     unsigned char* after_xpose = b_smem + b_region_bytes + (a.swap ? kXposeBytes : 0);
     float* xchg = reinterpret_cast<float*>(after_xpose);     // CLUSTER: [4 warps][xchg_slots][32 lanes][kXchgPitch] partial sums from the peer
@@ -340,7 +343,10 @@ general_tc_kernel(const KernelArgs a)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile unsigned long long* t_entry = reinterpret_cast<volatile unsigned long long*>(tmem_slot + 2);
     uint32_t* tap_shift = tmem_slot + 4;                   // [taps] r * row_pitch + s of every tap, in staged pixels
-    for (int t = tid; t < a.taps; t += kThreads) tap_shift[t] = (uint32_t)((t / a.s_slots) * a.row_pitch + (t % a.s_slots) * a.s_step);
+    // (bit 31: the slot is a lone tap held as a 64-row slice, see pair_compact)
+    for (int t = tid; t < a.taps; t += kThreads)
+        tap_shift[t] = (uint32_t)((t / a.s_slots) * a.row_pitch + (t % a.s_slots) * a.s_step) |
+                       ((a.pair_compact && (a.S & 1) && t % a.s_slots == a.s_slots - 1) ? 0x80000000u : 0u);
     if (kDiag && tid == 0) *t_entry = wall_ns();
 
     if (tid == 0) {
@@ -384,7 +390,7 @@ general_tc_kernel(const KernelArgs a)
                 // the whole filter bank (a single filter block in this mode), once, one bulk copy per channel
                 // block, all on one barrier
                 const unsigned char* src = reinterpret_cast<const unsigned char*>(a.wp);
-                const uint32_t piece = b_chunk_bytes * (uint32_t)a.taps;
+                const uint32_t piece = (uint32_t)a.cb_bytes;
                 mbar_arrive_expect_tx(&b_full[0], piece * (uint32_t)a.cblks);
                 for (int cb = 0; cb < a.cblks; ++cb)
                     bulk_g2s(b_smem + (size_t)cb * piece, src + (size_t)cb * piece, piece, &b_full[0]);
@@ -493,7 +499,7 @@ general_tc_kernel(const KernelArgs a)
                             const int nt = min(a.tps, a.taps - t0);
                             uint32_t b_lo;
                             if (a.resident) {
-                                b_lo = b_lo_fixed | ((smem_u32(b_smem + (size_t)(gr * a.cbg + g) * a.taps * b_chunk_bytes) >> 4) & 0x3FFFu);
+                                b_lo = b_lo_fixed | ((smem_u32(b_smem + (size_t)(gr * a.cbg + g) * a.cb_bytes) >> 4) & 0x3FFFu);
                             } else {
                                 if (!mbar_wait_bounded(&b_full[bs], b_phase, abort_flag, a.max_polls)) { alive = false; break; }
                                 tc_fence_after_sync();
@@ -507,6 +513,24 @@ general_tc_kernel(const KernelArgs a)
                                 // table, fetched one tap ahead.
                                 const uint32_t* shift = tap_shift + t0;
                                 uint32_t cur = shift[0];
+                                if (STACK && a.pair_compact) {
+                                    // pairs of taps as M = 128 slices, a lone last tap as an M = 64 slice of half the size
+                                    // (its chunk stride and K step are half as long too) onto the same accumulator lanes
+                                    const uint32_t idesc64 = B16 ? idesc_b16(64u, n_cols, a.fp16 != 0) : idesc_tf32(64u, n_cols);
+                                    for (int t = 0; t < nt; ++t) {
+                                        const uint32_t a_lo = a_lo_block + (cur & 0x7FFFFFFFu);
+                                        const bool lone = (cur >> 31) != 0u;
+                                        cur = shift[t + 1 < nt ? t + 1 : t];
+                                        if (lone) {
+                                            issue_tap<B16, 1>(d0, a_lo, b_lo - (64u << 16), a_kstep, b_kstep >> 1, n_mma, desc_hi, idesc64, accumulate);
+                                            b_lo += b_chunk_bytes >> 5;
+                                        } else {
+                                            issue_tap<B16, 1>(d0, a_lo, b_lo, a_kstep, b_kstep, n_mma, desc_hi, idesc, accumulate);
+                                            b_lo += b_chunk_bytes >> 4;
+                                        }
+                                        accumulate = 1;
+                                    }
+                                } else
 #pragma unroll 3
                                 for (int t = 0; t < nt; ++t, b_lo += b_chunk_bytes >> 4) {
                                     const uint32_t a_lo = a_lo_block + cur;
@@ -717,10 +741,13 @@ general_tc_kernel(const KernelArgs a)
             // tcgen05.ld is warp-collective: take the decision for the whole warp
             // (warps 8-15 come late and only for the last item: they wait on a barrier of its own, whose
             // phase they cannot have missed)
+            const long long t_wait0 = clock_now();
             alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(helper ? tail_full : &acc_full[buf],
                                                                        helper ? 0u : acc_phase, abort_flag, a.max_polls));
             if (!alive) break;
             tc_fence_after_sync();
+            const long long t_busy0 = clock_now();
+            if (kDiag && blockIdx.x == 0 && warp == 4 && lane == 0) a.status[10] += (unsigned)(t_busy0 - t_wait0);   // waited for accumulators
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * acc_cols);
             if (a.swap) {
                 // Lanes are filters, columns pixels: this thread holds adjacent pixels of ONE map.  A
@@ -884,6 +911,7 @@ general_tc_kernel(const KernelArgs a)
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0 && !helper) mbar_arrive(&acc_empty[buf]);
+                if (kDiag && blockIdx.x == 0 && warp == 4 && lane == 0) a.status[11] += (unsigned)(clock_now() - t_busy0);   // drained one item
                 continue;
             }
             int cur_m = -1;

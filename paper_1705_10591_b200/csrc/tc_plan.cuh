@@ -65,6 +65,8 @@ struct Plan {
     int resident;     // 1: the whole filter block stays in shared memory for the life of the thread block
     int swap;         // 1: filters are the MMA's M operand, 256 pixels its N operand (K <= 128)
     int pair_taps;    // 1: at most 64 filters, horizontally adjacent taps stacked in one M = 128 operand (see make_plan)
+    int pair_compact; // 1 (with pair_taps): a lone last tap of a filter row is a 64-row slice issued as M = 64 (resident bank only)
+    size_t cb_bytes;  // bytes of one channel block of the re-ordered bank (all taps of one filter block)
     int s_slots;      // shift-table entries per filter row: S, or ceil(S / 2) with stacked taps
     int ovl;          // pixels by which consecutive flat items overlap (4 with stacked taps, else 0)
     int ksplit;       // 2: the channel blocks of a tile are shared by two work items that add into y
@@ -93,7 +95,7 @@ size_t smem_need(int a_stages, int npix, int n_tile, int b_stages, int tps, int 
 
 // b16: the operands are 16-bit floats, bf16 or fp16 (16-byte unit = 8 channels, 32 channels per staged block, K = 16 per MMA); the
 // byte layout of every stage is the same as for TF32 (16 channels of 4 bytes).
-Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
+Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w, bool allow_compact = true)
 {
     Plan p{};
     p.ok = false;
@@ -158,6 +160,21 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
     const int pair_mode = env_int("CONV2D_B200_TF32_PAIR_TAPS", 1);
     p.pair_taps = (p.swap && kp16 <= 64 && p.fold_r * p.fold_s == 1 && s_eff >= 2 && pair_mode != 0 &&
                    (pair_mode == 2 || (long long)r_eff * s_eff * p.cblks >= 48)) ? 1 : 0;
+    // Compact stacking for banks that can stay in shared memory: pairs of taps as 128-row slices, the lone last tap of
+    // an odd filter row as a 64-row slice that an M = 64 instruction adds onto the same accumulator lanes.  The bank
+    // is then as large as the unstacked one, so a short contraction keeps its resident filters and still issues two
+    // instructions per three taps instead of three at half rate (64 filters of 64 x 3 x 3 on 56 x 56 images).
+    // Measured on that shape: the MMA thread's issue time per 256-pixel item falls from 9.4k to 7.4k cycles, but the
+    // four write-back warps need 10.4k cycles for the item (8.9k unstacked: every map is the sum of two tile rows), and
+    // with two accumulator sets the slower of the two sets the pace: 36.5 -> 39.4 us.  Off by default
+    // (CONV2D_B200_TF32_PAIR_COMPACT = 1 turns it on) until the write-back is faster than the MMAs.
+    p.pair_compact = 0;
+    const size_t compact_cb_bytes = (size_t)r_eff * ((s_eff / 2) * 128 + (s_eff & 1) * 64) * kCB * 4;
+    if (allow_compact && !p.pair_taps && p.swap && kp16 <= 64 && p.fold_r * p.fold_s == 1 && s_eff >= 2 && pair_mode != 0 &&
+        !padded && (size_t)((c_eff + cbc - 1) / cbc) * compact_cb_bytes <= 152 * 1024 && env_int("CONV2D_B200_TF32_PAIR_COMPACT", 0) != 0) {
+        p.pair_taps = 1;
+        p.pair_compact = 1;
+    }
     if (p.pair_taps) p.n_tile = 128;
     p.s_slots = p.pair_taps ? (s_eff + 1) / 2 : s_eff;
     p.taps = r_eff * p.s_slots;
@@ -204,7 +221,8 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
     const int sms = sm_count();
 
     const int forced_mt = env_int("CONV2D_B200_TF32_MT", 0);      // benchmark ablations only
-    const size_t wbytes = (size_t)p.cblks * p.taps * chunk;        // re-ordered filters of one filter block
+    p.cb_bytes = p.pair_compact ? compact_cb_bytes : (size_t)p.taps * chunk;
+    const size_t wbytes = (size_t)p.cblks * p.cb_bytes;            // re-ordered filters of one filter block
     auto npix_of = [&](int tile_px) { return (int)(((long long)tile_px + halo + 7) / 8 * 8); };
 
     // Light problems (1x1-like: few taps x channel blocks) with a small filter bank keep it resident in
@@ -222,12 +240,13 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
         if (p.swap && !p.patch_w && !forced_mt) {
             // When all pixels fit in one round of items of at most 512 pixels, one item per block is the better
             // cut (64 x 32 x 32 pixels with 1 x 1 filters: 448 pixels per item 19.9 us, 256 per item 22.1 us).
+            // (compact stacking issues one MMA per K step: at most 256 pixels per item)
             const long long one_round = ((total_pix + sms - 1) / sms + p.ovl + 31) / 32 * 32;
-            if (one_round >= 64 && one_round <= 512) res_px = (int)one_round;
+            if (one_round >= 64 && one_round <= (p.pair_compact ? 256 : 512)) res_px = (int)one_round;
         }
         {
             const int want = env_int("CONV2D_B200_TF32_TILE_PX", 0);
-            if (p.swap && want >= 64 && want <= 512 && want % 32 == 0 && pixel_items(want) > 0) res_px = want;
+            if (p.swap && want >= 64 && want <= (p.pair_compact ? 256 : 512) && want % 32 == 0 && pixel_items(want) > 0) res_px = want;
         }
         const int npix = npix_of(res_px);
         if ((p.swap ? res_px : mt * set_cols) <= 512 && npix <= 16000 && wbytes + extra + (size_t)2 * kCB * chunk_stride(npix) * 4 + kBookBytes <= kSmemLimit) {
@@ -247,6 +266,7 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
         }
     }
 
+    if (p.pair_compact && !p.resident) return plan_with_patch_width(sh, b16, want_patch_w, false);    // compact stacking needs the resident bank
     if (!p.resident) {
         // Streamed filters.  Measured: all SMs together draw filter stages from L2 at no more than
         // ~5-6 TB/s, i.e. a 8 KB stage costs ~120 cycles on top of the MMAs that consume it unless it is
@@ -339,6 +359,7 @@ Plan plan_with_patch_width(const Shape& sh, bool b16, int want_patch_w)
         const int want = env_int("CONV2D_B200_TF32_PX_GROUPS", 0);
         if (p.swap && want > 0 && want <= 2 && p.tile_px % (16 * want) == 0 && p.tile_px / want <= 256) p.px_groups = want;
     }
+    if (p.pair_compact) p.px_groups = 1;
     p.nbuf = (2 * item_cols <= 512 && env_int("CONV2D_B200_TF32_NBUF", 2) != 1) ? 2 : 1;
     if (p.patch_w) p.patch_rows = (sh.P + p.tile_px / p.patch_w - 1) / (p.tile_px / p.patch_w);
     if (pixel_items(p.tile_px) <= 0 || pixel_items(p.tile_px) > 0x7fffffffLL) return p;
@@ -396,7 +417,7 @@ Plan make_plan(const Shape& sh, bool b16 = false)
 
 size_t packed_floats(const Plan& p)
 {
-    return (size_t)p.n_blocks * p.cblks * p.taps * kCB * p.n_tile;
+    return (size_t)p.n_blocks * p.cblks * (p.cb_bytes / 4);
 }
 
 }  // namespace

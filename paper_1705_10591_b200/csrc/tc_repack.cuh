@@ -34,6 +34,8 @@ struct FoldedFilter {
 // 16-bit pattern with 8.
 // stacked = 1: half of the rows of the 128-row block are the filters' tap (r, 2u), the other half their tap
 // (r, 2u + 1) (zeros where S is odd and 2u + 1 = S); tap index t = r * ceil(S / 2) + u.
+// stacked = 2 (compact): the same, but where S is odd the lone last tap of a filter row is a slice of 64 rows in
+// natural filter order and half the size, so a channel block takes R * (floor(S / 2) * 128 + (S odd) * 64) rows.
 template <typename T, int EPC>
 __global__ void repack_filters_kernel(const T* __restrict__ w, T* __restrict__ wp, unsigned* __restrict__ status,
                                       int K, FoldedFilter ff, int taps, int n_tile, int cblks, long long threads_total,
@@ -62,6 +64,32 @@ __global__ void repack_filters_kernel(const T* __restrict__ w, T* __restrict__ w
         T* dst = wp + ((((size_t)nb * cblks + cb) * taps * kChunks + chunk) * n_tile + f) * EPC + e;
         const size_t tap_stride = (size_t)kChunks * n_tile * EPC;
         const bool live = k < K && (folded ? vc < ff.C * ff.fold_r * ff.fold_s : vc < ff.C);
+        if (stacked == 2) {
+            // compact bank of one filter block: per filter row `pairs` slices of 128 rows, then the lone tap's 64 rows
+            const int pairs = ff.S / 2, odd = ff.S & 1;
+            const size_t row_elems = (size_t)(pairs * n_tile + odd * (n_tile / 2)) * kChunks * EPC;
+            T* base = wp + (size_t)cb * ff.R * row_elems;
+            const bool chan = vc < ff.C;
+            for (int r = 0; r < ff.R; ++r, base += row_elems) {
+                for (int u = 0; u < pairs; ++u) {
+                    T v = T(0);
+                    if (k < K && chan) {
+                        v = __ldg(src + (vc * ff.R + r) * ff.S + 2 * u + upper);
+                        if (sizeof(T) == 4) v = (T)to_tf32_rna((float)v);
+                    }
+                    base[((size_t)(u * kChunks + chunk) * n_tile + f) * EPC + e] = v;
+                }
+                if (odd && f < n_tile / 2) {           // natural order: row f is filter f
+                    T v = T(0);
+                    if (f < K && chan) {
+                        v = __ldg(w + ((size_t)f * ff.C * ff.R + (size_t)vc * ff.R + r) * ff.S + ff.S - 1);
+                        if (sizeof(T) == 4) v = (T)to_tf32_rna((float)v);
+                    }
+                    base[(size_t)pairs * kChunks * n_tile * EPC + ((size_t)chunk * (n_tile / 2) + f) * EPC + e] = v;
+                }
+            }
+            continue;
+        }
         for (int t = 0; t < taps; ++t, dst += tap_stride) {
             T v = T(0);
             if (live) {

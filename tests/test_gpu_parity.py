@@ -383,3 +383,42 @@ def test_stacked_taps_for_few_filters(oracle, monkeypatch, dims, entry):
     y_plain = run_library(x, w, entry=entry, algo=ALGO_TF32)
     assert_parity(y_plain, y_ref, yabs, tol, f"unstacked {entry} {dims}")
     assert_parity(y_stacked, y_plain.astype(np.float64), yabs, 2e-5, f"stacked vs unstacked {entry} {dims}")
+
+
+COMPACT_STACK_SHAPES = [
+    # N, C, H, W, K, R, S      (at most 64 filters and a bank that stays in shared memory: pairs of taps as 128-row
+    #                           slices, a lone last tap of a row as a 64-row slice issued as M = 64)
+    (2, 64, 20, 20, 64, 3, 3),       # the early-layer benchmark shape in small: 4 channel blocks, lone third tap
+    (2, 16, 10, 10, 64, 3, 2),       # even taps per row: pairs only
+    (2, 8, 30, 30, 16, 3, 3),        # half a channel block, 16 filters: one lane quarter's worth
+    (3, 20, 15, 17, 40, 3, 3),       # odd image width, 40 filters, partial second channel block
+    (1, 16, 12, 40, 64, 1, 3),       # a single row of taps
+    (1, 8, 9, 9, 24, 5, 5),          # two pairs and a lone tap per row
+    (5, 32, 24, 24, 64, 3, 3),       # several items per block
+]
+
+
+@pytest.mark.parametrize("dims", COMPACT_STACK_SHAPES)
+@pytest.mark.parametrize("entry", ["general", "bf16"])
+def test_compact_stacked_taps(oracle, monkeypatch, dims, entry):
+    """Exact on integers, within tolerance, and equal (up to summation order) to the unstacked kernel."""
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K, R, S = dims
+    algo_q = ALGO_TF32 if entry == "general" else 3
+    monkeypatch.setenv("CONV2D_B200_TF32_PAIR_COMPACT", "1")       # (measured slower on the benchmark shape: off by default)
+    assert lib.conv2d_fwd_plan_describe(*dims, algo_q).get("stacked_compact") == 1, "meant to take compact stacking"
+    xi, wi = small_integers((N, C, H, W), 481), small_integers((K, C, R, S), 482)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry=entry, algo=ALGO_TF32).astype(np.float64), yi_ref)
+    x, w = uniform((N, C, H, W), 483), uniform((K, C, R, S), 484)
+    if entry == "bf16":
+        from helpers import bf16_values
+        x, w = bf16_values(x)[0], bf16_values(w)[0]
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    tol = TF32_TOL if entry == "general" else 1e-5
+    y_compact = run_library(x, w, entry=entry, algo=ALGO_TF32)
+    assert_parity(y_compact, y_ref, yabs, tol, f"compact stacking {entry} {dims}")
+    monkeypatch.setenv("CONV2D_B200_TF32_PAIR_COMPACT", "0")
+    monkeypatch.setenv("CONV2D_B200_TF32_PAIR_TAPS", "0")
+    y_plain = run_library(x, w, entry=entry, algo=ALGO_TF32)
+    assert_parity(y_compact, y_plain.astype(np.float64), yabs, 2e-5, f"compact vs unstacked {entry} {dims}")
