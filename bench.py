@@ -206,7 +206,7 @@ GENERAL_COLS = ["us_cold", "us_cold_after_flush", "us_warm", "us_warm_prepacked"
 L2_BYTES = 126 * 1024 * 1024
 
 
-def bench_general(torch, lib, peaks, flush, sampler, detail):
+def bench_general(torch, lib, peaks, flush, sampler, detail, with_sustained=True):
     """Times every general-case configuration: tensor cores on fp32 (TF32) and bf16 inputs, and the fp32 kernel.
 
     Per (configuration, algorithm) one row of GENERAL_COLS.  All times are complete calls (filter re-ordering
@@ -287,7 +287,10 @@ def bench_general(torch, lib, peaks, flush, sampler, detail):
             del xs, ys
             warm = event_ms(call, torch, iters=20)
             packed = event_ms(lambda: call(lib.FLAG_WEIGHTS_PACKED), torch, iters=20) if tensor_core else None
-            sust, sust_mhz, sust_iters = sustained_ms(call, torch, sampler, 1.0 if algo_name != "ffma" else 0.3)
+            if with_sustained:
+                sust, sust_mhz, sust_iters = sustained_ms(call, torch, sampler, 1.0 if algo_name != "ffma" else 0.3)
+            else:
+                sust, sust_mhz, sust_iters = warm, None, 0
             lib.conv2d_get_status(ws.data_ptr(), stream)
             t_flush = statistics.median(cold)
             t_cold = t_rot
@@ -559,7 +562,7 @@ def main():
             result["sustained"]["hbm_frac_of_measured"] = algorithmic_bytes / (sust * 1e-3) / 1e9 / peaks["hbm_gbs"]
         if not args.no_general:
             result["cfg1"] = bench_cfg1(torch, lib)
-            result["general"] = bench_general(torch, lib, peaks, flush, sampler2, detail)
+            result["general"] = bench_general(torch, lib, peaks, flush, sampler2, detail, not args.no_sustained)
         sampler2.stop()
         if not args.no_cpu_baseline:
             result["cpu_baseline"] = time_oracle_sample(cfg, 12.0)

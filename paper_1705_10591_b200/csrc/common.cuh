@@ -122,10 +122,10 @@ conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, co
 
 // 1 x 1 filters with every operand moved by tensor-map (TMA) copies; `workspace` only holds the status block.
 // CONV2D_ERR_UNSUPPORTED when the shape or its alignment has no such instance (the caller then takes the general kernel).
-bool pointwise_tma_supported(const Shape& sh);
-conv2d_status_t launch_pointwise_tma(const float* x, const float* w, float* y, const Shape& sh,
+bool pointwise_tma_supported(const Shape& sh, bool b16);
+conv2d_status_t launch_pointwise_tma(const void* x, const void* w, float* y, const Shape& sh, bool b16, bool fp16,
                                      void* workspace, size_t workspace_bytes, cudaStream_t stream);
-int describe_pointwise_tma_plan(const Shape& sh, char* text, size_t text_bytes);   // -1: no such instance
+int describe_pointwise_tma_plan(const Shape& sh, bool b16, char* text, size_t text_bytes);   // -1: no such instance
 
 // Text description of the tensor-core plan of a shape (snprintf semantics: returns the length it needs).
 int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text_bytes);

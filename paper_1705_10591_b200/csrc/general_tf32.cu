@@ -60,7 +60,7 @@ namespace conv2d_b200 {
 
 bool tf32_supported(const Shape& sh)
 {
-    return make_plan(sh).ok || pointwise_tma_supported(sh);
+    return make_plan(sh).ok || pointwise_tma_supported(sh, false);
 }
 
 size_t tf32_workspace_bytes(const Shape& sh)
@@ -72,7 +72,7 @@ size_t tf32_workspace_bytes(const Shape& sh)
 
 bool b16_supported(const Shape& sh)
 {
-    return make_plan(sh, true).ok;
+    return make_plan(sh, true).ok || pointwise_tma_supported(sh, true);
 }
 
 size_t b16_workspace_bytes(const Shape& sh)
@@ -88,8 +88,8 @@ size_t b16_workspace_bytes(const Shape& sh)
 // (this also counts filter rows, channels and stacked taps that are zero padding).
 int describe_tensor_core_plan(const Shape& sh, bool b16, char* text, size_t text_bytes)
 {
-    if (!b16) {
-        const int n = describe_pointwise_tma_plan(sh, text, text_bytes);
+    {
+        const int n = describe_pointwise_tma_plan(sh, b16, text, text_bytes);
         if (n >= 0) return n;
     }
     const Plan p = make_plan(sh, b16);
@@ -120,9 +120,9 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
 {
     const float* x = static_cast<const float*>(x_any);   // 16-bit operands: re-read as such inside the kernel
     const float* w = static_cast<const float*>(w_any);
-    if (!b16) {
+    {
         // 1 x 1 filters on suitably aligned tensors: the kernel whose operands and output all move by tensor-map copies
-        const conv2d_status_t st = launch_pointwise_tma(x, w, y, sh, workspace, workspace_bytes, stream);
+        const conv2d_status_t st = launch_pointwise_tma(x_any, w_any, y, sh, b16, fp16, workspace, workspace_bytes, stream);
         if (st != CONV2D_ERR_UNSUPPORTED) return st;
     }
     const Plan p = make_plan(sh, b16);

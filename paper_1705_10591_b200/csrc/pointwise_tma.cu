@@ -1,4 +1,5 @@
-// General case with 1 x 1 filters on the tcgen05 tensor cores, every operand and the output moved by tiled TMA
+// General case with 1 x 1 filters on the tcgen05 tensor cores (fp32 inputs as TF32, or bf16 / fp16 inputs), every
+// operand and the output moved by tiled TMA
 // copies (the staging and the prefetch of Algorithm 2, lines 4-5 and 8-9, done by the copy engine; its write-back,
 // line 20, as well).
 //
@@ -18,6 +19,7 @@
 //   * Output: accumulators (lanes = filters, columns = pixels) go tensor memory -> registers -> a swizzled
 //     32-filter x 32-pixel shared-memory tile per warp -> one tensor-map store per tile.  Out-of-range rows and
 //     pixels are clipped by the copy engine, so ragged images and filter counts need no predicates.
+// (16-bit operands: 64 pixels or channels per 128-byte row, K steps of 16, the ordinary 128-byte swizzle on both operands.)
 // The tensor core reads fp32 bits as TF32 by dropping the low 13 mantissa bits, so on this path both operands are
 // truncated, not rounded: |error| <= (2^-10 + 2^-10 + 2^-20) * sum|x*w| plus fp32 accumulation over at most 256
 // channels, (C + 1) * 2^-24 * sum|x*w|: below 1.97e-3 * sum|x*w|, inside the 2e-3 bound of CONV2D_ALGO_TF32.
@@ -42,39 +44,51 @@ using namespace ptx;
 
 constexpr int kPwThreads = 320;           // warp 0: loads, warp 1: MMAs, warps 2-9: write-back
 constexpr int kPwEpiWarps = 8;
-constexpr int kAtomPx = 32;               // pixels per 128-byte row of a swizzle atom
-constexpr int kStageCh = 32;              // channels per activation stage: four K steps of 8
-constexpr int kAtomBytes = kAtomPx * kStageCh * 4;     // one box of 32 pixels x 32 channels
-constexpr int kMaxAtoms = 8;              // atoms per work item: N <= 256 columns per MMA
 constexpr int kPwMaxStages = 8;
 constexpr int kAccCols = 256;             // tensor-memory columns of one accumulator set
-constexpr int kMaxChannels = 256;         // the filter bank of a block must stay resident
-constexpr int kMaxChunks = kMaxChannels / kStageCh;
+constexpr int kMaxChunks = 8;             // 128-byte channel chunks of the resident filter bank (at most 128 KB)
+
+// Sizes that depend on the operand type: fp32 (read by the tensor core as TF32) or a 16-bit float.  A 128-byte row
+// holds 32 or 64 elements; a stage holds four K steps (of 8 or 16 channels) for all pixels of a work item.
+template <bool B16>
+struct Geom {
+    static constexpr int kElem = B16 ? 2 : 4;
+    static constexpr int kAtomPx = 128 / kElem;            // pixels per 128-byte row of a swizzle atom
+    static constexpr int kKStep = B16 ? 16 : 8;            // channels per MMA
+    static constexpr int kStageCh = 4 * kKStep;            // channels per activation stage = per 128-byte filter row
+    static constexpr int kAtomBytes = 128 * kStageCh;      // one box of kAtomPx pixels x kStageCh channels
+    static constexpr int kMaxAtoms = kAccCols / kAtomPx;   // atoms per work item: N <= 256 columns per MMA
+    static constexpr int kMaxChannels = kMaxChunks * kStageCh;   // the filter bank of a block must stay resident
+};
 constexpr size_t kPwSmemLimit = 227 * 1024;
 constexpr size_t kPwBookBytes = 512;      // barriers, tensor-memory slot, abort flag
 
 struct PwArgs {
     unsigned* status;
     int K;
-    int apb;             // atoms per image: ceil(HW / 32)
+    int fp16;            // 16-bit operands only: 1 = IEEE half, 0 = bf16
+    int apb;             // atoms per image: ceil(HW / pixels per atom)
     int total_atoms;     // N * apb
     int a_item;          // atoms per work item
     int tiles;           // work items along the pixels
     int n_blocks;        // filter blocks of m_rows filters
     int m_rows;          // rows of the M operand: 64 (at most 64 filters) or 128
     int items;           // tiles * n_blocks, numbered filter block-major
-    int cchunks;         // 32-channel chunks: ceil(C / 32)
-    int ksteps;          // K steps of 8 channels: ceil(C / 8)
+    int cchunks;         // channel chunks of one stage each: ceil(C / channels per stage)
+    int ksteps;          // K steps: ceil(C / channels per MMA)
     int stages;          // activation ring depth
     unsigned max_polls;  // bound of every barrier wait
     int test_drop_stage; // test hook: the activation stage with this ordinal is armed but never copied (-1: none)
     FastDiv div_apb, div_tiles;
 };
 
+template <bool B16>
 __global__ void __launch_bounds__(kPwThreads, 1)
 pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                      const __grid_constant__ CUtensorMap map_y, const PwArgs a)
 {
+    using G = Geom<B16>;
+    constexpr int kAtomPx = G::kAtomPx, kStageCh = G::kStageCh, kAtomBytes = G::kAtomBytes;
     extern __shared__ unsigned char smem_raw[];
     // swizzle atoms must start on 1024 bytes
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -191,7 +205,8 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 cur_nb = nb;
                 if (!mbar_wait_bounded(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                 tc_fence_after_sync();
-                const uint32_t idesc = idesc_tf32((uint32_t)a.m_rows, (uint32_t)(atoms * kAtomPx)) | kIdescBMajorMN;
+                const uint32_t idesc = (B16 ? idesc_b16((uint32_t)a.m_rows, (uint32_t)(atoms * kAtomPx), a.fp16 != 0)
+                                            : idesc_tf32((uint32_t)a.m_rows, (uint32_t)(atoms * kAtomPx))) | kIdescBMajorMN;
                 const uint32_t d = tmem + (uint32_t)(buf * kAccCols);
                 bool accumulate = false;
                 for (int st = 0; st < a.cchunks && alive; ++st) {
@@ -200,11 +215,14 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     tc_fence_after_sync();
                     const uint32_t a_chunk = a_base + (uint32_t)st * a_chunk_bytes;
                     const uint32_t b_stage = b_base + (uint32_t)slot * b_stage_bytes;
-                    const int ks = min(kStageCh / 8, a.ksteps - st * (kStageCh / 8));
+                    const int ks = min(4, a.ksteps - st * 4);
                     for (int kk = 0; kk < ks; ++kk) {
-                        // filters: 32 bytes further inside the 128-byte rows; pixels: the next atom of 8 channel rows
-                        mma_tf32(d, smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u),
-                                 smem_desc_mn_sw128_32b(b_stage + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u), idesc, accumulate);
+                        // filters: 32 bytes further inside the 128-byte rows; pixels: the next 8 (fp32) or 16 (16-bit) channel rows
+                        const uint64_t a_desc = smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u);
+                        if (B16)
+                            mma_b16(d, a_desc, smem_desc_sw128(b_stage + (uint32_t)kk * 2048u, (uint32_t)kStageCh * 128u, 1024u), idesc, accumulate);
+                        else
+                            mma_tf32(d, a_desc, smem_desc_mn_sw128_32b(b_stage + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u), idesc, accumulate);
                         accumulate = true;
                     }
                     mma_commit(&b_empty[slot]);
@@ -244,9 +262,10 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             tc_fence_after_sync();
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccCols);
             const int k0 = nb * a.m_rows + quarter * rows_q;
-            for (int i = half; i < atoms; i += 2) {
+            constexpr int kBpa = kAtomPx / 32;                  // 32-column blocks per atom
+            for (int i = half; i < atoms * kBpa; i += 2) {
                 uint32_t v[32];
-                tmem_ld32(lane_base + (uint32_t)(i * kAtomPx), v);
+                tmem_ld32(lane_base + (uint32_t)(i * 32), v);
                 tmem_ld_wait();
                 if (lane == 0) bulk_wait_group_read<0>();       // the previous store has read the tile
                 __syncwarp();
@@ -261,8 +280,8 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 __syncwarp();
                 if (lane == 0 && k0 < a.K) {
                     int blk;
-                    const int n = a.div_apb.divmod(first + i, blk);
-                    tma_store_3d(&map_y, blk * kAtomPx, k0, n, tile);
+                    const int n = a.div_apb.divmod(first + i / kBpa, blk);
+                    tma_store_3d(&map_y, blk * kAtomPx + (i % kBpa) * 32, k0, n, tile);
                     bulk_commit_group();
                 }
             }
@@ -299,15 +318,15 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// fp32 tensor of `rank` dimensions (innermost first), zeros for out-of-range elements.  `swizzle`: 128-byte rows
+// Tensor of `rank` dimensions (innermost first), zeros for out-of-range elements.  `swizzle`: 128-byte rows
 // with 16-byte chunks swizzled (K-major operands, output tiles) or with 32-byte chunks (the MN-major TF32 operand).
-bool encode_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
-                const cuuint32_t* box, CUtensorMapSwizzle swizzle)
+bool encode_map(CUtensorMap* map, CUtensorMapDataType type, const void* base, int rank, const cuuint64_t* dims,
+                const cuuint64_t* strides_bytes, const cuuint32_t* box, CUtensorMapSwizzle swizzle)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint32_t ones[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, ones,
+    return fn(map, type, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, ones,
               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -319,33 +338,36 @@ struct PwPlan {
     size_t smem_bytes;
 };
 
+template <bool B16>
 PwPlan make_pw_plan(const Shape& sh)
 {
+    using G = Geom<B16>;
     PwPlan p{};
     p.ok = false;
     if (sh.R != 1 || sh.S != 1 || sh.pad_h || sh.pad_w) return p;
     const long long HW = (long long)sh.H * sh.W;
     // tensor-map strides are multiples of 16 bytes; the filter bank of a block stays in shared memory
-    if (HW % 4 != 0 || sh.C % 4 != 0 || sh.C > kMaxChannels) return p;
+    constexpr int kPer16 = 16 / G::kElem;
+    if (HW % kPer16 != 0 || sh.C % kPer16 != 0 || sh.C > G::kMaxChannels) return p;
     if (env_int("CONV2D_B200_TF32_TMA", 1) == 0) return p;
     p.m_rows = sh.K <= 64 ? 64 : 128;
     p.n_blocks = (sh.K + p.m_rows - 1) / p.m_rows;
-    p.apb = (int)((HW + kAtomPx - 1) / kAtomPx);
+    p.apb = (int)((HW + G::kAtomPx - 1) / G::kAtomPx);
     p.total_atoms = (long long)sh.N * p.apb;
     if (p.total_atoms > 0x3fffffffLL) return p;
-    p.cchunks = (sh.C + kStageCh - 1) / kStageCh;
+    p.cchunks = (sh.C + G::kStageCh - 1) / G::kStageCh;
     const int sms = sm_count();
     // Atoms per item: the fewest rounds of items over the SMs, counted in atoms, plus half an atom of fixed cost per
-    // item; ties go to the larger item (wider MMAs).  64 x 32 x 32 pixels = 2048 atoms: 7 per item = 293 items = two
-    // rounds of 7, where 8 per item would be two rounds of 8.
+    // item; ties go to the larger item (wider MMAs).  64 x 32 x 32 pixels = 2048 atoms of 32: 7 per item = 293 items =
+    // two rounds of 7, where 8 per item would be two rounds of 8.
     double best = 0;
     p.a_item = 0;
     const int forced = env_int("CONV2D_B200_TMA_ATOMS", 0);
-    for (int at = kMaxAtoms; at >= 1; --at) {
-        if (forced ? at != forced : false) continue;
+    for (int at = G::kMaxAtoms; at >= 1; --at) {
+        if (forced && at != (forced < G::kMaxAtoms ? forced : G::kMaxAtoms)) continue;
         const long long tiles = (p.total_atoms + at - 1) / at;
         const long long rounds = (tiles * p.n_blocks + sms - 1) / sms;
-        const double cost = (double)rounds * (at + 0.5);
+        const double cost = (double)rounds * (at + 0.5 * 32 / G::kAtomPx);
         if (p.a_item == 0 || cost < best - 1e-9) { best = cost; p.a_item = at; }
     }
     if (p.a_item == 0) return p;
@@ -353,7 +375,7 @@ PwPlan make_pw_plan(const Shape& sh)
     const long long items = (long long)p.tiles * p.n_blocks;
     if (items > 0x7fffffffLL) return p;
     const size_t fixed = (size_t)p.cchunks * p.m_rows * 128 + (size_t)kPwEpiWarps * 4096 + kPwBookBytes + 1024;
-    const size_t stage = (size_t)p.a_item * kAtomBytes;
+    const size_t stage = (size_t)p.a_item * G::kAtomBytes;
     if (fixed + 2 * stage > kPwSmemLimit) return p;
     p.stages = (int)((kPwSmemLimit - fixed) / stage);
     if (p.stages > kPwMaxStages) p.stages = kPwMaxStages;
@@ -366,70 +388,97 @@ PwPlan make_pw_plan(const Shape& sh)
     return p;
 }
 
-}  // namespace
-
-bool pointwise_tma_supported(const Shape& sh) { return make_pw_plan(sh).ok; }
-
-int describe_pointwise_tma_plan(const Shape& sh, char* text, size_t text_bytes)
+template <bool B16>
+int describe_pw(const Shape& sh, char* text, size_t text_bytes)
 {
-    const PwPlan p = make_pw_plan(sh);
+    using G = Geom<B16>;
+    const PwPlan p = make_pw_plan<B16>(sh);
     if (!p.ok) return -1;
     const double px = (double)sh.N * sh.H * sh.W;
-    const double cols = (double)p.total_atoms * kAtomPx;
-    const double issued = 2.0 * p.m_rows * p.n_blocks * cols * ((sh.C + 7) / 8 * 8);
+    const double cols = (double)p.total_atoms * G::kAtomPx;
+    const double issued = 2.0 * p.m_rows * p.n_blocks * cols * ((sh.C + G::kKStep - 1) / G::kKStep * G::kKStep);
     return snprintf(text, text_bytes,
                     "tensor_core=1 kernel=pointwise_tma addressing=atoms filters_as=M m_rows=%d tile_px=%d acc_sets=2 items=%lld "
                     "grid=%d stages=%d resident_filters=1 smem_bytes=%zu mma_useful_px=%.4f mma_useful_flops=%.4f",
-                    p.m_rows, p.a_item * kAtomPx, (long long)p.tiles * p.n_blocks, p.grid, p.stages, p.smem_bytes,
+                    p.m_rows, p.a_item * G::kAtomPx, (long long)p.tiles * p.n_blocks, p.grid, p.stages, p.smem_bytes,
                     px / cols, 2.0 * px * sh.K * sh.C / issued);
 }
 
-conv2d_status_t launch_pointwise_tma(const float* x, const float* w, float* y, const Shape& sh,
-                                     void* workspace, size_t workspace_bytes, cudaStream_t stream)
+template <bool B16>
+conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& sh, bool fp16,
+                          void* workspace, size_t workspace_bytes, cudaStream_t stream)
 {
-    const PwPlan p = make_pw_plan(sh);
+    using G = Geom<B16>;
+    const PwPlan p = make_pw_plan<B16>(sh);
     if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < kStatusBytes) return CONV2D_ERR_WORKSPACE;
     const cuuint64_t HW = (cuuint64_t)sh.H * sh.W;
+    const cuuint64_t es = G::kElem;
+    const CUtensorMapDataType in_type = !B16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                      : (fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     CUtensorMap map_w, map_x, map_y;
     {
         const cuuint64_t dims[2] = {(cuuint64_t)sh.C, (cuuint64_t)sh.K};
-        const cuuint64_t strides[1] = {(cuuint64_t)sh.C * 4};
-        const cuuint32_t box[2] = {(cuuint32_t)kStageCh, (cuuint32_t)p.m_rows};
-        if (!encode_map(&map_w, w, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return CONV2D_ERR_UNSUPPORTED;
+        const cuuint64_t strides[1] = {(cuuint64_t)sh.C * es};
+        const cuuint32_t box[2] = {(cuuint32_t)G::kStageCh, (cuuint32_t)p.m_rows};
+        if (!encode_map(&map_w, in_type, w, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return CONV2D_ERR_UNSUPPORTED;
     }
     {
+        // pixels contiguous: the MN-major operand; 4-byte elements need the 32-byte-atom flavour of the 128-byte swizzle
         const cuuint64_t dims[3] = {HW, (cuuint64_t)sh.C, (cuuint64_t)sh.N};
-        const cuuint64_t strides[2] = {HW * 4, HW * 4 * (cuuint64_t)sh.C};
-        const cuuint32_t box[3] = {(cuuint32_t)kAtomPx, (cuuint32_t)kStageCh, 1};
-        if (!encode_map(&map_x, x, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) return CONV2D_ERR_UNSUPPORTED;
+        const cuuint64_t strides[2] = {HW * es, HW * es * (cuuint64_t)sh.C};
+        const cuuint32_t box[3] = {(cuuint32_t)G::kAtomPx, (cuuint32_t)G::kStageCh, 1};
+        if (!encode_map(&map_x, in_type, x, 3, dims, strides, box,
+                        B16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+            return CONV2D_ERR_UNSUPPORTED;
     }
     {
         const cuuint64_t dims[3] = {HW, (cuuint64_t)sh.K, (cuuint64_t)sh.N};
         const cuuint64_t strides[2] = {HW * 4, HW * 4 * (cuuint64_t)sh.K};
-        const cuuint32_t box[3] = {(cuuint32_t)kAtomPx, (cuuint32_t)(p.m_rows / 4), 1};
-        if (!encode_map(&map_y, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return CONV2D_ERR_UNSUPPORTED;
+        const cuuint32_t box[3] = {32u, (cuuint32_t)(p.m_rows / 4), 1};
+        if (!encode_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+            return CONV2D_ERR_UNSUPPORTED;
     }
     static size_t smem_done[64] = {};
-    if (raise_smem_limit(reinterpret_cast<const void*>(pointwise_tma_kernel), p.smem_bytes, smem_done) != cudaSuccess)
+    if (raise_smem_limit(reinterpret_cast<const void*>(pointwise_tma_kernel<B16>), p.smem_bytes, smem_done) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     PwArgs a{};
     a.status = static_cast<unsigned*>(workspace);
     a.K = sh.K;
+    a.fp16 = fp16 ? 1 : 0;
     a.apb = p.apb; a.total_atoms = (int)p.total_atoms; a.a_item = p.a_item; a.tiles = p.tiles;
     a.n_blocks = p.n_blocks; a.m_rows = p.m_rows; a.items = p.tiles * p.n_blocks;
-    a.cchunks = p.cchunks; a.ksteps = (sh.C + 7) / 8; a.stages = p.stages;
+    a.cchunks = p.cchunks; a.ksteps = (sh.C + G::kKStep - 1) / G::kKStep; a.stages = p.stages;
     a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
     a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
     a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles);
     if (env_int("CONV2D_B200_TF32_VERBOSE", 0) != 0)
-        fprintf(stderr, "conv2d plan: pointwise_tma m_rows %d n_blocks %d atoms/item %d tiles %d stages %d grid %d smem %zu\n",
-                p.m_rows, p.n_blocks, p.a_item, p.tiles, p.stages, p.grid, p.smem_bytes);
-    if (launch_pdl(pointwise_tma_kernel, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
+        fprintf(stderr, "conv2d plan: pointwise_tma%s m_rows %d n_blocks %d atoms/item %d tiles %d stages %d grid %d smem %zu\n",
+                B16 ? " (16-bit)" : "", p.m_rows, p.n_blocks, p.a_item, p.tiles, p.stages, p.grid, p.smem_bytes);
+    if (launch_pdl(pointwise_tma_kernel<B16>, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
                    map_w, map_x, map_y, a) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;
+}
+
+}  // namespace
+
+bool pointwise_tma_supported(const Shape& sh, bool b16)
+{
+    return b16 ? make_pw_plan<true>(sh).ok : make_pw_plan<false>(sh).ok;
+}
+
+int describe_pointwise_tma_plan(const Shape& sh, bool b16, char* text, size_t text_bytes)
+{
+    return b16 ? describe_pw<true>(sh, text, text_bytes) : describe_pw<false>(sh, text, text_bytes);
+}
+
+conv2d_status_t launch_pointwise_tma(const void* x, const void* w, float* y, const Shape& sh, bool b16, bool fp16,
+                                     void* workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    return b16 ? launch_pw<true>(x, w, y, sh, fp16, workspace, workspace_bytes, stream)
+               : launch_pw<false>(x, w, y, sh, false, workspace, workspace_bytes, stream);
 }
 
 }  // namespace conv2d_b200

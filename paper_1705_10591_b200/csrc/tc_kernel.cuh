@@ -898,16 +898,22 @@ general_tc_kernel(const KernelArgs a)
                 const int b_step = split ? 3 : 1;
                 int b = split ? share : 0;
                 if (b < blocks) load_block(va0, va1, vax, b);
+                long long t_ld = 0;       // (diagnostics build: cycles spent waiting for tensor-memory loads)
                 while (b < blocks) {
+                    long long t0 = clock_now();
                     tmem_ld_wait();
+                    t_ld += clock_now() - t0;
                     if (b + b_step < blocks) load_block(vb0, vb1, vbx, b + b_step);
                     store_block(va0, va1, vax, b);
                     if ((b += b_step) >= blocks) break;
+                    t0 = clock_now();
                     tmem_ld_wait();
+                    t_ld += clock_now() - t0;
                     if (b + b_step < blocks) load_block(va0, va1, vax, b + b_step);
                     store_block(vb0, vb1, vbx, b);
                     b += b_step;
                 }
+                if (kDiag && blockIdx.x == 0 && warp == 4 && lane == 0) a.status[12] += (unsigned)t_ld;
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0 && !helper) mbar_arrive(&acc_empty[buf]);

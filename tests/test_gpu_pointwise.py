@@ -105,3 +105,31 @@ def test_pointwise_expired_wait_is_reported(oracle, monkeypatch):
     monkeypatch.delenv("CONV2D_B200_TF32_TEST_DROP_STAGE")
     y_ref, yabs = oracle.conv2d_oracle(x, w)
     assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, "after a time-out")
+
+
+SHAPES_16BIT = [
+    # N, C, H, W, K      (16-bit operands: 64 pixels per atom, 64 channels per stage, K steps of 16)
+    (2, 32, 8, 8, 16),          # one atom per image, half a stage of channels, 64-row operand
+    (1, 64, 12, 10, 200),       # HW = 120: second atom holds 56 pixels; two filter blocks
+    (5, 104, 10, 16, 64),       # C = 104: second stage holds 40 channels (2.5 MMA steps: zero-filled rows)
+    (4, 512, 8, 8, 300),        # most channels the resident bank takes; three filter blocks
+    (3, 128, 32, 32, 128),      # the benchmark's per-image shape
+    (40, 16, 20, 24, 24),       # 320 atoms: several rounds of items per block
+]
+
+
+@pytest.mark.parametrize("kind", ["bf16", "fp16"])
+@pytest.mark.parametrize("dims", SHAPES_16BIT)
+def test_pointwise_16bit_operands(oracle, dims, kind):
+    import paper_1705_10591_b200 as lib
+    from helpers import B16_TOL, bf16_values, fp16_values
+    N, C, H, W, K = dims
+    assert lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, 3).get("kernel") == "pointwise_tma"
+    xi, wi = small_integers((N, C, H, W), 981), small_integers((K, C, 1, 1), 982)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry=kind).astype(np.float64), yi_ref)
+    conv = bf16_values if kind == "bf16" else fp16_values
+    x, w = conv(uniform((N, C, H, W), 983))[0], conv(uniform((K, C, 1, 1), 984))[0]
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    r = assert_parity(run_library(x, w, entry=kind), y_ref, yabs, B16_TOL, f"pointwise {kind} {dims}")
+    print(f"pointwise {kind} {dims} max ratio {r:.3e}")
