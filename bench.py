@@ -200,9 +200,8 @@ def sustained_ms(fn, torch, sampler, seconds=1.0):
     return ms, mhz, iters
 
 
-GENERAL_COLS = ["us_cold", "us_cold_after_flush", "us_warm", "us_warm_prepacked", "frac_cold", "frac_warm_prepacked",
-                "frac_cold_of_nominal", "us_sustained_1s", "mhz_sustained", "frac_sustained",
-                "mma_useful_px", "mma_useful_flops"]
+GENERAL_COLS = ["us_cold", "us_cold_flushed", "us_warm", "us_warm_prepacked", "frac_cold", "frac_warm_prepacked",
+                "frac_cold_nominal", "us_sustained", "mhz_sustained", "frac_sustained", "useful_px", "useful_flops"]
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -215,10 +214,10 @@ def bench_general(torch, lib, peaks, flush, sampler, detail, with_sustained=True
                          to exceed twice the 126 MB L2, so no call finds its image in L2 and every call evicts an
                          earlier call's output: DRAM traffic per call = the algorithmic bytes.  `frac_cold` is the
                          roofline fraction of this time.
-      us_cold_after_flush  one call after a 256 MB fill: L2 then holds only dirty lines of the fill, so every line
+      us_cold_flushed    one call after a 256 MB fill: L2 then holds only dirty lines of the fill, so every line
                          the call brings in also costs a write-back that is not the call's own traffic
       us_warm, us_warm_prepacked   same buffers back to back (L2 resident); with the filters already re-ordered
-      us_sustained_1s    at least one second of back-to-back calls, SM clock sampled during the loop
+      us_sustained       at least one second of back-to-back calls, SM clock sampled during the loop
     """
     rows = {}
     dev = torch.device("cuda")
@@ -315,16 +314,15 @@ def bench_general(torch, lib, peaks, flush, sampler, detail, with_sustained=True
                    roof_ms(pipe_peak) / t_cold, roof_ms(pipe_peak) / packed if packed else None,
                    roof_ms(pipe_nominal, t_hbm_nominal) / t_cold, sust * 1e3, sust_mhz, roof_ms(pipe_sustained) / sust,
                    plan.get("mma_useful_px"), plan.get("mma_useful_flops")]
-            rows[name][algo_name] = [sig(v) for v in row]
+            rows[name][algo_name] = [sig(v, 3) if i in (5, 6, 8, 9, 10, 11) else sig(v) for i, v in enumerate(row)]
             detail.append({"workload": name, "algo": algo_name, "bound": bound, "cold_after_flush_us_all": [sig(c * 1e3) for c in cold], "rotating_sets": n_sets,
                            "sustained_iters": sust_iters, "pipe_peak_tflops": pipe_peak, "pipe_nominal_tflops": pipe_nominal,
                            "pipe_sustained_tflops": pipe_sustained, "t_hbm_us": sig(t_hbm * 1e3), "plan": plan,
                            "gflops_cold": sig(cfg.flops / t_cold / 1e6)})
         del xd, wd, yd, xd16, wd16
     return {"cols": GENERAL_COLS, "rows": rows,
-            "peaks": {"tf32": "bf16 burst/2", "bf16": "bf16 burst", "ffma": "148x128x2x1.965GHz", "hbm": peaks["hbm_gbs"],
-                      "nominal": "1125 tf32 / 2250 bf16 TFLOP/s, 8 TB/s", "sustained": "bf16_tflops_sustained (/2 for tf32)",
-                      "source": peaks["source"]}}
+            "peaks": {"tf32": "bf16/2", "ffma": "148x128x2x1.965GHz", "nominal": "1125/2250 TF, 8 TB/s",
+                      "sustained": "bf16_sustained(/2)", "source": peaks["source"]}}
 
 
 def bench_cfg1(torch, lib):
@@ -523,8 +521,7 @@ def main():
         "hbm_gbs_achieved": algorithmic_bytes / t_kernel_s / 1e9,
         "hbm_frac_of_measured": algorithmic_bytes / t_kernel_s / 1e9 / peaks["hbm_gbs"],
         "hbm_frac_of_nominal_8tbs": algorithmic_bytes / t_kernel_s / 1e9 / 8000.0,
-        "alu_tflops_achieved": cfg.flops / t_kernel_s / 1e12,
-        "alu_frac_at_max_clock": cfg.flops / t_kernel_s / 1e12 / fp32_peak,
+        "tflops_achieved": cfg.flops / t_kernel_s / 1e12,
     })
     if not (single or ffma):
         nominal = NOMINAL_BF16_TFLOPS if b16 else NOMINAL_TF32_TFLOPS
