@@ -67,3 +67,71 @@ def test_the_random_shapes_reach_the_planner_branches():
     assert any(R == 1 and S == 1 for (*_, R, S) in SHAPES)
     assert any(C >= 64 for (_, C, _, _, _, _, _) in SHAPES)
     assert len(SHAPES) >= 60
+
+
+def _draw_pointwise(seed):
+    """A 1 x 1 shape the kernel fed by tensor-map copies takes: H*W and C multiples of 8 (so that both operand
+    types qualify), at most 256 channels."""
+    u = uniform((8,), 9500 + seed, 0.0, 1.0)
+
+    def log_int(t, lo, hi):
+        return int(round(lo * (hi / lo) ** float(t)))
+
+    N = log_int(u[0], 1, 24)
+    C = 8 * log_int(u[1], 1, 32)
+    H = log_int(u[2], 1, 40)
+    W = 8 * log_int(u[3], 1, 12)
+    K = log_int(u[4], 1, 400)
+    while N * K * C * H * W > 4e8 and N > 1:
+        N = max(1, N // 2)
+    return N, C, H, W, K, 1, 1
+
+
+POINTWISE_SHAPES = sorted({_draw_pointwise(s) for s in range(40)})
+
+
+@pytest.mark.parametrize("dims", POINTWISE_SHAPES)
+def test_random_pointwise_shapes(oracle, dims):
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K, R, S = dims
+    assert lib.conv2d_fwd_plan_describe(*dims, ALGO_TF32).get("kernel") == "pointwise_tma"
+    assert lib.conv2d_fwd_plan_describe(*dims, 3).get("kernel") == "pointwise_tma"
+    x, w = uniform((N, C, H, W), 463), uniform((K, C, R, S), 464)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, f"tf32 {dims}")
+    xb, wb = bf16_values(x)[0], bf16_values(w)[0]
+    yb_ref, yb_abs = oracle.conv2d_oracle(xb, wb)
+    assert_parity(run_library(xb, wb, entry="bf16"), yb_ref, yb_abs, 1e-5, f"bf16 {dims}")
+
+
+def _draw_few_tiles(seed):
+    """Small images with many channels and filters: the shapes whose contraction is split over a two-block cluster."""
+    u = uniform((8,), 9700 + seed, 0.0, 1.0)
+    taps = (1, 2, 3, 5)
+    R, S = taps[int(u[0] * 4) % 4], taps[int(u[1] * 4) % 4]
+    if R == 1 and S == 1:
+        S = 3
+    N = 1 + int(u[2] * 8)
+    C = 16 * (2 + int(u[3] * 30))
+    H = max(R, 5 + int(u[4] * 12))
+    W = max(S, 5 + int(u[5] * 12))
+    K = 65 + int(u[6] * 300)
+    while N * K * C * R * S * (H - R + 1) * (W - S + 1) > 6e8 and C > 32:
+        C //= 2
+    return N, C, H, W, K, R, S
+
+
+FEW_TILE_SHAPES = sorted({_draw_few_tiles(s) for s in range(30)})
+
+
+@pytest.mark.parametrize("dims", FEW_TILE_SHAPES)
+def test_random_few_tile_shapes(oracle, dims):
+    N, C, H, W, K, R, S = dims
+    x, w = uniform((N, C, H, W), 465), uniform((K, C, R, S), 466)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, f"tf32 {dims}")
+
+
+def test_the_few_tile_stream_reaches_the_cluster():
+    import paper_1705_10591_b200 as lib
+    assert sum(lib.conv2d_fwd_plan_describe(*d, ALGO_TF32).get("cluster") == 1 for d in FEW_TILE_SHAPES) >= 8
