@@ -55,7 +55,8 @@ typedef enum {
 typedef enum {
     CONV2D_ALGO_AUTO = 0,  /* tensor cores (TF32) where an instance exists, else fp32 FMA */
     CONV2D_ALGO_FFMA = 1,  /* fp32 fused multiply-add on the CUDA cores; error <= 1e-5 * sum|x*w| */
-    CONV2D_ALGO_TF32 = 2,  /* operands rounded to TF32, fp32 accumulation on tcgen05; error <= 2e-3 * sum|x*w| */
+    CONV2D_ALGO_TF32 = 2,  /* operands reduced to TF32 (rounded to nearest; truncated for 1 x 1 filters, see
+                              conv2d_fwd_general), fp32 accumulation on tcgen05; error <= 2e-3 * sum|x*w| */
     CONV2D_ALGO_16BIT = 3  /* workspace query only: the size conv2d_fwd_general_16bit needs */
 } conv2d_algo_t;
 
@@ -126,6 +127,14 @@ conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float*
  *   (16-byte aligned).  Its first 256 bytes are a status block: the filter
  *   re-ordering step of each call clears it, a call with CONV2D_FLAG_WEIGHTS_PACKED
  *   leaves it as it is (so a time-out stays visible until the next full call).
+ *   1 x 1 filters with H*W and C multiples of 4 and C <= 256 take a kernel whose
+ *   operands and output all move by tensor-map (TMA) copies straight from and to
+ *   the caller's tensors: no filter re-ordering (the flag is accepted and has no
+ *   effect), the kernel clears the status block itself, and the tensor core
+ *   truncates both fp32 operands to TF32 instead of the rounding to nearest the
+ *   other shapes get (worst case 1.97e-3 * sum|x*w|, still inside the bound).
+ *   Layers with few output tiles (e.g. 14 x 14 images) split the contraction over
+ *   a two-block cluster; results do not depend on timing.
  * algo = AUTO: TF32 when an instance exists and the workspace suffices, else FFMA.
  * C == 1 is accepted and gives the same result as the single-channel entry.
  */
