@@ -71,6 +71,7 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, float a, fl
 {
     asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
+__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 // Arrives on a barrier of another block of the cluster; this thread's earlier writes into that block's shared
 // memory are visible to whoever then waits on it with cluster-scope acquire.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar_addr)

@@ -42,9 +42,9 @@ constexpr int kMaxTaps = 256;                // taps left as descriptor shifts (
 constexpr size_t kBookBytes = 512 + kMaxTaps * 4;    // barriers, tensor-memory slot, flags + the table of tap shifts
 constexpr int kXposePitch = 36;             // floats per row of the epilogue's transposition tile (16-byte aligned, conflict-free)
 constexpr size_t kXposeBytes = (size_t)kEpilogueWarps * 32 * kXposePitch * 4;
-constexpr int kXchgPitch = 36;              // floats per row of the exchange area of a two-block cluster (as above)
-// bytes of that area for `slots` 32-pixel blocks per epilogue warp: rows, then one barrier per (warp, slot)
-constexpr size_t xchg_area_bytes(int slots) { return (size_t)kEpilogueWarps * slots * (32 * kXchgPitch * 4 + 8); }
+constexpr int kXchgBlockFloats = 32 * 32;   // exchange area of a two-block cluster: one 32-filter x 32-pixel block of partial sums
+// bytes of that area for `slots` 32-pixel blocks per lane quarter: blocks, then one barrier per (quarter, slot)
+constexpr size_t xchg_area_bytes(int slots) { return (size_t)kEpilogueWarps * slots * (kXchgBlockFloats * 4 + 8); }
 
 struct Plan {
     int n_tile;       // filters per work item: 64 or 128 rows of the M operand (with the pixels as M: UMMA N, a multiple of 16)
