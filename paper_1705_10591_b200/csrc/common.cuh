@@ -120,11 +120,14 @@ size_t tf32_workspace_bytes(const Shape& sh);   // includes the status block
 conv2d_status_t launch_general_tf32(const float* x, const float* w, float* y, const Shape& sh,
                                     void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream);
 
-// 1 x 1 filters with every operand moved by tensor-map (TMA) copies; `workspace` only holds the status block.
+// 1 x 1 filters with every operand moved by tensor-map (TMA) copies; `workspace` holds the status block and, for fp32
+// shapes with more channels than a resident filter bank takes, the filters rounded to TF32 (`weights_packed`: they
+// are there already).
 // CONV2D_ERR_UNSUPPORTED when the shape or its alignment has no such instance (the caller then takes the general kernel).
 bool pointwise_tma_supported(const Shape& sh, bool b16);
 conv2d_status_t launch_pointwise_tma(const void* x, const void* w, float* y, const Shape& sh, bool b16, bool fp16,
-                                     void* workspace, size_t workspace_bytes, cudaStream_t stream);
+                                     void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream);
+size_t pointwise_tma_workspace_extra(const Shape& sh, bool b16);   // bytes after the status block, 0 if none
 int describe_pointwise_tma_plan(const Shape& sh, bool b16, char* text, size_t text_bytes);   // -1: no such instance
 
 // Text description of the tensor-core plan of a shape (snprintf semantics: returns the length it needs).

@@ -66,8 +66,9 @@ bool tf32_supported(const Shape& sh)
 size_t tf32_workspace_bytes(const Shape& sh)
 {
     const Plan p = make_plan(sh);
-    if (!p.ok) return kStatusBytes;
-    return kStatusBytes + packed_floats(p) * sizeof(float);
+    const size_t general = p.ok ? packed_floats(p) * sizeof(float) : 0;
+    const size_t pointwise = pointwise_tma_workspace_extra(sh, false);
+    return kStatusBytes + (general > pointwise ? general : pointwise);
 }
 
 bool b16_supported(const Shape& sh)
@@ -122,7 +123,7 @@ conv2d_status_t launch_tensor_core(const void* x_any, const void* w_any, float* 
     const float* w = static_cast<const float*>(w_any);
     {
         // 1 x 1 filters on suitably aligned tensors: the kernel whose operands and output all move by tensor-map copies
-        const conv2d_status_t st = launch_pointwise_tma(x_any, w_any, y, sh, b16, fp16, workspace, workspace_bytes, stream);
+        const conv2d_status_t st = launch_pointwise_tma(x_any, w_any, y, sh, b16, fp16, workspace, workspace_bytes, weights_packed, stream);
         if (st != CONV2D_ERR_UNSUPPORTED) return st;
     }
     const Plan p = make_plan(sh, b16);

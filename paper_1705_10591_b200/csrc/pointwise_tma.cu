@@ -62,6 +62,7 @@ struct Geom {
 };
 constexpr size_t kPwSmemLimit = 227 * 1024;
 constexpr size_t kPwBookBytes = 512;      // barriers, tensor-memory slot, abort flag
+constexpr int kPwMaxStreamChannels = 8192;  // streamed filters: keeps the fp32 accumulation term of the error bound small
 
 struct PwArgs {
     unsigned* status;
@@ -77,9 +78,10 @@ struct PwArgs {
     int cchunks;         // channel chunks of one stage each: ceil(C / channels per stage)
     int ksteps;          // K steps: ceil(C / channels per MMA)
     int stages;          // activation ring depth
+    int stream_a;        // 1: too many channels for a resident bank; every ring stage carries its filter chunk too
     unsigned max_polls;  // bound of every barrier wait
     int test_drop_stage; // test hook: the activation stage with this ordinal is armed but never copied (-1: none)
-    FastDiv div_apb, div_tiles;
+    FastDiv div_apb, div_tiles, div_nb;
 };
 
 template <bool B16>
@@ -93,9 +95,11 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     // swizzle atoms must start on 1024 bytes
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const uint32_t a_chunk_bytes = (uint32_t)a.m_rows * 128u;                 // filters x 32 channels
-    const uint32_t b_stage_bytes = (uint32_t)a.a_item * kAtomBytes;
+    const bool stream_a = a.stream_a != 0;
+    const uint32_t b_off = stream_a ? a_chunk_bytes : 0u;                     // a stage: [its filter chunk,] the pixel boxes
+    const uint32_t b_stage_bytes = b_off + (uint32_t)a.a_item * kAtomBytes;
     unsigned char* a_smem = smem;
-    unsigned char* b_smem = a_smem + (size_t)a.cchunks * a_chunk_bytes;
+    unsigned char* b_smem = a_smem + (stream_a ? (size_t)0 : (size_t)a.cchunks * a_chunk_bytes);
     unsigned char* o_smem = b_smem + (size_t)a.stages * b_stage_bytes;      // [kPwEpiWarps][32 rows x 128 bytes]
     uint64_t* bars = reinterpret_cast<uint64_t*>(o_smem + (size_t)kPwEpiWarps * 4096);
     uint64_t* a_full = bars;                       // [kMaxChunks] 32-channel chunk i of the current filter block has landed
@@ -113,7 +117,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         prefetch_tensormap(&map_w);
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_y);
-        for (int i = 0; i < a.cchunks; ++i) mbar_init(&a_full[i], 1);
+        for (int i = 0; i < (stream_a ? 0 : a.cchunks); ++i) mbar_init(&a_full[i], 1);
         mbar_init(a_empty, 1);
         for (int i = 0; i < a.stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kPwEpiWarps); }
@@ -133,10 +137,13 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     grid_dep_wait();
     if (blockIdx.x == 0 && tid == 0) *a.status = 0u;       // (a block that gives up raises it at its very end)
 
-    // item -> (filter block, first atom, atoms): filter block-major, so that a block rarely changes its bank
+    // item -> (filter block, first atom, atoms): filter block-major, so that a block rarely changes its resident bank;
+    // with streamed filters pixel tile-major, so that the blocks that read the same pixels do so at the same time
+    // and all but the first find them in L2
     auto decode = [&](int item, int& nb, int& first, int& atoms) {
         int tile;
-        nb = a.div_tiles.divmod(item, tile);
+        if (stream_a) tile = a.div_nb.divmod(item, nb);
+        else nb = a.div_tiles.divmod(item, tile);
         first = tile * a.a_item;
         atoms = min(a.a_item, a.total_atoms - first);
     };
@@ -150,7 +157,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
                 int nb, first, atoms;
                 decode(item, nb, first, atoms);
-                const bool new_bank = nb != cur_nb;
+                const bool new_bank = !stream_a && nb != cur_nb;
                 if (new_bank) {
                     // the bank of another filter block: wait until the MMAs on the old one are done
                     if (a_loads && !mbar_wait_bounded(a_empty, (a_loads - 1u) & 1u, abort_flag, a.max_polls)) { alive = false; break; }
@@ -165,9 +172,11 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                         tma_load_2d(a_smem + (size_t)st * a_chunk_bytes, &map_w, st * kStageCh, nb * a.m_rows, &a_full[st]);
                     }
                     if (!mbar_wait_bounded(&b_empty[slot], ph ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                    mbar_arrive_expect_tx(&b_full[slot], (uint32_t)atoms * kAtomBytes);
+                    unsigned char* stage = b_smem + (size_t)slot * b_stage_bytes;
+                    mbar_arrive_expect_tx(&b_full[slot], b_off + (uint32_t)atoms * kAtomBytes);
+                    if (stream_a) tma_load_2d(stage, &map_w, st * kStageCh, nb * a.m_rows, &b_full[slot]);
                     if (issued != a.test_drop_stage) {
-                        unsigned char* dst = b_smem + (size_t)slot * b_stage_bytes;
+                        unsigned char* dst = stage + b_off;
                         int blk;
                         int n = a.div_apb.divmod(first, blk);
                         for (int i = 0; i < atoms; ++i, dst += kAtomBytes) {
@@ -201,7 +210,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
                 int nb, first, atoms;
                 decode(item, nb, first, atoms);
-                const bool new_bank = nb != cur_nb;
+                const bool new_bank = !stream_a && nb != cur_nb;
                 cur_nb = nb;
                 if (!mbar_wait_bounded(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                 tc_fence_after_sync();
@@ -213,8 +222,9 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     if (new_bank && !mbar_wait_bounded(&a_full[st], a_waits & 1u, abort_flag, a.max_polls)) { alive = false; break; }
                     if (!mbar_wait_bounded(&b_full[slot], ph, abort_flag, a.max_polls)) { alive = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a_chunk = a_base + (uint32_t)st * a_chunk_bytes;
-                    const uint32_t b_stage = b_base + (uint32_t)slot * b_stage_bytes;
+                    const uint32_t stage = b_base + (uint32_t)slot * b_stage_bytes;
+                    const uint32_t a_chunk = stream_a ? stage : a_base + (uint32_t)st * a_chunk_bytes;
+                    const uint32_t b_stage = stage + b_off;
                     const int ks = min(4, a.ksteps - st * 4);
                     for (int kk = 0; kk < ks; ++kk) {
                         // filters: 32 bytes further inside the 128-byte rows; pixels: the next 8 (fp32) or 16 (16-bit) channel rows
@@ -233,7 +243,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 mma_commit(&acc_full[buf]);
                 // the next item of this block uses another filter block: tell the loader when this bank is free
                 const int next = item + (int)gridDim.x;
-                if (next < a.items && a.div_tiles.div(next) != nb) mma_commit(a_empty);
+                if (!stream_a && next < a.items && a.div_tiles.div(next) != nb) mma_commit(a_empty);
                 acc_phase[buf] ^= 1u;
                 buf ^= 1;
             }
@@ -298,6 +308,21 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
 }
 
+// Streamed filters, fp32 only: the filters rounded to the nearest TF32 value, into the workspace, so that only the
+// image is truncated by the tensor core and the error bound holds for any channel count.  Also clears the status
+// block, like the re-ordering kernels of the other tensor-core path.
+__global__ void round_filters_tf32_kernel(const float4* __restrict__ w, float4* __restrict__ wp, long long n4,
+                                          unsigned* __restrict__ status)
+{
+    grid_dep_launch();      // the convolution kernel may set itself up while this one runs
+    if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / sizeof(unsigned)) status[threadIdx.x] = 0u;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        const float4 v = w[i];
+        wp[i] = make_float4(to_tf32_rna(v.x), to_tf32_rna(v.y), to_tf32_rna(v.z), to_tf32_rna(v.w));
+    }
+}
+
 // ---------------------------------------------------------------- host side
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -334,6 +359,8 @@ bool encode_map(CUtensorMap* map, CUtensorMapDataType type, const void* base, in
 struct PwPlan {
     bool ok;
     int m_rows, n_blocks, apb, a_item, tiles, cchunks, stages, grid;
+    bool stream_a;         // the filter bank does not fit: filter chunks travel through the ring with the pixels
+    bool round_filters;    // ... and (fp32) are first rounded to TF32 into the workspace
     long long total_atoms;
     size_t smem_bytes;
 };
@@ -348,8 +375,11 @@ PwPlan make_pw_plan(const Shape& sh)
     const long long HW = (long long)sh.H * sh.W;
     // tensor-map strides are multiples of 16 bytes; the filter bank of a block stays in shared memory
     constexpr int kPer16 = 16 / G::kElem;
-    if (HW % kPer16 != 0 || sh.C % kPer16 != 0 || sh.C > G::kMaxChannels) return p;
+    if (HW % kPer16 != 0 || sh.C % kPer16 != 0 || sh.C > kPwMaxStreamChannels) return p;
     if (env_int("CONV2D_B200_TF32_TMA", 1) == 0) return p;
+    p.stream_a = sh.C > G::kMaxChannels;
+    if (p.stream_a && env_int("CONV2D_B200_TMA_STREAM", 1) == 0) return p;
+    p.round_filters = p.stream_a && !B16;
     p.m_rows = sh.K <= 64 ? 64 : 128;
     p.n_blocks = (sh.K + p.m_rows - 1) / p.m_rows;
     p.apb = (int)((HW + G::kAtomPx - 1) / G::kAtomPx);
@@ -374,8 +404,9 @@ PwPlan make_pw_plan(const Shape& sh)
     p.tiles = (int)((p.total_atoms + p.a_item - 1) / p.a_item);
     const long long items = (long long)p.tiles * p.n_blocks;
     if (items > 0x7fffffffLL) return p;
-    const size_t fixed = (size_t)p.cchunks * p.m_rows * 128 + (size_t)kPwEpiWarps * 4096 + kPwBookBytes + 1024;
-    const size_t stage = (size_t)p.a_item * G::kAtomBytes;
+    const size_t bank = (size_t)p.m_rows * 128;           // one channel chunk of a filter block
+    const size_t fixed = (p.stream_a ? 0 : (size_t)p.cchunks * bank) + (size_t)kPwEpiWarps * 4096 + kPwBookBytes + 1024;
+    const size_t stage = (p.stream_a ? bank : 0) + (size_t)p.a_item * G::kAtomBytes;
     if (fixed + 2 * stage > kPwSmemLimit) return p;
     p.stages = (int)((kPwSmemLimit - fixed) / stage);
     if (p.stages > kPwMaxStages) p.stages = kPwMaxStages;
@@ -399,19 +430,37 @@ int describe_pw(const Shape& sh, char* text, size_t text_bytes)
     const double issued = 2.0 * p.m_rows * p.n_blocks * cols * ((sh.C + G::kKStep - 1) / G::kKStep * G::kKStep);
     return snprintf(text, text_bytes,
                     "tensor_core=1 kernel=pointwise_tma addressing=atoms filters_as=M m_rows=%d tile_px=%d acc_sets=2 items=%lld "
-                    "grid=%d stages=%d resident_filters=1 smem_bytes=%zu mma_useful_px=%.4f mma_useful_flops=%.4f",
-                    p.m_rows, p.a_item * G::kAtomPx, (long long)p.tiles * p.n_blocks, p.grid, p.stages, p.smem_bytes,
+                    "grid=%d stages=%d resident_filters=%d filters_rounded_first=%d smem_bytes=%zu mma_useful_px=%.4f "
+                    "mma_useful_flops=%.4f",
+                    p.m_rows, p.a_item * G::kAtomPx, (long long)p.tiles * p.n_blocks, p.grid, p.stages, p.stream_a ? 0 : 1,
+                    p.round_filters ? 1 : 0, p.smem_bytes,
                     px / cols, 2.0 * px * sh.K * sh.C / issued);
 }
 
 template <bool B16>
 conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& sh, bool fp16,
-                          void* workspace, size_t workspace_bytes, cudaStream_t stream)
+                          void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream)
 {
     using G = Geom<B16>;
     const PwPlan p = make_pw_plan<B16>(sh);
     if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
-    if (!workspace || workspace_bytes < kStatusBytes) return CONV2D_ERR_WORKSPACE;
+    const size_t rounded_bytes = p.round_filters ? (size_t)sh.K * sh.C * sizeof(float) : 0;
+    if (!workspace || workspace_bytes < kStatusBytes + rounded_bytes) return CONV2D_ERR_WORKSPACE;
+    if (p.round_filters) {
+        float* wp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
+        if ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(wp)) & 15u) return CONV2D_ERR_UNSUPPORTED;
+        if (!weights_packed) {
+            const long long n4 = (long long)sh.K * sh.C / 4;
+            long long blocks = (n4 + 255) / 256;
+            if (blocks > sm_count() * 8LL) blocks = sm_count() * 8LL;
+            // (launched the ordinary way: it starts only when the previous kernel on the stream, which may still be
+            // reading the workspace, has finished)
+            round_filters_tf32_kernel<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const float4*>(w), reinterpret_cast<float4*>(wp),
+                                                                            n4, static_cast<unsigned*>(workspace));
+            count_launch();
+        }
+        w = wp;
+    }
     const cuuint64_t HW = (cuuint64_t)sh.H * sh.W;
     const cuuint64_t es = G::kElem;
     const CUtensorMapDataType in_type = !B16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
@@ -449,12 +498,13 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
     a.apb = p.apb; a.total_atoms = (int)p.total_atoms; a.a_item = p.a_item; a.tiles = p.tiles;
     a.n_blocks = p.n_blocks; a.m_rows = p.m_rows; a.items = p.tiles * p.n_blocks;
     a.cchunks = p.cchunks; a.ksteps = (sh.C + G::kKStep - 1) / G::kKStep; a.stages = p.stages;
+    a.stream_a = p.stream_a ? 1 : 0;
     a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
     a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
-    a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles);
+    a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles); a.div_nb = FastDiv(p.n_blocks);
     if (env_int("CONV2D_B200_TF32_VERBOSE", 0) != 0)
-        fprintf(stderr, "conv2d plan: pointwise_tma%s m_rows %d n_blocks %d atoms/item %d tiles %d stages %d grid %d smem %zu\n",
-                B16 ? " (16-bit)" : "", p.m_rows, p.n_blocks, p.a_item, p.tiles, p.stages, p.grid, p.smem_bytes);
+        fprintf(stderr, "conv2d plan: pointwise_tma%s%s m_rows %d n_blocks %d atoms/item %d tiles %d stages %d grid %d smem %zu\n",
+                B16 ? " (16-bit)" : "", p.stream_a ? " (streamed filters)" : "", p.m_rows, p.n_blocks, p.a_item, p.tiles, p.stages, p.grid, p.smem_bytes);
     if (launch_pdl(pointwise_tma_kernel<B16>, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
                    map_w, map_x, map_y, a) != cudaSuccess)
         return CONV2D_ERR_CUDA;
@@ -474,11 +524,19 @@ int describe_pointwise_tma_plan(const Shape& sh, bool b16, char* text, size_t te
     return b16 ? describe_pw<true>(sh, text, text_bytes) : describe_pw<false>(sh, text, text_bytes);
 }
 
-conv2d_status_t launch_pointwise_tma(const void* x, const void* w, float* y, const Shape& sh, bool b16, bool fp16,
-                                     void* workspace, size_t workspace_bytes, cudaStream_t stream)
+// Workspace bytes the kernel needs beyond the status block (the rounded filters), 0 if none or not supported.
+size_t pointwise_tma_workspace_extra(const Shape& sh, bool b16)
 {
-    return b16 ? launch_pw<true>(x, w, y, sh, fp16, workspace, workspace_bytes, stream)
-               : launch_pw<false>(x, w, y, sh, false, workspace, workspace_bytes, stream);
+    if (b16) return 0;
+    const PwPlan p = make_pw_plan<false>(sh);
+    return p.ok && p.round_filters ? (size_t)sh.K * sh.C * sizeof(float) : 0;
+}
+
+conv2d_status_t launch_pointwise_tma(const void* x, const void* w, float* y, const Shape& sh, bool b16, bool fp16,
+                                     void* workspace, size_t workspace_bytes, bool weights_packed, cudaStream_t stream)
+{
+    return b16 ? launch_pw<true>(x, w, y, sh, fp16, workspace, workspace_bytes, weights_packed, stream)
+               : launch_pw<false>(x, w, y, sh, false, workspace, workspace_bytes, weights_packed, stream);
 }
 
 }  // namespace conv2d_b200

@@ -133,3 +133,121 @@ def test_pointwise_16bit_operands(oracle, dims, kind):
     y_ref, yabs = oracle.conv2d_oracle(x, w)
     r = assert_parity(run_library(x, w, entry=kind), y_ref, yabs, B16_TOL, f"pointwise {kind} {dims}")
     print(f"pointwise {kind} {dims} max ratio {r:.3e}")
+
+
+# More channels than a resident filter bank holds (256 fp32, 512 16-bit): every ring stage carries its chunk of the
+# filters with the pixels, and fp32 filters are first rounded to TF32 by a small kernel.
+STREAM_SHAPES = [
+    # N, C, H, W, K
+    (4, 512, 14, 14, 300),      # three filter blocks, ragged atoms, items tile-major
+    (2, 1024, 8, 8, 64),        # 64-row operand, 32 stages per item
+    (1, 260, 12, 10, 130),      # C = 260: ninth stage holds 4 channels; second filter block holds 2 filters
+    (3, 2048, 7, 8, 128),       # the deepest layers of a residual network
+    (20, 320, 16, 16, 256),     # more work items than SMs
+]
+
+STREAM_SHAPES_16BIT = [
+    (4, 1024, 8, 8, 300),
+    (2, 520, 12, 10, 64),       # C = 520: ninth stage holds 8 channels (half an MMA step)
+    (3, 2048, 8, 8, 128),
+    (20, 640, 16, 16, 256),
+]
+
+
+def _round_to_tf32(a):
+    """fp32 -> nearest value with a 10-bit mantissa, ties away from zero (what cvt.rna.tf32.f32 does)."""
+    bits = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    return ((bits + np.uint32(0x1000)) & np.uint32(0xFFFFE000)).view(np.float32)
+
+
+@pytest.mark.parametrize("dims", STREAM_SHAPES)
+def test_pointwise_streamed_filters(oracle, dims):
+    import paper_1705_10591_b200 as lib
+    from oracle.conv2d_oracle import MODE_TF32_TRUNC
+    N, C, H, W, K = dims
+    plan = lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, ALGO_TF32)
+    assert plan.get("kernel") == "pointwise_tma" and plan.get("resident_filters") == 0 and plan.get("filters_rounded_first") == 1
+    xi, wi = small_integers((N, C, H, W), 971), small_integers((K, C, 1, 1), 972)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry="general", algo=ALGO_TF32).astype(np.float64), yi_ref)
+    x, w = uniform((N, C, H, W), 973), uniform((K, C, 1, 1), 974)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    y = run_library(x, w, entry="general", algo=ALGO_TF32)
+    r = assert_parity(y, y_ref, yabs, TF32_TOL, f"pointwise, streamed filters {dims}")
+    # filters rounded to nearest by the library, image truncated by the tensor core: against the oracle fed such
+    # operands (truncating a rounded filter changes nothing) only the order of the fp32 additions differs
+    y_t, yabs_t = oracle.conv2d_oracle(x, _round_to_tf32(w), mode=MODE_TF32_TRUNC)
+    assert_parity(y, y_t, yabs_t, 2e-5, f"pointwise, streamed filters vs TF32-operand oracle {dims}")
+    print(f"pointwise streamed {dims} max ratio {r:.3e}")
+
+
+@pytest.mark.parametrize("kind", ["bf16", "fp16"])
+@pytest.mark.parametrize("dims", STREAM_SHAPES_16BIT)
+def test_pointwise_streamed_filters_16bit(oracle, dims, kind):
+    import paper_1705_10591_b200 as lib
+    from helpers import B16_TOL, bf16_values, fp16_values
+    N, C, H, W, K = dims
+    plan = lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, 3)
+    assert plan.get("kernel") == "pointwise_tma" and plan.get("resident_filters") == 0 and plan.get("filters_rounded_first") == 0
+    xi, wi = small_integers((N, C, H, W), 985), small_integers((K, C, 1, 1), 986)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry=kind).astype(np.float64), yi_ref)
+    conv = bf16_values if kind == "bf16" else fp16_values
+    x, w = conv(uniform((N, C, H, W), 987))[0], conv(uniform((K, C, 1, 1), 988))[0]
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry=kind), y_ref, yabs, B16_TOL, f"pointwise, streamed filters {kind} {dims}")
+
+
+def test_pointwise_streamed_filters_prepacked(oracle):
+    """CONV2D_FLAG_WEIGHTS_PACKED: the second call finds the rounded filters in the workspace and launches one
+    kernel less; the result is the same bits."""
+    import torch
+    import paper_1705_10591_b200 as lib
+
+    N, C, H, W, K = 2, 512, 8, 8, 96
+    x, w = uniform((N, C, H, W), 975), uniform((K, C, 1, 1), 976)
+    dev = torch.device("cuda:0")
+    xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
+    ws_bytes = lib.conv2d_fwd_workspace_size(N, C, H, W, K, 1, 1, ALGO_TF32)
+    assert ws_bytes >= 256 + K * C * 4
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    ys = []
+    for flags in (0, 1):
+        y = torch.zeros((N, K, H, W), device=dev)
+        before = lib.conv2d_launch_count()
+        lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), y.data_ptr(), N, C, H, W, K, 1, 1, ALGO_TF32,
+                               ws.data_ptr(), ws_bytes, flags, stream)
+        lib.conv2d_get_status(ws.data_ptr(), stream)
+        assert lib.conv2d_launch_count() - before == 2 - flags
+        ys.append(y.cpu().numpy())
+    np.testing.assert_array_equal(ys[0], ys[1])
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(ys[1], y_ref, yabs, TF32_TOL, "streamed filters, prepacked")
+
+
+def test_pointwise_streamed_filters_expired_wait_is_reported(oracle, monkeypatch):
+    """The same host-side injection as above on the streamed-filter variant: a stage whose pixels never arrive."""
+    import torch
+    import paper_1705_10591_b200 as lib
+
+    N, C, H, W, K = 2, 512, 16, 16, 128
+    x, w = uniform((N, C, H, W), 977), uniform((K, C, 1, 1), 978)
+    dev = torch.device("cuda:0")
+    xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
+    y = torch.zeros((N, K, H, W), device=dev)
+    ws_bytes = lib.conv2d_fwd_workspace_size(N, C, H, W, K, 1, 1, ALGO_TF32)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    monkeypatch.setenv("CONV2D_B200_TF32_MAX_POLLS", "2048")
+    monkeypatch.setenv("CONV2D_B200_TF32_TEST_DROP_STAGE", "5")
+    lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), y.data_ptr(), N, C, H, W, K, 1, 1, ALGO_TF32,
+                           ws.data_ptr(), ws_bytes, 0, stream)
+    with pytest.raises(lib.Conv2dError) as e:
+        lib.conv2d_get_status(ws.data_ptr(), stream)
+    assert e.value.status == 8                       # CONV2D_ERR_DEVICE_TIMEOUT
+    torch.cuda.synchronize()
+    monkeypatch.delenv("CONV2D_B200_TF32_MAX_POLLS")
+    monkeypatch.delenv("CONV2D_B200_TF32_TEST_DROP_STAGE")
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, "after a time-out")
