@@ -30,6 +30,7 @@
 // Work items are runs of `a_item` 32-pixel atoms of the flat atom sequence (image-major; an image has
 // ceil(HW / 32) atoms, the last one may be ragged and is zero-filled on load and clipped on store).
 // Every wait is bounded; on expiry the block stops, frees its tensor memory and raises the status word.
+#include <algorithm>
 #include <cstdio>
 #include <cuda.h>
 
@@ -62,6 +63,7 @@ struct Geom {
 };
 constexpr size_t kPwSmemLimit = 227 * 1024;
 constexpr size_t kPwBookBytes = 512;      // barriers, tensor-memory slot, abort flag
+constexpr double kPwPairBias = 1.03;      // planner: the two-SM form is taken when its estimate is at least 3 % shorter
 constexpr int kPwMaxStreamChannels = 8192;  // streamed filters: keeps the fp32 accumulation term of the error bound small
 
 struct PwArgs {
@@ -308,6 +310,242 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
 }
 
+// ---------------------------------------------------------------- two-SM variant
+// More than 128 filters: the two blocks of a cluster work as a pair on 256 filters x `a_item` atoms of pixels with
+// two-SM MMAs (cta_group::2, M = 256).  Block r of the pair holds filter block 2 * pair + r (its 128 rows of the M
+// operand) and the r-th half of the item's pixels (its half of the N operand), so every byte of the image is
+// fetched once per 256 filters instead of once per 128, and each SM's tensor core reads half of the pixel operand
+// from its own shared memory.  The first block issues the MMAs; its `full` barriers collect the bytes of both
+// blocks' copies, its commits arrive on the `empty` / `acc_full` barriers of both blocks, and the write-back warps
+// of both blocks (each drains its own 128 accumulator lanes) arrive on its `acc_empty` barriers.  Items always
+// span `a_item` atoms: atoms past the end of the batch are zero-filled by the loads and skipped by the stores.
+template <bool B16>
+__global__ void __launch_bounds__(kPwThreads, 1)
+pointwise_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+                      const __grid_constant__ CUtensorMap map_y, const PwArgs a)
+{
+    using G = Geom<B16>;
+    constexpr int kAtomPx = G::kAtomPx, kStageCh = G::kStageCh, kAtomBytes = G::kAtomBytes;
+    constexpr int kRows = 128;                                                // filters per block of the pair
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const bool stream_a = a.stream_a != 0;
+    const int half_atoms = a.a_item >> 1;                                     // atoms this block loads per stage
+    const uint32_t a_chunk_bytes = (uint32_t)kRows * 128u;
+    const uint32_t b_off = stream_a ? a_chunk_bytes : 0u;
+    const uint32_t stage_tx = b_off + (uint32_t)half_atoms * kAtomBytes;      // bytes one block's copies bring per stage
+    const uint32_t b_stage_bytes = stage_tx;
+    unsigned char* a_smem = smem;
+    unsigned char* b_smem = a_smem + (stream_a ? (size_t)0 : (size_t)a.cchunks * a_chunk_bytes);
+    unsigned char* o_smem = b_smem + (size_t)a.stages * b_stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(o_smem + (size_t)kPwEpiWarps * 4096);
+    uint64_t* a_full = bars;                       // [kMaxChunks]   (waited on in the first block only)
+    uint64_t* a_empty = a_full + kMaxChunks;       // [1]
+    uint64_t* b_full = a_empty + 1;                // [kPwMaxStages] (first block only)
+    uint64_t* b_empty = b_full + kPwMaxStages;     // [kPwMaxStages]
+    uint64_t* acc_full = b_empty + kPwMaxStages;   // [2]
+    uint64_t* acc_empty = acc_full + 2;            // [2]            (first block only; both blocks' warps arrive)
+    uint64_t* drain_bar = acc_empty + 2;           // [1]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool first_block = rank == 0;
+    const int pair_id = (int)(blockIdx.x >> 1), n_pairs_running = (int)(gridDim.x >> 1);
+    if (tid == 0) {
+        prefetch_tensormap(&map_w);
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_y);
+        for (int i = 0; i < (stream_a ? 0 : a.cchunks); ++i) mbar_init(&a_full[i], 1);
+        mbar_init(a_empty, 1);
+        for (int i = 0; i < a.stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 2 * kPwEpiWarps); }
+        mbar_init(drain_bar, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    cluster_sync_all();             // the peer's barriers exist before a copy or a commit can signal them
+    if (warp == 1) { tmem_alloc_pair(tmem_slot, 2 * kAccCols); tmem_relinquish_pair(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    grid_dep_launch();
+    grid_dep_wait();
+    if (blockIdx.x == 0 && tid == 0) *a.status = 0u;
+
+    // item -> (pair of filter blocks, first atom): as in the one-SM kernel, with pairs in place of filter blocks
+    auto decode = [&](int item, int& pr, int& first) {
+        int tile;
+        if (stream_a) tile = a.div_nb.divmod(item, pr);
+        else pr = a.div_tiles.divmod(item, tile);
+        first = tile * a.a_item;
+    };
+
+    if (warp == 0) {
+        // ---------------- loads (one thread per block): this block's filter rows and its half of the pixels
+        if (lane == 0) {
+            const uint32_t a_full_first = map_to_cta(smem_u32(a_full), 0);     // the first block's barriers
+            const uint32_t b_full_first = map_to_cta(smem_u32(b_full), 0);
+            int cur_pr = -1, slot = 0, issued = 0;
+            uint32_t ph = 0, a_loads = 0;
+            bool alive = true;
+            for (int item = pair_id; item < a.items && alive; item += n_pairs_running) {
+                int pr, first;
+                decode(item, pr, first);
+                const int k_row = (2 * pr + (int)rank) * kRows;
+                const bool new_bank = !stream_a && pr != cur_pr;
+                if (new_bank) {
+                    if (a_loads && !mbar_wait_bounded(a_empty, (a_loads - 1u) & 1u, abort_flag, a.max_polls)) { alive = false; break; }
+                    cur_pr = pr;
+                    ++a_loads;
+                }
+                for (int st = 0; st < a.cchunks; ++st) {
+                    if (new_bank) {
+                        if (first_block) mbar_arrive_expect_tx(&a_full[st], 2u * a_chunk_bytes);
+                        tma_load_2d_pair(a_smem + (size_t)st * a_chunk_bytes, &map_w, st * kStageCh, k_row, a_full_first + 8u * (uint32_t)st);
+                    }
+                    if (!mbar_wait_bounded(&b_empty[slot], ph ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
+                    unsigned char* stage = b_smem + (size_t)slot * b_stage_bytes;
+                    const uint32_t bar = b_full_first + 8u * (uint32_t)slot;
+                    if (first_block) mbar_arrive_expect_tx(&b_full[slot], 2u * stage_tx);
+                    if (stream_a) tma_load_2d_pair(stage, &map_w, st * kStageCh, k_row, bar);
+                    if (!(first_block && issued == a.test_drop_stage)) {
+                        unsigned char* dst = stage + b_off;
+                        int blk;
+                        int n = a.div_apb.divmod(first + (int)rank * half_atoms, blk);
+                        for (int i = 0; i < half_atoms; ++i, dst += kAtomBytes) {
+                            tma_load_3d_pair(dst, &map_x, blk * kAtomPx, st * kStageCh, n, bar);   // (n past the batch: zeros)
+                            if (++blk == a.apb) { blk = 0; ++n; }
+                        }
+                    }
+                    ++issued;
+                    if (++slot == a.stages) { slot = 0; ph ^= 1u; }
+                }
+            }
+            if (*abort_flag && first_block) {
+                // let copies already in flight (of both blocks: they signal these barriers) land before the blocks leave
+                uint32_t dummy = 0;
+                for (int cb = 0; cb < (stream_a ? 0 : a.cchunks) && a_loads; ++cb)
+                    mbar_wait_bounded(&a_full[cb], (a_loads - 1u) & 1u, &dummy, 1u << 14);
+                const int pending = issued < a.stages ? issued : a.stages;
+                for (int i = 0; i < pending; ++i) {
+                    const int it = issued - 1 - i;
+                    mbar_wait_bounded(&b_full[it % a.stages], (uint32_t)(it / a.stages) & 1u, &dummy, 1u << 14);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issue (one thread of the first block)
+        if (lane == 0 && first_block) {
+            const uint32_t a_base = smem_u32(a_smem), b_base = smem_u32(b_smem);
+            int cur_pr = -1, slot = 0, buf = 0;
+            uint32_t ph = 0, a_waits = 0, acc_phase[2] = {0u, 0u};
+            bool alive = true;
+            const uint32_t n_cols = (uint32_t)(a.a_item * kAtomPx);
+            const uint32_t idesc = (B16 ? idesc_b16(256u, n_cols, a.fp16 != 0) : idesc_tf32(256u, n_cols)) | kIdescBMajorMN;
+            for (int item = pair_id; item < a.items && alive; item += n_pairs_running) {
+                int pr, first;
+                decode(item, pr, first);
+                const bool new_bank = !stream_a && pr != cur_pr;
+                cur_pr = pr;
+                if (!mbar_wait_bounded_cluster(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d = tmem + (uint32_t)(buf * kAccCols);
+                bool accumulate = false;
+                for (int st = 0; st < a.cchunks && alive; ++st) {
+                    if (new_bank && !mbar_wait_bounded(&a_full[st], a_waits & 1u, abort_flag, a.max_polls)) { alive = false; break; }
+                    if (!mbar_wait_bounded(&b_full[slot], ph, abort_flag, a.max_polls)) { alive = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t stage = b_base + (uint32_t)slot * b_stage_bytes;
+                    const uint32_t a_chunk = stream_a ? stage : a_base + (uint32_t)st * a_chunk_bytes;
+                    const uint32_t b_stage = stage + b_off;
+                    const int ks = min(4, a.ksteps - st * 4);
+                    for (int kk = 0; kk < ks; ++kk) {
+                        const uint64_t a_desc = smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u);
+                        if (B16)
+                            mma_b16_pair(d, a_desc, smem_desc_sw128(b_stage + (uint32_t)kk * 2048u, (uint32_t)kStageCh * 128u, 1024u), idesc, accumulate);
+                        else
+                            mma_tf32_pair(d, a_desc, smem_desc_mn_sw128_32b(b_stage + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u), idesc, accumulate);
+                        accumulate = true;
+                    }
+                    mma_commit_pair_both(&b_empty[slot]);
+                    if (++slot == a.stages) { slot = 0; ph ^= 1u; }
+                }
+                if (!alive) break;
+                if (new_bank) ++a_waits;
+                mma_commit_pair_both(&acc_full[buf]);
+                const int next = item + n_pairs_running;
+                if (!stream_a && next < a.items && a.div_tiles.div(next) != pr) mma_commit_pair_both(a_empty);
+                acc_phase[buf] ^= 1u;
+                buf ^= 1;
+            }
+            if (!alive) {
+                mma_commit_pair(drain_bar);
+                uint32_t dummy = 0;
+                mbar_wait_bounded(drain_bar, 0u, &dummy, 1u << 16);
+            }
+        }
+    } else {
+        // ---------------- write-back (both blocks): this block's 128 filters, all pixels of the item
+        const int ew = warp - 2;
+        const int quarter = warp & 3;
+        const int half = ew >> 2;
+        unsigned char* tile = o_smem + (size_t)ew * 4096;
+        const uint32_t acc_empty_first = map_to_cta(smem_u32(acc_empty), 0);
+        bool alive = true;
+        int li = 0;
+        for (int item = pair_id; item < a.items; item += n_pairs_running, ++li) {
+            int pr, first;
+            decode(item, pr, first);
+            const int atoms = min(a.a_item, a.total_atoms - first);
+            const int buf = li & 1;
+            const uint32_t acc_phase = (uint32_t)(li >> 1) & 1u;
+            alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag, a.max_polls));
+            if (!alive) break;
+            tc_fence_after_sync();
+            const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccCols);
+            const int k0 = (2 * pr + (int)rank) * kRows + quarter * 32;
+            constexpr int kBpa = kAtomPx / 32;
+            if (k0 < a.K)
+                for (int i = half; i < atoms * kBpa; i += 2) {
+                    uint32_t v[32];
+                    tmem_ld32(lane_base + (uint32_t)(i * 32), v);
+                    tmem_ld_wait();
+                    if (lane == 0) bulk_wait_group_read<0>();
+                    __syncwarp();
+                    unsigned char* row = tile + lane * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4*>(row + ((c ^ (lane & 7)) << 4)) = make_uint4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        int blk;
+                        const int n = a.div_apb.divmod(first + i / kBpa, blk);
+                        tma_store_3d(&map_y, blk * kAtomPx + (i % kBpa) * 32, k0, n, tile);
+                        bulk_commit_group();
+                    }
+                }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                if (first_block) mbar_arrive(&acc_empty[buf]);
+                else mbar_arrive_remote(acc_empty_first + 8u * (uint32_t)buf);
+            }
+        }
+        if (lane == 0) bulk_wait_group<0>();
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();             // neither block leaves while the peer may still signal its barriers or read its operands
+    if (warp == 1) tmem_dealloc_pair(tmem, 2 * kAccCols);
+    if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
+}
+
 // Streamed filters, fp32 only: the filters rounded to the nearest TF32 value, into the workspace, so that only the
 // image is truncated by the tensor core and the error bound holds for any channel count.  Also clears the status
 // block, like the re-ordering kernels of the other tensor-core path.
@@ -361,52 +599,64 @@ struct PwPlan {
     int m_rows, n_blocks, apb, a_item, tiles, cchunks, stages, grid;
     bool stream_a;         // the filter bank does not fit: filter chunks travel through the ring with the pixels
     bool round_filters;    // ... and (fp32) are first rounded to TF32 into the workspace
+    bool pair;             // two-SM MMAs: work items are (pixel tile, pair of 128-filter blocks), one per two-block cluster
+    int n_units;           // filter blocks, or pairs of them
     long long total_atoms;
+    long long items;
+    double cost;           // planner's estimate of the kernel time in SM cycles (compares the one-SM and the two-SM form)
     size_t smem_bytes;
 };
 
+// Plan for the one-SM (`pair` = false) or the two-SM form.
 template <bool B16>
-PwPlan make_pw_plan(const Shape& sh)
+PwPlan make_pw_variant(const Shape& sh, bool pair)
 {
     using G = Geom<B16>;
     PwPlan p{};
     p.ok = false;
-    if (sh.R != 1 || sh.S != 1 || sh.pad_h || sh.pad_w) return p;
-    const long long HW = (long long)sh.H * sh.W;
-    // tensor-map strides are multiples of 16 bytes; the filter bank of a block stays in shared memory
-    constexpr int kPer16 = 16 / G::kElem;
-    if (HW % kPer16 != 0 || sh.C % kPer16 != 0 || sh.C > kPwMaxStreamChannels) return p;
-    if (env_int("CONV2D_B200_TF32_TMA", 1) == 0) return p;
+    p.pair = pair;
     p.stream_a = sh.C > G::kMaxChannels;
-    if (p.stream_a && env_int("CONV2D_B200_TMA_STREAM", 1) == 0) return p;
     p.round_filters = p.stream_a && !B16;
-    p.m_rows = sh.K <= 64 ? 64 : 128;
+    p.m_rows = (sh.K <= 64 && !pair) ? 64 : 128;
     p.n_blocks = (sh.K + p.m_rows - 1) / p.m_rows;
+    if (pair && p.n_blocks < 2) return p;
+    p.n_units = pair ? (p.n_blocks + 1) / 2 : p.n_blocks;
+    const long long HW = (long long)sh.H * sh.W;
     p.apb = (int)((HW + G::kAtomPx - 1) / G::kAtomPx);
     p.total_atoms = (long long)sh.N * p.apb;
     if (p.total_atoms > 0x3fffffffLL) return p;
     p.cchunks = (sh.C + G::kStageCh - 1) / G::kStageCh;
     const int sms = sm_count();
-    // Atoms per item: the fewest rounds of items over the SMs, counted in atoms, plus half an atom of fixed cost per
-    // item; ties go to the larger item (wider MMAs).  64 x 32 x 32 pixels = 2048 atoms of 32: 7 per item = 293 items =
-    // two rounds of 7, where 8 per item would be two rounds of 8.
-    double best = 0;
+    const int workers = pair ? sms / 2 : sms;            // blocks, or pairs of blocks
+    if (workers < 1) return p;
+    // Atoms per item, one-SM form: the fewest rounds of items over the SMs, counted in atoms, plus half an atom of
+    // fixed cost per item; ties go to the larger item (wider MMAs).  64 x 32 x 32 pixels = 2048 atoms of 32: 7 per
+    // item = 293 items = two rounds of 7, where 8 per item would be two rounds of 8.
+    // Two-SM form (an even number, half for each block): the widest MMAs that still leave an item for at least half
+    // of the pairs; measured, narrower items only pay when most of the machine would otherwise idle.
     p.a_item = 0;
     const int forced = env_int("CONV2D_B200_TMA_ATOMS", 0);
+    double best = 0;
     for (int at = G::kMaxAtoms; at >= 1; --at) {
+        if (pair && (at & 1)) continue;
         if (forced && at != (forced < G::kMaxAtoms ? forced : G::kMaxAtoms)) continue;
         const long long tiles = (p.total_atoms + at - 1) / at;
-        const long long rounds = (tiles * p.n_blocks + sms - 1) / sms;
+        if (pair) {
+            p.a_item = at;
+            if (2 * tiles * p.n_units >= workers) break;
+            continue;
+        }
+        const long long rounds = (tiles * p.n_units + workers - 1) / workers;
         const double cost = (double)rounds * (at + 0.5 * 32 / G::kAtomPx);
         if (p.a_item == 0 || cost < best - 1e-9) { best = cost; p.a_item = at; }
     }
     if (p.a_item == 0) return p;
     p.tiles = (int)((p.total_atoms + p.a_item - 1) / p.a_item);
-    const long long items = (long long)p.tiles * p.n_blocks;
-    if (items > 0x7fffffffLL) return p;
+    p.items = (long long)p.tiles * p.n_units;
+    if (p.items > 0x7fffffffLL) return p;
     const size_t bank = (size_t)p.m_rows * 128;           // one channel chunk of a filter block
     const size_t fixed = (p.stream_a ? 0 : (size_t)p.cchunks * bank) + (size_t)kPwEpiWarps * 4096 + kPwBookBytes + 1024;
-    const size_t stage = (p.stream_a ? bank : 0) + (size_t)p.a_item * G::kAtomBytes;
+    const size_t stage = (p.stream_a ? bank : 0) + (size_t)(pair ? p.a_item / 2 : p.a_item) * G::kAtomBytes;
     if (fixed + 2 * stage > kPwSmemLimit) return p;
     p.stages = (int)((kPwSmemLimit - fixed) / stage);
     if (p.stages > kPwMaxStages) p.stages = kPwMaxStages;
@@ -414,9 +664,48 @@ PwPlan make_pw_plan(const Shape& sh)
     // more than half of an SM's shared memory, so that two of these blocks, which both want all 512 tensor-memory
     // columns, never share an SM
     if (p.smem_bytes < 116 * 1024) p.smem_bytes = 116 * 1024;
-    p.grid = (int)(items < sms ? items : sms);
+    p.grid = (int)(p.items < workers ? p.items : workers) * (pair ? 2 : 1);
+    // Estimated time in SM cycles, used only to choose between the two forms (constants fitted to measurements on
+    // B200): the longest of (a) the busiest block's items, a stage taking the longest of its MMAs (at least 120
+    // cycles each), its bytes at 40 B/clk and the copy latency spread over the ring, (b) all stages' bytes through
+    // L2 at 7 TB/s, (c) the image, read once per filter block (pair) when it does not stay in L2 between the
+    // filter block-major passes of a resident bank, and the output through HBM.
+    {
+        const double rounds = (double)((p.items + workers - 1) / workers);
+        const double mma = 4.0 * std::max((double)p.a_item * 16.0 * G::kAtomPx / 32.0, 120.0);
+        const double stage_time = std::max({mma, (double)stage / 40.0, 2500.0 / std::max(p.stages - 1, 1)});
+        const double crit = rounds * (p.cchunks * stage_time + 2500.0);
+        const double l2 = (double)p.items * (pair ? 2 : 1) * p.cchunks * (double)stage / 3700.0;
+        const double x_bytes = (double)sh.N * sh.C * (double)HW * G::kElem, y_bytes = (double)sh.N * sh.K * (double)HW * 4.0;
+        const double passes = (!p.stream_a && x_bytes > 100e6) ? p.n_units : 1;
+        const double hbm = (y_bytes + x_bytes * passes) / 3400.0;
+        p.cost = std::max({crit, l2, hbm});
+    }
     p.ok = true;
     return p;
+}
+
+template <bool B16>
+PwPlan make_pw_plan(const Shape& sh)
+{
+    using G = Geom<B16>;
+    PwPlan none{};
+    none.ok = false;
+    if (sh.R != 1 || sh.S != 1 || sh.pad_h || sh.pad_w) return none;
+    const long long HW = (long long)sh.H * sh.W;
+    // tensor-map strides are multiples of 16 bytes
+    constexpr int kPer16 = 16 / G::kElem;
+    if (HW % kPer16 != 0 || sh.C % kPer16 != 0 || sh.C > kPwMaxStreamChannels) return none;
+    if (env_int("CONV2D_B200_TF32_TMA", 1) == 0) return none;
+    if (sh.C > G::kMaxChannels && env_int("CONV2D_B200_TMA_STREAM", 1) == 0) return none;
+    const PwPlan one = make_pw_variant<B16>(sh, false);
+    // CONV2D_B200_TMA_PAIR: 0 never, 1 where the planner expects it to be faster, 2 wherever it exists
+    const int want = env_int("CONV2D_B200_TMA_PAIR", 1);
+    if (want == 0 || sh.K <= 128) return one;
+    const PwPlan two = make_pw_variant<B16>(sh, true);
+    if (!two.ok) return one;
+    if (!one.ok || want == 2) return two;
+    return two.cost * kPwPairBias <= one.cost ? two : one;
 }
 
 template <bool B16>
@@ -427,14 +716,16 @@ int describe_pw(const Shape& sh, char* text, size_t text_bytes)
     if (!p.ok) return -1;
     const double px = (double)sh.N * sh.H * sh.W;
     const double cols = (double)p.total_atoms * G::kAtomPx;
-    const double issued = 2.0 * p.m_rows * p.n_blocks * cols * ((sh.C + G::kKStep - 1) / G::kKStep * G::kKStep);
+    const double cols_issued = (double)p.tiles * p.a_item * G::kAtomPx;   // (a pair's last item is computed in full)
+    const double issued = 2.0 * p.m_rows * (p.pair ? 2 * p.n_units : p.n_blocks) * (p.pair ? cols_issued : cols) *
+                          ((sh.C + G::kKStep - 1) / G::kKStep * G::kKStep);
     return snprintf(text, text_bytes,
-                    "tensor_core=1 kernel=pointwise_tma addressing=atoms filters_as=M m_rows=%d tile_px=%d acc_sets=2 items=%lld "
+                    "tensor_core=1 kernel=pointwise_tma addressing=atoms filters_as=M two_sm=%d m_rows=%d tile_px=%d acc_sets=2 items=%lld "
                     "grid=%d stages=%d resident_filters=%d filters_rounded_first=%d smem_bytes=%zu mma_useful_px=%.4f "
                     "mma_useful_flops=%.4f",
-                    p.m_rows, p.a_item * G::kAtomPx, (long long)p.tiles * p.n_blocks, p.grid, p.stages, p.stream_a ? 0 : 1,
+                    p.pair ? 1 : 0, p.pair ? 256 : p.m_rows, p.a_item * G::kAtomPx, p.items, p.grid, p.stages, p.stream_a ? 0 : 1,
                     p.round_filters ? 1 : 0, p.smem_bytes,
-                    px / cols, 2.0 * px * sh.K * sh.C / issued);
+                    px / (p.pair ? cols_issued : cols), 2.0 * px * sh.K * sh.C / issued);
 }
 
 template <bool B16>
@@ -488,25 +779,51 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
         if (!encode_map(&map_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
             return CONV2D_ERR_UNSUPPORTED;
     }
-    static size_t smem_done[64] = {};
-    if (raise_smem_limit(reinterpret_cast<const void*>(pointwise_tma_kernel<B16>), p.smem_bytes, smem_done) != cudaSuccess)
+    static size_t smem_done[64] = {}, smem_done_pair[64] = {};
+    if ((p.pair ? raise_smem_limit(reinterpret_cast<const void*>(pointwise_pair_kernel<B16>), p.smem_bytes, smem_done_pair)
+                : raise_smem_limit(reinterpret_cast<const void*>(pointwise_tma_kernel<B16>), p.smem_bytes, smem_done)) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     PwArgs a{};
     a.status = static_cast<unsigned*>(workspace);
     a.K = sh.K;
     a.fp16 = fp16 ? 1 : 0;
     a.apb = p.apb; a.total_atoms = (int)p.total_atoms; a.a_item = p.a_item; a.tiles = p.tiles;
-    a.n_blocks = p.n_blocks; a.m_rows = p.m_rows; a.items = p.tiles * p.n_blocks;
+    a.n_blocks = p.n_blocks; a.m_rows = p.m_rows; a.items = (int)p.items;
     a.cchunks = p.cchunks; a.ksteps = (sh.C + G::kKStep - 1) / G::kKStep; a.stages = p.stages;
     a.stream_a = p.stream_a ? 1 : 0;
     a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
     a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
-    a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles); a.div_nb = FastDiv(p.n_blocks);
+    a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles); a.div_nb = FastDiv(p.n_units);
     if (env_int("CONV2D_B200_TF32_VERBOSE", 0) != 0)
-        fprintf(stderr, "conv2d plan: pointwise_tma%s%s m_rows %d n_blocks %d atoms/item %d tiles %d stages %d grid %d smem %zu\n",
-                B16 ? " (16-bit)" : "", p.stream_a ? " (streamed filters)" : "", p.m_rows, p.n_blocks, p.a_item, p.tiles, p.stages, p.grid, p.smem_bytes);
-    if (launch_pdl(pointwise_tma_kernel<B16>, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
-                   map_w, map_x, map_y, a) != cudaSuccess)
+        fprintf(stderr, "conv2d plan: pointwise_tma%s%s%s m_rows %d n_blocks %d atoms/item %d tiles %d stages %d grid %d smem %zu\n",
+                B16 ? " (16-bit)" : "", p.stream_a ? " (streamed filters)" : "", p.pair ? " (two-SM)" : "", p.m_rows, p.n_blocks, p.a_item, p.tiles, p.stages, p.grid, p.smem_bytes);
+    if (p.pair) {
+        // no more pairs than the device runs at once: the items are dealt out to the pairs of the grid in turn
+        static int max_pairs[64] = {};
+        const int slot = (int)((p.smem_bytes >> 12) & 63);
+        if (max_pairs[slot] == 0) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)(sm_count() / 2 * 2));
+            cfg.blockDim = dim3(kPwThreads);
+            cfg.dynamicSmemBytes = p.smem_bytes;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, pointwise_pair_kernel<B16>, &cfg) != cudaSuccess || n < 1) {
+                (void)cudaGetLastError();
+                n = sm_count() / 2;
+            }
+            max_pairs[slot] = n;
+        }
+        const int pairs = p.grid / 2 < max_pairs[slot] ? p.grid / 2 : max_pairs[slot];
+        if (launch_pdl_cluster(pointwise_pair_kernel<B16>, dim3((unsigned)(2 * pairs)), dim3(kPwThreads), p.smem_bytes, stream, 2u,
+                               map_w, map_x, map_y, a) != cudaSuccess)
+            return CONV2D_ERR_CUDA;
+    } else if (launch_pdl(pointwise_tma_kernel<B16>, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
+                          map_w, map_x, map_y, a) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;

@@ -104,6 +104,42 @@ def test_random_pointwise_shapes(oracle, dims):
     assert_parity(run_library(xb, wb, entry="bf16"), yb_ref, yb_abs, 1e-5, f"bf16 {dims}")
 
 
+def _draw_pointwise_deep(seed):
+    """1 x 1 shapes with up to 1024 channels and 600 filters: streamed filter banks and the two-SM form."""
+    u = uniform((8,), 9600 + seed, 0.0, 1.0)
+
+    def log_int(t, lo, hi):
+        return int(round(lo * (hi / lo) ** float(t)))
+
+    N = log_int(u[0], 1, 16)
+    C = 8 * log_int(u[1], 16, 128)
+    H = log_int(u[2], 1, 24)
+    W = 8 * log_int(u[3], 1, 6)
+    K = log_int(u[4], 100, 600)
+    while N * K * C * H * W > 6e8 and N > 1:
+        N = max(1, N // 2)
+    return N, C, H, W, K, 1, 1
+
+
+POINTWISE_DEEP_SHAPES = sorted({_draw_pointwise_deep(s) for s in range(30)})
+
+
+@pytest.mark.parametrize("dims", POINTWISE_DEEP_SHAPES)
+def test_random_deep_pointwise_shapes(oracle, dims, monkeypatch):
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K, R, S = dims
+    # the planner's own choice, the one-SM form and the two-SM form in turn
+    monkeypatch.setenv("CONV2D_B200_TMA_PAIR", str((N + C // 8 + H + K) % 3))
+    assert lib.conv2d_fwd_plan_describe(*dims, ALGO_TF32).get("kernel") == "pointwise_tma"
+    assert lib.conv2d_fwd_plan_describe(*dims, 3).get("kernel") == "pointwise_tma"
+    x, w = uniform((N, C, H, W), 465), uniform((K, C, R, S), 466)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, f"tf32 {dims}")
+    xb, wb = bf16_values(x)[0], bf16_values(w)[0]
+    yb_ref, yb_abs = oracle.conv2d_oracle(xb, wb)
+    assert_parity(run_library(xb, wb, entry="bf16"), yb_ref, yb_abs, 1e-5, f"bf16 {dims}")
+
+
 def _draw_few_tiles(seed):
     """Small images with many channels and filters: the shapes whose contraction is split over a two-block cluster."""
     u = uniform((8,), 9700 + seed, 0.0, 1.0)

@@ -251,3 +251,118 @@ def test_pointwise_streamed_filters_expired_wait_is_reported(oracle, monkeypatch
     monkeypatch.delenv("CONV2D_B200_TF32_TEST_DROP_STAGE")
     y_ref, yabs = oracle.conv2d_oracle(x, w)
     assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, "after a time-out")
+
+
+# More than 128 filters: two-SM MMAs (cta_group::2) by the two blocks of a cluster, each holding one 128-filter block
+# and half of the item's pixels.  CONV2D_B200_TMA_PAIR=2 takes that form wherever it exists, so that the small
+# shapes below meet its edges: an odd number of filter blocks (the last pair's second block has no filters), a
+# ragged filter count, items that end past the batch (atoms the loads zero-fill and the stores skip), items that
+# straddle images, the resident and the streamed filter bank.
+PAIR_SHAPES = [
+    # N, C, H, W, K
+    (2, 32, 8, 8, 256),         # one pair, one ragged item
+    (1, 64, 12, 10, 200),       # second block holds 72 filters; HW = 120: ragged atoms
+    (4, 256, 14, 14, 300),      # three filter blocks = two pairs; largest resident bank
+    (3, 128, 32, 32, 256),      # items straddle images
+    (4, 512, 14, 14, 300),      # streamed filters
+    (1, 260, 12, 10, 130),      # streamed, ninth stage holds 4 channels, second block holds 2 filters
+    (40, 16, 20, 20, 384),      # several rounds of items per pair
+    (5, 100, 10, 10, 129),      # second block holds one filter
+]
+
+
+def _two_sm(dims, algo=ALGO_TF32):
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K = dims
+    plan = lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, algo)
+    return plan.get("kernel") == "pointwise_tma" and plan.get("two_sm") == 1
+
+
+@pytest.mark.parametrize("dims", PAIR_SHAPES)
+def test_pointwise_two_sm(oracle, dims, monkeypatch):
+    from oracle.conv2d_oracle import MODE_TF32_TRUNC
+    monkeypatch.setenv("CONV2D_B200_TMA_PAIR", "2")
+    assert _two_sm(dims)
+    N, C, H, W, K = dims
+    xi, wi = small_integers((N, C, H, W), 991), small_integers((K, C, 1, 1), 992)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry="general", algo=ALGO_TF32).astype(np.float64), yi_ref)
+    x, w = uniform((N, C, H, W), 993), uniform((K, C, 1, 1), 994)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    y = run_library(x, w, entry="general", algo=ALGO_TF32)
+    assert_parity(y, y_ref, yabs, TF32_TOL, f"pointwise, two-SM {dims}")
+    w_seen = _round_to_tf32(w) if C > 256 else w          # streamed fp32 filters are rounded first
+    y_t, yabs_t = oracle.conv2d_oracle(x, w_seen, mode=MODE_TF32_TRUNC)
+    assert_parity(y, y_t, yabs_t, 2e-5, f"pointwise, two-SM vs TF32-operand oracle {dims}")
+
+
+@pytest.mark.parametrize("kind", ["bf16", "fp16"])
+@pytest.mark.parametrize("dims", [(2, 32, 8, 8, 256), (1, 64, 12, 10, 200), (4, 512, 8, 8, 300), (2, 520, 12, 10, 130),
+                                  (3, 128, 32, 32, 256)])
+def test_pointwise_two_sm_16bit(oracle, dims, kind, monkeypatch):
+    from helpers import B16_TOL, bf16_values, fp16_values
+    monkeypatch.setenv("CONV2D_B200_TMA_PAIR", "2")
+    assert _two_sm(dims, 3)
+    N, C, H, W, K = dims
+    xi, wi = small_integers((N, C, H, W), 995), small_integers((K, C, 1, 1), 996)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry=kind).astype(np.float64), yi_ref)
+    conv = bf16_values if kind == "bf16" else fp16_values
+    x, w = conv(uniform((N, C, H, W), 997))[0], conv(uniform((K, C, 1, 1), 998))[0]
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry=kind), y_ref, yabs, B16_TOL, f"pointwise, two-SM {kind} {dims}")
+
+
+def test_pointwise_two_sm_item_sizes_agree(oracle, monkeypatch):
+    """Every item size of the two-SM form (2, 4, 6, 8 atoms) gives the same bits on integer inputs."""
+    dims = (3, 40, 16, 12, 200)
+    N, C, H, W, K = dims
+    monkeypatch.setenv("CONV2D_B200_TMA_PAIR", "2")
+    x, w = small_integers((N, C, H, W), 999), small_integers((K, C, 1, 1), 1000)
+    y_ref, _ = oracle.conv2d_oracle(x, w)
+    for atoms in (2, 4, 6, 8):
+        monkeypatch.setenv("CONV2D_B200_TMA_ATOMS", str(atoms))
+        assert _two_sm(dims)
+        np.testing.assert_array_equal(run_library(x, w, entry="general", algo=ALGO_TF32).astype(np.float64), y_ref)
+
+
+def test_pointwise_two_sm_is_the_default_for_deep_wide_layers(oracle):
+    """Without any switch the planner takes the two-SM form for a layer with many channels and filters."""
+    dims = (16, 512, 16, 16, 512)
+    assert _two_sm(dims)
+    N, C, H, W, K = dims
+    x, w = uniform((N, C, H, W), 1001), uniform((K, C, 1, 1), 1002)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, f"two-SM by default {dims}")
+
+
+@pytest.mark.parametrize("dims", [(2, 64, 16, 16, 256), (2, 512, 16, 16, 256)])
+def test_pointwise_two_sm_expired_wait_is_reported(oracle, dims, monkeypatch):
+    """Host-side injection on the two-SM form (resident and streamed filters): the first block of a pair never
+    copies one stage of pixels.  Both blocks of every pair give up within their bounds and meet at the closing
+    cluster barrier; the status word reports it; the next call is correct."""
+    import torch
+    import paper_1705_10591_b200 as lib
+
+    N, C, H, W, K = dims
+    monkeypatch.setenv("CONV2D_B200_TMA_PAIR", "2")
+    assert _two_sm(dims)
+    x, w = uniform((N, C, H, W), 1003), uniform((K, C, 1, 1), 1004)
+    dev = torch.device("cuda:0")
+    xd, wd = torch.from_numpy(x).to(dev), torch.from_numpy(w).to(dev)
+    y = torch.zeros((N, K, H, W), device=dev)
+    ws_bytes = lib.conv2d_fwd_workspace_size(N, C, H, W, K, 1, 1, ALGO_TF32)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    monkeypatch.setenv("CONV2D_B200_TF32_MAX_POLLS", "2048")
+    monkeypatch.setenv("CONV2D_B200_TF32_TEST_DROP_STAGE", "1")
+    lib.conv2d_fwd_general(xd.data_ptr(), wd.data_ptr(), y.data_ptr(), N, C, H, W, K, 1, 1, ALGO_TF32,
+                           ws.data_ptr(), ws_bytes, 0, stream)
+    with pytest.raises(lib.Conv2dError) as e:
+        lib.conv2d_get_status(ws.data_ptr(), stream)
+    assert e.value.status == 8                       # CONV2D_ERR_DEVICE_TIMEOUT
+    torch.cuda.synchronize()
+    monkeypatch.delenv("CONV2D_B200_TF32_MAX_POLLS")
+    monkeypatch.delenv("CONV2D_B200_TF32_TEST_DROP_STAGE")
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, "after a time-out")
