@@ -66,6 +66,9 @@ constexpr size_t kPwBookBytes = 512;      // barriers, tensor-memory slot, abort
 constexpr double kPwPairBias = 1.03;      // planner: the two-SM form is taken when its estimate is at least 3 % shorter
 constexpr int kPwMaxStreamChannels = 8192;  // streamed filters: keeps the fp32 accumulation term of the error bound small
 
+// Tensor maps over the image as (pixel in atom, channel, atom, image) whose boxes hold 1 .. 8 atoms: box i + 1 atoms.
+struct XMaps { CUtensorMap m[8]; };
+
 struct PwArgs {
     unsigned* status;
     int K;
@@ -81,6 +84,7 @@ struct PwArgs {
     int ksteps;          // K steps: ceil(C / channels per MMA)
     int stages;          // activation ring depth
     int stream_a;        // 1: too many channels for a resident bank; every ring stage carries its filter chunk too
+    int multi;           // 1: H*W is a whole number of atoms: one copy brings all atoms of an item that lie in one image
     unsigned max_polls;  // bound of every barrier wait
     int test_drop_stage; // test hook: the activation stage with this ordinal is armed but never copied (-1: none)
     FastDiv div_apb, div_tiles, div_nb;
@@ -89,7 +93,7 @@ struct PwArgs {
 template <bool B16>
 __global__ void __launch_bounds__(kPwThreads, 1)
 pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-                     const __grid_constant__ CUtensorMap map_y, const PwArgs a)
+                     const __grid_constant__ CUtensorMap map_y, const __grid_constant__ XMaps maps_x, const PwArgs a)
 {
     using G = Geom<B16>;
     constexpr int kAtomPx = G::kAtomPx, kStageCh = G::kStageCh, kAtomBytes = G::kAtomBytes;
@@ -181,6 +185,15 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                         unsigned char* dst = stage + b_off;
                         int blk;
                         int n = a.div_apb.divmod(first, blk);
+                        if (a.multi) {
+                            // one copy per image the item touches
+                            for (int left = atoms; left > 0; ++n, blk = 0) {
+                                const int cnt = min(left, a.apb - blk);
+                                tma_load_4d(dst, &maps_x.m[cnt - 1], 0, st * kStageCh, blk, n, &b_full[slot]);
+                                dst += (size_t)cnt * kAtomBytes;
+                                left -= cnt;
+                            }
+                        } else
                         for (int i = 0; i < atoms; ++i, dst += kAtomBytes) {
                             tma_load_3d(dst, &map_x, blk * kAtomPx, st * kStageCh, n, &b_full[slot]);
                             if (++blk == a.apb) { blk = 0; ++n; }
@@ -322,7 +335,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
 template <bool B16>
 __global__ void __launch_bounds__(kPwThreads, 1)
 pointwise_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-                      const __grid_constant__ CUtensorMap map_y, const PwArgs a)
+                      const __grid_constant__ CUtensorMap map_y, const __grid_constant__ XMaps maps_x, const PwArgs a)
 {
     using G = Geom<B16>;
     constexpr int kAtomPx = G::kAtomPx, kStageCh = G::kStageCh, kAtomBytes = G::kAtomBytes;
@@ -416,6 +429,14 @@ pointwise_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_co
                         unsigned char* dst = stage + b_off;
                         int blk;
                         int n = a.div_apb.divmod(first + (int)rank * half_atoms, blk);
+                        if (a.multi) {
+                            for (int left = half_atoms; left > 0; ++n, blk = 0) {
+                                const int cnt = min(left, a.apb - blk);
+                                tma_load_4d_pair(dst, &maps_x.m[cnt - 1], 0, st * kStageCh, blk, n, bar);   // (n past the batch: zeros)
+                                dst += (size_t)cnt * kAtomBytes;
+                                left -= cnt;
+                            }
+                        } else
                         for (int i = 0; i < half_atoms; ++i, dst += kAtomBytes) {
                             tma_load_3d_pair(dst, &map_x, blk * kAtomPx, st * kStageCh, n, bar);   // (n past the batch: zeros)
                             if (++blk == a.apb) { blk = 0; ++n; }
@@ -588,7 +609,7 @@ bool encode_map(CUtensorMap* map, CUtensorMapDataType type, const void* base, in
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    const cuuint32_t ones[3] = {1, 1, 1};
+    const cuuint32_t ones[4] = {1, 1, 1, 1};
     return fn(map, type, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, ones,
               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -660,6 +681,10 @@ PwPlan make_pw_variant(const Shape& sh, bool pair)
     if (fixed + 2 * stage > kPwSmemLimit) return p;
     p.stages = (int)((kPwSmemLimit - fixed) / stage);
     if (p.stages > kPwMaxStages) p.stages = kPwMaxStages;
+    {
+        const int cap = env_int("CONV2D_B200_TMA_STAGES", 0);      // tuning: a shallower ring
+        if (cap >= 2 && cap < p.stages) p.stages = cap;
+    }
     p.smem_bytes = fixed + (size_t)p.stages * stage;
     // more than half of an SM's shared memory, so that two of these blocks, which both want all 512 tensor-memory
     // columns, never share an SM
@@ -772,6 +797,20 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
                         B16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
             return CONV2D_ERR_UNSUPPORTED;
     }
+    XMaps maps_x{};
+    const bool multi = HW % G::kAtomPx == 0 && env_int("CONV2D_B200_TMA_MULTI", 1) != 0;
+    if (multi) {
+        // the image as (pixel in atom, channel, atom, image): a box of i + 1 atoms lands as i + 1 consecutive
+        // [channel][pixel] blocks, which is how the MMA descriptor walks along the pixels
+        const cuuint64_t dims[4] = {(cuuint64_t)G::kAtomPx, (cuuint64_t)sh.C, HW / G::kAtomPx, (cuuint64_t)sh.N};
+        const cuuint64_t strides[3] = {HW * es, 128, HW * es * (cuuint64_t)sh.C};
+        for (int i = 0; i < G::kMaxAtoms; ++i) {
+            const cuuint32_t box[4] = {(cuuint32_t)G::kAtomPx, (cuuint32_t)G::kStageCh, (cuuint32_t)(i + 1), 1};
+            if (!encode_map(&maps_x.m[i], in_type, x, 4, dims, strides, box,
+                            B16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+                return CONV2D_ERR_UNSUPPORTED;
+        }
+    }
     {
         const cuuint64_t dims[3] = {HW, (cuuint64_t)sh.K, (cuuint64_t)sh.N};
         const cuuint64_t strides[2] = {HW * 4, HW * 4 * (cuuint64_t)sh.K};
@@ -791,6 +830,7 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
     a.n_blocks = p.n_blocks; a.m_rows = p.m_rows; a.items = (int)p.items;
     a.cchunks = p.cchunks; a.ksteps = (sh.C + G::kKStep - 1) / G::kKStep; a.stages = p.stages;
     a.stream_a = p.stream_a ? 1 : 0;
+    a.multi = multi ? 1 : 0;
     a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
     a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
     a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles); a.div_nb = FastDiv(p.n_units);
@@ -820,10 +860,10 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
         }
         const int pairs = p.grid / 2 < max_pairs[slot] ? p.grid / 2 : max_pairs[slot];
         if (launch_pdl_cluster(pointwise_pair_kernel<B16>, dim3((unsigned)(2 * pairs)), dim3(kPwThreads), p.smem_bytes, stream, 2u,
-                               map_w, map_x, map_y, a) != cudaSuccess)
+                               map_w, map_x, map_y, maps_x, a) != cudaSuccess)
             return CONV2D_ERR_CUDA;
     } else if (launch_pdl(pointwise_tma_kernel<B16>, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
-                          map_w, map_x, map_y, a) != cudaSuccess)
+                          map_w, map_x, map_y, maps_x, a) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? CONV2D_OK : CONV2D_ERR_CUDA;

@@ -138,6 +138,11 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const void* map, int
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
                  ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* map, int c0, int c1, int c2, int c3, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar)) : "memory");
+}
 // The same loads for a pair of blocks that run two-SM MMAs (cta_group::2): the box lands in this block's shared
 // memory, the bytes are signalled on `cluster_bar`, a shared::cluster address that may name a barrier of the peer
 // block (the block that issues the pair's MMAs waits for both blocks' boxes on one barrier).
@@ -150,6 +155,11 @@ __device__ __forceinline__ void tma_load_3d_pair(void* smem_dst, const void* map
 {
     asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
                  ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(void* smem_dst, const void* map, int c0, int c1, int c2, int c3, uint32_t cluster_bar)
+{
+    asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(cluster_bar) : "memory");
 }
 // Store of one box shared -> global (elements outside the tensor are dropped); completion is tracked per thread
 // in bulk groups.

@@ -4,6 +4,9 @@
     python sweep.py special   # one input channel: filter 1x1 / 3x3 / 5x5, image size and filter count swept (Fig. 7)
     python sweep.py general   # many channels: filter 3x3 / 5x5 / 7x7, image size, channels, filters swept (Fig. 9)
     python sweep.py unit      # per-thread unit float / float2 / float4 on the 3x3 special case (matched vs unmatched)
+    python sweep.py point N C H W K R S tf32|bf16|fp32   # one shape of the general case (what the profiles capture)
+    python sweep.py pointwise # many channels, 1x1 filters: channels and filters swept up to 1024 / 512 (which form of
+                              # the kernel fed by tensor-map copies the planner took is part of each record)
 
 The swept values of the paper's figures were not published as numbers, so the grids below are this
 repository's own.  Prints one JSON line per point: shape, time, GFLOP/s and the fraction of the roofline
@@ -105,6 +108,22 @@ def main():
                         n = max(1, 65536 // (size * size))
                         for algo, name in ((lib.ALGO_TF32, "tf32"), (lib.ALGO_16BIT, "bf16"), (lib.ALGO_FFMA, "fp32")):
                             run_point(torch, lib, peaks, flush, n, c, size, size, k, r, r, algo, "general", {"algo": name})
+    elif which == "point":
+        n, c, h, w_, k, r, s_ = (int(v) for v in sys.argv[2:9])
+        name = sys.argv[9] if len(sys.argv) > 9 else "tf32"
+        algo = {"tf32": lib.ALGO_TF32, "bf16": lib.ALGO_16BIT, "fp32": lib.ALGO_FFMA}[name]
+        plan = lib.conv2d_fwd_plan_describe(n, c, h, w_, k, r, s_, algo) if algo != lib.ALGO_FFMA else {}
+        run_point(torch, lib, peaks, flush, n, c, h, w_, k, r, s_, algo, "point", {"algo": name, "plan": plan})
+    elif which == "pointwise":
+        for size in (16, 32, 64):
+            for c in (128, 256, 512, 1024):
+                for k in (128, 256, 512):
+                    n = max(1, 65536 // (size * size))
+                    for algo, name in ((lib.ALGO_TF32, "tf32"), (lib.ALGO_16BIT, "bf16")):
+                        plan = lib.conv2d_fwd_plan_describe(n, c, size, size, k, 1, 1, algo)
+                        run_point(torch, lib, peaks, flush, n, c, size, size, k, 1, 1, algo, "pointwise",
+                                  {"algo": name, "kernel": plan.get("kernel"), "two_sm": plan.get("two_sm"),
+                                   "resident_filters": plan.get("resident_filters")})
     elif which == "unit":
         os.environ["CONV2D_B200_TUNING"] = "1"      # must be set before the library's first call
         for size in (2048, 4096):
