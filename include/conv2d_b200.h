@@ -127,12 +127,17 @@ conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float*
  *   (16-byte aligned).  Its first 256 bytes are a status block: the filter
  *   re-ordering step of each call clears it, a call with CONV2D_FLAG_WEIGHTS_PACKED
  *   leaves it as it is (so a time-out stays visible until the next full call).
- *   1 x 1 filters with H*W and C multiples of 4 and C <= 256 take a kernel whose
+ *   1 x 1 filters with H*W and C multiples of 4 (C <= 8192) take a kernel whose
  *   operands and output all move by tensor-map (TMA) copies straight from and to
- *   the caller's tensors: no filter re-ordering (the flag is accepted and has no
- *   effect), the kernel clears the status block itself, and the tensor core
- *   truncates both fp32 operands to TF32 instead of the rounding to nearest the
- *   other shapes get (worst case 1.97e-3 * sum|x*w|, still inside the bound).
+ *   the caller's tensors.  Up to 256 channels: no filter re-ordering (the flag is
+ *   accepted and has no effect), the kernel clears the status block itself, and the
+ *   tensor core truncates both fp32 operands to TF32 instead of the rounding to
+ *   nearest the other shapes get (worst case 1.97e-3 * sum|x*w|, still inside the
+ *   bound).  More channels: a short kernel first rounds the filters to nearest TF32
+ *   into the workspace (what CONV2D_FLAG_WEIGHTS_PACKED then skips) and only the
+ *   image is truncated (worst case below 1.6e-3 * sum|x*w|).  With more than 128
+ *   filters the blocks may work in cluster pairs on two-SM MMAs; results do not
+ *   depend on which form runs beyond the order of the fp32 additions.
  *   Layers with few output tiles (e.g. 14 x 14 images) split the contraction over
  *   a two-block cluster; results do not depend on timing.
  * algo = AUTO: TF32 when an instance exists and the workspace suffices, else FFMA.
