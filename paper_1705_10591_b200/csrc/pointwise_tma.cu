@@ -90,35 +90,86 @@ struct PwArgs {
     FastDiv div_apb, div_tiles, div_nb;
 };
 
-template <bool B16>
+// The copy, allocation, MMA and commit instructions of the one-SM and of the two-SM (cta_group::2) form.
+template <bool PAIR>
+struct Ops {
+    // `bar`: shared::cluster address of the barrier that collects the bytes (a barrier of the pair's first block, PAIR)
+    static __device__ __forceinline__ void load_2d(void* dst, const void* map, int c0, int c1, uint32_t bar)
+    {
+        if (PAIR) tma_load_2d_pair(dst, map, c0, c1, bar); else tma_load_2d(dst, map, c0, c1, bar);
+    }
+    static __device__ __forceinline__ void load_3d(void* dst, const void* map, int c0, int c1, int c2, uint32_t bar)
+    {
+        if (PAIR) tma_load_3d_pair(dst, map, c0, c1, c2, bar); else tma_load_3d(dst, map, c0, c1, c2, bar);
+    }
+    static __device__ __forceinline__ void load_4d(void* dst, const void* map, int c0, int c1, int c2, int c3, uint32_t bar)
+    {
+        if (PAIR) tma_load_4d_pair(dst, map, c0, c1, c2, c3, bar); else tma_load_4d(dst, map, c0, c1, c2, c3, bar);
+    }
+    static __device__ __forceinline__ void alloc(uint32_t* slot, uint32_t cols)
+    {
+        if (PAIR) { tmem_alloc_pair(slot, cols); tmem_relinquish_pair(); } else { tmem_alloc(slot, cols); tmem_relinquish(); }
+    }
+    static __device__ __forceinline__ void dealloc(uint32_t taddr, uint32_t cols)
+    {
+        if (PAIR) tmem_dealloc_pair(taddr, cols); else tmem_dealloc(taddr, cols);
+    }
+    template <bool B16>
+    static __device__ __forceinline__ void mma(uint32_t d, uint64_t ad, uint64_t bd, uint32_t idesc, bool accumulate)
+    {
+        if (PAIR) { if (B16) mma_b16_pair(d, ad, bd, idesc, accumulate); else mma_tf32_pair(d, ad, bd, idesc, accumulate); }
+        else { if (B16) mma_b16(d, ad, bd, idesc, accumulate); else mma_tf32(d, ad, bd, idesc, accumulate); }
+    }
+    // arrives on `bar` (of both blocks of a pair) when the MMAs issued so far have completed
+    static __device__ __forceinline__ void commit(uint64_t* bar) { if (PAIR) mma_commit_pair_both(bar); else mma_commit(bar); }
+    static __device__ __forceinline__ void commit_local(uint64_t* bar) { if (PAIR) mma_commit_pair(bar); else mma_commit(bar); }
+};
+
+// PAIR = false: one block per work item (a pixel tile x one block of `m_rows` filters).
+// PAIR = true (more than 128 filters): the two blocks of a cluster work as a pair on 256 filters x `a_item` atoms of
+// pixels with two-SM MMAs (cta_group::2, M = 256).  Block r of the pair holds filter block 2 * pair + r (its 128 rows
+// of the M operand) and the r-th half of the item's pixels (its half of the N operand), so every byte of the image is
+// fetched once per 256 filters instead of once per 128, and each SM's tensor core reads half of the pixel operand
+// from its own shared memory.  The first block issues the MMAs; its `full` barriers collect the bytes of both
+// blocks' copies, its commits arrive on the `empty` / `acc_full` barriers of both blocks, and the write-back warps
+// of both blocks (each drains its own 128 accumulator lanes) arrive on its `acc_empty` barriers.  A pair's items
+// always span `a_item` atoms: atoms past the end of the batch are zero-filled by the loads and skipped by the stores.
+template <bool B16, bool PAIR>
 __global__ void __launch_bounds__(kPwThreads, 1)
 pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                      const __grid_constant__ CUtensorMap map_y, const __grid_constant__ XMaps maps_x, const PwArgs a)
 {
     using G = Geom<B16>;
+    using Op = Ops<PAIR>;
     constexpr int kAtomPx = G::kAtomPx, kStageCh = G::kStageCh, kAtomBytes = G::kAtomBytes;
+    constexpr uint32_t kBlocks = PAIR ? 2u : 1u;                              // blocks that work on one item
     extern __shared__ unsigned char smem_raw[];
     // swizzle atoms must start on 1024 bytes
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    const uint32_t a_chunk_bytes = (uint32_t)a.m_rows * 128u;                 // filters x 32 channels
     const bool stream_a = a.stream_a != 0;
+    const int my_atoms_max = PAIR ? a.a_item >> 1 : a.a_item;                 // atoms this block loads per stage
+    const uint32_t a_chunk_bytes = (uint32_t)a.m_rows * 128u;                 // filters x 32 channels
     const uint32_t b_off = stream_a ? a_chunk_bytes : 0u;                     // a stage: [its filter chunk,] the pixel boxes
-    const uint32_t b_stage_bytes = b_off + (uint32_t)a.a_item * kAtomBytes;
+    const uint32_t b_stage_bytes = b_off + (uint32_t)my_atoms_max * kAtomBytes;
     unsigned char* a_smem = smem;
     unsigned char* b_smem = a_smem + (stream_a ? (size_t)0 : (size_t)a.cchunks * a_chunk_bytes);
     unsigned char* o_smem = b_smem + (size_t)a.stages * b_stage_bytes;      // [kPwEpiWarps][32 rows x 128 bytes]
     uint64_t* bars = reinterpret_cast<uint64_t*>(o_smem + (size_t)kPwEpiWarps * 4096);
-    uint64_t* a_full = bars;                       // [kMaxChunks] 32-channel chunk i of the current filter block has landed
+    uint64_t* a_full = bars;                       // [kMaxChunks] 32-channel chunk i of the current filter block has landed (*)
     uint64_t* a_empty = a_full + kMaxChunks;       // [1] all MMAs that read the bank have completed
-    uint64_t* b_full = a_empty + 1;                // [kPwMaxStages]
+    uint64_t* b_full = a_empty + 1;                // [kPwMaxStages] (*)
     uint64_t* b_empty = b_full + kPwMaxStages;     // [kPwMaxStages]
     uint64_t* acc_full = b_empty + kPwMaxStages;   // [2]
-    uint64_t* acc_empty = acc_full + 2;            // [2]
+    uint64_t* acc_empty = acc_full + 2;            // [2] (*)        (*) of a pair: waited on in its first block only
     uint64_t* drain_bar = acc_empty + 2;           // [1] time-out path: the MMAs issued so far have completed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+    const bool first_block = rank == 0;                                       // issues the MMAs of the item
+    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // block, or pair of blocks
+    const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     if (tid == 0) {
         prefetch_tensormap(&map_w);
         prefetch_tensormap(&map_x);
@@ -126,87 +177,98 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         for (int i = 0; i < (stream_a ? 0 : a.cchunks); ++i) mbar_init(&a_full[i], 1);
         mbar_init(a_empty, 1);
         for (int i = 0; i < a.stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kPwEpiWarps); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kBlocks * kPwEpiWarps); }
         mbar_init(drain_bar, 1);
         *abort_flag = 0;
         fence_mbar_init();
     }
     __syncthreads();
-    if (warp == 1) { tmem_alloc(tmem_slot, 2 * kAccCols); tmem_relinquish(); }
+    if (PAIR) cluster_sync_all();       // the peer's barriers exist before a copy or a commit can signal them
+    if (warp == 1) Op::alloc(tmem_slot, 2 * kAccCols);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
-    // Everything above touched only this block's shared and tensor memory and may overlap the tail of the
+    // Everything above touched only this block's (pair's) shared and tensor memory and may overlap the tail of the
     // preceding kernel on the stream; global memory is read and written from here on.
     grid_dep_launch();
     grid_dep_wait();
     if (blockIdx.x == 0 && tid == 0) *a.status = 0u;       // (a block that gives up raises it at its very end)
 
-    // item -> (filter block, first atom, atoms): filter block-major, so that a block rarely changes its resident bank;
-    // with streamed filters pixel tile-major, so that the blocks that read the same pixels do so at the same time
-    // and all but the first find them in L2
-    auto decode = [&](int item, int& nb, int& first, int& atoms) {
+    // item -> (filter block or pair of filter blocks, first atom): filter block-major, so that a block rarely changes
+    // its resident bank; with streamed filters pixel tile-major, so that the blocks that read the same pixels do so at
+    // the same time and all but the first find them in L2
+    auto decode = [&](int item, int& unit, int& first) {
         int tile;
-        if (stream_a) tile = a.div_nb.divmod(item, nb);
-        else nb = a.div_tiles.divmod(item, tile);
+        if (stream_a) tile = a.div_nb.divmod(item, unit);
+        else unit = a.div_tiles.divmod(item, tile);
         first = tile * a.a_item;
-        atoms = min(a.a_item, a.total_atoms - first);
     };
+    // first filter row of this block for a unit
+    auto filter_row = [&](int unit) { return (PAIR ? 2 * unit + (int)rank : unit) * a.m_rows; };
 
     if (warp == 0) {
-        // ---------------- loads (one thread)
+        // ---------------- loads (one thread per block): this block's filter rows and its (half of the) pixels
         if (lane == 0) {
-            int cur_nb = -1, slot = 0, issued = 0;
+            const uint32_t a_full_addr = PAIR ? map_to_cta(smem_u32(a_full), 0) : smem_u32(a_full);   // the first block's barriers
+            const uint32_t b_full_addr = PAIR ? map_to_cta(smem_u32(b_full), 0) : smem_u32(b_full);
+            int cur_unit = -1, slot = 0, issued = 0;
             uint32_t ph = 0, a_loads = 0;
             bool alive = true;
-            for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
-                int nb, first, atoms;
-                decode(item, nb, first, atoms);
-                const bool new_bank = !stream_a && nb != cur_nb;
+            for (int item = worker; item < a.items && alive; item += n_workers) {
+                int unit, first;
+                decode(item, unit, first);
+                const int k_row = filter_row(unit);
+                // a lone block loads the atoms that exist; a block of a pair always its half of the item (past the batch: zeros)
+                const int my_atoms = PAIR ? my_atoms_max : min(a.a_item, a.total_atoms - first);
+                const int my_first = first + (PAIR ? (int)rank * my_atoms_max : 0);
+                const uint32_t stage_tx = kBlocks * (b_off + (uint32_t)my_atoms * kAtomBytes);
+                const bool new_bank = !stream_a && unit != cur_unit;
                 if (new_bank) {
                     // the bank of another filter block: wait until the MMAs on the old one are done
                     if (a_loads && !mbar_wait_bounded(a_empty, (a_loads - 1u) & 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                    cur_nb = nb;
+                    cur_unit = unit;
                     ++a_loads;
                 }
                 for (int st = 0; st < a.cchunks; ++st) {
                     if (new_bank) {
                         // chunk st of the bank goes out just ahead of the activation stage that needs it, so the
                         // first MMA waits for 16 KB of filters, not for the whole bank
-                        mbar_arrive_expect_tx(&a_full[st], a_chunk_bytes);
-                        tma_load_2d(a_smem + (size_t)st * a_chunk_bytes, &map_w, st * kStageCh, nb * a.m_rows, &a_full[st]);
+                        if (first_block) mbar_arrive_expect_tx(&a_full[st], kBlocks * a_chunk_bytes);
+                        Op::load_2d(a_smem + (size_t)st * a_chunk_bytes, &map_w, st * kStageCh, k_row, a_full_addr + 8u * (uint32_t)st);
                     }
                     if (!mbar_wait_bounded(&b_empty[slot], ph ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                     unsigned char* stage = b_smem + (size_t)slot * b_stage_bytes;
-                    mbar_arrive_expect_tx(&b_full[slot], b_off + (uint32_t)atoms * kAtomBytes);
-                    if (stream_a) tma_load_2d(stage, &map_w, st * kStageCh, nb * a.m_rows, &b_full[slot]);
-                    if (issued != a.test_drop_stage) {
+                    const uint32_t bar = b_full_addr + 8u * (uint32_t)slot;
+                    if (first_block) mbar_arrive_expect_tx(&b_full[slot], stage_tx);
+                    if (stream_a) Op::load_2d(stage, &map_w, st * kStageCh, k_row, bar);
+                    if (!(first_block && issued == a.test_drop_stage)) {     // (test hook: the first block's pixels never arrive)
                         unsigned char* dst = stage + b_off;
                         int blk;
-                        int n = a.div_apb.divmod(first, blk);
+                        int n = a.div_apb.divmod(my_first, blk);
                         if (a.multi) {
-                            // one copy per image the item touches
-                            for (int left = atoms; left > 0; ++n, blk = 0) {
+                            // one copy per image the atoms touch
+                            for (int left = my_atoms; left > 0; ++n, blk = 0) {
                                 const int cnt = min(left, a.apb - blk);
-                                tma_load_4d(dst, &maps_x.m[cnt - 1], 0, st * kStageCh, blk, n, &b_full[slot]);
+                                Op::load_4d(dst, &maps_x.m[cnt - 1], 0, st * kStageCh, blk, n, bar);
                                 dst += (size_t)cnt * kAtomBytes;
                                 left -= cnt;
                             }
                         } else
-                        for (int i = 0; i < atoms; ++i, dst += kAtomBytes) {
-                            tma_load_3d(dst, &map_x, blk * kAtomPx, st * kStageCh, n, &b_full[slot]);
-                            if (++blk == a.apb) { blk = 0; ++n; }
-                        }
+                            for (int i = 0; i < my_atoms; ++i, dst += kAtomBytes) {
+                                Op::load_3d(dst, &map_x, blk * kAtomPx, st * kStageCh, n, bar);
+                                if (++blk == a.apb) { blk = 0; ++n; }
+                            }
                     }
                     ++issued;
                     if (++slot == a.stages) { slot = 0; ph ^= 1u; }
                 }
             }
-            if (*abort_flag) {
-                // let copies already in flight land before the block's shared memory is released
+            if (*abort_flag && first_block) {
+                // let copies already in flight (of both blocks of a pair: they signal these barriers) land before the
+                // block's shared memory is released
                 uint32_t dummy = 0;
-                for (int cb = 0; cb < a.cchunks && a_loads; ++cb)
+                for (int cb = 0; cb < (stream_a ? 0 : a.cchunks) && a_loads; ++cb)
                     mbar_wait_bounded(&a_full[cb], (a_loads - 1u) & 1u, &dummy, 1u << 14);
                 const int pending = issued < a.stages ? issued : a.stages;
                 for (int i = 0; i < pending; ++i) {
@@ -216,21 +278,24 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issue (one thread)
-        if (lane == 0) {
+        // ---------------- MMA issue (one thread; of a pair: of its first block)
+        if (lane == 0 && first_block) {
             const uint32_t a_base = smem_u32(a_smem), b_base = smem_u32(b_smem);
-            int cur_nb = -1, slot = 0, buf = 0;
+            int cur_unit = -1, slot = 0, buf = 0;
             uint32_t ph = 0, a_waits = 0, acc_phase[2] = {0u, 0u};
             bool alive = true;
-            for (int item = blockIdx.x; item < a.items && alive; item += gridDim.x) {
-                int nb, first, atoms;
-                decode(item, nb, first, atoms);
-                const bool new_bank = !stream_a && nb != cur_nb;
-                cur_nb = nb;
-                if (!mbar_wait_bounded(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
+            for (int item = worker; item < a.items && alive; item += n_workers) {
+                int unit, first;
+                decode(item, unit, first);
+                const bool new_bank = !stream_a && unit != cur_unit;
+                cur_unit = unit;
+                // (of a pair: both blocks' write-back warps arrive here, the peer's with cluster-scope release)
+                if (!(PAIR ? mbar_wait_bounded_cluster(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)
+                           : mbar_wait_bounded(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls))) { alive = false; break; }
                 tc_fence_after_sync();
-                const uint32_t idesc = (B16 ? idesc_b16((uint32_t)a.m_rows, (uint32_t)(atoms * kAtomPx), a.fp16 != 0)
-                                            : idesc_tf32((uint32_t)a.m_rows, (uint32_t)(atoms * kAtomPx))) | kIdescBMajorMN;
+                const uint32_t n_cols = (uint32_t)((PAIR ? a.a_item : min(a.a_item, a.total_atoms - first)) * kAtomPx);
+                const uint32_t m = PAIR ? 256u : (uint32_t)a.m_rows;
+                const uint32_t idesc = (B16 ? idesc_b16(m, n_cols, a.fp16 != 0) : idesc_tf32(m, n_cols)) | kIdescBMajorMN;
                 const uint32_t d = tmem + (uint32_t)(buf * kAccCols);
                 bool accumulate = false;
                 for (int st = 0; st < a.cchunks && alive; ++st) {
@@ -244,303 +309,66 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     for (int kk = 0; kk < ks; ++kk) {
                         // filters: 32 bytes further inside the 128-byte rows; pixels: the next 8 (fp32) or 16 (16-bit) channel rows
                         const uint64_t a_desc = smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u);
-                        if (B16)
-                            mma_b16(d, a_desc, smem_desc_sw128(b_stage + (uint32_t)kk * 2048u, (uint32_t)kStageCh * 128u, 1024u), idesc, accumulate);
-                        else
-                            mma_tf32(d, a_desc, smem_desc_mn_sw128_32b(b_stage + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u), idesc, accumulate);
+                        const uint64_t b_desc = B16 ? smem_desc_sw128(b_stage + (uint32_t)kk * 2048u, (uint32_t)kStageCh * 128u, 1024u)
+                                                    : smem_desc_mn_sw128_32b(b_stage + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u);
+                        Op::template mma<B16>(d, a_desc, b_desc, idesc, accumulate);
                         accumulate = true;
                     }
-                    mma_commit(&b_empty[slot]);
+                    Op::commit(&b_empty[slot]);
                     if (++slot == a.stages) { slot = 0; ph ^= 1u; }
                 }
                 if (!alive) break;
                 if (new_bank) ++a_waits;
-                mma_commit(&acc_full[buf]);
-                // the next item of this block uses another filter block: tell the loader when this bank is free
-                const int next = item + (int)gridDim.x;
-                if (!stream_a && next < a.items && a.div_tiles.div(next) != nb) mma_commit(a_empty);
+                Op::commit(&acc_full[buf]);
+                // the next item of this block uses another filter block: tell the loaders when this bank is free
+                const int next = item + n_workers;
+                if (!stream_a && next < a.items && a.div_tiles.div(next) != unit) Op::commit(a_empty);
                 acc_phase[buf] ^= 1u;
                 buf ^= 1;
             }
             if (!alive) {
-                mma_commit(drain_bar);
+                Op::commit_local(drain_bar);
                 uint32_t dummy = 0;
                 mbar_wait_bounded(drain_bar, 0u, &dummy, 1u << 16);
             }
         }
     } else {
         // ---------------- write-back: tensor memory -> registers -> swizzled tile -> tensor-map store
+        // (of a pair: both blocks, each its own 128 filters and all pixels of the item)
         const int ew = warp - 2;
         const int quarter = warp & 3;                       // tensor-memory lanes this warp may read
-        const int half = ew >> 2;                           // the two warps of a quarter take alternate atoms
+        const int half = ew >> 2;                           // the two warps of a quarter take alternate 32-pixel blocks
         unsigned char* tile = o_smem + (size_t)ew * 4096;
         const int rows_q = a.m_rows / 4;                    // filters per lane quarter: 32, or 16 (M = 64: lanes 0-15)
+        const uint32_t acc_empty_first = PAIR ? map_to_cta(smem_u32(acc_empty), 0) : 0u;
         bool alive = true;
         int li = 0;
-        for (int item = blockIdx.x; item < a.items; item += gridDim.x, ++li) {
-            int nb, first, atoms;
-            decode(item, nb, first, atoms);
+        for (int item = worker; item < a.items; item += n_workers, ++li) {
+            int unit, first;
+            decode(item, unit, first);
+            const int atoms = min(a.a_item, a.total_atoms - first);          // atoms of the item that exist
             const int buf = li & 1;
             const uint32_t acc_phase = (uint32_t)(li >> 1) & 1u;
             alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag, a.max_polls));
             if (!alive) break;
             tc_fence_after_sync();
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccCols);
-            const int k0 = nb * a.m_rows + quarter * rows_q;
+            const int k0 = filter_row(unit) + quarter * rows_q;
             constexpr int kBpa = kAtomPx / 32;                  // 32-column blocks per atom
-            for (int i = half; i < atoms * kBpa; i += 2) {
-                uint32_t v[32];
-                tmem_ld32(lane_base + (uint32_t)(i * 32), v);
-                tmem_ld_wait();
-                if (lane == 0) bulk_wait_group_read<0>();       // the previous store has read the tile
-                __syncwarp();
-                if (lane < rows_q) {
-                    // row = this lane's filter, 32 pixels = eight 16-byte chunks, chunk c stored at c ^ (row & 7)
-                    unsigned char* row = tile + lane * 128;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        *reinterpret_cast<uint4*>(row + ((c ^ (lane & 7)) << 4)) = make_uint4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0 && k0 < a.K) {
-                    int blk;
-                    const int n = a.div_apb.divmod(first + i / kBpa, blk);
-                    tma_store_3d(&map_y, blk * kAtomPx + (i % kBpa) * 32, k0, n, tile);
-                    bulk_commit_group();
-                }
-            }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[buf]);
-        }
-        if (lane == 0) bulk_wait_group<0>();                 // this thread's stores are complete
-    }
-
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 2 * kAccCols);
-    if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
-}
-
-// ---------------------------------------------------------------- two-SM variant
-// More than 128 filters: the two blocks of a cluster work as a pair on 256 filters x `a_item` atoms of pixels with
-// two-SM MMAs (cta_group::2, M = 256).  Block r of the pair holds filter block 2 * pair + r (its 128 rows of the M
-// operand) and the r-th half of the item's pixels (its half of the N operand), so every byte of the image is
-// fetched once per 256 filters instead of once per 128, and each SM's tensor core reads half of the pixel operand
-// from its own shared memory.  The first block issues the MMAs; its `full` barriers collect the bytes of both
-// blocks' copies, its commits arrive on the `empty` / `acc_full` barriers of both blocks, and the write-back warps
-// of both blocks (each drains its own 128 accumulator lanes) arrive on its `acc_empty` barriers.  Items always
-// span `a_item` atoms: atoms past the end of the batch are zero-filled by the loads and skipped by the stores.
-template <bool B16>
-__global__ void __launch_bounds__(kPwThreads, 1)
-pointwise_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-                      const __grid_constant__ CUtensorMap map_y, const __grid_constant__ XMaps maps_x, const PwArgs a)
-{
-    using G = Geom<B16>;
-    constexpr int kAtomPx = G::kAtomPx, kStageCh = G::kStageCh, kAtomBytes = G::kAtomBytes;
-    constexpr int kRows = 128;                                                // filters per block of the pair
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    const bool stream_a = a.stream_a != 0;
-    const int half_atoms = a.a_item >> 1;                                     // atoms this block loads per stage
-    const uint32_t a_chunk_bytes = (uint32_t)kRows * 128u;
-    const uint32_t b_off = stream_a ? a_chunk_bytes : 0u;
-    const uint32_t stage_tx = b_off + (uint32_t)half_atoms * kAtomBytes;      // bytes one block's copies bring per stage
-    const uint32_t b_stage_bytes = stage_tx;
-    unsigned char* a_smem = smem;
-    unsigned char* b_smem = a_smem + (stream_a ? (size_t)0 : (size_t)a.cchunks * a_chunk_bytes);
-    unsigned char* o_smem = b_smem + (size_t)a.stages * b_stage_bytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(o_smem + (size_t)kPwEpiWarps * 4096);
-    uint64_t* a_full = bars;                       // [kMaxChunks]   (waited on in the first block only)
-    uint64_t* a_empty = a_full + kMaxChunks;       // [1]
-    uint64_t* b_full = a_empty + 1;                // [kPwMaxStages] (first block only)
-    uint64_t* b_empty = b_full + kPwMaxStages;     // [kPwMaxStages]
-    uint64_t* acc_full = b_empty + kPwMaxStages;   // [2]
-    uint64_t* acc_empty = acc_full + 2;            // [2]            (first block only; both blocks' warps arrive)
-    uint64_t* drain_bar = acc_empty + 2;           // [1]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
-    volatile uint32_t* abort_flag = tmem_slot + 1;
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t rank = cluster_ctarank();
-    const bool first_block = rank == 0;
-    const int pair_id = (int)(blockIdx.x >> 1), n_pairs_running = (int)(gridDim.x >> 1);
-    if (tid == 0) {
-        prefetch_tensormap(&map_w);
-        prefetch_tensormap(&map_x);
-        prefetch_tensormap(&map_y);
-        for (int i = 0; i < (stream_a ? 0 : a.cchunks); ++i) mbar_init(&a_full[i], 1);
-        mbar_init(a_empty, 1);
-        for (int i = 0; i < a.stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 2 * kPwEpiWarps); }
-        mbar_init(drain_bar, 1);
-        *abort_flag = 0;
-        fence_mbar_init();
-    }
-    __syncthreads();
-    cluster_sync_all();             // the peer's barriers exist before a copy or a commit can signal them
-    if (warp == 1) { tmem_alloc_pair(tmem_slot, 2 * kAccCols); tmem_relinquish_pair(); }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem = *tmem_slot;
-    grid_dep_launch();
-    grid_dep_wait();
-    if (blockIdx.x == 0 && tid == 0) *a.status = 0u;
-
-    // item -> (pair of filter blocks, first atom): as in the one-SM kernel, with pairs in place of filter blocks
-    auto decode = [&](int item, int& pr, int& first) {
-        int tile;
-        if (stream_a) tile = a.div_nb.divmod(item, pr);
-        else pr = a.div_tiles.divmod(item, tile);
-        first = tile * a.a_item;
-    };
-
-    if (warp == 0) {
-        // ---------------- loads (one thread per block): this block's filter rows and its half of the pixels
-        if (lane == 0) {
-            const uint32_t a_full_first = map_to_cta(smem_u32(a_full), 0);     // the first block's barriers
-            const uint32_t b_full_first = map_to_cta(smem_u32(b_full), 0);
-            int cur_pr = -1, slot = 0, issued = 0;
-            uint32_t ph = 0, a_loads = 0;
-            bool alive = true;
-            for (int item = pair_id; item < a.items && alive; item += n_pairs_running) {
-                int pr, first;
-                decode(item, pr, first);
-                const int k_row = (2 * pr + (int)rank) * kRows;
-                const bool new_bank = !stream_a && pr != cur_pr;
-                if (new_bank) {
-                    if (a_loads && !mbar_wait_bounded(a_empty, (a_loads - 1u) & 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                    cur_pr = pr;
-                    ++a_loads;
-                }
-                for (int st = 0; st < a.cchunks; ++st) {
-                    if (new_bank) {
-                        if (first_block) mbar_arrive_expect_tx(&a_full[st], 2u * a_chunk_bytes);
-                        tma_load_2d_pair(a_smem + (size_t)st * a_chunk_bytes, &map_w, st * kStageCh, k_row, a_full_first + 8u * (uint32_t)st);
-                    }
-                    if (!mbar_wait_bounded(&b_empty[slot], ph ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                    unsigned char* stage = b_smem + (size_t)slot * b_stage_bytes;
-                    const uint32_t bar = b_full_first + 8u * (uint32_t)slot;
-                    if (first_block) mbar_arrive_expect_tx(&b_full[slot], 2u * stage_tx);
-                    if (stream_a) tma_load_2d_pair(stage, &map_w, st * kStageCh, k_row, bar);
-                    if (!(first_block && issued == a.test_drop_stage)) {
-                        unsigned char* dst = stage + b_off;
-                        int blk;
-                        int n = a.div_apb.divmod(first + (int)rank * half_atoms, blk);
-                        if (a.multi) {
-                            for (int left = half_atoms; left > 0; ++n, blk = 0) {
-                                const int cnt = min(left, a.apb - blk);
-                                tma_load_4d_pair(dst, &maps_x.m[cnt - 1], 0, st * kStageCh, blk, n, bar);   // (n past the batch: zeros)
-                                dst += (size_t)cnt * kAtomBytes;
-                                left -= cnt;
-                            }
-                        } else
-                        for (int i = 0; i < half_atoms; ++i, dst += kAtomBytes) {
-                            tma_load_3d_pair(dst, &map_x, blk * kAtomPx, st * kStageCh, n, bar);   // (n past the batch: zeros)
-                            if (++blk == a.apb) { blk = 0; ++n; }
-                        }
-                    }
-                    ++issued;
-                    if (++slot == a.stages) { slot = 0; ph ^= 1u; }
-                }
-            }
-            if (*abort_flag && first_block) {
-                // let copies already in flight (of both blocks: they signal these barriers) land before the blocks leave
-                uint32_t dummy = 0;
-                for (int cb = 0; cb < (stream_a ? 0 : a.cchunks) && a_loads; ++cb)
-                    mbar_wait_bounded(&a_full[cb], (a_loads - 1u) & 1u, &dummy, 1u << 14);
-                const int pending = issued < a.stages ? issued : a.stages;
-                for (int i = 0; i < pending; ++i) {
-                    const int it = issued - 1 - i;
-                    mbar_wait_bounded(&b_full[it % a.stages], (uint32_t)(it / a.stages) & 1u, &dummy, 1u << 14);
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ---------------- MMA issue (one thread of the first block)
-        if (lane == 0 && first_block) {
-            const uint32_t a_base = smem_u32(a_smem), b_base = smem_u32(b_smem);
-            int cur_pr = -1, slot = 0, buf = 0;
-            uint32_t ph = 0, a_waits = 0, acc_phase[2] = {0u, 0u};
-            bool alive = true;
-            const uint32_t n_cols = (uint32_t)(a.a_item * kAtomPx);
-            const uint32_t idesc = (B16 ? idesc_b16(256u, n_cols, a.fp16 != 0) : idesc_tf32(256u, n_cols)) | kIdescBMajorMN;
-            for (int item = pair_id; item < a.items && alive; item += n_pairs_running) {
-                int pr, first;
-                decode(item, pr, first);
-                const bool new_bank = !stream_a && pr != cur_pr;
-                cur_pr = pr;
-                if (!mbar_wait_bounded_cluster(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                tc_fence_after_sync();
-                const uint32_t d = tmem + (uint32_t)(buf * kAccCols);
-                bool accumulate = false;
-                for (int st = 0; st < a.cchunks && alive; ++st) {
-                    if (new_bank && !mbar_wait_bounded(&a_full[st], a_waits & 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                    if (!mbar_wait_bounded(&b_full[slot], ph, abort_flag, a.max_polls)) { alive = false; break; }
-                    tc_fence_after_sync();
-                    const uint32_t stage = b_base + (uint32_t)slot * b_stage_bytes;
-                    const uint32_t a_chunk = stream_a ? stage : a_base + (uint32_t)st * a_chunk_bytes;
-                    const uint32_t b_stage = stage + b_off;
-                    const int ks = min(4, a.ksteps - st * 4);
-                    for (int kk = 0; kk < ks; ++kk) {
-                        const uint64_t a_desc = smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u);
-                        if (B16)
-                            mma_b16_pair(d, a_desc, smem_desc_sw128(b_stage + (uint32_t)kk * 2048u, (uint32_t)kStageCh * 128u, 1024u), idesc, accumulate);
-                        else
-                            mma_tf32_pair(d, a_desc, smem_desc_mn_sw128_32b(b_stage + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u), idesc, accumulate);
-                        accumulate = true;
-                    }
-                    mma_commit_pair_both(&b_empty[slot]);
-                    if (++slot == a.stages) { slot = 0; ph ^= 1u; }
-                }
-                if (!alive) break;
-                if (new_bank) ++a_waits;
-                mma_commit_pair_both(&acc_full[buf]);
-                const int next = item + n_pairs_running;
-                if (!stream_a && next < a.items && a.div_tiles.div(next) != pr) mma_commit_pair_both(a_empty);
-                acc_phase[buf] ^= 1u;
-                buf ^= 1;
-            }
-            if (!alive) {
-                mma_commit_pair(drain_bar);
-                uint32_t dummy = 0;
-                mbar_wait_bounded(drain_bar, 0u, &dummy, 1u << 16);
-            }
-        }
-    } else {
-        // ---------------- write-back (both blocks): this block's 128 filters, all pixels of the item
-        const int ew = warp - 2;
-        const int quarter = warp & 3;
-        const int half = ew >> 2;
-        unsigned char* tile = o_smem + (size_t)ew * 4096;
-        const uint32_t acc_empty_first = map_to_cta(smem_u32(acc_empty), 0);
-        bool alive = true;
-        int li = 0;
-        for (int item = pair_id; item < a.items; item += n_pairs_running, ++li) {
-            int pr, first;
-            decode(item, pr, first);
-            const int atoms = min(a.a_item, a.total_atoms - first);
-            const int buf = li & 1;
-            const uint32_t acc_phase = (uint32_t)(li >> 1) & 1u;
-            alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag, a.max_polls));
-            if (!alive) break;
-            tc_fence_after_sync();
-            const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccCols);
-            const int k0 = (2 * pr + (int)rank) * kRows + quarter * 32;
-            constexpr int kBpa = kAtomPx / 32;
             if (k0 < a.K)
                 for (int i = half; i < atoms * kBpa; i += 2) {
                     uint32_t v[32];
                     tmem_ld32(lane_base + (uint32_t)(i * 32), v);
                     tmem_ld_wait();
-                    if (lane == 0) bulk_wait_group_read<0>();
+                    if (lane == 0) bulk_wait_group_read<0>();       // the previous store has read the tile
                     __syncwarp();
-                    unsigned char* row = tile + lane * 128;
+                    if (lane < rows_q) {
+                        // row = this lane's filter, 32 pixels = eight 16-byte chunks, chunk c stored at c ^ (row & 7)
+                        unsigned char* row = tile + lane * 128;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        *reinterpret_cast<uint4*>(row + ((c ^ (lane & 7)) << 4)) = make_uint4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                        for (int c = 0; c < 8; ++c)
+                            *reinterpret_cast<uint4*>(row + ((c ^ (lane & 7)) << 4)) = make_uint4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                    }
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
@@ -557,15 +385,16 @@ pointwise_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_co
                 else mbar_arrive_remote(acc_empty_first + 8u * (uint32_t)buf);
             }
         }
-        if (lane == 0) bulk_wait_group<0>();
+        if (lane == 0) bulk_wait_group<0>();                 // this thread's stores are complete
     }
 
     tc_fence_before_sync();
     __syncthreads();
-    cluster_sync_all();             // neither block leaves while the peer may still signal its barriers or read its operands
-    if (warp == 1) tmem_dealloc_pair(tmem, 2 * kAccCols);
+    if (PAIR) cluster_sync_all();       // neither block leaves while the peer may still signal its barriers or read its operands
+    if (warp == 1) Op::dealloc(tmem, 2 * kAccCols);
     if (tid == 0 && *abort_flag) atomicExch(a.status, 1u);
 }
+
 
 // Streamed filters, fp32 only: the filters rounded to the nearest TF32 value, into the workspace, so that only the
 // image is truncated by the tensor core and the error bound holds for any channel count.  Also clears the status
@@ -819,8 +648,8 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
             return CONV2D_ERR_UNSUPPORTED;
     }
     static size_t smem_done[64] = {}, smem_done_pair[64] = {};
-    if ((p.pair ? raise_smem_limit(reinterpret_cast<const void*>(pointwise_pair_kernel<B16>), p.smem_bytes, smem_done_pair)
-                : raise_smem_limit(reinterpret_cast<const void*>(pointwise_tma_kernel<B16>), p.smem_bytes, smem_done)) != cudaSuccess)
+    if ((p.pair ? raise_smem_limit(reinterpret_cast<const void*>(pointwise_tma_kernel<B16, true>), p.smem_bytes, smem_done_pair)
+                : raise_smem_limit(reinterpret_cast<const void*>(pointwise_tma_kernel<B16, false>), p.smem_bytes, smem_done)) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     PwArgs a{};
     a.status = static_cast<unsigned*>(workspace);
@@ -852,17 +681,17 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
             cfg.attrs = attr;
             cfg.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, pointwise_pair_kernel<B16>, &cfg) != cudaSuccess || n < 1) {
+            if (cudaOccupancyMaxActiveClusters(&n, pointwise_tma_kernel<B16, true>, &cfg) != cudaSuccess || n < 1) {
                 (void)cudaGetLastError();
                 n = sm_count() / 2;
             }
             max_pairs[slot] = n;
         }
         const int pairs = p.grid / 2 < max_pairs[slot] ? p.grid / 2 : max_pairs[slot];
-        if (launch_pdl_cluster(pointwise_pair_kernel<B16>, dim3((unsigned)(2 * pairs)), dim3(kPwThreads), p.smem_bytes, stream, 2u,
+        if (launch_pdl_cluster(pointwise_tma_kernel<B16, true>, dim3((unsigned)(2 * pairs)), dim3(kPwThreads), p.smem_bytes, stream, 2u,
                                map_w, map_x, map_y, maps_x, a) != cudaSuccess)
             return CONV2D_ERR_CUDA;
-    } else if (launch_pdl(pointwise_tma_kernel<B16>, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
+    } else if (launch_pdl(pointwise_tma_kernel<B16, false>, dim3((unsigned)p.grid), dim3(kPwThreads), p.smem_bytes, stream,
                           map_w, map_x, map_y, maps_x, a) != cudaSuccess)
         return CONV2D_ERR_CUDA;
     count_launch();
