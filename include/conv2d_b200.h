@@ -137,7 +137,10 @@ conv2d_status_t conv2d_fwd_single_channel(const float* x, const float* w, float*
  *   into the workspace (what CONV2D_FLAG_WEIGHTS_PACKED then skips) and only the
  *   image is truncated (worst case below 1.6e-3 * sum|x*w|).  With more than 128
  *   filters the blocks may work in cluster pairs on two-SM MMAs; results do not
- *   depend on which form runs beyond the order of the fp32 additions.
+ *   depend on which form runs beyond the order of the fp32 additions.  Very deep
+ *   layers on few pixels (1536 channels or more) may be computed as two halves of
+ *   the contraction that are added into y after the call has zero-filled it; the
+ *   result does not depend on timing.
  *   Layers with few output tiles (e.g. 14 x 14 images) split the contraction over
  *   a two-block cluster; results do not depend on timing.
  * algo = AUTO: TF32 when an instance exists and the workspace suffices, else FFMA.

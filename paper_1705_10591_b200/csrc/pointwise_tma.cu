@@ -59,7 +59,6 @@ struct Geom {
     static constexpr int kStageCh = 4 * kKStep;            // channels per activation stage = per 128-byte filter row
     static constexpr int kAtomBytes = 128 * kStageCh;      // one box of kAtomPx pixels x kStageCh channels
     static constexpr int kMaxAtoms = kAccCols / kAtomPx;   // atoms per work item: N <= 256 columns per MMA
-    static constexpr int kMaxChannels = kMaxChunks * kStageCh;   // the filter bank of a block must stay resident
 };
 constexpr size_t kPwSmemLimit = 227 * 1024;
 constexpr size_t kPwBookBytes = 512;      // barriers, tensor-memory slot, abort flag
@@ -81,6 +80,8 @@ struct PwArgs {
     int m_rows;          // rows of the M operand: 64 (at most 64 filters) or 128
     int items;           // tiles * n_blocks, numbered filter block-major
     int cchunks;         // channel chunks of one stage each: ceil(C / channels per stage)
+    int ksplit;          // 1, or 2: the channel chunks of a tile are shared out to two work items that both add into a zeroed y
+    int cpart;           // channel chunks per work item: ceil(cchunks / ksplit)
     int ksteps;          // K steps: ceil(C / channels per MMA)
     int stages;          // activation ring depth
     int stream_a;        // 1: too many channels for a resident bank; every ring stage carries its filter chunk too
@@ -152,7 +153,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     const uint32_t b_off = stream_a ? a_chunk_bytes : 0u;                     // a stage: [its filter chunk,] the pixel boxes
     const uint32_t b_stage_bytes = b_off + (uint32_t)my_atoms_max * kAtomBytes;
     unsigned char* a_smem = smem;
-    unsigned char* b_smem = a_smem + (stream_a ? (size_t)0 : (size_t)a.cchunks * a_chunk_bytes);
+    unsigned char* b_smem = a_smem + (stream_a ? (size_t)0 : (size_t)a.cpart * a_chunk_bytes);
     unsigned char* o_smem = b_smem + (size_t)a.stages * b_stage_bytes;      // [kPwEpiWarps][32 rows x 128 bytes]
     uint64_t* bars = reinterpret_cast<uint64_t*>(o_smem + (size_t)kPwEpiWarps * 4096);
     uint64_t* a_full = bars;                       // [kMaxChunks] 32-channel chunk i of the current filter block has landed (*)
@@ -174,7 +175,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         prefetch_tensormap(&map_w);
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_y);
-        for (int i = 0; i < (stream_a ? 0 : a.cchunks); ++i) mbar_init(&a_full[i], 1);
+        for (int i = 0; i < (stream_a ? 0 : a.cpart); ++i) mbar_init(&a_full[i], 1);
         mbar_init(a_empty, 1);
         for (int i = 0; i < a.stages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kBlocks * kPwEpiWarps); }
@@ -195,14 +196,20 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     grid_dep_wait();
     if (blockIdx.x == 0 && tid == 0) *a.status = 0u;       // (a block that gives up raises it at its very end)
 
-    // item -> (filter block or pair of filter blocks, first atom): filter block-major, so that a block rarely changes
-    // its resident bank; with streamed filters pixel tile-major, so that the blocks that read the same pixels do so at
-    // the same time and all but the first find them in L2
-    auto decode = [&](int item, int& unit, int& first) {
+    // item -> (bank = (filter block or pair of filter blocks) * ksplit + part of the channels, first atom): bank-major,
+    // so that a block rarely changes its resident bank; with streamed filters pixel tile-major, so that the blocks
+    // that read the same pixels do so at the same time and all but the first find them in L2
+    auto decode = [&](int item, int& bank, int& first) {
         int tile;
-        if (stream_a) tile = a.div_nb.divmod(item, unit);
-        else unit = a.div_tiles.divmod(item, tile);
+        if (stream_a) tile = a.div_nb.divmod(item, bank);
+        else bank = a.div_tiles.divmod(item, tile);
         first = tile * a.a_item;
+    };
+    // bank -> filter unit, first channel chunk and number of chunks of its part of the contraction
+    auto split = [&](int bank, int& unit, int& c_lo, int& c_n) {
+        unit = a.ksplit == 2 ? bank >> 1 : bank;
+        c_lo = a.ksplit == 2 ? (bank & 1) * a.cpart : 0;
+        c_n = min(a.cpart, a.cchunks - c_lo);
     };
     // first filter row of this block for a unit
     auto filter_row = [&](int unit) { return (PAIR ? 2 * unit + (int)rank : unit) * a.m_rows; };
@@ -212,36 +219,38 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         if (lane == 0) {
             const uint32_t a_full_addr = PAIR ? map_to_cta(smem_u32(a_full), 0) : smem_u32(a_full);   // the first block's barriers
             const uint32_t b_full_addr = PAIR ? map_to_cta(smem_u32(b_full), 0) : smem_u32(b_full);
-            int cur_unit = -1, slot = 0, issued = 0;
+            int cur_bank = -1, slot = 0, issued = 0;
             uint32_t ph = 0, a_loads = 0;
             bool alive = true;
             for (int item = worker; item < a.items && alive; item += n_workers) {
-                int unit, first;
-                decode(item, unit, first);
+                int bank, first, unit, c_lo, c_n;
+                decode(item, bank, first);
+                split(bank, unit, c_lo, c_n);
                 const int k_row = filter_row(unit);
                 // a lone block loads the atoms that exist; a block of a pair always its half of the item (past the batch: zeros)
                 const int my_atoms = PAIR ? my_atoms_max : min(a.a_item, a.total_atoms - first);
                 const int my_first = first + (PAIR ? (int)rank * my_atoms_max : 0);
                 const uint32_t stage_tx = kBlocks * (b_off + (uint32_t)my_atoms * kAtomBytes);
-                const bool new_bank = !stream_a && unit != cur_unit;
+                const bool new_bank = !stream_a && bank != cur_bank;
                 if (new_bank) {
-                    // the bank of another filter block: wait until the MMAs on the old one are done
+                    // another bank: wait until the MMAs on the old one are done
                     if (a_loads && !mbar_wait_bounded(a_empty, (a_loads - 1u) & 1u, abort_flag, a.max_polls)) { alive = false; break; }
-                    cur_unit = unit;
+                    cur_bank = bank;
                     ++a_loads;
                 }
-                for (int st = 0; st < a.cchunks; ++st) {
+                for (int st = 0; st < c_n; ++st) {
+                    const int ch = (c_lo + st) * kStageCh;       // first channel of this stage
                     if (new_bank) {
                         // chunk st of the bank goes out just ahead of the activation stage that needs it, so the
                         // first MMA waits for 16 KB of filters, not for the whole bank
                         if (first_block) mbar_arrive_expect_tx(&a_full[st], kBlocks * a_chunk_bytes);
-                        Op::load_2d(a_smem + (size_t)st * a_chunk_bytes, &map_w, st * kStageCh, k_row, a_full_addr + 8u * (uint32_t)st);
+                        Op::load_2d(a_smem + (size_t)st * a_chunk_bytes, &map_w, ch, k_row, a_full_addr + 8u * (uint32_t)st);
                     }
                     if (!mbar_wait_bounded(&b_empty[slot], ph ^ 1u, abort_flag, a.max_polls)) { alive = false; break; }
                     unsigned char* stage = b_smem + (size_t)slot * b_stage_bytes;
                     const uint32_t bar = b_full_addr + 8u * (uint32_t)slot;
                     if (first_block) mbar_arrive_expect_tx(&b_full[slot], stage_tx);
-                    if (stream_a) Op::load_2d(stage, &map_w, st * kStageCh, k_row, bar);
+                    if (stream_a) Op::load_2d(stage, &map_w, ch, k_row, bar);
                     if (!(first_block && issued == a.test_drop_stage)) {     // (test hook: the first block's pixels never arrive)
                         unsigned char* dst = stage + b_off;
                         int blk;
@@ -250,13 +259,13 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                             // one copy per image the atoms touch
                             for (int left = my_atoms; left > 0; ++n, blk = 0) {
                                 const int cnt = min(left, a.apb - blk);
-                                Op::load_4d(dst, &maps_x.m[cnt - 1], 0, st * kStageCh, blk, n, bar);
+                                Op::load_4d(dst, &maps_x.m[cnt - 1], 0, ch, blk, n, bar);
                                 dst += (size_t)cnt * kAtomBytes;
                                 left -= cnt;
                             }
                         } else
                             for (int i = 0; i < my_atoms; ++i, dst += kAtomBytes) {
-                                Op::load_3d(dst, &map_x, blk * kAtomPx, st * kStageCh, n, bar);
+                                Op::load_3d(dst, &map_x, blk * kAtomPx, ch, n, bar);
                                 if (++blk == a.apb) { blk = 0; ++n; }
                             }
                     }
@@ -268,7 +277,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 // let copies already in flight (of both blocks of a pair: they signal these barriers) land before the
                 // block's shared memory is released
                 uint32_t dummy = 0;
-                for (int cb = 0; cb < (stream_a ? 0 : a.cchunks) && a_loads; ++cb)
+                for (int cb = 0; cb < (stream_a ? 0 : a.cpart) && a_loads; ++cb)
                     mbar_wait_bounded(&a_full[cb], (a_loads - 1u) & 1u, &dummy, 1u << 14);
                 const int pending = issued < a.stages ? issued : a.stages;
                 for (int i = 0; i < pending; ++i) {
@@ -281,14 +290,15 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         // ---------------- MMA issue (one thread; of a pair: of its first block)
         if (lane == 0 && first_block) {
             const uint32_t a_base = smem_u32(a_smem), b_base = smem_u32(b_smem);
-            int cur_unit = -1, slot = 0, buf = 0;
+            int cur_bank = -1, slot = 0, buf = 0;
             uint32_t ph = 0, a_waits = 0, acc_phase[2] = {0u, 0u};
             bool alive = true;
             for (int item = worker; item < a.items && alive; item += n_workers) {
-                int unit, first;
-                decode(item, unit, first);
-                const bool new_bank = !stream_a && unit != cur_unit;
-                cur_unit = unit;
+                int bank, first, unit, c_lo, c_n;
+                decode(item, bank, first);
+                split(bank, unit, c_lo, c_n);
+                const bool new_bank = !stream_a && bank != cur_bank;
+                cur_bank = bank;
                 // (of a pair: both blocks' write-back warps arrive here, the peer's with cluster-scope release)
                 if (!(PAIR ? mbar_wait_bounded_cluster(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)
                            : mbar_wait_bounded(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls))) { alive = false; break; }
@@ -298,14 +308,14 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 const uint32_t idesc = (B16 ? idesc_b16(m, n_cols, a.fp16 != 0) : idesc_tf32(m, n_cols)) | kIdescBMajorMN;
                 const uint32_t d = tmem + (uint32_t)(buf * kAccCols);
                 bool accumulate = false;
-                for (int st = 0; st < a.cchunks && alive; ++st) {
+                for (int st = 0; st < c_n && alive; ++st) {
                     if (new_bank && !mbar_wait_bounded(&a_full[st], a_waits & 1u, abort_flag, a.max_polls)) { alive = false; break; }
                     if (!mbar_wait_bounded(&b_full[slot], ph, abort_flag, a.max_polls)) { alive = false; break; }
                     tc_fence_after_sync();
                     const uint32_t stage = b_base + (uint32_t)slot * b_stage_bytes;
                     const uint32_t a_chunk = stream_a ? stage : a_base + (uint32_t)st * a_chunk_bytes;
                     const uint32_t b_stage = stage + b_off;
-                    const int ks = min(4, a.ksteps - st * 4);
+                    const int ks = min(4, a.ksteps - (c_lo + st) * 4);
                     for (int kk = 0; kk < ks; ++kk) {
                         // filters: 32 bytes further inside the 128-byte rows; pixels: the next 8 (fp32) or 16 (16-bit) channel rows
                         const uint64_t a_desc = smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u);
@@ -322,7 +332,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 Op::commit(&acc_full[buf]);
                 // the next item of this block uses another filter block: tell the loaders when this bank is free
                 const int next = item + n_workers;
-                if (!stream_a && next < a.items && a.div_tiles.div(next) != unit) Op::commit(a_empty);
+                if (!stream_a && next < a.items && a.div_tiles.div(next) != bank) Op::commit(a_empty);
                 acc_phase[buf] ^= 1u;
                 buf ^= 1;
             }
@@ -344,8 +354,9 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         bool alive = true;
         int li = 0;
         for (int item = worker; item < a.items; item += n_workers, ++li) {
-            int unit, first;
-            decode(item, unit, first);
+            int bank, first, unit, c_lo, c_n;
+            decode(item, bank, first);
+            split(bank, unit, c_lo, c_n);
             const int atoms = min(a.a_item, a.total_atoms - first);          // atoms of the item that exist
             const int buf = li & 1;
             const uint32_t acc_phase = (uint32_t)(li >> 1) & 1u;
@@ -374,7 +385,9 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     if (lane == 0) {
                         int blk;
                         const int n = a.div_apb.divmod(first + i / kBpa, blk);
-                        tma_store_3d(&map_y, blk * kAtomPx + (i % kBpa) * 32, k0, n, tile);
+                        // (split contraction: both parts add into y, which the launcher zeroed; a + b = b + a)
+                        if (a.ksplit == 2) tma_reduce_add_3d(&map_y, blk * kAtomPx + (i % kBpa) * 32, k0, n, tile);
+                        else tma_store_3d(&map_y, blk * kAtomPx + (i % kBpa) * 32, k0, n, tile);
                         bulk_commit_group();
                     }
                 }
@@ -447,6 +460,7 @@ bool encode_map(CUtensorMap* map, CUtensorMapDataType type, const void* base, in
 struct PwPlan {
     bool ok;
     int m_rows, n_blocks, apb, a_item, tiles, cchunks, stages, grid;
+    int ksplit, cpart;     // split of the contraction over two work items (1: none), channel chunks per item
     bool stream_a;         // the filter bank does not fit: filter chunks travel through the ring with the pixels
     bool round_filters;    // ... and (fp32) are first rounded to TF32 into the workspace
     bool pair;             // two-SM MMAs: work items are (pixel tile, pair of 128-filter blocks), one per two-block cluster
@@ -465,8 +479,6 @@ PwPlan make_pw_variant(const Shape& sh, bool pair)
     PwPlan p{};
     p.ok = false;
     p.pair = pair;
-    p.stream_a = sh.C > G::kMaxChannels;
-    p.round_filters = p.stream_a && !B16;
     p.m_rows = (sh.K <= 64 && !pair) ? 64 : 128;
     p.n_blocks = (sh.K + p.m_rows - 1) / p.m_rows;
     if (pair && p.n_blocks < 2) return p;
@@ -479,33 +491,62 @@ PwPlan make_pw_variant(const Shape& sh, bool pair)
     const int sms = sm_count();
     const int workers = pair ? sms / 2 : sms;            // blocks, or pairs of blocks
     if (workers < 1) return p;
-    // Atoms per item, one-SM form: the fewest rounds of items over the SMs, counted in atoms, plus half an atom of
-    // fixed cost per item; ties go to the larger item (wider MMAs).  64 x 32 x 32 pixels = 2048 atoms of 32: 7 per
-    // item = 293 items = two rounds of 7, where 8 per item would be two rounds of 8.
-    // Two-SM form (an even number, half for each block): the widest MMAs that still leave an item for at least half
-    // of the pairs; measured, narrower items only pay when most of the machine would otherwise idle.
-    p.a_item = 0;
+    // Atoms per item and split of the contraction.
+    // One-SM form: the fewest rounds of items over the SMs, counted in atoms, plus half an atom of fixed cost per
+    // item; ties go to the larger item (wider MMAs).  64 x 32 x 32 pixels = 2048 atoms of 32: 7 per item = 293 items =
+    // two rounds of 7, where 8 per item would be two rounds of 8.
+    // Two-SM form (an even number of atoms, half for each block): the widest MMAs that still leave an item for at
+    // least half of the pairs; measured, narrower items only pay when most of the machine would otherwise idle.
+    // Very long contractions (48 channel chunks or more: 1536 fp32 channels) on few pixels leave most SMs without
+    // an item however small the items are; there the channel chunks of a tile may be shared out to two items that
+    // both add into a zeroed y.  An item's time then counts as max(atoms, 3) (MMAs narrower than three atoms are as
+    // short as their issue) and halves with the split, which costs 0.75 atoms (the zero-fill, adds instead of
+    // stores).  Measured: 32 x 2048 x 7 x 8, 512 filters 31.6 -> 25.1 us, 128 filters 31.3 -> 22.3; with 512 or 1024
+    // channels the split never paid (32 x 512 x 14 x 14, 128 filters: 11.2 -> 14.4 us).
+    // CONV2D_B200_TMA_KSPLIT: 0 never split, 1 where the estimate says so, 2 wherever there are two chunks.
     const int forced = env_int("CONV2D_B200_TMA_ATOMS", 0);
+    const int want_ks = env_int("CONV2D_B200_TMA_KSPLIT", 1);
+    const bool deep = p.cchunks >= 48;
+    const int ks_lo = (want_ks == 2 && p.cchunks >= 2) ? 2 : 1;
+    const int ks_hi = (want_ks == 2 && p.cchunks >= 2) || (want_ks == 1 && deep) ? 2 : 1;
+    p.a_item = 0;
+    p.ksplit = 1;
     double best = 0;
-    for (int at = G::kMaxAtoms; at >= 1; --at) {
-        if (pair && (at & 1)) continue;
-        if (forced && at != (forced < G::kMaxAtoms ? forced : G::kMaxAtoms)) continue;
-        const long long tiles = (p.total_atoms + at - 1) / at;
-        if (pair) {
-            p.a_item = at;
-            if (2 * tiles * p.n_units >= workers) break;
-            continue;
+    for (int ks = ks_lo; ks <= ks_hi; ++ks) {
+        int at_pair = 0;
+        for (int at = G::kMaxAtoms; at >= 1; --at) {
+            if (pair && (at & 1)) continue;
+            if (forced && at != (forced < G::kMaxAtoms ? forced : G::kMaxAtoms)) continue;
+            const long long tiles = (p.total_atoms + at - 1) / at;
+            const long long items = tiles * p.n_units * ks;
+            if (pair) {
+                at_pair = at;
+                if (2 * items >= workers) break;
+                continue;
+            }
+            const long long rounds = (items + workers - 1) / workers;
+            const double unit = 32.0 / G::kAtomPx;                       // an fp32 atom; a 16-bit atom counts double
+            const double cost = (double)rounds * ((deep || ks == 2 ? std::max((double)at, 3.0 * unit) : (double)at) + 0.5 * unit) / ks +
+                                (ks == 2 ? 0.75 * unit : 0.0);
+            if (p.a_item == 0 || cost < best - 1e-9) { best = cost; p.a_item = at; p.ksplit = ks; }
         }
-        const long long rounds = (tiles * p.n_units + workers - 1) / workers;
-        const double cost = (double)rounds * (at + 0.5 * 32 / G::kAtomPx);
-        if (p.a_item == 0 || cost < best - 1e-9) { best = cost; p.a_item = at; }
+        if (pair && at_pair) {
+            const long long tiles = (p.total_atoms + at_pair - 1) / at_pair;
+            const long long rounds = (tiles * p.n_units * ks + workers - 1) / workers;
+            const double cost = (double)rounds * (at_pair + 2.0) / ks + (ks == 2 ? 0.75 : 0.0);
+            if (p.a_item == 0 || cost < best - 1e-9) { best = cost; p.a_item = at_pair; p.ksplit = ks; }
+        }
     }
     if (p.a_item == 0) return p;
+    p.cpart = (p.cchunks + p.ksplit - 1) / p.ksplit;
+    p.stream_a = p.cpart > kMaxChunks;
+    if (p.stream_a && env_int("CONV2D_B200_TMA_STREAM", 1) == 0) return p;
+    p.round_filters = p.stream_a && !B16;
     p.tiles = (int)((p.total_atoms + p.a_item - 1) / p.a_item);
-    p.items = (long long)p.tiles * p.n_units;
+    p.items = (long long)p.tiles * p.n_units * p.ksplit;
     if (p.items > 0x7fffffffLL) return p;
     const size_t bank = (size_t)p.m_rows * 128;           // one channel chunk of a filter block
-    const size_t fixed = (p.stream_a ? 0 : (size_t)p.cchunks * bank) + (size_t)kPwEpiWarps * 4096 + kPwBookBytes + 1024;
+    const size_t fixed = (p.stream_a ? 0 : (size_t)p.cpart * bank) + (size_t)kPwEpiWarps * 4096 + kPwBookBytes + 1024;
     const size_t stage = (p.stream_a ? bank : 0) + (size_t)(pair ? p.a_item / 2 : p.a_item) * G::kAtomBytes;
     if (fixed + 2 * stage > kPwSmemLimit) return p;
     p.stages = (int)((kPwSmemLimit - fixed) / stage);
@@ -528,11 +569,11 @@ PwPlan make_pw_variant(const Shape& sh, bool pair)
         const double rounds = (double)((p.items + workers - 1) / workers);
         const double mma = 4.0 * std::max((double)p.a_item * 16.0 * G::kAtomPx / 32.0, 120.0);
         const double stage_time = std::max({mma, (double)stage / 40.0, 2500.0 / std::max(p.stages - 1, 1)});
-        const double crit = rounds * (p.cchunks * stage_time + 2500.0);
-        const double l2 = (double)p.items * (pair ? 2 : 1) * p.cchunks * (double)stage / 3700.0;
+        const double crit = rounds * (p.cpart * stage_time + 2500.0);
+        const double l2 = (double)p.items * (pair ? 2 : 1) * p.cpart * (double)stage / 3700.0;
         const double x_bytes = (double)sh.N * sh.C * (double)HW * G::kElem, y_bytes = (double)sh.N * sh.K * (double)HW * 4.0;
         const double passes = (!p.stream_a && x_bytes > 100e6) ? p.n_units : 1;
-        const double hbm = (y_bytes + x_bytes * passes) / 3400.0;
+        const double hbm = (y_bytes * (p.ksplit == 2 ? 2.0 : 1.0) + x_bytes * passes) / 3400.0;
         p.cost = std::max({crit, l2, hbm});
     }
     p.ok = true;
@@ -551,7 +592,6 @@ PwPlan make_pw_plan(const Shape& sh)
     constexpr int kPer16 = 16 / G::kElem;
     if (HW % kPer16 != 0 || sh.C % kPer16 != 0 || sh.C > kPwMaxStreamChannels) return none;
     if (env_int("CONV2D_B200_TF32_TMA", 1) == 0) return none;
-    if (sh.C > G::kMaxChannels && env_int("CONV2D_B200_TMA_STREAM", 1) == 0) return none;
     const PwPlan one = make_pw_variant<B16>(sh, false);
     // CONV2D_B200_TMA_PAIR: 0 never, 1 where the planner expects it to be faster, 2 wherever it exists
     const int want = env_int("CONV2D_B200_TMA_PAIR", 1);
@@ -575,9 +615,9 @@ int describe_pw(const Shape& sh, char* text, size_t text_bytes)
                           ((sh.C + G::kKStep - 1) / G::kKStep * G::kKStep);
     return snprintf(text, text_bytes,
                     "tensor_core=1 kernel=pointwise_tma addressing=atoms filters_as=M two_sm=%d m_rows=%d tile_px=%d acc_sets=2 items=%lld "
-                    "grid=%d stages=%d resident_filters=%d filters_rounded_first=%d smem_bytes=%zu mma_useful_px=%.4f "
+                    "grid=%d stages=%d ksplit=%d resident_filters=%d filters_rounded_first=%d smem_bytes=%zu mma_useful_px=%.4f "
                     "mma_useful_flops=%.4f",
-                    p.pair ? 1 : 0, p.pair ? 256 : p.m_rows, p.a_item * G::kAtomPx, p.items, p.grid, p.stages, p.stream_a ? 0 : 1,
+                    p.pair ? 1 : 0, p.pair ? 256 : p.m_rows, p.a_item * G::kAtomPx, p.items, p.grid, p.stages, p.ksplit, p.stream_a ? 0 : 1,
                     p.round_filters ? 1 : 0, p.smem_bytes,
                     px / (p.pair ? cols_issued : cols), 2.0 * px * sh.K * sh.C / issued);
 }
@@ -591,6 +631,10 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
     if (!p.ok) return CONV2D_ERR_UNSUPPORTED;
     const size_t rounded_bytes = p.round_filters ? (size_t)sh.K * sh.C * sizeof(float) : 0;
     if (!workspace || workspace_bytes < kStatusBytes + rounded_bytes) return CONV2D_ERR_WORKSPACE;
+    if (p.ksplit == 2) {
+        // both parts of the contraction add into y
+        if (cudaMemsetAsync(y, 0, (size_t)sh.N * sh.K * sh.H * sh.W * sizeof(float), stream) != cudaSuccess) return CONV2D_ERR_CUDA;
+    }
     if (p.round_filters) {
         float* wp = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
         if ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(wp)) & 15u) return CONV2D_ERR_UNSUPPORTED;
@@ -659,10 +703,11 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
     a.n_blocks = p.n_blocks; a.m_rows = p.m_rows; a.items = (int)p.items;
     a.cchunks = p.cchunks; a.ksteps = (sh.C + G::kKStep - 1) / G::kKStep; a.stages = p.stages;
     a.stream_a = p.stream_a ? 1 : 0;
+    a.ksplit = p.ksplit; a.cpart = p.cpart;
     a.multi = multi ? 1 : 0;
     a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);
     a.test_drop_stage = env_int("CONV2D_B200_TF32_TEST_DROP_STAGE", -1);
-    a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles); a.div_nb = FastDiv(p.n_units);
+    a.div_apb = FastDiv(p.apb); a.div_tiles = FastDiv(p.tiles); a.div_nb = FastDiv(p.n_units * p.ksplit);
     if (env_int("CONV2D_B200_TF32_VERBOSE", 0) != 0)
         fprintf(stderr, "conv2d plan: pointwise_tma%s%s%s m_rows %d n_blocks %d atoms/item %d tiles %d stages %d grid %d smem %zu\n",
                 B16 ? " (16-bit)" : "", p.stream_a ? " (streamed filters)" : "", p.pair ? " (two-SM)" : "", p.m_rows, p.n_blocks, p.a_item, p.tiles, p.stages, p.grid, p.smem_bytes);

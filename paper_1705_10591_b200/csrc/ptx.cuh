@@ -169,6 +169,13 @@ __device__ __forceinline__ void tma_store_3d(const void* map, int c0, int c1, in
     asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
                  ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(smem_src)) : "memory");
 }
+// The same with the box added to what global memory holds (element-wise, type as in the tensor map) instead of
+// replacing it.
+__device__ __forceinline__ void tma_reduce_add_3d(const void* map, int c0, int c1, int c2, const void* smem_src)
+{
+    asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(smem_src)) : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // all but the newest `N` groups of this thread have finished READING their shared-memory source
 template <int N>

@@ -130,6 +130,7 @@ def test_random_deep_pointwise_shapes(oracle, dims, monkeypatch):
     N, C, H, W, K, R, S = dims
     # the planner's own choice, the one-SM form and the two-SM form in turn
     monkeypatch.setenv("CONV2D_B200_TMA_PAIR", str((N + C // 8 + H + K) % 3))
+    monkeypatch.setenv("CONV2D_B200_TMA_KSPLIT", str(1 + (C // 8 + W + K) % 2))     # the planner's choice / split wherever possible
     assert lib.conv2d_fwd_plan_describe(*dims, ALGO_TF32).get("kernel") == "pointwise_tma"
     assert lib.conv2d_fwd_plan_describe(*dims, 3).get("kernel") == "pointwise_tma"
     x, w = uniform((N, C, H, W), 465), uniform((K, C, R, S), 466)

@@ -366,3 +366,60 @@ def test_pointwise_two_sm_expired_wait_is_reported(oracle, dims, monkeypatch):
     monkeypatch.delenv("CONV2D_B200_TF32_TEST_DROP_STAGE")
     y_ref, yabs = oracle.conv2d_oracle(x, w)
     assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, "after a time-out")
+
+
+# Split contraction: the channel chunks of a tile are shared out to two work items that both add their partial sums
+# into a zeroed y with tensor-map reduce copies (a + b = b + a, so the result does not depend on which comes first).
+# The planner takes it for very long contractions on few pixels; CONV2D_B200_TMA_KSPLIT=2 forces it wherever a
+# shape has two channel chunks.
+KSPLIT_SHAPES = [
+    # N, C, H, W, K
+    (2, 64, 8, 8, 16),          # two chunks, one each; 64-row operand
+    (1, 100, 12, 10, 200),      # four chunks (the last holds 4 channels) as 2 + 2; ragged atoms; two filter blocks
+    (4, 256, 14, 14, 300),      # resident banks of four chunks
+    (3, 288, 16, 16, 128),      # nine chunks as 5 + 4
+    (4, 1024, 8, 8, 96),        # 16 + 16 chunks; streamed filters either way
+    (2, 2048, 7, 8, 130),       # the planner's own pick
+]
+
+
+@pytest.mark.parametrize("pair", ["0", "2"])
+@pytest.mark.parametrize("dims", KSPLIT_SHAPES)
+def test_pointwise_split_contraction(oracle, dims, pair, monkeypatch):
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K = dims
+    monkeypatch.setenv("CONV2D_B200_TMA_KSPLIT", "2")
+    monkeypatch.setenv("CONV2D_B200_TMA_PAIR", pair)
+    plan = lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, ALGO_TF32)
+    assert plan.get("kernel") == "pointwise_tma" and plan.get("ksplit") == 2
+    xi, wi = small_integers((N, C, H, W), 1101), small_integers((K, C, 1, 1), 1102)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry="general", algo=ALGO_TF32).astype(np.float64), yi_ref)
+    x, w = uniform((N, C, H, W), 1103), uniform((K, C, 1, 1), 1104)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    y1 = run_library(x, w, entry="general", algo=ALGO_TF32)
+    assert_parity(y1, y_ref, yabs, TF32_TOL, f"pointwise, split contraction {dims}")
+    # the same bits every time: neither the order of the two adds nor the timing matters
+    np.testing.assert_array_equal(run_library(x, w, entry="general", algo=ALGO_TF32), y1)
+
+
+@pytest.mark.parametrize("kind", ["bf16", "fp16"])
+def test_pointwise_split_contraction_16bit(oracle, kind, monkeypatch):
+    from helpers import B16_TOL, bf16_values, fp16_values
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K = 3, 320, 8, 8, 200
+    monkeypatch.setenv("CONV2D_B200_TMA_KSPLIT", "2")
+    assert lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, 3).get("ksplit") == 2
+    xi, wi = small_integers((N, C, H, W), 1105), small_integers((K, C, 1, 1), 1106)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry=kind).astype(np.float64), yi_ref)
+    conv = bf16_values if kind == "bf16" else fp16_values
+    x, w = conv(uniform((N, C, H, W), 1107))[0], conv(uniform((K, C, 1, 1), 1108))[0]
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry=kind), y_ref, yabs, B16_TOL, f"pointwise, split contraction {kind}")
+
+
+def test_pointwise_split_contraction_is_the_planners_pick_for_deep_layers():
+    import paper_1705_10591_b200 as lib
+    assert lib.conv2d_fwd_plan_describe(32, 2048, 7, 8, 512, 1, 1, ALGO_TF32).get("ksplit") == 2
+    assert lib.conv2d_fwd_plan_describe(32, 512, 14, 14, 128, 1, 1, ALGO_TF32).get("ksplit") == 1
