@@ -13,7 +13,9 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libconv2d_b200.so"
-SOURCES = ["conv2d_api.cu", "single_channel.cu", "general_ffma.cu", "general_tf32.cu", "pointwise_tma.cu"]
+SOURCES = ["conv2d_api.cu", "single_channel.cu", "general_ffma.cu", "general_ffma_r1.cu", "general_ffma_r2.cu",
+           "general_ffma_r3.cu", "general_ffma_r4.cu", "general_ffma_r5.cu", "general_ffma_r7.cu", "general_tf32.cu",
+           "pointwise_tma.cu"]
 
 
 def _stale() -> bool:
