@@ -19,6 +19,8 @@ CASES = [
     (2, 6, 9, 9, 5, 2, 4, 1, 2, 2),          # rectangular, even taps
     (1, 5, 12, 12, 7, 3, 3, 1, 1, 1),        # stride 1 degenerates to the padded convolution
     (1, 2, 11, 11, 3, 3, 3, 0, 0, 4),        # stride larger than the filter
+    (2, 512, 14, 16, 96, 1, 1, 0, 0, 2),     # 1 x 1, stride 2: 2048 channels on 7 x 8 pixels after the rewriting (streamed, split contraction)
+    (1, 128, 16, 16, 200, 1, 1, 0, 0, 2),    # 512 channels, 200 filters after the rewriting (streamed filters, two-SM form)
 ]
 
 
