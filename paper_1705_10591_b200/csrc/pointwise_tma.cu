@@ -86,6 +86,8 @@ struct PwArgs {
     int stages;          // activation ring depth
     int stream_a;        // 1: too many channels for a resident bank; every ring stage carries its filter chunk too
     int multi;           // 1: H*W is a whole number of atoms: one copy brings all atoms of an item that lie in one image
+    int wide;            // pairs only: an item spans two MMA widths of pixels and uses both accumulator sets at once, so
+                         // that a filter chunk serves twice the pixels (no write-back under the next item's MMAs then)
     unsigned max_polls;  // bound of every barrier wait
     int test_drop_stage; // test hook: the activation stage with this ordinal is armed but never copied (-1: none)
     FastDiv div_apb, div_tiles, div_nb;
@@ -303,11 +305,11 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 if (!(PAIR ? mbar_wait_bounded_cluster(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls)
                            : mbar_wait_bounded(&acc_empty[buf], acc_phase[buf] ^ 1u, abort_flag, a.max_polls))) { alive = false; break; }
                 tc_fence_after_sync();
-                const uint32_t n_cols = (uint32_t)((PAIR ? a.a_item : min(a.a_item, a.total_atoms - first)) * kAtomPx);
+                const int groups = (PAIR && a.wide) ? 2 : 1;                 // MMA widths per item
+                const uint32_t n_cols = (uint32_t)((PAIR ? a.a_item / groups : min(a.a_item, a.total_atoms - first)) * kAtomPx);
                 const uint32_t m = PAIR ? 256u : (uint32_t)a.m_rows;
                 const uint32_t idesc = (B16 ? idesc_b16(m, n_cols, a.fp16 != 0) : idesc_tf32(m, n_cols)) | kIdescBMajorMN;
                 const uint32_t d = tmem + (uint32_t)(buf * kAccCols);
-                bool accumulate = false;
                 for (int st = 0; st < c_n && alive; ++st) {
                     if (new_bank && !mbar_wait_bounded(&a_full[st], a_waits & 1u, abort_flag, a.max_polls)) { alive = false; break; }
                     if (!mbar_wait_bounded(&b_full[slot], ph, abort_flag, a.max_polls)) { alive = false; break; }
@@ -316,13 +318,16 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     const uint32_t a_chunk = stream_a ? stage : a_base + (uint32_t)st * a_chunk_bytes;
                     const uint32_t b_stage = stage + b_off;
                     const int ks = min(4, a.ksteps - (c_lo + st) * 4);
-                    for (int kk = 0; kk < ks; ++kk) {
-                        // filters: 32 bytes further inside the 128-byte rows; pixels: the next 8 (fp32) or 16 (16-bit) channel rows
-                        const uint64_t a_desc = smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u);
-                        const uint64_t b_desc = B16 ? smem_desc_sw128(b_stage + (uint32_t)kk * 2048u, (uint32_t)kStageCh * 128u, 1024u)
-                                                    : smem_desc_mn_sw128_32b(b_stage + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u);
-                        Op::template mma<B16>(d, a_desc, b_desc, idesc, accumulate);
-                        accumulate = true;
+                    for (int g = 0; g < groups; ++g) {
+                        // group g: this block's atoms [g * q, (g + 1) * q) of the stage, accumulator set g
+                        const uint32_t b_grp = b_stage + (uint32_t)g * (uint32_t)(my_atoms_max / groups) * kAtomBytes;
+                        for (int kk = 0; kk < ks; ++kk) {
+                            // filters: 32 bytes further inside the 128-byte rows; pixels: the next 8 (fp32) or 16 (16-bit) channel rows
+                            const uint64_t a_desc = smem_desc_sw128(a_chunk + (uint32_t)kk * 32u, 16u, 1024u);
+                            const uint64_t b_desc = B16 ? smem_desc_sw128(b_grp + (uint32_t)kk * 2048u, (uint32_t)kStageCh * 128u, 1024u)
+                                                        : smem_desc_mn_sw128_32b(b_grp + (uint32_t)kk * 1024u, (uint32_t)kStageCh * 128u, 512u);
+                            Op::template mma<B16>(d + (uint32_t)(g * kAccCols), a_desc, b_desc, idesc, st > 0 || kk > 0);
+                        }
                     }
                     Op::commit(&b_empty[slot]);
                     if (++slot == a.stages) { slot = 0; ph ^= 1u; }
@@ -334,7 +339,7 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 const int next = item + n_workers;
                 if (!stream_a && next < a.items && a.div_tiles.div(next) != bank) Op::commit(a_empty);
                 acc_phase[buf] ^= 1u;
-                buf ^= 1;
+                if (!(PAIR && a.wide)) buf ^= 1;         // (a wide item uses both sets: one logical buffer)
             }
             if (!alive) {
                 Op::commit_local(drain_bar);
@@ -357,19 +362,27 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             int bank, first, unit, c_lo, c_n;
             decode(item, bank, first);
             split(bank, unit, c_lo, c_n);
-            const int atoms = min(a.a_item, a.total_atoms - first);          // atoms of the item that exist
-            const int buf = li & 1;
-            const uint32_t acc_phase = (uint32_t)(li >> 1) & 1u;
+            const bool wide = PAIR && a.wide;
+            const int buf = wide ? 0 : li & 1;
+            const uint32_t acc_phase = (uint32_t)(wide ? li : li >> 1) & 1u;
             alive = __all_sync(0xffffffffu, alive && mbar_wait_bounded(&acc_full[buf], acc_phase, abort_flag, a.max_polls));
             if (!alive) break;
             tc_fence_after_sync();
             const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccCols);
             const int k0 = filter_row(unit) + quarter * rows_q;
             constexpr int kBpa = kAtomPx / 32;                  // 32-column blocks per atom
+            // Accumulator column -> atom of the item.  One MMA width holds the atoms of block 0 of a pair, then those of
+            // block 1; a wide item has two widths (accumulator sets 0 and 1), each with half of either block's atoms.
+            const int q_atoms = PAIR ? my_atoms_max / (wide ? 2 : 1) : a.a_item;     // atoms of one block in one width
+            const int width_blocks = (PAIR ? 2 : 1) * q_atoms * kBpa;               // 32-column blocks of one width
             if (k0 < a.K)
-                for (int i = half; i < atoms * kBpa; i += 2) {
+                for (int i = half; i < (wide ? 2 : 1) * width_blocks; i += 2) {
+                    const int g = i >= width_blocks ? 1 : 0, ib = i - g * width_blocks;    // width, block inside it
+                    const int hb = ib / (q_atoms * kBpa), jb = ib - hb * (q_atoms * kBpa); // block of the pair, block inside its part
+                    const int atom = first + hb * my_atoms_max + g * q_atoms + jb / kBpa;
+                    if (atom >= a.total_atoms) continue;            // (past the batch: zero-filled on load, never stored)
                     uint32_t v[32];
-                    tmem_ld32(lane_base + (uint32_t)(i * 32), v);
+                    tmem_ld32(lane_base + (uint32_t)(g * kAccCols + ib * 32), v);
                     tmem_ld_wait();
                     if (lane == 0) bulk_wait_group_read<0>();       // the previous store has read the tile
                     __syncwarp();
@@ -384,10 +397,10 @@ pointwise_tma_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     __syncwarp();
                     if (lane == 0) {
                         int blk;
-                        const int n = a.div_apb.divmod(first + i / kBpa, blk);
+                        const int n = a.div_apb.divmod(atom, blk);
                         // (split contraction: both parts add into y, which the launcher zeroed; a + b = b + a)
-                        if (a.ksplit == 2) tma_reduce_add_3d(&map_y, blk * kAtomPx + (i % kBpa) * 32, k0, n, tile);
-                        else tma_store_3d(&map_y, blk * kAtomPx + (i % kBpa) * 32, k0, n, tile);
+                        if (a.ksplit == 2) tma_reduce_add_3d(&map_y, blk * kAtomPx + (jb % kBpa) * 32, k0, n, tile);
+                        else tma_store_3d(&map_y, blk * kAtomPx + (jb % kBpa) * 32, k0, n, tile);
                         bulk_commit_group();
                     }
                 }
@@ -464,6 +477,7 @@ struct PwPlan {
     bool stream_a;         // the filter bank does not fit: filter chunks travel through the ring with the pixels
     bool round_filters;    // ... and (fp32) are first rounded to TF32 into the workspace
     bool pair;             // two-SM MMAs: work items are (pixel tile, pair of 128-filter blocks), one per two-block cluster
+    bool wide;             // ... whose items span two MMA widths of pixels (both accumulator sets at once)
     int n_units;           // filter blocks, or pairs of them
     long long total_atoms;
     long long items;
@@ -512,7 +526,24 @@ PwPlan make_pw_variant(const Shape& sh, bool pair)
     p.a_item = 0;
     p.ksplit = 1;
     double best = 0;
-    for (int ks = ks_lo; ks <= ks_hi; ++ks) {
+    // Wide items of a pair (twice the atoms, both accumulator sets for one item): a streamed filter chunk then serves
+    // twice the pixels, but the write-back no longer runs under the next item's MMAs.  Measured, that pays only for
+    // long contractions (32 chunks or more: 1024 fp32 channels) and only where the wide items need no more rounds
+    // over the pairs, counted in pixels, than the ordinary ones (16 x 1024 x 14 x 14, 2048 filters: 43.4 -> 36.6 us;
+    // 64 x 1024 x 16 x 16, 1024 filters: 74.4 -> 66.6; 64 x 512 x 32 x 32, 512 filters: 70.7 -> 79.9, not taken).
+    // CONV2D_B200_TMA_WIDE: 0 never, 1 so, 2 wherever a pair runs.
+    const int want_wide = env_int("CONV2D_B200_TMA_WIDE", 1);
+    {
+        const long long tiles_w = (p.total_atoms + 2 * G::kMaxAtoms - 1) / (2 * G::kMaxAtoms);
+        const long long tiles_n = (p.total_atoms + G::kMaxAtoms - 1) / G::kMaxAtoms;
+        const long long rounds_w = (tiles_w * p.n_units + workers - 1) / workers, rounds_n = (tiles_n * p.n_units + workers - 1) / workers;
+        p.wide = pair && !forced && (want_wide == 2 || (want_wide == 1 && p.cchunks >= 32 && 2 * rounds_w <= rounds_n));
+    }
+    if (p.wide) {
+        p.a_item = 2 * G::kMaxAtoms;
+        p.ksplit = 1;
+    }
+    for (int ks = ks_lo; ks <= ks_hi && !p.wide; ++ks) {
         int at_pair = 0;
         for (int at = G::kMaxAtoms; at >= 1; --at) {
             if (pair && (at & 1)) continue;
@@ -614,10 +645,10 @@ int describe_pw(const Shape& sh, char* text, size_t text_bytes)
     const double issued = 2.0 * p.m_rows * (p.pair ? 2 * p.n_units : p.n_blocks) * (p.pair ? cols_issued : cols) *
                           ((sh.C + G::kKStep - 1) / G::kKStep * G::kKStep);
     return snprintf(text, text_bytes,
-                    "tensor_core=1 kernel=pointwise_tma addressing=atoms filters_as=M two_sm=%d m_rows=%d tile_px=%d acc_sets=2 items=%lld "
+                    "tensor_core=1 kernel=pointwise_tma addressing=atoms filters_as=M two_sm=%d m_rows=%d tile_px=%d acc_sets=%d items=%lld "
                     "grid=%d stages=%d ksplit=%d resident_filters=%d filters_rounded_first=%d smem_bytes=%zu mma_useful_px=%.4f "
                     "mma_useful_flops=%.4f",
-                    p.pair ? 1 : 0, p.pair ? 256 : p.m_rows, p.a_item * G::kAtomPx, p.items, p.grid, p.stages, p.ksplit, p.stream_a ? 0 : 1,
+                    p.pair ? 1 : 0, p.pair ? 256 : p.m_rows, p.a_item * G::kAtomPx, p.wide ? 1 : 2, p.items, p.grid, p.stages, p.ksplit, p.stream_a ? 0 : 1,
                     p.round_filters ? 1 : 0, p.smem_bytes,
                     px / (p.pair ? cols_issued : cols), 2.0 * px * sh.K * sh.C / issued);
 }
@@ -703,6 +734,7 @@ conv2d_status_t launch_pw(const void* x, const void* w, float* y, const Shape& s
     a.n_blocks = p.n_blocks; a.m_rows = p.m_rows; a.items = (int)p.items;
     a.cchunks = p.cchunks; a.ksteps = (sh.C + G::kKStep - 1) / G::kKStep; a.stages = p.stages;
     a.stream_a = p.stream_a ? 1 : 0;
+    a.wide = p.wide ? 1 : 0;
     a.ksplit = p.ksplit; a.cpart = p.cpart;
     a.multi = multi ? 1 : 0;
     a.max_polls = (unsigned)env_int("CONV2D_B200_TF32_MAX_POLLS", 1 << 22);

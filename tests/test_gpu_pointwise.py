@@ -423,3 +423,39 @@ def test_pointwise_split_contraction_is_the_planners_pick_for_deep_layers():
     import paper_1705_10591_b200 as lib
     assert lib.conv2d_fwd_plan_describe(32, 2048, 7, 8, 512, 1, 1, ALGO_TF32).get("ksplit") == 2
     assert lib.conv2d_fwd_plan_describe(32, 512, 14, 14, 128, 1, 1, ALGO_TF32).get("ksplit") == 1
+
+
+@pytest.mark.parametrize("dims", [(2, 32, 8, 8, 256), (1, 64, 12, 10, 200), (4, 512, 14, 14, 300), (3, 128, 32, 32, 256),
+                                  (1, 260, 12, 10, 130), (20, 320, 16, 16, 256)])
+def test_pointwise_two_sm_wide_items(oracle, dims, monkeypatch):
+    """Items of a pair that span two MMA widths of pixels (both accumulator sets for one item): CONV2D_B200_TMA_WIDE=2
+    takes them wherever a pair runs, so that ragged items and odd filter-block counts meet this form too."""
+    import paper_1705_10591_b200 as lib
+    N, C, H, W, K = dims
+    monkeypatch.setenv("CONV2D_B200_TMA_PAIR", "2")
+    monkeypatch.setenv("CONV2D_B200_TMA_WIDE", "2")
+    plan = lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, ALGO_TF32)
+    assert plan.get("two_sm") == 1 and plan.get("acc_sets") == 1 and plan.get("tile_px") == 512
+    xi, wi = small_integers((N, C, H, W), 1111), small_integers((K, C, 1, 1), 1112)
+    yi_ref, _ = oracle.conv2d_oracle(xi, wi)
+    np.testing.assert_array_equal(run_library(xi, wi, entry="general", algo=ALGO_TF32).astype(np.float64), yi_ref)
+    x, w = uniform((N, C, H, W), 1113), uniform((K, C, 1, 1), 1114)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, f"pointwise, wide two-SM items {dims}")
+    if (H * W) % 8 == 0 and C % 8 == 0:        # (what the 16-bit operands need for this kernel)
+        from helpers import B16_TOL, bf16_values
+        assert lib.conv2d_fwd_plan_describe(N, C, H, W, K, 1, 1, 3).get("acc_sets") == 1
+        xb, wb = bf16_values(x)[0], bf16_values(w)[0]
+        yb_ref, yb_abs = oracle.conv2d_oracle(xb, wb)
+        assert_parity(run_library(xb, wb, entry="bf16"), yb_ref, yb_abs, B16_TOL, f"pointwise, wide two-SM items bf16 {dims}")
+
+
+def test_pointwise_wide_items_are_the_planners_pick_for_long_contractions(oracle):
+    import paper_1705_10591_b200 as lib
+    dims = (16, 1024, 14, 14, 2048)
+    assert lib.conv2d_fwd_plan_describe(*dims, 1, 1, ALGO_TF32).get("acc_sets") == 1
+    assert lib.conv2d_fwd_plan_describe(64, 512, 32, 32, 512, 1, 1, ALGO_TF32).get("acc_sets") == 2
+    N, C, H, W, K = dims
+    x, w = uniform((N, C, H, W), 1115), uniform((K, C, 1, 1), 1116)
+    y_ref, yabs = oracle.conv2d_oracle(x, w)
+    assert_parity(run_library(x, w, entry="general", algo=ALGO_TF32), y_ref, yabs, TF32_TOL, f"wide items by default {dims}")
